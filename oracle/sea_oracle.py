@@ -1,0 +1,196 @@
+"""fp64 CPU oracle for the SEA attention hot path.  TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plain statement of what the CUDA library computes.  It
+is imported by the tests, by the smoke check and by the benchmark's CPU
+baseline leg, and by nothing on the product path.  It shares no code with the
+CUDA kernels and never imports them.
+
+Every function works on one attention head (2-D arrays) in float64 and follows
+the paper's steps in the paper's order:
+
+    favor_features      Sec. 3 "Performer (FAVOR+)": positive random features of
+                        the softmax kernel (the paper omits the projection; the
+                        benchmark definition fixes it: x = u * d^(-1/4),
+                        phi_f(u) = exp(w_f . x - |x|^2 / 2) / sqrt(m)).
+    favor_attention     Sec. 3 "Performer (FAVOR+)": phi(Q) (phi(K)^T V), with
+                        the row normaliser phi(Q) (phi(K)^T 1); the causal form
+                        keeps running prefix sums over phi(k) v^T and phi(k).
+    decode_estimate     Sec. 3.1 "CNN Decoder", replaced by one linear head:
+                        A_hat = C_perf W_dec.
+    topk_select         Sec. 3.1 "Grouped Top-k Selection", per-query grouping:
+                        the k_hat largest entries of each row of A_hat; equal
+                        values go to the lower column.
+    expand_mask         Sec. 3.1 "Linear Sparse Attention Mask Generation" and
+                        App. "Sparse Interpolation": nearest-neighbour
+                        up-sampling of the compressed mask done on indices; a
+                        selected column c covers keys c*r .. c*r+r-1, r = T/Kc;
+                        causal rows drop keys j > i.  Output is a flat CSR.
+    sparse_attention    Sec. 3.1.1 "Sparse Attention Mechanism": rho (scores at
+                        mask positions), sigma (softmax over a row's non-zeros),
+                        then C = A* V.
+    sea_attention_head  the four steps chained.
+
+Pins (tests/test_oracle_*.py): k_hat = Kc reproduces dense (causal) softmax
+attention from a library routine; top-k equals a brute-force ordering;
+expansion equals a library nearest-neighbour resize; the feature form equals
+the normalised T x T kernel-matrix product and its expectation equals
+exp(q.k / sqrt(d)); rows of A* sum to one; causal outputs do not depend on
+later tokens.
+
+Parity unpinned: the particular omega / W_dec draws (only their seed is
+fixed), and the choice of a linear head in place of the paper's trained
+MLP + CNN decoder (a definition of this benchmark, nothing to check against).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+__all__ = [
+    "favor_features",
+    "favor_attention",
+    "decode_estimate",
+    "estimate_head",
+    "topk_select",
+    "expand_mask",
+    "sparse_attention",
+    "sea_attention_head",
+    "k_hat_from_k",
+]
+
+
+def _f64(a) -> np.ndarray:
+    return np.asarray(a, dtype=np.float64)
+
+
+def k_hat_from_k(k: int, Kc: int, T: int) -> int:
+    """Sec. 3.1: k_hat = max(1, round(k * K / T)); halves round to even."""
+    return max(1, int(np.rint(k * Kc / T)))
+
+
+def favor_features(U, omega) -> np.ndarray:
+    """Positive softmax-kernel features of the rows of U [T, d] -> [T, m]."""
+    U = _f64(U)
+    omega = _f64(omega)
+    d = U.shape[1]
+    m = omega.shape[0]
+    X = U * d ** (-0.25)
+    proj = X @ omega.T  # [T, m]
+    sq = np.sum(X * X, axis=1, keepdims=True)  # [T, 1]
+    return np.exp(proj - 0.5 * sq) / np.sqrt(m)
+
+
+def favor_attention(Q, K, V, omega, causal: bool) -> np.ndarray:
+    """Normalised linear attention C_perf [T, d]."""
+    V = _f64(V)
+    phi_q = favor_features(Q, omega)  # [T, m]
+    phi_k = favor_features(K, omega)  # [T, m]
+    T, d = V.shape
+    if not causal:
+        S = phi_k.T @ V  # [m, d]
+        z = phi_k.T @ np.ones(T)  # [m]
+        return (phi_q @ S) / (phi_q @ z)[:, None]
+    m = phi_k.shape[1]
+    S = np.zeros((m, d))
+    z = np.zeros(m)
+    C = np.empty((T, d))
+    for i in range(T):
+        S += np.outer(phi_k[i], V[i])
+        z += phi_k[i]
+        C[i] = (phi_q[i] @ S) / (phi_q[i] @ z)
+    return C
+
+
+def decode_estimate(C_perf, W_dec) -> np.ndarray:
+    """A_hat [T, Kc] = C_perf [T, d] W_dec [d, Kc]."""
+    return _f64(C_perf) @ _f64(W_dec)
+
+
+def estimate_head(Q, K, V, omega, W_dec, causal: bool) -> np.ndarray:
+    return decode_estimate(favor_attention(Q, K, V, omega, causal), W_dec)
+
+
+def topk_select(A_hat, k_hat: int) -> np.ndarray:
+    """Columns of the k_hat largest entries of each row, ascending.  [T, k_hat] int64."""
+    A_hat = _f64(A_hat)
+    T, Kc = A_hat.shape
+    if not 1 <= k_hat <= Kc:
+        raise ValueError("k_hat out of range")
+    sel = np.empty((T, k_hat), dtype=np.int64)
+    for i in range(T):
+        # descending by value; a stable sort leaves equal values in column order
+        order = np.argsort(-A_hat[i], kind="stable")
+        sel[i] = np.sort(order[:k_hat])
+    return sel
+
+
+def expand_mask(sel, T: int, Kc: int, causal: bool):
+    """Flat CSR (row_ptr [T+1], col_idx [nnz]) of the up-sampled mask of one head."""
+    sel = np.asarray(sel)
+    if T % Kc != 0:
+        raise ValueError("T must be a multiple of Kc")
+    r = T // Kc
+    row_ptr = np.zeros(T + 1, dtype=np.int64)
+    cols = []
+    for i in range(T):
+        row = []
+        for c in sel[i]:
+            for j in range(int(c) * r, int(c) * r + r):
+                if causal and j > i:
+                    continue
+                row.append(j)
+        cols.extend(row)
+        row_ptr[i + 1] = row_ptr[i] + len(row)
+    return row_ptr, np.asarray(cols, dtype=np.int64)
+
+
+def sparse_attention(Q, K, V, row_ptr, col_idx, scale: float):
+    """O [T, d] and the CSR probabilities P [nnz] of one head."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    T, d = Q.shape
+    O = np.zeros((T, d))
+    P = np.zeros(len(col_idx))
+    for i in range(T):
+        lo, hi = int(row_ptr[i]), int(row_ptr[i + 1])
+        if hi == lo:
+            continue  # an empty row keeps O_i = 0
+        js = col_idx[lo:hi]
+        s = (K[js] @ Q[i]) * scale
+        e = np.exp(s - np.max(s))
+        p = e / np.sum(e)
+        P[lo:hi] = p
+        O[i] = p @ V[js]
+    return O, P
+
+
+def sea_attention_head(Q, K, V, k_hat: int, Kc: int, causal: bool, scale: float,
+                       A_hat=None, omega=None, W_dec=None):
+    """All stages for one head.  Returns a dict with A_hat, sel, row_ptr, col_idx, O, P."""
+    T = np.asarray(Q).shape[0]
+    if A_hat is None:
+        A_hat = estimate_head(Q, K, V, omega, W_dec, causal)
+    sel = topk_select(A_hat, k_hat)
+    row_ptr, col_idx = expand_mask(sel, T, Kc, causal)
+    O, P = sparse_attention(Q, K, V, row_ptr, col_idx, scale)
+    return dict(A_hat=_f64(A_hat), sel=sel, row_ptr=row_ptr, col_idx=col_idx, O=O, P=P)
+
+
+def flatten_heads(per_head, T: int):
+    """Join per-head results in flat row order ((b*H + h)*T + i).
+
+    ``per_head`` is the list of ``sea_attention_head`` dicts in (b, h) order.
+    Row pointers become global offsets into the concatenated col_idx / P.
+    """
+    row_ptr = [np.zeros(1, dtype=np.int64)]
+    base = 0
+    for r in per_head:
+        row_ptr.append(r["row_ptr"][1:] + base)
+        base += int(r["row_ptr"][-1])
+    out = dict(
+        row_ptr=np.concatenate(row_ptr),
+        col_idx=np.concatenate([r["col_idx"] for r in per_head]),
+        P=np.concatenate([r["P"] for r in per_head]),
+        sel=np.concatenate([r["sel"] for r in per_head], axis=0),
+        O=np.concatenate([r["O"] for r in per_head], axis=0),
+        A_hat=np.concatenate([r["A_hat"] for r in per_head], axis=0),
+    )
+    return out
