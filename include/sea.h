@@ -1,0 +1,162 @@
+/*
+ * libsea -- the deployed attention layer of SEA ("Sparse linear attention with
+ * Estimated Attention mask"), as a C ABI over hand-written sm_100a kernels.
+ *
+ * The layer has the paper's two phases (Sec. 3.1): (1) a linear-cost estimate
+ * A_hat [T x Kc] of the attention matrix from a kernel-based (FAVOR+) attention
+ * followed by a decoder; (2) a per-row top-k_hat selection on A_hat that is
+ * interpolated to a sparse T x T mask and drives a sparse attention
+ * (scores at mask positions, row softmax, product with V).
+ *
+ * Conventions for every call
+ *   - Pointers named Q, K, V, O, P, A_hat, sel, row_ptr, col_idx, omega, W_dec
+ *     and ws are DEVICE pointers owned by the caller, 16-byte aligned, dense and
+ *     row-major with the last index fastest.  The library never allocates or
+ *     frees device memory and keeps no state between calls except inside `ws`.
+ *   - Q, K, V, O are [B, H, T, d] in the dtype `shape->io`; d must be 64.
+ *   - A "row" is one query: row = (b*H + h)*T + i, rows = B*H*T.
+ *   - r = T / Kc keys are covered by one compressed column (T % Kc == 0).
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *     the default stream) and the call returns without synchronising.
+ *   - Host-detectable errors (null pointer, bad shape, too small a workspace or
+ *     nnz_cap, sizes beyond int32 indexing) return a code and launch nothing.
+ *     Anomalies only visible on the device (a row longer than nnz_cap allows, a
+ *     non-finite normaliser) set bits in a status word inside `ws`, the kernel
+ *     finishes safely, and sea_device_status() reads the word back.
+ *   - Inputs must be finite.
+ *   - Calls that share a workspace must be ordered on one stream.
+ */
+#ifndef SEA_H_
+#define SEA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SEA_OK = 0,
+  SEA_ERR_INVALID_ARG = 1, /* null pointer, misaligned pointer, non-positive size */
+  SEA_ERR_UNSUPPORTED = 2, /* d != 64, T % Kc != 0, m or Kc outside the built range */
+  SEA_ERR_WORKSPACE = 3,   /* ws_bytes below sea_workspace_bytes() */
+  SEA_ERR_TOO_LARGE = 4,   /* an index would not fit int32, or nnz_cap too small */
+  SEA_ERR_CUDA = 5         /* a CUDA runtime call failed (launch, copy) */
+} sea_status;
+
+typedef enum { SEA_F32 = 0, SEA_BF16 = 1 } sea_dtype;
+
+/* Bits of the device status word (sea_device_status). */
+enum {
+  SEA_DEV_ROW_OVERFLOW = 1, /* a CSR row did not fit below nnz_cap and was truncated */
+  SEA_DEV_NONFINITE = 2     /* the estimator met a zero or non-finite normaliser */
+};
+
+typedef struct sea_shape {
+  int32_t B, H, T, d; /* batch, heads, sequence length, head width (64) */
+  int32_t m;          /* FAVOR+ random features, a multiple of 16 in [16, 128]; 0 when the estimator is not used */
+  int32_t Kc;         /* width of the compressed estimate (the paper's K), 1 <= Kc <= 2048 */
+  int32_t k_hat;      /* columns kept per row in the compressed space, 1 <= k_hat <= Kc */
+  int32_t causal;     /* 0 or 1 */
+  int32_t io;         /* sea_dtype of Q, K, V, O and P */
+  float scale;        /* softmax scale applied to q.k; 0 selects 1/sqrt(d) */
+} sea_shape;
+
+/* Bytes of device workspace that are enough for any call with this shape.
+ * The first 256 bytes of a workspace hold the device status word; the caller
+ * zeroes them once (cudaMemset) before first use. */
+sea_status sea_workspace_bytes(const sea_shape* shape, size_t* bytes);
+
+/*
+ * Attention estimation, Sec. 3.1 "Attention Matrix Estimation" with the FAVOR+
+ * attention of Sec. 3 "Performer (FAVOR+)" and one linear head in place of the
+ * trained MLP + CNN decoder of "CNN Decoder":
+ *
+ *   x = u * d^(-1/4),  phi_f(u) = exp(omega_f . x - |x|^2 / 2) / sqrt(m)
+ *   C_i = sum_j phi(q_i).phi(k_j) v_j / sum_j phi(q_i).phi(k_j)
+ *         (all j when causal == 0, j <= i when causal == 1)
+ *   A_hat = C W_dec
+ *
+ * omega [m, d] fp32 and W_dec [d, Kc] fp32 are shared by all (b, h).
+ * A_hat [B, H, T, Kc] fp32 is written in full.
+ */
+sea_status sea_estimate(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                        const float* omega, const float* W_dec, float* A_hat,
+                        void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Mask generation, Sec. 3.1 "Grouped Top-k Selection" (per-query grouping) and
+ * "Linear Sparse Attention Mask Generation" / App. "Sparse Interpolation".
+ *
+ * For every row the k_hat largest entries of A_hat[row, :] are selected; equal
+ * values (including -0 and +0) go to the lower column.  sel [rows, k_hat] int32
+ * receives the selected columns in ascending order (may be NULL).  Each selected
+ * column c is up-sampled by nearest neighbour to the keys c*r .. c*r+r-1; causal
+ * rows drop keys j > i.  The result is a flat CSR over all rows: row_ptr
+ * [rows+1] int32, col_idx [row_ptr[rows]] int32 ascending within a row.
+ * nnz_cap is the capacity of col_idx in elements; rows*k_hat*r always suffices.
+ * col_idx may be NULL (only sel and row_ptr are produced).
+ */
+sea_status sea_topk_mask(const sea_shape* shape, const float* A_hat, int32_t* sel,
+                         int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                         void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Sparse attention, Sec. 3.1.1 "Sparse Attention Mechanism": rho (q_i . k_j * scale
+ * at the mask's positions), sigma (softmax over the non-zeros of each row, so that
+ * every non-empty row of A* sums to 1) and C = A* V, fused.  The learned
+ * re-scaling s_prob is not applied.
+ *
+ * The mask is the CSR (row_ptr, col_idx).  When `sel` is given (the output of
+ * sea_topk_mask for the same shape) the kernel walks the selected runs of r keys
+ * directly and col_idx may be NULL.  O [B, H, T, d] is written in full; a row
+ * without entries gives O = 0.  P, when not NULL, receives the CSR probabilities
+ * aligned with col_idx (P[row_ptr[row] + n] belongs to the row's n-th key), in
+ * the io dtype, rounded once from fp32; O is accumulated from the unrounded
+ * probabilities.
+ */
+sea_status sea_sparse_attn(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                           const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
+                           void* O, void* P, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * The whole layer: sea_estimate -> sea_topk_mask -> sea_sparse_attn on one stream.
+ * A_hat, sel, row_ptr, col_idx and P are optional outputs (NULL = kept inside the
+ * workspace or not materialised).  When A_hat_in is not NULL the estimator stage
+ * is skipped and that estimate is used (shape->m may then be 0 and omega, W_dec
+ * may be NULL).
+ */
+sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                         const float* omega, const float* W_dec, const float* A_hat_in,
+                         void* O, float* A_hat, int32_t* sel, int32_t* row_ptr,
+                         int32_t* col_idx, int64_t nnz_cap, void* P,
+                         void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * sea_attention for callers whose tensors live in HOST memory (pinned memory
+ * gives asynchronous copies).  hQ, hK, hV, homega, hW_dec are copied to staging
+ * areas inside `ws` on the stream, the layer runs, and O is copied back to hO.
+ * Bytes needed: sea_workspace_host_bytes().  The call returns after the stream
+ * has been synchronised, so hO is valid on return.  The paper has no
+ * counterpart; this is the end-to-end form of the call above.
+ */
+sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes);
+sea_status sea_attention_host(const sea_shape* shape, const void* hQ, const void* hK,
+                              const void* hV, const float* homega, const float* hW_dec,
+                              void* hO, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Copies the device status word of `ws` to *out (host) and synchronises the
+ * stream; with `clear` != 0 the word is reset to zero afterwards. */
+sea_status sea_device_status(void* ws, int32_t* out, int32_t clear, void* cuda_stream);
+
+/* Number of kernel launches the last call of each entry point enqueued from
+ * this thread (for benchmark bookkeeping). */
+int32_t sea_last_launch_count(void);
+
+const char* sea_status_string(sea_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEA_H_ */

@@ -123,23 +123,30 @@ def topk_select(A_hat, k_hat: int) -> np.ndarray:
     return sel
 
 
-def expand_mask(sel, T: int, Kc: int, causal: bool):
-    """Flat CSR (row_ptr [T+1], col_idx [nnz]) of the up-sampled mask of one head."""
+def expand_mask(sel, T: int, Kc: int, causal: bool, query_index=None):
+    """Flat CSR (row_ptr [n+1], col_idx [nnz]) of the up-sampled mask of one head.
+
+    Row t of ``sel`` belongs to query ``query_index[t]`` (default: t, all T queries).
+    """
     sel = np.asarray(sel)
     if T % Kc != 0:
         raise ValueError("T must be a multiple of Kc")
     r = T // Kc
-    row_ptr = np.zeros(T + 1, dtype=np.int64)
+    n = sel.shape[0]
+    if query_index is None:
+        query_index = np.arange(n)
+    row_ptr = np.zeros(n + 1, dtype=np.int64)
     cols = []
-    for i in range(T):
+    for t in range(n):
+        i = int(query_index[t])
         row = []
-        for c in sel[i]:
+        for c in sel[t]:
             for j in range(int(c) * r, int(c) * r + r):
                 if causal and j > i:
                     continue
                 row.append(j)
         cols.extend(row)
-        row_ptr[i + 1] = row_ptr[i] + len(row)
+        row_ptr[t + 1] = row_ptr[t] + len(row)
     return row_ptr, np.asarray(cols, dtype=np.int64)
 
 

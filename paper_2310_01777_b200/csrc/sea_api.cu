@@ -1,0 +1,234 @@
+// C ABI of libsea: argument checks, workspace carve-up and the chaining of the stages.
+#include "sea_common.cuh"
+
+namespace sea {
+
+namespace {
+constexpr int kScanTileRows = 2048;
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+size_t io_bytes(const sea_shape& s) { return s.io == SEA_BF16 ? 2 : 4; }
+}  // namespace
+
+sea_status validate_shape(const sea_shape* s, bool need_estimator) {
+  if (s == nullptr) return SEA_ERR_INVALID_ARG;
+  if (s->B <= 0 || s->H <= 0 || s->T <= 0 || s->Kc <= 0 || s->k_hat <= 0) return SEA_ERR_INVALID_ARG;
+  if (s->causal != 0 && s->causal != 1) return SEA_ERR_INVALID_ARG;
+  if (s->io != SEA_F32 && s->io != SEA_BF16) return SEA_ERR_INVALID_ARG;
+  if (!(s->scale >= 0.f) || s->scale > 3.0e38f) return SEA_ERR_INVALID_ARG;
+  if (s->m < 0) return SEA_ERR_INVALID_ARG;
+  if (s->k_hat > s->Kc) return SEA_ERR_INVALID_ARG;
+  if (s->d != kHeadDim) return SEA_ERR_UNSUPPORTED;
+  if (s->T % s->Kc != 0) return SEA_ERR_UNSUPPORTED;
+  if (s->Kc > 2048) return SEA_ERR_UNSUPPORTED;
+  if (need_estimator && (s->m < 16 || s->m > 128 || s->m % 16 != 0)) return SEA_ERR_UNSUPPORTED;
+  const long long rows = (long long)s->B * s->H * s->T;
+  const long long r = s->T / s->Kc;
+  const long long lim = 2147483647ll;
+  if (rows + 1 > lim || rows * s->k_hat * r > lim) return SEA_ERR_TOO_LARGE;
+  return SEA_OK;
+}
+
+WsLayout ws_layout(const sea_shape& s) {
+  WsLayout L{};
+  const size_t rows = (size_t)s.B * s.H * s.T;
+  const size_t BH = (size_t)s.B * s.H;
+  const size_t nchunk = ((size_t)s.T + kEstChunk - 1) / kEstChunk;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off += align_up(bytes, 256);
+    return at;
+  };
+  L.status = take(kStatusBytes);
+  L.est_state = take(s.m > 0 ? BH * nchunk * (size_t)s.m * (kHeadDim + 1) * sizeof(float) : 0);
+  L.row_counts = take(rows * sizeof(int32_t));
+  L.tile_sums = take(((rows + kScanTileRows - 1) / kScanTileRows + 1) * sizeof(int32_t));
+  L.a_hat = take(rows * (size_t)s.Kc * sizeof(float));
+  L.sel = take(rows * (size_t)s.k_hat * sizeof(int32_t));
+  L.row_ptr = take((rows + 1) * sizeof(int32_t));
+  L.total = off;
+  return L;
+}
+
+}  // namespace sea
+
+using namespace sea;
+
+extern "C" {
+
+sea_status sea_workspace_bytes(const sea_shape* shape, size_t* bytes) {
+  if (bytes == nullptr) return SEA_ERR_INVALID_ARG;
+  const sea_status rc = validate_shape(shape, false);
+  if (rc != SEA_OK) return rc;
+  *bytes = ws_layout(*shape).total;
+  return SEA_OK;
+}
+
+sea_status sea_estimate(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                        const float* omega, const float* W_dec, float* A_hat, void* ws,
+                        size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  const sea_status rc = validate_shape(shape, true);
+  if (rc != SEA_OK) return rc;
+  if (!Q || !K || !V || !omega || !W_dec || !A_hat || !ws) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(omega) || !aligned16(W_dec) ||
+      !aligned16(A_hat) || !aligned16(ws))
+    return SEA_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*shape);
+  if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  return launch_estimate(*shape, Q, K, V, omega, W_dec, A_hat, reinterpret_cast<float*>(w + L.est_state),
+                         reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
+}
+
+sea_status sea_topk_mask(const sea_shape* shape, const float* A_hat, int32_t* sel, int32_t* row_ptr,
+                         int32_t* col_idx, int64_t nnz_cap, void* ws, size_t ws_bytes,
+                         void* cuda_stream) {
+  Launch::count() = 0;
+  const sea_status rc = validate_shape(shape, false);
+  if (rc != SEA_OK) return rc;
+  if (!A_hat || !row_ptr || !ws) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(A_hat) || !aligned16(row_ptr) || !aligned16(ws) || (sel && !aligned16(sel)) ||
+      (col_idx && !aligned16(col_idx)))
+    return SEA_ERR_INVALID_ARG;
+  if (col_idx && nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
+  if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  const WsLayout L = ws_layout(*shape);
+  if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
+  return launch_topk_mask(*shape, A_hat, sel_buf, row_ptr, col_idx, nnz_cap,
+                          reinterpret_cast<int32_t*>(w + L.row_counts),
+                          reinterpret_cast<int32_t*>(w + L.tile_sums),
+                          reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
+}
+
+sea_status sea_sparse_attn(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                           const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel, void* O,
+                           void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  (void)ws;
+  (void)ws_bytes;
+  const sea_status rc = validate_shape(shape, false);
+  if (rc != SEA_OK) return rc;
+  if (!Q || !K || !V || !row_ptr || !O || (!col_idx && !sel)) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(row_ptr) ||
+      (P && !aligned16(P)) || (sel && !aligned16(sel)) || (col_idx && !aligned16(col_idx)))
+    return SEA_ERR_INVALID_ARG;
+  return launch_sparse_attn(*shape, Q, K, V, row_ptr, col_idx, sel, O, P, static_cast<cudaStream_t>(cuda_stream));
+}
+
+sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                         const float* omega, const float* W_dec, const float* A_hat_in, void* O,
+                         float* A_hat, int32_t* sel, int32_t* row_ptr, int32_t* col_idx,
+                         int64_t nnz_cap, void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  const bool estimate = A_hat_in == nullptr;
+  sea_status rc = validate_shape(shape, estimate);
+  if (rc != SEA_OK) return rc;
+  if (!Q || !K || !V || !O || !ws) return SEA_ERR_INVALID_ARG;
+  if (estimate && (!omega || !W_dec)) return SEA_ERR_INVALID_ARG;
+  if (P && !col_idx) return SEA_ERR_INVALID_ARG;  // probabilities are only meaningful beside their indices
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(ws) ||
+      (omega && !aligned16(omega)) || (W_dec && !aligned16(W_dec)) || (A_hat_in && !aligned16(A_hat_in)) ||
+      (A_hat && !aligned16(A_hat)) || (sel && !aligned16(sel)) || (row_ptr && !aligned16(row_ptr)) ||
+      (col_idx && !aligned16(col_idx)) || (P && !aligned16(P)))
+    return SEA_ERR_INVALID_ARG;
+  if (col_idx && nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
+  if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  const WsLayout L = ws_layout(*shape);
+  if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
+
+  const float* a_use = A_hat_in;
+  if (estimate) {
+    float* a_out = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
+    rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state), status, st);
+    if (rc != SEA_OK) return rc;
+    a_use = a_out;
+  }
+  int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
+  int32_t* rp_buf = row_ptr ? row_ptr : reinterpret_cast<int32_t*>(w + L.row_ptr);
+  rc = launch_topk_mask(*shape, a_use, sel_buf, rp_buf, col_idx, nnz_cap,
+                        reinterpret_cast<int32_t*>(w + L.row_counts),
+                        reinterpret_cast<int32_t*>(w + L.tile_sums), status, st);
+  if (rc != SEA_OK) return rc;
+  return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P, st);
+}
+
+sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes) {
+  if (bytes == nullptr) return SEA_ERR_INVALID_ARG;
+  const sea_status rc = validate_shape(shape, true);
+  if (rc != SEA_OK) return rc;
+  const size_t qkv = align_up((size_t)shape->B * shape->H * shape->T * kHeadDim * io_bytes(*shape), 256);
+  const size_t om = align_up((size_t)shape->m * kHeadDim * sizeof(float), 256);
+  const size_t wd = align_up((size_t)kHeadDim * shape->Kc * sizeof(float), 256);
+  *bytes = ws_layout(*shape).total + 4 * qkv + om + wd;
+  return SEA_OK;
+}
+
+sea_status sea_attention_host(const sea_shape* shape, const void* hQ, const void* hK, const void* hV,
+                              const float* homega, const float* hW_dec, void* hO, void* ws,
+                              size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  size_t need = 0;
+  sea_status rc = sea_workspace_host_bytes(shape, &need);
+  if (rc != SEA_OK) return rc;
+  if (!hQ || !hK || !hV || !homega || !hW_dec || !hO || !ws || !aligned16(ws)) return SEA_ERR_INVALID_ARG;
+  if (ws_bytes < need) return SEA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t inner = ws_layout(*shape).total;
+  const size_t qkv_b = (size_t)shape->B * shape->H * shape->T * kHeadDim * io_bytes(*shape);
+  const size_t qkv = align_up(qkv_b, 256);
+  const size_t om_b = (size_t)shape->m * kHeadDim * sizeof(float);
+  const size_t wd_b = (size_t)kHeadDim * shape->Kc * sizeof(float);
+  char* w = static_cast<char*>(ws);
+  char* dQ = w + inner;
+  char* dK = dQ + qkv;
+  char* dV = dK + qkv;
+  char* dO = dV + qkv;
+  char* dOm = dO + qkv;
+  char* dWd = dOm + align_up(om_b, 256);
+  if (cudaMemcpyAsync(dQ, hQ, qkv_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(dK, hK, qkv_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(dV, hV, qkv_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(dOm, homega, om_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(dWd, hW_dec, wd_b, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return SEA_ERR_CUDA;
+  const int keep = Launch::count();
+  rc = sea_attention(shape, dQ, dK, dV, reinterpret_cast<const float*>(dOm),
+                     reinterpret_cast<const float*>(dWd), nullptr, dO, nullptr, nullptr, nullptr, nullptr,
+                     0, nullptr, ws, inner, cuda_stream);
+  (void)keep;
+  if (rc != SEA_OK) return rc;
+  if (cudaMemcpyAsync(hO, dO, qkv_b, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SEA_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SEA_ERR_CUDA;
+  return SEA_OK;
+}
+
+sea_status sea_device_status(void* ws, int32_t* out, int32_t clear, void* cuda_stream) {
+  if (!ws || !out) return SEA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(out, ws, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SEA_ERR_CUDA;
+  if (clear && cudaMemsetAsync(ws, 0, sizeof(int32_t), st) != cudaSuccess) return SEA_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SEA_ERR_CUDA;
+  return SEA_OK;
+}
+
+int32_t sea_last_launch_count(void) { return Launch::count(); }
+
+const char* sea_status_string(sea_status s) {
+  switch (s) {
+    case SEA_OK: return "ok";
+    case SEA_ERR_INVALID_ARG: return "invalid argument";
+    case SEA_ERR_UNSUPPORTED: return "unsupported shape";
+    case SEA_ERR_WORKSPACE: return "workspace too small";
+    case SEA_ERR_TOO_LARGE: return "size exceeds int32 indexing or nnz_cap";
+    case SEA_ERR_CUDA: return "CUDA runtime error";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

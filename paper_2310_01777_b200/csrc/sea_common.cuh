@@ -1,0 +1,116 @@
+// Shared device/host helpers of libsea (internal; the public interface is include/sea.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sea.h"
+
+namespace sea {
+
+constexpr int kHeadDim = 64;        // d, fixed by the interface
+constexpr int kStatusBytes = 256;   // head of every workspace: the device status word
+constexpr int kEstChunk = 64;       // rows per estimator chunk (prefix-state granularity)
+
+struct Launch {  // per-thread launch bookkeeping behind sea_last_launch_count()
+  static int& count() {
+    static thread_local int c = 0;
+    return c;
+  }
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Workspace carve-up shared by the entry points (all offsets 256-byte aligned).
+struct WsLayout {
+  size_t status;      // int32 status word
+  size_t est_state;   // float [BH][nchunk][m*(d+1)]  chunk states of the estimator
+  size_t row_counts;  // int32 [rows]                 per-row nnz before the scan
+  size_t tile_sums;   // int32 [ceil(rows/2048)]      scan partials
+  size_t a_hat;       // float [rows][Kc]             estimate when the caller keeps none
+  size_t sel;         // int32 [rows][k_hat]
+  size_t row_ptr;     // int32 [rows+1]
+  size_t total;
+};
+
+WsLayout ws_layout(const sea_shape& s);
+sea_status validate_shape(const sea_shape* s, bool need_estimator);
+
+// Stage launchers (defined one per .cu file).  All are asynchronous on `st`.
+sea_status launch_estimate(const sea_shape& s, const void* Q, const void* K, const void* V,
+                           const float* omega, const float* W_dec, float* A_hat,
+                           float* est_state, int32_t* status, cudaStream_t st);
+sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel,
+                            int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                            int32_t* row_counts, int32_t* tile_sums, int32_t* status,
+                            cudaStream_t st);
+sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, const void* V,
+                              const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
+                              void* O, void* P, cudaStream_t st);
+
+inline sea_status check_launch() {
+  Launch::count()++;
+  return cudaGetLastError() == cudaSuccess ? SEA_OK : SEA_ERR_CUDA;
+}
+
+#ifdef __CUDACC__
+// ---- 16-byte vector access to a row of d elements in the io dtype ------------------
+template <typename T>
+struct Io;
+
+template <>
+struct Io<float> {
+  static constexpr int kElemsPerLane = 4;   // one 16-byte load
+  static constexpr int kLanesPerRow = 16;   // 64 floats = 256 B
+  __device__ static void load(const float* p, float (&v)[4]) {
+    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  }
+  __device__ static void store(float* p, const float (&v)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+  __device__ static float to_io(float x) { return x; }
+  __device__ static float from_io(float x) { return x; }
+};
+
+template <>
+struct Io<__nv_bfloat16> {
+  static constexpr int kElemsPerLane = 8;
+  static constexpr int kLanesPerRow = 8;    // 64 bf16 = 128 B
+  __device__ static void load(const __nv_bfloat16* p, float (&v)[8]) {
+    const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  __device__ static void store(__nv_bfloat16* p, const float (&v)[8]) {
+    uint4 t;
+    uint32_t* w = reinterpret_cast<uint32_t*>(&t);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      w[i] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(p) = t;
+  }
+  __device__ static __nv_bfloat16 to_io(float x) { return __float2bfloat16_rn(x); }
+  __device__ static float from_io(__nv_bfloat16 x) { return __bfloat162float(x); }
+};
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+#endif  // __CUDACC__
+
+}  // namespace sea

@@ -1,0 +1,237 @@
+// Mask generation: per-row top-k_hat over the compressed estimate (Sec. 3.1 "Grouped Top-k
+// Selection", per-query grouping) and nearest-neighbour expansion of the selected columns to
+// a flat CSR (Sec. 3.1 "Linear Sparse Attention Mask Generation", App. "Sparse Interpolation").
+//
+// Selection is exact and unique: every value is mapped to a 32-bit key whose unsigned order
+// is the float order (with -0 folded onto +0), the k_hat-th largest key is found by a
+// bit-by-bit search with warp-wide counts, and columns holding exactly that key are taken
+// in ascending column order until k_hat are chosen.
+#include "sea_common.cuh"
+
+namespace sea {
+namespace {
+
+constexpr int kWarpsPerCta = 8;
+constexpr int kScanThreads = 256;
+constexpr int kScanPerThread = 8;
+constexpr int kScanTile = kScanThreads * kScanPerThread;
+
+__device__ __forceinline__ uint32_t order_key(float v) {
+  uint32_t u = __float_as_uint(v);
+  if (u == 0x80000000u) u = 0u;  // -0 ties with +0
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// One warp per row; lane l holds columns l, l+32, ... (VPL of them).
+template <int VPL>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
+                 int32_t* __restrict__ row_counts, int rows, int Kc, int k_hat, int seq_len, int r,
+                 int causal) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kWarpsPerCta + warp;
+  if (row >= rows) return;
+  const float* a = A_hat + (size_t)row * Kc;
+  uint32_t key[VPL];
+#pragma unroll
+  for (int t = 0; t < VPL; ++t) {
+    const int col = lane + 32 * t;
+    key[t] = col < Kc ? order_key(__ldg(a + col)) : 0u;  // padding sorts below every real value
+  }
+  // k_hat-th largest key: the largest tau with |{key >= tau}| >= k_hat
+  uint32_t tau = 0u;
+#pragma unroll 1
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t cand = tau | (1u << bit);
+    int c = 0;
+#pragma unroll
+    for (int t = 0; t < VPL; ++t) c += key[t] >= cand;
+    c = __reduce_add_sync(0xffffffffu, c);
+    if (c >= k_hat) tau = cand;
+  }
+  int n_gt = 0;
+#pragma unroll
+  for (int t = 0; t < VPL; ++t) n_gt += key[t] > tau;
+  n_gt = __reduce_add_sync(0xffffffffu, n_gt);
+  const int need = k_hat - n_gt;  // how many columns equal to tau are taken (lowest first)
+
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  const int i = row % seq_len;
+  int out_base = 0, tie_seen = 0, cnt = 0;
+  int32_t* my_sel = sel + (size_t)row * k_hat;
+#pragma unroll
+  for (int t = 0; t < VPL; ++t) {
+    const bool tie = key[t] == tau;
+    const uint32_t tb = __ballot_sync(0xffffffffu, tie);
+    const bool take = key[t] > tau || (tie && tie_seen + __popc(tb & lt_mask) < need);
+    const uint32_t sb = __ballot_sync(0xffffffffu, take);
+    if (take) {
+      const int col = lane + 32 * t;
+      my_sel[out_base + __popc(sb & lt_mask)] = col;
+      cnt += causal ? max(0, min(r, i + 1 - col * r)) : r;
+    }
+    tie_seen += __popc(tb);
+    out_base += __popc(sb);
+  }
+  if (row_counts != nullptr) {
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if (lane == 0) row_counts[row] = cnt;
+  }
+}
+
+// ---- exclusive scan of row_counts -> row_ptr (three small kernels) -------------------
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int& block_total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  const int nwarps = blockDim.x >> 5;
+  if (warp == 0) {
+    int w = lane < nwarps ? warp_tot[lane] : 0;
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    if (lane < nwarps) warp_tot[lane] = winc - w;  // exclusive offset of each warp
+    if (lane == 31) warp_tot[32] = winc;           // block total
+  }
+  __syncthreads();
+  block_total = warp_tot[32];
+  const int res = inc - v + warp_tot[warp];
+  __syncthreads();
+  return res;
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+scan_tile_sums_kernel(const int32_t* __restrict__ counts, int32_t* __restrict__ tile_sums, int rows) {
+  __shared__ int warp_tot[33];
+  const int base = blockIdx.x * kScanTile + threadIdx.x * kScanPerThread;
+  int s = 0;
+#pragma unroll
+  for (int e = 0; e < kScanPerThread; ++e) s += (base + e < rows) ? counts[base + e] : 0;
+  int total;
+  block_exclusive_scan(s, warp_tot, total);
+  if (threadIdx.x == 0) tile_sums[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(1024)
+scan_tile_offsets_kernel(int32_t* __restrict__ tile_sums, int ntiles) {
+  __shared__ int warp_tot[33];
+  int carry = 0;
+  for (int c0 = 0; c0 < ntiles; c0 += 1024) {
+    const int idx = c0 + threadIdx.x;
+    const int v = idx < ntiles ? tile_sums[idx] : 0;
+    int total;
+    const int ex = block_exclusive_scan(v, warp_tot, total);
+    if (idx < ntiles) tile_sums[idx] = carry + ex;
+    carry += total;
+  }
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+scan_write_row_ptr_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ tile_offs,
+                          int32_t* __restrict__ row_ptr, int rows) {
+  __shared__ int warp_tot[33];
+  const int base = blockIdx.x * kScanTile + threadIdx.x * kScanPerThread;
+  int v[kScanPerThread];
+  int s = 0;
+#pragma unroll
+  for (int e = 0; e < kScanPerThread; ++e) {
+    v[e] = (base + e < rows) ? counts[base + e] : 0;
+    s += v[e];
+  }
+  int total;
+  int run = block_exclusive_scan(s, warp_tot, total) + tile_offs[blockIdx.x];
+#pragma unroll
+  for (int e = 0; e < kScanPerThread; ++e) {
+    if (base + e < rows) row_ptr[base + e] = run;
+    run += v[e];
+    if (base + e == rows - 1) row_ptr[rows] = run;
+  }
+}
+
+__global__ void uniform_row_ptr_kernel(int32_t* __restrict__ row_ptr, int rows, int per_row) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i <= rows) row_ptr[i] = i * per_row;
+}
+
+// One warp per row: col_idx[row_ptr[row] + n] = sel[n / r] * r + n % r.  For a causal row the
+// kept keys are a prefix of that sequence, because sel is ascending and only the run that
+// contains the diagonal is cut.
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+fill_col_idx_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__ row_ptr,
+                    int32_t* __restrict__ col_idx, long long nnz_cap, int rows, int k_hat, int r,
+                    int32_t* __restrict__ status) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kWarpsPerCta + warp;
+  if (row >= rows) return;
+  const int base = row_ptr[row];
+  int n = row_ptr[row + 1] - base;
+  if ((long long)base + n > nnz_cap) {
+    if (lane == 0) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
+    n = (int)max(0ll, min((long long)n, nnz_cap - base));
+  }
+  const int32_t* my_sel = sel + (size_t)row * k_hat;
+  for (int pos = lane; pos < n; pos += 32) {
+    const int b = pos / r;
+    col_idx[(size_t)base + pos] = __ldg(my_sel + b) * r + (pos - b * r);
+  }
+}
+
+template <int VPL>
+void launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, int rows, const sea_shape& s,
+                 cudaStream_t st) {
+  const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+  topk_rows_kernel<VPL><<<grid, kWarpsPerCta * 32, 0, st>>>(A_hat, sel, counts, rows, s.Kc, s.k_hat,
+                                                             s.T, s.T / s.Kc, s.causal);
+}
+
+}  // namespace
+
+sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel, int32_t* row_ptr,
+                            int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts,
+                            int32_t* tile_sums, int32_t* status, cudaStream_t st) {
+  const int rows = s.B * s.H * s.T;
+  const int r = s.T / s.Kc;
+  int32_t* counts = s.causal ? row_counts : nullptr;
+  const int vpl = (s.Kc + 31) / 32;
+  if (vpl <= 1) launch_topk<1>(A_hat, sel, counts, rows, s, st);
+  else if (vpl <= 2) launch_topk<2>(A_hat, sel, counts, rows, s, st);
+  else if (vpl <= 4) launch_topk<4>(A_hat, sel, counts, rows, s, st);
+  else if (vpl <= 8) launch_topk<8>(A_hat, sel, counts, rows, s, st);
+  else if (vpl <= 16) launch_topk<16>(A_hat, sel, counts, rows, s, st);
+  else if (vpl <= 32) launch_topk<32>(A_hat, sel, counts, rows, s, st);
+  else if (vpl <= 64) launch_topk<64>(A_hat, sel, counts, rows, s, st);
+  else return SEA_ERR_UNSUPPORTED;
+  sea_status rc = check_launch();
+  if (rc != SEA_OK) return rc;
+
+  if (s.causal) {
+    const int ntiles = (rows + kScanTile - 1) / kScanTile;
+    scan_tile_sums_kernel<<<ntiles, kScanThreads, 0, st>>>(row_counts, tile_sums, rows);
+    if ((rc = check_launch()) != SEA_OK) return rc;
+    scan_tile_offsets_kernel<<<1, 1024, 0, st>>>(tile_sums, ntiles);
+    if ((rc = check_launch()) != SEA_OK) return rc;
+    scan_write_row_ptr_kernel<<<ntiles, kScanThreads, 0, st>>>(row_counts, tile_sums, row_ptr, rows);
+    if ((rc = check_launch()) != SEA_OK) return rc;
+  } else {
+    uniform_row_ptr_kernel<<<(rows + 1 + 255) / 256, 256, 0, st>>>(row_ptr, rows, s.k_hat * r);
+    if ((rc = check_launch()) != SEA_OK) return rc;
+  }
+  if (col_idx != nullptr) {
+    const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+    fill_col_idx_kernel<<<grid, kWarpsPerCta * 32, 0, st>>>(sel, row_ptr, col_idx, (long long)nnz_cap,
+                                                            rows, s.k_hat, r, status);
+    if ((rc = check_launch()) != SEA_OK) return rc;
+  }
+  return SEA_OK;
+}
+
+}  // namespace sea

@@ -1,0 +1,238 @@
+"""GPU parity: libsea (through its C ABI) against the fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2310_01777_b200 as sea
+from oracle import sea_oracle as orc
+from paper_2310_01777_b200 import binding
+from paper_2310_01777_b200.inputs import WORKLOADS, Workload, make_inputs
+from tests.helpers import (GpuRun, check_a_hat, check_float, check_head_against_oracle,
+                           global_mask_properties, head_slices, np64, scale_of)
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name, **kw):
+    base = dict(name=name, B=1, H=2, T=128, d=64, m=32, Kc=32, k_hat=4, causal=False, dtype="f32", seed=7)
+    base.update(kw)
+    return Workload(**base)
+
+
+SMALL_CASES = [
+    small("nc_f32"),
+    small("c_f32", causal=True),
+    small("nc_bf16", dtype="bf16", B=2, H=3, T=256, Kc=64, k_hat=8, m=64),
+    small("c_bf16", dtype="bf16", causal=True, B=2, H=2, T=320, Kc=80, k_hat=10, m=128),  # Kc % 32 != 0, several chunks
+    small("ragged_T", causal=True, T=96, Kc=32, k_hat=5, m=16),       # T % 64 != 0, r = 3
+    small("ragged_nc", T=200, Kc=40, k_hat=7, m=48, dtype="bf16"),    # r = 5, last chunk of 8 rows
+    small("r1", causal=True, T=64, Kc=64, k_hat=64),                  # r = 1 and k_hat = Kc: dense causal
+    small("k1", causal=True, T=128, Kc=8, k_hat=1),                   # one column, many empty rows
+    small("dense_nc", T=128, Kc=16, k_hat=16, dtype="bf16"),          # k_hat = Kc: dense attention
+    small("long_rows", T=2048, Kc=64, k_hat=40, H=1, causal=True, dtype="bf16"),  # 1280 keys per row > one smem chunk
+    small("wide_Kc", T=1024, Kc=1024, k_hat=33, H=1, causal=True, dtype="bf16", m=64),  # 32 values per lane in the select
+]
+
+
+@pytest.mark.parametrize("w", SMALL_CASES, ids=lambda w: w.name)
+def test_stages_match_oracle_on_small_shapes(w):
+    run = GpuRun(w)
+    run.estimate()
+    run.topk_mask()
+    run.sparse_attn()
+    run.sync()
+    assert run.status() == 0
+    for b in range(w.B):
+        for h in range(w.H):
+            check_head_against_oracle(run, b, h, check_estimate=True)
+    global_mask_properties(run)
+
+
+@pytest.mark.parametrize("w", SMALL_CASES[:6], ids=lambda w: w.name)
+def test_fused_call_equals_stage_calls_bitwise(w):
+    a = GpuRun(w)
+    a.estimate(); a.topk_mask(); a.sparse_attn(); a.sync()
+    b = GpuRun(w)
+    b.attention(); b.sync()
+    assert b.status() == 0
+    nnz = int(a.row_ptr[-1])
+    for name in ("A_hat", "sel", "row_ptr", "O"):
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+    assert torch.equal(a.col_idx[:nnz], b.col_idx[:nnz])
+    assert torch.equal(a.P[:nnz].view(torch.int16 if w.dtype == "bf16" else torch.int32),
+                       b.P[:nnz].view(torch.int16 if w.dtype == "bf16" else torch.int32))
+    # running it again gives the same bits (fixed-order reductions, no atomics on data)
+    c = GpuRun(w)
+    c.attention(); c.sync()
+    assert torch.equal(b.O, c.O) and torch.equal(b.A_hat, c.A_hat)
+
+
+def test_fused_call_with_optional_outputs_omitted():
+    w = small("opt_out", causal=True, dtype="bf16", T=256, Kc=32, k_hat=6)
+    full = GpuRun(w)
+    full.attention(); full.sync()
+    lean = GpuRun(w, want_col=False)
+    sea.sea_attention(lean.shape, lean.d["Q"], lean.d["K"], lean.d["V"], lean.d["omega"], lean.d["W_dec"],
+                      lean.O, lean.ws)
+    lean.sync()
+    assert torch.equal(full.O, lean.O)
+
+
+def test_csr_path_equals_sel_path_and_generic_csr_matches_oracle():
+    w = small("csr", causal=True, dtype="bf16", T=256, Kc=32, k_hat=6)
+    run = GpuRun(w)
+    run.estimate(); run.topk_mask(); run.sparse_attn(use_sel=True); run.sync()
+    O_sel, P_sel = run.O.clone(), run.P.clone()
+    run.O.fill_(float("nan")); run.P.fill_(float("nan"))
+    run.sparse_attn(use_sel=False); run.sync()
+    nnz = int(run.row_ptr[-1])
+    assert torch.equal(O_sel, run.O)
+    assert torch.equal(P_sel[:nnz].view(torch.int16), run.P[:nnz].view(torch.int16))
+
+    # an arbitrary CSR (unsorted columns, repeated keys, empty rows, one very long row)
+    for dtype in ("f32", "bf16"):
+        w2 = small("anycsr", dtype=dtype, B=1, H=2, T=192, Kc=192, k_hat=192)
+        g = np.random.default_rng(5)
+        host = make_inputs(w2)
+        counts = g.integers(0, 40, size=w2.rows)
+        counts[3] = 0
+        counts[17] = 1500  # longer than the 1024-entry shared-memory chunk
+        row_ptr = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+        col_idx = g.integers(0, w2.T, size=int(row_ptr[-1])).astype(np.int32)
+        dev = "cuda:0"
+        io = torch.bfloat16 if dtype == "bf16" else torch.float32
+        O = torch.empty((w2.B, w2.H, w2.T, w2.d), dtype=io, device=dev)
+        P = torch.empty(int(row_ptr[-1]), dtype=io, device=dev)
+        d = {k: v.to(dev) for k, v in host.items()}
+        sea.sea_sparse_attn(sea.make_shape(w2), d["Q"], d["K"], d["V"], torch.from_numpy(row_ptr).to(dev),
+                            torch.from_numpy(col_idx).to(dev), None, O, P)
+        torch.cuda.synchronize()
+        for h in range(w2.H):
+            rp = row_ptr[h * w2.T:(h + 1) * w2.T + 1].astype(np.int64)
+            refO, refP = orc.sparse_attention(np64(host["Q"][0, h]), np64(host["K"][0, h]), np64(host["V"][0, h]),
+                                              rp - rp[0], col_idx[rp[0]:rp[-1]].astype(np.int64), scale_of(w2))
+            check_float(np64(O[0, h]), refO, dtype, "O")
+            check_float(np64(P[rp[0]:rp[-1]]), refP, dtype, "P")
+
+
+def test_topk_ties_and_signed_zeros_are_bit_exact():
+    w = small("ties", T=256, Kc=128, k_hat=16, m=0, H=1)
+    host = make_inputs(w)
+    a = host["A_hat"]
+    a[:] = torch.round(a * 2) / 2          # heavy duplication: ties everywhere
+    a[0, 0, 0, :] = 0.0                    # an all-equal row
+    a[0, 0, 1, ::2] = -0.0                 # +0 / -0 must tie
+    a[0, 0, 1, 1::2] = 0.0
+    a[0, 0, 2, :] = -1.0
+    a[0, 0, 2, 100:120] = 5.0              # more maxima than k_hat
+    run = GpuRun(w, inputs=host)
+    run.topk_mask(); run.sparse_attn(); run.sync()
+    check_head_against_oracle(run, 0, 0, check_estimate=False)
+
+
+def test_small_nnz_cap_sets_status_and_stays_in_bounds():
+    w = small("cap", causal=False, T=128, Kc=32, k_hat=4, H=1, m=0)
+    run = GpuRun(w)
+    cap = w.nnz_cap // 2 + 3
+    guard = torch.full((w.nnz_cap,), -7, dtype=torch.int32, device=run.dev)
+    sea.sea_topk_mask(run.shape, run.A_hat, run.sel, run.row_ptr, guard, run.ws, nnz_cap=cap)
+    run.sync()
+    assert run.status() & binding.SEA_DEV_ROW_OVERFLOW
+    assert run.status() == 0  # cleared by the read above
+    assert bool((guard[cap:] == -7).all()) and bool((guard[:cap] >= 0).all())
+
+
+def test_causality_by_perturbation_on_device():
+    w = small("perturb", causal=True, dtype="bf16", T=256, Kc=32, k_hat=6, m=64, H=1)
+    t = 140
+    a = GpuRun(w)
+    a.attention(); a.sync()
+    host2 = {k: v.clone() for k, v in a.host.items()}
+    g = torch.Generator().manual_seed(99)
+    for k in ("Q", "K", "V"):
+        host2[k][:, :, t + 1:] = torch.randn(host2[k][:, :, t + 1:].shape, generator=g).to(host2[k].dtype)
+    b = GpuRun(w, inputs=host2)
+    b.attention(); b.sync()
+    n = int(a.row_ptr[t + 1])
+    assert torch.equal(a.A_hat[:, :, :t + 1], b.A_hat[:, :, :t + 1])
+    assert torch.equal(a.sel[:t + 1], b.sel[:t + 1])
+    assert torch.equal(a.row_ptr[:t + 2], b.row_ptr[:t + 2])
+    assert torch.equal(a.col_idx[:n], b.col_idx[:n])
+    assert torch.equal(a.O[:, :, :t + 1], b.O[:, :, :t + 1])
+    assert torch.equal(a.P[:n].view(torch.int16), b.P[:n].view(torch.int16))
+
+
+def test_host_entry_point_matches_device_entry_point():
+    w = small("host", causal=True, dtype="bf16", T=256, Kc=32, k_hat=6, m=64)
+    dev_run = GpuRun(w)
+    dev_run.attention(); dev_run.sync()
+    shp = sea.make_shape(w)
+    ws = sea.new_workspace(shp, "cuda:0", host_staging=True)
+    h = {k: v.pin_memory() for k, v in dev_run.host.items()}
+    hO = torch.empty_like(h["Q"]).pin_memory()
+    sea.sea_attention_host(shp, h["Q"], h["K"], h["V"], h["omega"], h["W_dec"], hO, ws)
+    assert torch.equal(hO, dev_run.O.cpu())
+    assert sea.sea_last_launch_count() >= 3
+
+
+# ---------------------------------------------------------------------------------------
+# The five benchmark workloads at full size, in the launch configuration the benchmark times
+# (one sea_attention call).  The oracle checks a sample of heads element by element (all heads
+# for the tiny case); properties that hold at any size are checked over every row on the device.
+# ---------------------------------------------------------------------------------------
+FULL = [
+    ("tiny_f32", "all"),
+    ("bert_base", [(0, 0), (13, 5), (31, 11)]),
+    ("opt_125m", [(0, 0), (7, 11)]),
+    ("opt_1p3b", [(0, 0), (2, 17), (3, 31)]),
+    ("long_8k", [(0, 9)]),
+]
+
+
+@pytest.mark.parametrize("name,heads", FULL, ids=[f[0] for f in FULL])
+def test_benchmark_workloads_full_size(name, heads):
+    w = WORKLOADS[name]
+    run = GpuRun(w)
+    run.attention()
+    run.sync()
+    assert run.status() == 0
+    nnz = global_mask_properties(run)
+    if not w.causal:
+        assert nnz == w.rows * w.k_hat * w.r  # the paper's constant T*k non-zeros per head
+    if heads == "all":
+        heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    for b, h in heads:
+        check_head_against_oracle(run, b, h, check_estimate=w.m > 0)
+
+
+@pytest.mark.parametrize("name,head,n_rows", [("long_16k", (0, 3), 96), ("long_32k", (0, 30), 64)])
+def test_long_context_sampled_rows(name, head, n_rows):
+    """T = 16384 / 32768: the oracle computes the estimate for a whole head (linear cost) but the
+    mask and the attention only for a sample of rows, one by one."""
+    w = WORKLOADS[name]
+    run = GpuRun(w, want_P=True)
+    run.attention()
+    run.sync()
+    assert run.status() == 0
+    global_mask_properties(run)
+    b, h = head
+    bh = b * w.H + h
+    g = np.random.default_rng(11)
+    rows = np.unique(np.concatenate([[0, 1, 15, 16, 17, w.T - 1], g.integers(0, w.T, size=n_rows)]))
+    Q, K, V = (np64(run.host[k][b, h]) for k in ("Q", "K", "V"))
+    C = orc.favor_attention(Q, K, V, np64(run.host["omega"]), True)
+    ref_a = orc.decode_estimate(C[rows], np64(run.host["W_dec"]))
+    a_gpu = run.A_hat[b, h][torch.from_numpy(rows).to(run.dev)].cpu().numpy()
+    check_a_hat(a_gpu, ref_a)
+    sel_ref = orc.topk_select(a_gpu, w.k_hat)
+    sel_gpu = run.sel[bh * w.T + torch.from_numpy(rows).to(run.dev)].cpu().numpy()
+    np.testing.assert_array_equal(sel_gpu, sel_ref)
+    rp_ref, col_ref = orc.expand_mask(sel_ref, w.T, w.Kc, True, query_index=rows)
+    O_ref, P_ref = orc.sparse_attention(Q[rows], K, V, rp_ref, col_ref, scale_of(w))
+    rp_gpu = run.row_ptr.cpu().numpy().astype(np.int64)
+    for t, i in enumerate(rows):
+        lo, hi = rp_gpu[bh * w.T + i], rp_gpu[bh * w.T + i + 1]
+        assert hi - lo == rp_ref[t + 1] - rp_ref[t]
+        np.testing.assert_array_equal(run.col_idx[lo:hi].cpu().numpy(), col_ref[rp_ref[t]:rp_ref[t + 1]])
+        check_float(np64(run.P[lo:hi]), P_ref[rp_ref[t]:rp_ref[t + 1]], w.dtype, "P")
+    check_float(np64(run.O[b, h])[rows], O_ref, w.dtype, "O")
