@@ -41,6 +41,7 @@ WsLayout ws_layout(const sea_shape& s) {
   };
   L.status = take(kStatusBytes);
   L.est_state = take(s.m > 0 ? BH * nchunk * (size_t)s.m * (kHeadDim + 1) * sizeof(float) : 0);
+  L.est_split = take(s.m > 0 ? estimate_split_bytes(s) : 0);
   L.row_counts = take(rows * sizeof(int32_t));
   L.tile_sums = take(((rows + kScanTileRows - 1) / kScanTileRows + 1) * sizeof(int32_t));
   L.a_hat = take(rows * (size_t)s.Kc * sizeof(float));
@@ -78,7 +79,8 @@ sea_status sea_estimate(const sea_shape* shape, const void* Q, const void* K, co
   if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
   char* w = static_cast<char*>(ws);
   return launch_estimate(*shape, Q, K, V, omega, W_dec, A_hat, reinterpret_cast<float*>(w + L.est_state),
-                         reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
+                         w + L.est_split, reinterpret_cast<int32_t*>(w + L.status),
+                         static_cast<cudaStream_t>(cuda_stream));
 }
 
 sea_status sea_topk_mask(const sea_shape* shape, const float* A_hat, int32_t* sel, int32_t* row_ptr,
@@ -145,7 +147,8 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
   const float* a_use = A_hat_in;
   if (estimate) {
     float* a_out = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
-    rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state), status, st);
+    rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state),
+                         w + L.est_split, status, st);
     if (rc != SEA_OK) return rc;
     a_use = a_out;
   }

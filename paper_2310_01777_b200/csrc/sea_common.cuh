@@ -26,6 +26,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct WsLayout {
   size_t status;      // int32 status word
   size_t est_state;   // float [BH][nchunk][m*(d+1)]  chunk states of the estimator
+  size_t est_split;   // bf16 head/remainder copies of omega and W_dec (bf16 estimator)
   size_t row_counts;  // int32 [rows]                 per-row nnz before the scan
   size_t tile_sums;   // int32 [ceil(rows/2048)]      scan partials
   size_t a_hat;       // float [rows][Kc]             estimate when the caller keeps none
@@ -40,7 +41,14 @@ sea_status validate_shape(const sea_shape* s, bool need_estimator);
 // Stage launchers (defined one per .cu file).  All are asynchronous on `st`.
 sea_status launch_estimate(const sea_shape& s, const void* Q, const void* K, const void* V,
                            const float* omega, const float* W_dec, float* A_hat,
-                           float* est_state, int32_t* status, cudaStream_t st);
+                           float* est_state, void* est_split, int32_t* status, cudaStream_t st);
+sea_status launch_estimate_f32(const sea_shape& s, const void* Q, const void* K, const void* V,
+                               const float* omega, const float* W_dec, float* A_hat,
+                               float* est_state, int32_t* status, cudaStream_t st);
+sea_status launch_estimate_bf16(const sea_shape& s, const void* Q, const void* K, const void* V,
+                                const float* omega, const float* W_dec, float* A_hat,
+                                float* est_state, void* est_split, int32_t* status, cudaStream_t st);
+size_t estimate_split_bytes(const sea_shape& s);
 sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel,
                             int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
                             int32_t* row_counts, int32_t* tile_sums, int32_t* status,

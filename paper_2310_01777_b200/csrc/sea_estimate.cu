@@ -9,7 +9,8 @@
 // in a fixed order: an exclusive prefix for causal attention, the total otherwise.
 // Kernel 3 computes, per chunk, phi(Q_c) S + (phi(Q_c) phi(K_c)^T . tril) [V_c | 1]
 // (the second term only when causal), divides, applies W_dec and writes A_hat.
-// All arithmetic is fp32.
+// This file is the plain fp32 FMA form used for fp32 inputs; bf16 inputs take the tensor-core
+// form in sea_estimate_mma.cu.
 #include "sea_common.cuh"
 
 namespace sea {
@@ -313,15 +314,19 @@ sea_status launch_typed(const sea_shape& s, const T* Q, const T* K, const T* V, 
 
 }  // namespace
 
-sea_status launch_estimate(const sea_shape& s, const void* Q, const void* K, const void* V,
-                           const float* omega, const float* W_dec, float* A_hat, float* est_state,
-                           int32_t* status, cudaStream_t st) {
-  if (s.io == SEA_BF16) {
-    using T = __nv_bfloat16;
-    return launch_typed<T>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, status, st);
-  }
+sea_status launch_estimate_f32(const sea_shape& s, const void* Q, const void* K, const void* V,
+                               const float* omega, const float* W_dec, float* A_hat, float* est_state,
+                               int32_t* status, cudaStream_t st) {
   return launch_typed<float>(s, (const float*)Q, (const float*)K, (const float*)V, omega, W_dec, A_hat,
                              est_state, status, st);
+}
+
+sea_status launch_estimate(const sea_shape& s, const void* Q, const void* K, const void* V,
+                           const float* omega, const float* W_dec, float* A_hat, float* est_state,
+                           void* est_split, int32_t* status, cudaStream_t st) {
+  if (s.io == SEA_BF16)
+    return launch_estimate_bf16(s, Q, K, V, omega, W_dec, A_hat, est_state, est_split, status, st);
+  return launch_estimate_f32(s, Q, K, V, omega, W_dec, A_hat, est_state, status, st);
 }
 
 }  // namespace sea
