@@ -264,48 +264,74 @@ favor_key_state_mma_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloa
 }
 
 // Kernel 2: fixed-order combination of the chunk states of each head (exclusive prefix when
-// causal, total otherwise).
-__global__ void favor_state_scan_mma_kernel(float* __restrict__ state, int nchunk, int per_chunk,
-                                            long long total_threads, int causal) {
+// causal, total otherwise), written as the bf16 head / remainder operand that kernel 3 copies
+// straight into shared memory: per (head, chunk) two [MP][72] matrices, columns 0..63 the value
+// part, column 64 the normaliser part z, the rest (and feature rows >= m) zero.
+constexpr int kSLd = kHeadDim + 8;  // 72 columns: 144-byte pitch
+
+__global__ void favor_state_scan_mma_kernel(const float* __restrict__ state, __nv_bfloat16* __restrict__ split,
+                                            int nchunk, int m, int MP, long long total_threads, int causal) {
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= total_threads) return;
-  const long long bh = gid / per_chunk;
-  const int e = (int)(gid - bh * per_chunk);
-  float* p = state + (size_t)bh * nchunk * per_chunk + e;
-  float run = 0.f;
-  for (int c = 0; c < nchunk; ++c) {
-    const float v = p[(size_t)c * per_chunk];
-    if (causal) p[(size_t)c * per_chunk] = run;
-    run += v;
+  const int per_head = MP * (kSLd / 2);
+  const long long bh = gid / per_head;
+  const int v = (int)(gid - bh * per_head);
+  const int f = v / (kSLd / 2), c = (v - f * (kSLd / 2)) * 2;
+  const bool in0 = f < m && c < kStateCols, in1 = f < m && c + 1 < kStateCols;
+  const size_t per_chunk = (size_t)m * kStateCols;
+  const float* p = state + (size_t)bh * nchunk * per_chunk + (size_t)f * kStateCols + c;
+  const size_t out_chunk = 2 * (size_t)MP * kSLd;
+  __nv_bfloat16* q = split + (size_t)bh * nchunk * out_chunk + (size_t)f * kSLd + c;
+  float r0 = 0.f, r1 = 0.f;
+#pragma unroll 4
+  for (int ch = 0; ch < nchunk; ++ch) {
+    const float x = in0 ? p[ch * per_chunk] : 0.f;
+    const float y = in1 ? p[ch * per_chunk + 1] : 0.f;
+    if (causal) {
+      uint32_t hi, lo;
+      split2(r0, r1, hi, lo);
+      *reinterpret_cast<uint32_t*>(q + ch * out_chunk) = hi;
+      *reinterpret_cast<uint32_t*>(q + ch * out_chunk + (size_t)MP * kSLd) = lo;
+    }
+    r0 += x;
+    r1 += y;
   }
-  if (!causal) p[0] = run;
+  if (!causal) {
+    uint32_t hi, lo;
+    split2(r0, r1, hi, lo);
+    *reinterpret_cast<uint32_t*>(q) = hi;
+    *reinterpret_cast<uint32_t*>(q + (size_t)MP * kSLd) = lo;
+  }
 }
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src));
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
 
 template <int MP>
 struct SmemOutput {
-  // omega' during the projections, then the staged W_dec tile
-  __nv_bfloat16 om_hi[(MP * kLd64 > kHeadDim * (kWTile + kPad)) ? MP * kLd64 : kHeadDim * (kWTile + kPad)];
-  __nv_bfloat16 om_lo[(MP * kLd64 > kHeadDim * (kWTile + kPad)) ? MP * kLd64 : kHeadDim * (kWTile + kPad)];
+  // omega' (pitch 72) during the projections, then the prefix state S (pitch 72)
+  __nv_bfloat16 r1_hi[MP * kSLd], r1_lo[MP * kSLd];
   __nv_bfloat16 ph_hi[kC * (MP + kPad)], ph_lo[kC * (MP + kPad)];
   __nv_bfloat16 v[kC * kLd64];
-  __nv_bfloat16 s_hi[MP * (kHeadDim + 8)], s_lo[MP * (kHeadDim + 8)];  // [f][72]: value columns, z, zeros
 };
 
 // Kernel 3: per chunk, num = phi(Q) S + (phi(Q) phi(K)^T . tril) V, den likewise with the ones
-// column, C = num / den, A_hat = C W_dec.
+// column, C = num / den, written as bf16 head / remainder [rows][64] for the decoder product.
 template <int MP>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)
 favor_output_mma_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
                         const __nv_bfloat16* __restrict__ V, const __nv_bfloat16* __restrict__ om_hi_g,
-                        const __nv_bfloat16* __restrict__ om_lo_g, const __nv_bfloat16* __restrict__ w_hi_g,
-                        const __nv_bfloat16* __restrict__ w_lo_g, const float* __restrict__ state,
-                        float* __restrict__ A_hat, int32_t* __restrict__ status, int seq_len, int m, int Kc,
-                        int KcP, int nchunk, int causal) {
+                        const __nv_bfloat16* __restrict__ om_lo_g, const __nv_bfloat16* __restrict__ s_split,
+                        __nv_bfloat16* __restrict__ c_hi, __nv_bfloat16* __restrict__ c_lo,
+                        int32_t* __restrict__ status, int seq_len, int m, int nchunk, int causal) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SmemOutput<MP>& sm = *reinterpret_cast<SmemOutput<MP>*>(smem_raw);
   constexpr int LDP = MP + kPad;
-  constexpr int LDS = kHeadDim + 8;  // 72: 144-byte pitch
-  constexpr int LDW = kWTile + kPad;        // 136
+  constexpr int LDS = kSLd;
+  static_assert(kLd64 == kSLd, "omega' and S share one region and one pitch");
   const int chunk = blockIdx.x, bh = blockIdx.y, row0 = chunk * kC;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const size_t head = (size_t)bh * seq_len * kHeadDim;
@@ -313,24 +339,9 @@ favor_output_mma_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
   const int r0 = 16 * warp;
   const float inv_sqrt_m = rsqrtf((float)m);
 
-  stage_rows64(sm.om_hi, om_hi_g, MP, MP);
-  stage_rows64(sm.om_lo, om_lo_g, MP, MP);
+  stage_rows64(sm.r1_hi, om_hi_g, MP, MP);
+  stage_rows64(sm.r1_lo, om_lo_g, MP, MP);
   if (causal) stage_rows64(sm.v, V + head + (size_t)row0 * kHeadDim, kC, valid);
-  {  // prefix (or total) state: fp32 [m][65] -> bf16 head / remainder [MP][72], zero padded
-    const float* st = state + ((size_t)bh * nchunk + (causal ? chunk : 0)) * (size_t)m * kStateCols;
-    for (int v = threadIdx.x; v < MP * (LDS / 2); v += kThreads) {
-      const int f = v / (LDS / 2), c = (v - f * (LDS / 2)) * 2;
-      float x = 0.f, y = 0.f;
-      if (f < m) {
-        if (c < kStateCols) x = st[(size_t)f * kStateCols + c];
-        if (c + 1 < kStateCols) y = st[(size_t)f * kStateCols + c + 1];
-      }
-      uint32_t hi, lo;
-      split2(x, y, hi, lo);
-      *reinterpret_cast<uint32_t*>(sm.s_hi + f * LDS + c) = hi;
-      *reinterpret_cast<uint32_t*>(sm.s_lo + f * LDS + c) = lo;
-    }
-  }
   __syncthreads();
 
   uint32_t qh[MP / 16][4], ql[MP / 16][4];  // phi(Q) rows of this warp as A fragments
@@ -339,7 +350,7 @@ favor_output_mma_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
     float sq_g, sq_g8;
     load_rows_frag(a, sq_g, sq_g8, Q + head, row0 + r0 + g, seq_len, t);
     float acc[MP / 8][4];
-    project<MP>(acc, a, sm.om_hi, sm.om_lo, lane);
+    project<MP>(acc, a, sm.r1_hi, sm.r1_lo, lane);
     features_frag<MP>(qh, ql, acc, sq_g, sq_g8, true, true, m, inv_sqrt_m, t);
   }
   if (causal) {
@@ -347,12 +358,21 @@ favor_output_mma_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
     float sq_g, sq_g8;
     load_rows_frag(a, sq_g, sq_g8, K + head, row0 + r0 + g, seq_len, t);
     float acc[MP / 8][4];
-    project<MP>(acc, a, sm.om_hi, sm.om_lo, lane);
+    project<MP>(acc, a, sm.r1_hi, sm.r1_lo, lane);
     uint32_t fh[MP / 16][4], fl[MP / 16][4];
     features_frag<MP>(fh, fl, acc, sq_g, sq_g8, r0 + g < valid, r0 + g + 8 < valid, m, inv_sqrt_m, t);
     store_features<MP>(sm.ph_hi, sm.ph_lo, fh, fl, r0, g, t);
   }
-  __syncthreads();  // phi(K) visible; omega' no longer needed
+  __syncthreads();  // phi(K) visible; omega' no longer needed: its region takes the state S
+
+  {  // asynchronous copy of the prefix (or total) state, overlapped with the in-chunk part
+    const __nv_bfloat16* src = s_split + ((size_t)bh * nchunk + (causal ? chunk : 0)) * (2 * (size_t)MP * kSLd);
+    constexpr int kVecs = MP * kSLd / 8;  // 16-byte pieces per matrix
+    for (int v = threadIdx.x; v < kVecs; v += kThreads) {
+      cp_async16(sm.r1_hi + v * 8, src + v * 8);
+      cp_async16(sm.r1_lo + v * 8, src + (size_t)MP * kSLd + v * 8);
+    }
+  }
 
   // num[0..7] = 64 value columns, num[8] = normaliser column (n = 0 of the ninth tile)
   float num[9][4];
@@ -360,30 +380,6 @@ favor_output_mma_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
   for (int j = 0; j < 9; ++j)
 #pragma unroll
     for (int e = 0; e < 4; ++e) num[j][e] = 0.f;
-#pragma unroll
-  for (int ks = 0; ks < MP / 16; ++ks) {
-    const int brow = 16 * ks + (lane & 7) + 8 * ((lane >> 3) & 1);
-#pragma unroll
-    for (int np = 0; np < 4; ++np) {
-      uint32_t bh_[4], bl_[4];  // S stored [k = f][n = e]
-      const int off = brow * LDS + 16 * np + 8 * (lane >> 4);
-      ldsm_x4_t(bh_, sm.s_hi + off);
-      ldsm_x4_t(bl_, sm.s_lo + off);
-      mma16816(num[2 * np], qh[ks], bh_[0], bh_[1]);
-      mma16816(num[2 * np + 1], qh[ks], bh_[2], bh_[3]);
-      mma16816(num[2 * np], qh[ks], bl_[0], bl_[1]);
-      mma16816(num[2 * np + 1], qh[ks], bl_[2], bl_[3]);
-      mma16816(num[2 * np], ql[ks], bh_[0], bh_[1]);
-      mma16816(num[2 * np + 1], ql[ks], bh_[2], bh_[3]);
-    }
-    uint32_t zh[2], zl[2];
-    const int zoff = (16 * ks + (lane & 15)) * LDS + kHeadDim;
-    ldsm_x2_t(zh, sm.s_hi + zoff);
-    ldsm_x2_t(zl, sm.s_lo + zoff);
-    mma16816(num[8], qh[ks], zh[0], zh[1]);
-    mma16816(num[8], qh[ks], zl[0], zl[1]);
-    mma16816(num[8], ql[ks], zh[0], zh[1]);
-  }
 
   float den_g = 0.f, den_g8 = 0.f;  // this lane's share of the in-chunk normaliser
   if (causal) {
@@ -434,6 +430,34 @@ favor_output_mma_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
     den_g += __shfl_xor_sync(0xffffffffu, den_g, 1); den_g += __shfl_xor_sync(0xffffffffu, den_g, 2);
     den_g8 += __shfl_xor_sync(0xffffffffu, den_g8, 1); den_g8 += __shfl_xor_sync(0xffffffffu, den_g8, 2);
   }
+
+  cp_async_wait_all();
+  __syncthreads();  // S complete and visible to every warp
+#pragma unroll
+  for (int ks = 0; ks < MP / 16; ++ks) {
+    const int brow = 16 * ks + (lane & 7) + 8 * ((lane >> 3) & 1);
+#pragma unroll
+    for (int np = 0; np < 4; ++np) {
+      uint32_t bh_[4], bl_[4];  // S stored [k = f][n = e]
+      const int off = brow * LDS + 16 * np + 8 * (lane >> 4);
+      ldsm_x4_t(bh_, sm.r1_hi + off);
+      ldsm_x4_t(bl_, sm.r1_lo + off);
+      mma16816(num[2 * np], qh[ks], bh_[0], bh_[1]);
+      mma16816(num[2 * np + 1], qh[ks], bh_[2], bh_[3]);
+      mma16816(num[2 * np], qh[ks], bl_[0], bl_[1]);
+      mma16816(num[2 * np + 1], qh[ks], bl_[2], bl_[3]);
+      mma16816(num[2 * np], ql[ks], bh_[0], bh_[1]);
+      mma16816(num[2 * np + 1], ql[ks], bh_[2], bh_[3]);
+    }
+    uint32_t zh[2], zl[2];
+    const int zoff = (16 * ks + (lane & 15)) * LDS + kHeadDim;
+    ldsm_x2_t(zh, sm.r1_hi + zoff);
+    ldsm_x2_t(zl, sm.r1_lo + zoff);
+    mma16816(num[8], qh[ks], zh[0], zh[1]);
+    mma16816(num[8], qh[ks], zl[0], zl[1]);
+    mma16816(num[8], ql[ks], zh[0], zh[1]);
+  }
+
   // the prefix normaliser sits in column 0 of the ninth tile, i.e. in the lane with t == 0
   den_g += __shfl_sync(0xffffffffu, num[8][0], lane & ~3);
   den_g8 += __shfl_sync(0xffffffffu, num[8][2], lane & ~3);
@@ -442,20 +466,57 @@ favor_output_mma_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
     atomicOr(status, SEA_DEV_NONFINITE);
   const float inv_g = 1.f / den_g, inv_g8 = 1.f / den_g8;
 
-  uint32_t ch[4][4], cl[4][4];  // C rows as A fragments over e
+  const size_t o_g = ((size_t)bh * seq_len + row0 + r0 + g) * kHeadDim, o_g8 = o_g + 8 * kHeadDim;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    const int ks = j >> 1, o = (j & 1) * 2;
-    split2(num[j][0] * inv_g, num[j][1] * inv_g, ch[ks][o], cl[ks][o]);
-    split2(num[j][2] * inv_g8, num[j][3] * inv_g8, ch[ks][o + 1], cl[ks][o + 1]);
+    const int e = 8 * j + 2 * t;
+    uint32_t hi, lo;
+    if (ok_g) {
+      split2(num[j][0] * inv_g, num[j][1] * inv_g, hi, lo);
+      *reinterpret_cast<uint32_t*>(c_hi + o_g + e) = hi;
+      *reinterpret_cast<uint32_t*>(c_lo + o_g + e) = lo;
+    }
+    if (ok_g8) {
+      split2(num[j][2] * inv_g8, num[j][3] * inv_g8, hi, lo);
+      *reinterpret_cast<uint32_t*>(c_hi + o_g8 + e) = hi;
+      *reinterpret_cast<uint32_t*>(c_lo + o_g8 + e) = lo;
+    }
   }
+}
 
-  __nv_bfloat16* wt_hi = sm.om_hi;
-  __nv_bfloat16* wt_lo = sm.om_lo;
-  float* out_g = A_hat + ((size_t)bh * seq_len + row0 + r0 + g) * Kc;
+// Kernel 4: decoder head A_hat = C W_dec on the bf16 head / remainder operands.  A CTA of four
+// warps owns 64 rows (one warp per 16) and walks the Kc columns in tiles of 128.
+__global__ void __launch_bounds__(kThreads)
+favor_decoder_mma_kernel(const __nv_bfloat16* __restrict__ c_hi, const __nv_bfloat16* __restrict__ c_lo,
+                         const __nv_bfloat16* __restrict__ w_hi_g, const __nv_bfloat16* __restrict__ w_lo_g,
+                         float* __restrict__ A_hat, long long rows, int Kc, int KcP) {
+  constexpr int LDW = kWTile + kPad;  // 136: 272-byte pitch
+  __shared__ __align__(16) __nv_bfloat16 wt_hi[kHeadDim * LDW];
+  __shared__ __align__(16) __nv_bfloat16 wt_lo[kHeadDim * LDW];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const long long row_g = (long long)blockIdx.x * kC + 16 * warp + g;
+  const bool ok_g = row_g < rows, ok_g8 = row_g + 8 < rows;
+  uint32_t ch[4][4], cl[4][4];
+  {
+    const uint32_t* h0 = reinterpret_cast<const uint32_t*>(c_hi + (size_t)row_g * kHeadDim) + t;
+    const uint32_t* l0 = reinterpret_cast<const uint32_t*>(c_lo + (size_t)row_g * kHeadDim) + t;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      ch[s][0] = ok_g ? __ldg(h0 + 8 * s) : 0u;
+      ch[s][1] = ok_g8 ? __ldg(h0 + 256 + 8 * s) : 0u;
+      ch[s][2] = ok_g ? __ldg(h0 + 8 * s + 4) : 0u;
+      ch[s][3] = ok_g8 ? __ldg(h0 + 256 + 8 * s + 4) : 0u;
+      cl[s][0] = ok_g ? __ldg(l0 + 8 * s) : 0u;
+      cl[s][1] = ok_g8 ? __ldg(l0 + 256 + 8 * s) : 0u;
+      cl[s][2] = ok_g ? __ldg(l0 + 8 * s + 4) : 0u;
+      cl[s][3] = ok_g8 ? __ldg(l0 + 256 + 8 * s + 4) : 0u;
+    }
+  }
+  float* out_g = A_hat + (size_t)row_g * Kc;
   float* out_g8 = out_g + (size_t)8 * Kc;
+  const bool vec2 = (Kc & 1) == 0;
   for (int c0 = 0; c0 < Kc; c0 += kWTile) {
-    __syncthreads();  // previous users of the region are done
+    if (c0 > 0) __syncthreads();  // the previous tile is no longer being read
     for (int v = threadIdx.x; v < kHeadDim * (kWTile / 8); v += kThreads) {
       const int e = v / (kWTile / 8), cc = (v - e * (kWTile / 8)) * 8;
       uint4 xh = make_uint4(0u, 0u, 0u, 0u), xl = xh;
@@ -490,13 +551,18 @@ favor_output_mma_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
         const int c = c0 + 16 * np + 8 * u + 2 * t;
-        if (ok_g) {
-          if (c < Kc) out_g[c] = acc[u][0];
-          if (c + 1 < Kc) out_g[c + 1] = acc[u][1];
-        }
-        if (ok_g8) {
-          if (c < Kc) out_g8[c] = acc[u][2];
-          if (c + 1 < Kc) out_g8[c + 1] = acc[u][3];
+        if (vec2) {
+          if (ok_g && c < Kc) *reinterpret_cast<float2*>(out_g + c) = make_float2(acc[u][0], acc[u][1]);
+          if (ok_g8 && c < Kc) *reinterpret_cast<float2*>(out_g8 + c) = make_float2(acc[u][2], acc[u][3]);
+        } else {
+          if (ok_g) {
+            if (c < Kc) out_g[c] = acc[u][0];
+            if (c + 1 < Kc) out_g[c + 1] = acc[u][1];
+          }
+          if (ok_g8) {
+            if (c < Kc) out_g8[c] = acc[u][2];
+            if (c + 1 < Kc) out_g8[c + 1] = acc[u][3];
+          }
         }
       }
     }
@@ -509,11 +575,16 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
                      __nv_bfloat16* split_buf, int32_t* status, cudaStream_t st) {
   const int BH = s.B * s.H, m = s.m;
   const int nchunk = (s.T + kC - 1) / kC;
+  const long long rows = (long long)BH * s.T;
   const int KcP = (s.Kc + 15) / 16 * 16;
+  // carve-up of the split buffer (see estimate_split_bytes)
   __nv_bfloat16* om_hi = split_buf;
-  __nv_bfloat16* om_lo = om_hi + MP * kHeadDim;
-  __nv_bfloat16* w_hi = om_lo + MP * kHeadDim;
+  __nv_bfloat16* om_lo = om_hi + 128 * kHeadDim;
+  __nv_bfloat16* w_hi = om_lo + 128 * kHeadDim;
   __nv_bfloat16* w_lo = w_hi + (size_t)kHeadDim * KcP;
+  __nv_bfloat16* c_hi = w_lo + (size_t)kHeadDim * KcP;
+  __nv_bfloat16* c_lo = c_hi + (size_t)rows * kHeadDim;
+  __nv_bfloat16* s_split = c_lo + (size_t)rows * kHeadDim;
   const size_t smem1 = sizeof(SmemKeyState<MP>), smem3 = sizeof(SmemOutput<MP>);
   if (cudaFuncSetAttribute(favor_key_state_mma_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
       cudaFuncSetAttribute(favor_output_mma_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem3) != cudaSuccess)
@@ -526,20 +597,27 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   const dim3 grid(nchunk, BH);
   favor_key_state_mma_kernel<MP><<<grid, kThreads, smem1, st>>>(K, V, om_hi, om_lo, state, s.T, m, nchunk);
   if ((rc = check_launch()) != SEA_OK) return rc;
-  const int per_chunk = m * kStateCols;
-  const long long total = (long long)BH * per_chunk;
-  favor_state_scan_mma_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(state, nchunk, per_chunk, total, s.causal);
+  const long long total = (long long)BH * MP * (kSLd / 2);
+  favor_state_scan_mma_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(state, s_split, nchunk, m, MP, total, s.causal);
   if ((rc = check_launch()) != SEA_OK) return rc;
-  favor_output_mma_kernel<MP><<<grid, kThreads, smem3, st>>>(Q, K, V, om_hi, om_lo, w_hi, w_lo, state, A_hat, status,
-                                                             s.T, m, s.Kc, KcP, nchunk, s.causal);
+  favor_output_mma_kernel<MP><<<grid, kThreads, smem3, st>>>(Q, K, V, om_hi, om_lo, s_split, c_hi, c_lo, status, s.T, m,
+                                                             nchunk, s.causal);
+  if ((rc = check_launch()) != SEA_OK) return rc;
+  favor_decoder_mma_kernel<<<(unsigned)((rows + kC - 1) / kC), kThreads, 0, st>>>(c_hi, c_lo, w_hi, w_lo, A_hat, rows, s.Kc, KcP);
   return check_launch();
 }
 
 }  // namespace
 
+// bf16 scratch of the tensor-core estimator: omega' and W_dec (head / remainder), C (head /
+// remainder, [rows][64]) and the scanned chunk states ([BH][nchunk][2][128][72]).
 size_t estimate_split_bytes(const sea_shape& s) {
   const size_t KcP = ((size_t)s.Kc + 15) / 16 * 16;
-  return (2 * (size_t)128 * kHeadDim + 2 * (size_t)kHeadDim * KcP) * sizeof(__nv_bfloat16);
+  const size_t rows = (size_t)s.B * s.H * s.T;
+  const size_t nchunk = ((size_t)s.T + kC - 1) / kC;
+  const size_t elems = 2 * (size_t)128 * kHeadDim + 2 * (size_t)kHeadDim * KcP + 2 * rows * kHeadDim +
+                       (size_t)s.B * s.H * nchunk * 2 * 128 * kSLd;
+  return elems * sizeof(__nv_bfloat16);
 }
 
 sea_status launch_estimate_bf16(const sea_shape& s, const void* Q, const void* K, const void* V,
