@@ -50,7 +50,8 @@ typedef enum { SEA_F32 = 0, SEA_BF16 = 1 } sea_dtype;
 /* Bits of the device status word (sea_device_status). */
 enum {
   SEA_DEV_ROW_OVERFLOW = 1, /* a CSR row did not fit below nnz_cap and was truncated */
-  SEA_DEV_NONFINITE = 2     /* the estimator met a zero or non-finite normaliser */
+  SEA_DEV_NONFINITE = 2,    /* the estimator met a zero or non-finite normaliser */
+  SEA_DEV_TIMEOUT = 4       /* a bounded wait on an asynchronous copy ran out; the affected rows of O are zero */
 };
 
 typedef struct sea_shape {

@@ -109,15 +109,18 @@ sea_status sea_sparse_attn(const sea_shape* shape, const void* Q, const void* K,
                            const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel, void* O,
                            void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
   Launch::count() = 0;
-  (void)ws;
-  (void)ws_bytes;
   const sea_status rc = validate_shape(shape, false);
   if (rc != SEA_OK) return rc;
   if (!Q || !K || !V || !row_ptr || !O || (!col_idx && !sel)) return SEA_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(row_ptr) ||
       (P && !aligned16(P)) || (sel && !aligned16(sel)) || (col_idx && !aligned16(col_idx)))
     return SEA_ERR_INVALID_ARG;
-  return launch_sparse_attn(*shape, Q, K, V, row_ptr, col_idx, sel, O, P, static_cast<cudaStream_t>(cuda_stream));
+  if (ws && !aligned16(ws)) return SEA_ERR_INVALID_ARG;
+  if (ws && ws_bytes < (size_t)kStatusBytes) return SEA_ERR_WORKSPACE;
+  // the status word at the head of ws is all this stage needs; without ws it runs the kernels
+  // that have no device-side waits
+  return launch_sparse_attn(*shape, Q, K, V, row_ptr, col_idx, sel, O, P, static_cast<int32_t*>(ws),
+                            static_cast<cudaStream_t>(cuda_stream));
 }
 
 sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, const void* V,
@@ -158,7 +161,7 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
                         reinterpret_cast<int32_t*>(w + L.row_counts),
                         reinterpret_cast<int32_t*>(w + L.tile_sums), status, st);
   if (rc != SEA_OK) return rc;
-  return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P, st);
+  return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P, status, st);
 }
 
 sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes) {

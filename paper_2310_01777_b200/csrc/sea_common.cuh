@@ -55,7 +55,11 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
                             cudaStream_t st);
 sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, const void* V,
                               const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
-                              void* O, void* P, cudaStream_t st);
+                              void* O, void* P, int32_t* status, cudaStream_t st);
+bool sparse_attn_tma_applicable(const sea_shape& s, const int32_t* sel, const int32_t* status);
+sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void* K, const void* V,
+                                  const int32_t* row_ptr, const int32_t* sel, void* O, void* P,
+                                  int32_t* status, cudaStream_t st);
 
 inline sea_status check_launch() {
   Launch::count()++;

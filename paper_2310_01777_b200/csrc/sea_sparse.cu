@@ -369,7 +369,9 @@ sea_status launch_typed(const sea_shape& s, const T* Q, const T* K, const T* V,
 
 sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, const void* V,
                               const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
-                              void* O, void* P, cudaStream_t st) {
+                              void* O, void* P, int32_t* status, cudaStream_t st) {
+  if (sparse_attn_tma_applicable(s, sel, status))
+    return launch_sparse_attn_tma(s, Q, K, V, row_ptr, sel, O, P, status, st);
   if (s.io == SEA_BF16) {
     using T = __nv_bfloat16;
     const int rows = s.B * s.H * s.T;

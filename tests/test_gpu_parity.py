@@ -31,6 +31,9 @@ SMALL_CASES = [
     small("dense_nc", T=128, Kc=16, k_hat=16, dtype="bf16"),          # k_hat = Kc: dense attention
     small("long_rows", T=2048, Kc=64, k_hat=40, H=1, causal=True, dtype="bf16"),  # 1280 keys per row > one smem chunk
     small("wide_Kc", T=1024, Kc=1024, k_hat=33, H=1, causal=True, dtype="bf16", m=64),  # 32 values per lane in the select
+    small("runs16", T=512, Kc=32, k_hat=5, causal=True, dtype="bf16", m=64),   # r = 16: runs staged by TMA
+    small("runs32", T=512, Kc=16, k_hat=3, causal=False, dtype="bf16"),        # r = 32: two TMA blocks per column
+    small("runs16_full", T=256, Kc=16, k_hat=16, causal=True, dtype="bf16"),   # every block selected, ring wraps
 ]
 
 
