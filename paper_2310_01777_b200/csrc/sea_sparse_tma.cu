@@ -1,4 +1,4 @@
-// Sparse attention over runs of keys, staged by TMA (bf16, mask given as `sel`, r % 16 == 0).
+// Sparse attention over runs of keys, staged by TMA (bf16, mask given as `sel`, r = 16, 32, 64, ...).
 //
 // Same arithmetic as the gather kernel in sea_sparse.cu (Sec. 3.1.1: scores at the mask's
 // positions, row softmax, product with V; one warp per query row, tensor-core tiles with 16
@@ -8,11 +8,13 @@
 // pipe, whose wavefront rate bounded the gather kernel (a fragment-shaped global load touches
 // 2 to 4 lines per quarter-warp), and leaves one 128-byte wavefront per 128 bytes of K or V.
 //
-// Each warp drives its own ring: lane 0 issues the copies, every lane waits on the slot's
-// mbarrier, and a slot is refilled right after the warp has read it.  All K blocks of the row
-// are consumed first (scores), then all V blocks, so V streams in during the softmax.  Waits
-// are bounded: a wait that runs out sets SEA_DEV_TIMEOUT in the status word and the warp
-// leaves its row zeroed.
+// The grid is persistent: every warp walks rows wg, wg + W, wg + 2W, ... (W = warps in the
+// grid) and keeps ONE stream of block copies running across row boundaries - for each row all
+// its K blocks, then all its V blocks - so the ring stays full while a row's softmax runs and
+// while the next row starts.  The warp is its own producer: after a block has been read, lane 0
+// issues the copy that is kSlots ahead in the stream; the row metadata that the producer needs
+// (row_ptr pair, selected columns) is fetched one row early into registers.  Waits are bounded:
+// a wait that runs out sets SEA_DEV_TIMEOUT in the status word and the warp stops.
 #include <cuda.h>
 
 #include "sea_common.cuh"
@@ -21,9 +23,9 @@ namespace sea {
 namespace {
 
 constexpr int kWarps = 8;
-constexpr int kSlots = 4;              // ring depth per warp
+constexpr int kSlots = 4;              // ring depth per warp (power of two)
 constexpr int kSlotBytes = 16 * 128;   // 16 keys x 64 bf16
-constexpr int kMaxBlocks = 64;         // 16-key blocks per row (k_hat * r <= 1024)
+constexpr int kMaxBlocks = 64;         // 16-key blocks per row (k_hat * r <= 1024, so k_hat <= 64)
 constexpr uint32_t kWaitPolls = 1u << 16;
 
 struct alignas(1024) WarpRing {
@@ -32,28 +34,35 @@ struct alignas(1024) WarpRing {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count));
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
 }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
 }
 // Bounded wait for the given phase parity; false when the poll budget ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  const uint32_t a = smem_u32(bar);
-  for (uint32_t i = 0; i < kWaitPolls; ++i) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok) : "r"(a), "r"(parity) : "memory");
-    if (ok) return true;
-  }
+__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try(bar, parity)) return true;  // the usual case: the copy landed long ago
+  for (uint32_t i = 0; i < kWaitPolls; ++i)
+    if (mbar_try(bar, parity)) return true;
   return false;
 }
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+__device__ __forceinline__ float ex2(float x) {  // 2^x for x <= 0 (flushes denormal results to zero)
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void ldsm4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -75,8 +84,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// Dynamic shared memory: kWarps rings (1024-byte aligned), then per warp: scores / packed
-// probabilities (chunk floats), block starts (kMaxBlocks ints), barriers (kSlots).
+// Dynamic shared memory: kWarps rings (1024-byte aligned), then per warp the scores / packed
+// probabilities (chunk floats) and the ring's barriers.
 template <bool kWriteP>
 __global__ void __launch_bounds__(kWarps * 32)
 sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -88,163 +97,207 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
   // the swizzle pattern is a function of the shared-memory address: slots start on 1024-byte lines
   unsigned char* smem_raw = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  WarpRing& ring = reinterpret_cast<WarpRing*>(smem_raw)[warp];
+  const uint32_t ring = smem_u32(smem_raw) + warp * (uint32_t)sizeof(WarpRing);
   unsigned char* tail = smem_raw + sizeof(WarpRing) * kWarps;
   float* sc = reinterpret_cast<float*>(tail) + warp * chunk;
-  int32_t* jstart = reinterpret_cast<int32_t*>(tail + sizeof(float) * kWarps * chunk) + warp * kMaxBlocks;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tail + sizeof(float) * kWarps * chunk + sizeof(int32_t) * kWarps * kMaxBlocks) +
-                   warp * kSlots;
+  const uint32_t bars = smem_u32(tail + sizeof(float) * kWarps * chunk) + warp * kSlots * 8;
   uint2* pairs = reinterpret_cast<uint2*>(sc);
 
   if (lane == 0) {
 #pragma unroll
-    for (int s = 0; s < kSlots; ++s) mbar_init(bars + s, 1);
+    for (int s = 0; s < kSlots; ++s) mbar_init(bars + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   __syncthreads();
 
-  const int row = blockIdx.x * kWarps + warp;
-  if (row >= rows) return;
+  const int stride = gridDim.x * kWarps;
+  const int wg = blockIdx.x * kWarps + warp;
+  if (wg >= rows) return;
   const int g = lane >> 2, t = lane & 3;
-  const int bh = row / seq_len;
-  const int base = __ldg(row_ptr + row);
-  const int n = __ldg(row_ptr + row + 1) - base;
-  __nv_bfloat16* out = O + (size_t)row * kHeadDim;
-  auto zero_row = [&]() {
-    if (t == 0) *reinterpret_cast<uint4*>(out + 8 * g) = make_uint4(0u, 0u, 0u, 0u);
+  const int rb_shift = 31 - __clz(r >> 4);  // log2 of the 16-key blocks per selected column
+
+  // ---- producer cursor: the next copy of this warp's stream ---------------------------------
+  int p_row = wg - stride;     // row whose copies are being issued (none yet)
+  int p_i = 0, p_nb = 0;       // next copy within the row: K blocks 0..nb-1, then V blocks
+  uint32_t p_s = 0;            // copies issued so far
+  int p_key0 = 0;              // first key row of the head in the [B*H*T][64] view
+  int p_sel0 = 0, p_sel1 = 0;  // lane c holds sel[c] and sel[c+32] of p_row
+  // metadata of the row after p_row, fetched early
+  int nf_rp0 = 0, nf_rp1 = 0, nf_sel0 = 0, nf_sel1 = 0;
+  auto fetch_meta = [&](int row) {
+    if (row < rows) {
+      nf_rp0 = __ldg(row_ptr + row);
+      nf_rp1 = __ldg(row_ptr + row + 1);
+      const int32_t* ms = sel + (size_t)row * k_hat;
+      nf_sel0 = lane < k_hat ? __ldg(ms + lane) : 0;
+      nf_sel1 = lane + 32 < k_hat ? __ldg(ms + lane + 32) : 0;
+    }
   };
-  if (n <= 0) {
-    zero_row();
-    return;
-  }
-  const int nb = (n + 15) >> 4;      // 16-key blocks of this row (only the last may be cut)
-  const int total = 2 * nb;          // K blocks, then V blocks
+  fetch_meta(wg);
+  uint32_t c_s = 0;  // copies consumed so far
+
+  // Issues the next copy of the stream if the ring has a free slot.  Executed by all lanes
+  // together; called once after every consumed block (and kSlots times to prime the ring).
+  auto pump = [&]() {
+    if (p_s - c_s >= (uint32_t)kSlots) return;
+    while (p_i == 2 * p_nb) {  // next row of the stream (rows without keys are skipped)
+      if (p_row >= rows - stride) { p_row = rows; p_nb = 0; p_i = 0; return; }
+      p_row += stride;
+      p_nb = (nf_rp1 - nf_rp0 + 15) >> 4;
+      p_i = 0;
+      p_sel0 = nf_sel0;
+      p_sel1 = nf_sel1;
+      p_key0 = (p_row / seq_len) * seq_len;
+      fetch_meta(p_row + stride);
+    }
+    const bool is_k = p_i < p_nb;
+    const int blk = is_k ? p_i : p_i - p_nb;
+    const int c = blk >> rb_shift;
+    const int col = __shfl_sync(0xffffffffu, c < 32 ? p_sel0 : p_sel1, c);
+    if (lane == 0) {
+      const uint32_t slot = p_s & (kSlots - 1);
+      const uint32_t bar = bars + 8 * slot;
+      mbar_expect_tx(bar, kSlotBytes);
+      tma_load_2d(ring + slot * kSlotBytes, is_k ? &map_k : &map_v, 0, p_key0 + col * r + ((blk - (c << rb_shift)) << 4), bar);
+    }
+    ++p_i;
+    ++p_s;
+  };
+
+  // ldmatrix lane roles.  K (plain): matrix mi -> rows 8*(mi&1).., chunk 2s + (mi>>1).
+  // V (transposed): matrix mi -> rows 8*(mi>>1).., chunk 2i + (mi&1).  Offsets inside a slot:
+  uint32_t k_off[4], v_off[4];
   {
-    const int rb = r >> 4;           // blocks per selected column
-    const int32_t* my_sel = sel + (size_t)row * k_hat;
-    for (int s = lane; s < nb; s += 32) {
-      const int c = s / rb;
-      jstart[s] = bh * seq_len + __ldg(my_sel + c) * r + (s - c * rb) * 16;
+    const int mi = lane >> 3, lr = lane & 7;
+    const int k_row = lr + 8 * (mi & 1), v_row = lr + 8 * (mi >> 1);
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      k_off[s] = k_row * 128 + (((2 * s + (mi >> 1)) ^ (k_row & 7)) << 4);
+      v_off[s] = v_row * 128 + (((2 * s + (mi & 1)) ^ (v_row & 7)) << 4);
     }
   }
-  __syncwarp();
-  auto issue = [&](int i) {  // lane 0 only
-    uint64_t* bar = bars + (i % kSlots);
-    mbar_expect_tx(bar, kSlotBytes);
-    const bool is_k = i < nb;
-    tma_load_2d(ring.slot[i % kSlots], is_k ? &map_k : &map_v, 0, jstart[is_k ? i : i - nb], bar);
-  };
-  if (lane == 0) {
-    for (int i = 0; i < min(kSlots, total); ++i) issue(i);
-  }
 
-  // q as the B operand of every k-step: b0 = dims 16s+2t.., b1 = dims 16s+8+2t..
-  uint32_t qw[8];
-  {
+  // consumer's own early fetch: row_ptr pair and q of the next row
+  int n_rp0 = __ldg(row_ptr + wg), n_rp1 = __ldg(row_ptr + wg + 1);
+  uint32_t n_qw[8];
+  auto fetch_q = [&](int row) {
     const uint32_t* qp = reinterpret_cast<const uint32_t*>(Q + (size_t)row * kHeadDim) + t;
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-      qw[2 * s] = __ldg(qp + 8 * s);
-      qw[2 * s + 1] = __ldg(qp + 8 * s + 4);
+      n_qw[2 * s] = __ldg(qp + 8 * s);
+      n_qw[2 * s + 1] = __ldg(qp + 8 * s + 4);
     }
-  }
+  };
+  fetch_q(wg);
+#pragma unroll
+  for (int i = 0; i < kSlots; ++i) pump();
 
-  const int cn16 = nb * 16;
   bool ok = true;
-  float mx = -INFINITY;
-  // ldmatrix lane roles.  K (plain): matrix mi -> rows 8*(mi&1).., chunk 2s + (mi>>1).
-  // V (transposed): matrix mi -> rows 8*(mi>>1).., chunk 2i + (mi&1).
-  const int mi = lane >> 3, lr = lane & 7;
-  const int k_row = lr + 8 * (mi & 1), k_chk = mi >> 1;
-  const int v_row = lr + 8 * (mi >> 1), v_chk = mi & 1;
-  for (int b = 0; b < nb; ++b) {
-    if (!__all_sync(0xffffffffu, mbar_wait(bars + (b % kSlots), (b / kSlots) & 1))) { ok = false; break; }
-    const uint32_t sbase = smem_u32(ring.slot[b % kSlots]) + k_row * 128;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int row = wg; row < rows && ok; row += stride) {
+    const int base = n_rp0, n = n_rp1 - n_rp0;
+    uint32_t qw[8];  // q as the B operand of every k-step: b0 = dims 16s+2t.., b1 = dims 16s+8+2t..
 #pragma unroll
-    for (int s = 0; s < 4; ++s) {
-      uint32_t a[4];
-      ldsm4(a, sbase + (((2 * s + k_chk) ^ (k_row & 7)) << 4));
-      mma16816(acc, a, qw[2 * s], qw[2 * s + 1]);
+    for (int i = 0; i < 8; ++i) qw[i] = n_qw[i];
+    if (row < rows - stride) {
+      n_rp0 = __ldg(row_ptr + row + stride);
+      n_rp1 = __ldg(row_ptr + row + stride + 1);
+      fetch_q(row + stride);
     }
-    const int p0 = 16 * b;
-    const float s0 = p0 + g < n ? acc[0] * scale_log2 : -INFINITY;
-    const float s1 = p0 + g + 8 < n ? acc[2] * scale_log2 : -INFINITY;
-    mx = fmaxf(mx, fmaxf(s0, s1));
-    if (t == 0) {
-      sc[p0 + g] = s0;
-      sc[p0 + g + 8] = s1;
+    __nv_bfloat16* out = O + (size_t)row * kHeadDim;
+    if (n <= 0) {
+      out[16 * t + g] = __float2bfloat16_rn(0.f);
+      out[16 * t + 8 + g] = __float2bfloat16_rn(0.f);
+      continue;
+    }
+    const int nb = (n + 15) >> 4;  // 16-key blocks of this row (only the last may be cut)
+    const int cn16 = nb * 16;
+    float mx = -INFINITY;
+    for (int b = 0; b < nb; ++b) {
+      const uint32_t slot = c_s & (kSlots - 1);
+      ok &= mbar_wait(bars + 8 * slot, (c_s / kSlots) & 1);
+      const uint32_t sbase = ring + slot * kSlotBytes;
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int s = 0; s < 4; ++s) {
+        uint32_t a[4];
+        ldsm4(a, sbase + k_off[s]);
+        mma16816(acc, a, qw[2 * s], qw[2 * s + 1]);
+      }
+      const int p0 = 16 * b;
+      const float s0 = p0 + g < n ? acc[0] * scale_log2 : -INFINITY;
+      const float s1 = p0 + g + 8 < n ? acc[2] * scale_log2 : -INFINITY;
+      mx = fmaxf(mx, fmaxf(s0, s1));
+      if (t == 0) {
+        sc[p0 + g] = s0;
+        sc[p0 + g + 8] = s1;
+      }
+      __syncwarp();
+      ++c_s;
+      pump();
+    }
+    ok = __all_sync(0xffffffffu, ok);  // a wait that ran out ends the warp's work after this row's K pass
+    if (!ok) break;
+    mx = warp_max(mx);
+
+    float part = 0.f;
+    for (int u = lane; u < cn16 / 2; u += 32) {
+      float2 s = reinterpret_cast<float2*>(sc)[u];
+      s.x = ex2(s.x - mx);
+      s.y = ex2(s.y - mx);
+      part += s.x + s.y;
+      reinterpret_cast<float2*>(sc)[u] = s;
+    }
+    const float inv = 1.f / warp_sum(part);
+    for (int u = lane; u < cn16 / 2; u += 32) {
+      const float2 e = reinterpret_cast<float2*>(sc)[u];
+      const float p0 = e.x * inv, p1 = e.y * inv;
+      const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+      const uint32_t hw = *reinterpret_cast<const uint32_t*>(&h);
+      const uint32_t lw = pack_bf16(p0 - __bfloat162float(h.x), p1 - __bfloat162float(h.y));
+      pairs[u] = make_uint2(hw, lw);
+      if (kWriteP) {
+        __nv_bfloat16* pp = P + (size_t)base + 2 * u;
+        if (2 * u < n) pp[0] = h.x;
+        if (2 * u + 1 < n) pp[1] = h.y;
+      }
     }
     __syncwarp();
-    if (lane == 0 && b + kSlots < total) issue(b + kSlots);
-  }
-  if (!ok) {
-    if (lane == 0) atomicOr(status, SEA_DEV_TIMEOUT);
-    zero_row();
-    return;
-  }
-  mx = warp_max(mx);
 
-  float part = 0.f;
-  for (int u = lane; u < cn16 / 2; u += 32) {
-    float2 s = reinterpret_cast<float2*>(sc)[u];
-    s.x = exp2f(s.x - mx);
-    s.y = exp2f(s.y - mx);
-    part += s.x + s.y;
-    reinterpret_cast<float2*>(sc)[u] = s;
-  }
-  const float inv = 1.f / warp_sum(part);
-  for (int u = lane; u < cn16 / 2; u += 32) {
-    const float2 e = reinterpret_cast<float2*>(sc)[u];
-    const float p0 = e.x * inv, p1 = e.y * inv;
-    const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-    const uint32_t hw = *reinterpret_cast<const uint32_t*>(&h);
-    const uint32_t lw = pack_bf16(p0 - __bfloat162float(h.x), p1 - __bfloat162float(h.y));
-    pairs[u] = make_uint2(hw, lw);
-    if (kWriteP) {
-      __nv_bfloat16* pp = P + (size_t)base + 2 * u;
-      if (2 * u < n) pp[0] = h.x;
-      if (2 * u + 1 < n) pp[1] = h.y;
+    float acc_o[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc_o[i][e] = 0.f;
+    for (int b = 0; b < nb; ++b) {
+      const uint32_t slot = c_s & (kSlots - 1);
+      ok &= mbar_wait(bars + 8 * slot, (c_s / kSlots) & 1);
+      const uint32_t sbase = ring + slot * kSlotBytes;
+      const uint2 pa = pairs[8 * b + t];      // positions 16b+2t, 16b+2t+1
+      const uint2 pb = pairs[8 * b + 4 + t];  // positions 16b+8+2t, 16b+9+2t
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {  // tile i: rows g / g+8 = dims 16i+g / 16i+8+g
+        uint32_t a[4];
+        ldsm4_t(a, sbase + v_off[i]);
+        mma16816(acc_o[i], a, pa.x, pb.x);
+        mma16816(acc_o[i], a, pa.y, pb.y);
+      }
+      __syncwarp();
+      ++c_s;
+      pump();
+    }
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) break;
+    // every lane of a quad holds the same sums; lane t writes tile t: dims 16t + g and 16t + 8 + g
+    {
+      float lo = acc_o[0][0], hi = acc_o[0][2];
+      if (t == 1) { lo = acc_o[1][0]; hi = acc_o[1][2]; }
+      if (t == 2) { lo = acc_o[2][0]; hi = acc_o[2][2]; }
+      if (t == 3) { lo = acc_o[3][0]; hi = acc_o[3][2]; }
+      out[16 * t + g] = __float2bfloat16_rn(lo);
+      out[16 * t + 8 + g] = __float2bfloat16_rn(hi);
     }
   }
-  __syncwarp();
-
-  float acc_o[4][4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) acc_o[i][e] = 0.f;
-  for (int b = 0; b < nb; ++b) {
-    const int i_load = nb + b;
-    if (!__all_sync(0xffffffffu, mbar_wait(bars + (i_load % kSlots), (i_load / kSlots) & 1))) { ok = false; break; }
-    const uint32_t sbase = smem_u32(ring.slot[i_load % kSlots]) + v_row * 128;
-    const uint2 pa = pairs[8 * b + t];      // positions 16b+2t, 16b+2t+1
-    const uint2 pb = pairs[8 * b + 4 + t];  // positions 16b+8+2t, 16b+9+2t
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {  // tile i: rows g / g+8 = dims 16i+g / 16i+8+g
-      uint32_t a[4];
-      ldsm4_t(a, sbase + (((2 * i + v_chk) ^ (v_row & 7)) << 4));
-      mma16816(acc_o[i], a, pa.x, pb.x);
-      mma16816(acc_o[i], a, pa.y, pb.y);
-    }
-    __syncwarp();
-    if (lane == 0 && i_load + kSlots < total) issue(i_load + kSlots);
-  }
-  if (!ok) {
-    if (lane == 0) atomicOr(status, SEA_DEV_TIMEOUT);
-    zero_row();
-    return;
-  }
-  // every lane of a quad holds the same sums; lane t writes the two 8-dim groups 2t and 2t+1:
-  // tile i = t (dims 16t + g and 16t + 8 + g)
-  {
-    float lo = acc_o[0][0], hi = acc_o[0][2];
-    if (t == 1) { lo = acc_o[1][0]; hi = acc_o[1][2]; }
-    if (t == 2) { lo = acc_o[2][0]; hi = acc_o[2][2]; }
-    if (t == 3) { lo = acc_o[3][0]; hi = acc_o[3][2]; }
-    out[16 * t + g] = __float2bfloat16_rn(lo);
-    out[16 * t + 8 + g] = __float2bfloat16_rn(hi);
-  }
+  if (!ok && lane == 0) atomicOr(status, SEA_DEV_TIMEOUT);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -276,11 +329,34 @@ bool make_rows_map(CUtensorMap* map, const void* ptr, unsigned long long total_r
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <bool kWriteP>
+sea_status launch_tma(const sea_shape& s, const CUtensorMap& map_k, const CUtensorMap& map_v, const __nv_bfloat16* Q,
+                      const int32_t* row_ptr, const int32_t* sel, __nv_bfloat16* O, __nv_bfloat16* P, int32_t* status,
+                      cudaStream_t st) {
+  const int rows = s.B * s.H * s.T;
+  const int r = s.T / s.Kc;
+  const int chunk = (s.k_hat * r + 63) / 64 * 64;
+  const size_t smem = 1024 + sizeof(WarpRing) * kWarps + sizeof(float) * kWarps * chunk + 8 * kWarps * kSlots;
+  auto kern = sparse_attn_blocks_tma_kernel<kWriteP>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SEA_ERR_CUDA;
+  int dev = 0, sms = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kWarps * 32, smem) != cudaSuccess || per_sm < 1)
+    return SEA_ERR_CUDA;
+  const int want = (rows + kWarps - 1) / kWarps;
+  const int grid = want < sms * per_sm ? want : sms * per_sm;  // persistent: one wave of CTAs
+  const float scale = s.scale != 0.f ? s.scale : 0.125f;
+  kern<<<grid, kWarps * 32, smem, st>>>(map_k, map_v, Q, row_ptr, sel, O, P, status, rows, s.T, r, s.k_hat,
+                                        scale * 1.4426950408889634f, chunk);
+  return check_launch();
+}
+
 }  // namespace
 
 bool sparse_attn_tma_applicable(const sea_shape& s, const int32_t* sel, const int32_t* status) {
   const int r = s.T / s.Kc;
-  return s.io == SEA_BF16 && sel != nullptr && status != nullptr && r % 16 == 0 &&
+  return s.io == SEA_BF16 && sel != nullptr && status != nullptr && r % 16 == 0 && ((r >> 4) & ((r >> 4) - 1)) == 0 && s.k_hat <= kMaxBlocks &&
          (long long)s.k_hat * r <= 16 * kMaxBlocks && encode_fn() != nullptr;
 }
 
@@ -288,29 +364,11 @@ sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void*
                                   const int32_t* row_ptr, const int32_t* sel, void* O, void* P,
                                   int32_t* status, cudaStream_t st) {
   using T = __nv_bfloat16;
-  const int rows = s.B * s.H * s.T;
-  const int r = s.T / s.Kc;
+  const unsigned long long rows = (unsigned long long)s.B * s.H * s.T;
   CUtensorMap map_k, map_v;
-  if (!make_rows_map(&map_k, K, (unsigned long long)rows) || !make_rows_map(&map_v, V, (unsigned long long)rows))
-    return SEA_ERR_CUDA;
-  const int chunk = (s.k_hat * r + 63) / 64 * 64;
-  const size_t smem = 1024 + sizeof(WarpRing) * kWarps + sizeof(float) * kWarps * chunk + sizeof(int32_t) * kWarps * kMaxBlocks +
-                      sizeof(uint64_t) * kWarps * kSlots;
-  const float scale = s.scale != 0.f ? s.scale : 0.125f;
-  const float scale_log2 = scale * 1.4426950408889634f;
-  const int grid = (rows + kWarps - 1) / kWarps;
-  if (P) {
-    if (cudaFuncSetAttribute(sparse_attn_blocks_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return SEA_ERR_CUDA;
-    sparse_attn_blocks_tma_kernel<true><<<grid, kWarps * 32, smem, st>>>(map_k, map_v, (const T*)Q, row_ptr, sel, (T*)O, (T*)P,
-                                                                         status, rows, s.T, r, s.k_hat, scale_log2, chunk);
-  } else {
-    if (cudaFuncSetAttribute(sparse_attn_blocks_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return SEA_ERR_CUDA;
-    sparse_attn_blocks_tma_kernel<false><<<grid, kWarps * 32, smem, st>>>(map_k, map_v, (const T*)Q, row_ptr, sel, (T*)O, nullptr,
-                                                                          status, rows, s.T, r, s.k_hat, scale_log2, chunk);
-  }
-  return check_launch();
+  if (!make_rows_map(&map_k, K, rows) || !make_rows_map(&map_v, V, rows)) return SEA_ERR_CUDA;
+  if (P) return launch_tma<true>(s, map_k, map_v, (const T*)Q, row_ptr, sel, (T*)O, (T*)P, status, st);
+  return launch_tma<false>(s, map_k, map_v, (const T*)Q, row_ptr, sel, (T*)O, nullptr, status, st);
 }
 
 }  // namespace sea
