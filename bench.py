@@ -36,8 +36,8 @@ if ROOT not in sys.path:
 METRIC = "SEA attention-layer tokens/s on 1 B200 (all stages)"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparse-attention launch, from the ncu capture
-# summarised under profiles/ (captured on a 16-head slice of the workload and scaled by heads).
-NCU_TRAFFIC_BYTES = {}
+# summarised in profiles/sparse_attn_tma_opt_1p3b.md (one launch covers the whole workload).
+NCU_TRAFFIC_BYTES = {"opt_1p3b": 183.9e6}
 
 
 def measured_peaks():
@@ -296,6 +296,7 @@ def main():
         peak, peak_kind = measured_peaks()
         alg_bytes = 2 * w.rows * w.d * elem + 2 * nnz * w.d * elem  # Q + O + gathered K and V
         sparse_s = stage_ms[2] / 1e3
+        unique_bytes = 4 * w.rows * w.d * elem + nnz * elem + w.rows * w.k_hat * 4 + (w.rows + 1) * 4
         achieved = alg_bytes / sparse_s / 1e9
         line = {
             "metric": METRIC, "value": tokens / (ms_per_step / 1e3), "unit": "tokens/s", "n_gpus": world,
@@ -308,10 +309,14 @@ def main():
             "clocks": clocks,
             "stages_ms": {"estimate": stage_ms[0], "topk_mask": stage_ms[1], "sparse_attn": stage_ms[2]},
             "nnz": nnz,
-            "roofline": {"kernel": "sparse_attn_rows_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+            "roofline": {"kernel": "sparse_attn_blocks_tma_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_source": f"{peak_kind} HBM copy bandwidth",
                          "algorithmic_bytes": alg_bytes, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
-                         "ms": stage_ms[2], "sparse_stage_tokens_per_s": w.B * w.T / sparse_s},
+                         "ms": stage_ms[2], "sparse_stage_tokens_per_s": w.B * w.T / sparse_s,
+                         # K and V of every head fit the L2 together, so the bytes that must cross HBM are
+                         # far fewer than the algorithmic ones: Q, K, V once, O and P once, sel and row_ptr
+                         "compulsory_hbm_bytes": unique_bytes,
+                         "compulsory_hbm_gbs": unique_bytes / sparse_s / 1e9},
         }
         if not args.no_cpu_baseline and world == 1:
             n = min(args.cpu_heads, w.B * w.H)
