@@ -104,6 +104,33 @@ sea_status sea_topk_mask(const sea_shape* shape, const float* A_hat, int32_t* se
                          void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * sea_topk_mask without a workspace (the paper has no counterpart; this is an
+ * interface variant of the call above, same kernels, same results).
+ *
+ * It is meant for callers that cannot allocate device memory and have no
+ * workspace to pass: an engine plugin whose memory plan is frozen, or a serving
+ * loop where cudaMalloc is off limits because it synchronises the device and can
+ * fail under a fixed budget.  The call itself allocates and frees nothing: the
+ * per-row counts and scan partials live in a static device array inside the
+ * library (4.2 MB, held by every GPU that loads the library until the process
+ * exits), which limits the call to rows = B*H*T <= 1 048 576; larger shapes
+ * return SEA_ERR_TOO_LARGE.
+ *
+ * Differences from sea_topk_mask: `sel` is required (it is an output the caller
+ * owns); when col_idx is given, nnz_cap must be at least rows*k_hat*r, otherwise
+ * SEA_ERR_TOO_LARGE (there is no status word through which a truncated row could
+ * be reported).  The first call on each device looks up the array's device
+ * address (with that device current); make that first call before any stream
+ * capture begins.  All calls on a device share the one array, which keeps the
+ * previous call's contents (the call clears what has to start at zero): two
+ * calls whose kernels overlap on the GPU race, so keep them on one stream or
+ * order them with events.
+ */
+sea_status sea_topk_mask_static(const sea_shape* shape, const float* A_hat, int32_t* sel,
+                                int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                                void* cuda_stream);
+
+/*
  * Sparse attention, Sec. 3.1.1 "Sparse Attention Mechanism": rho (q_i . k_j * scale
  * at the mask's positions), sigma (softmax over the non-zeros of each row, so that
  * every non-empty row of A* sums to 1) and C = A* V, fused.  The learned

@@ -28,7 +28,8 @@ SEA_DEV_ROW_OVERFLOW = 1
 SEA_DEV_NONFINITE = 2
 
 EXPORTS = (
-    "sea_workspace_bytes", "sea_estimate", "sea_topk_mask", "sea_sparse_attn", "sea_attention",
+    "sea_workspace_bytes", "sea_estimate", "sea_topk_mask", "sea_topk_mask_static", "sea_sparse_attn",
+    "sea_attention",
     "sea_workspace_host_bytes", "sea_attention_host", "sea_device_status", "sea_last_launch_count",
     "sea_status_string",
 )
@@ -67,6 +68,7 @@ def load_library() -> ctypes.CDLL:
     lib.sea_workspace_host_bytes.argtypes = [shp, ctypes.POINTER(sz)]
     lib.sea_estimate.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sea_topk_mask.argtypes = [shp, vp, vp, vp, vp, i64, vp, sz, vp]
+    lib.sea_topk_mask_static.argtypes = [shp, vp, vp, vp, vp, i64, vp]
     lib.sea_sparse_attn.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sea_attention.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
     lib.sea_attention_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -141,6 +143,15 @@ def sea_topk_mask(shape, A_hat, sel, row_ptr, col_idx, ws, nnz_cap: Optional[int
     _check(load_library().sea_topk_mask(ctypes.byref(shape), _ptr(A_hat), _ptr(sel), _ptr(row_ptr),
                                         _ptr(col_idx), nnz_cap, _ptr(ws), ws.numel(), _stream(ws.device)),
            "sea_topk_mask")
+
+
+def sea_topk_mask_static(shape, A_hat, sel, row_ptr, col_idx, nnz_cap: Optional[int] = None):
+    """sea_topk_mask for callers without a workspace: scratch lives in a static array of the library."""
+    if nnz_cap is None:
+        nnz_cap = col_idx.numel() if col_idx is not None else 0
+    _check(load_library().sea_topk_mask_static(ctypes.byref(shape), _ptr(A_hat), _ptr(sel), _ptr(row_ptr),
+                                               _ptr(col_idx), nnz_cap, _stream(A_hat.device)),
+           "sea_topk_mask_static")
 
 
 def sea_sparse_attn(shape, Q, K, V, row_ptr, col_idx, sel, O, P, ws=None):

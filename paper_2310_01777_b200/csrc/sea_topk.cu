@@ -235,3 +235,72 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
 }
 
 }  // namespace sea
+
+// ---- sea_topk_mask_static: the same stage without a caller-provided workspace ----------------
+//
+// For callers that can neither allocate device memory nor hand over a workspace: an inference
+// plugin whose memory plan was frozen when the engine was built, or a serving loop that must not
+// call cudaMalloc because it synchronises the device and can fail under a fixed memory budget.
+// The scratch the stage needs (per-row counts and the partial sums of their scan) lives in the
+// file-scope device array below, sized for at most kStaticMaxRows rows; every GPU that loads the
+// library holds these 4.2 MB until the process exits.
+#include <mutex>
+
+namespace sea {
+namespace {
+
+constexpr int kStaticMaxRows = 1 << 20;  // B*H*T limit of the static variant
+constexpr int kStaticTiles = kStaticMaxRows / kScanTile + 1;
+constexpr int kStaticHead = 64;  // int32 words reserved ahead of the counts (word 0: status)
+constexpr int kStaticMaxDevices = 64;
+
+static __device__ __align__(256) int32_t g_static_scratch[kStaticHead + kStaticMaxRows + kStaticTiles + 63];
+
+// In host code the array's name is only a handle; the device address is looked up once per
+// device, with that device current, and remembered here.
+std::mutex g_static_mutex;
+int32_t* g_static_ptr[kStaticMaxDevices] = {};
+
+sea_status static_scratch(int32_t** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return SEA_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_ptr[dev] == nullptr) {
+    int32_t* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_scratch) != cudaSuccess || p == nullptr)
+      return SEA_ERR_CUDA;
+    g_static_ptr[dev] = p;
+  }
+  *out = g_static_ptr[dev];
+  return SEA_OK;
+}
+
+}  // namespace
+}  // namespace sea
+
+extern "C" sea_status sea_topk_mask_static(const sea_shape* shape, const float* A_hat, int32_t* sel,
+                                           int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                                           void* cuda_stream) {
+  using namespace sea;
+  Launch::count() = 0;
+  const sea_status rc = validate_shape(shape, false);
+  if (rc != SEA_OK) return rc;
+  if (!A_hat || !sel || !row_ptr) return SEA_ERR_INVALID_ARG;
+  auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+  if (misaligned(A_hat) || misaligned(sel) || misaligned(row_ptr) || (col_idx && misaligned(col_idx)))
+    return SEA_ERR_INVALID_ARG;
+  const long long rows = (long long)shape->B * shape->H * shape->T;
+  if (rows > kStaticMaxRows) return SEA_ERR_TOO_LARGE;  // beyond the static scratch
+  const long long full = rows * shape->k_hat * (shape->T / shape->Kc);
+  // without a status word to report a truncated row, col_idx must be able to hold every row in full
+  if (col_idx && (nnz_cap < full || nnz_cap > 2147483647ll)) return SEA_ERR_TOO_LARGE;
+  int32_t* scratch = nullptr;
+  const sea_status rs = static_scratch(&scratch);
+  if (rs != SEA_OK) return rs;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // the array keeps the previous call's contents: counts and partial sums are rewritten in full
+  // by the kernels, the status word is the one thing that has to start at zero
+  if (cudaMemsetAsync(scratch, 0, sizeof(int32_t), st) != cudaSuccess) return SEA_ERR_CUDA;
+  return launch_topk_mask(*shape, A_hat, sel, row_ptr, col_idx, nnz_cap, scratch + kStaticHead,
+                          scratch + kStaticHead + kStaticMaxRows, scratch, st);
+}
