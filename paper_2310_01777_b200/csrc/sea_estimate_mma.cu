@@ -184,8 +184,9 @@ __device__ __forceinline__ void store_features(__nv_bfloat16* ph, __nv_bfloat16*
 
 template <int MP>
 struct SmemKeyState {
-  __nv_bfloat16 om_hi[MP * kLd64], om_lo[MP * kLd64];
-  __nv_bfloat16 ph_hi[kC * (MP + kPad)], ph_lo[kC * (MP + kPad)];
+  // one region holds omega' during the projection and phi(K) afterwards
+  static constexpr int kR = (MP * kLd64 > kC * (MP + kPad)) ? MP * kLd64 : kC * (MP + kPad);
+  __nv_bfloat16 r_hi[kR], r_lo[kR];
   __nv_bfloat16 v[kC * kLd64];
 };
 
@@ -203,8 +204,8 @@ favor_key_state_mma_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloa
   const size_t head = (size_t)bh * seq_len * kHeadDim;
   const int valid = min(kC, seq_len - row0);
 
-  stage_rows64(sm.om_hi, om_hi_g, MP, MP);
-  stage_rows64(sm.om_lo, om_lo_g, MP, MP);
+  stage_rows64(sm.r_hi, om_hi_g, MP, MP);
+  stage_rows64(sm.r_lo, om_lo_g, MP, MP);
   stage_rows64(sm.v, V + head + (size_t)row0 * kHeadDim, kC, valid);
   __syncthreads();
 
@@ -214,10 +215,11 @@ favor_key_state_mma_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloa
     const int r0 = 16 * warp;
     load_rows_frag(a, sq_g, sq_g8, K + head, row0 + r0 + g, seq_len, t);
     float acc[MP / 8][4];
-    project<MP>(acc, a, sm.om_hi, sm.om_lo, lane);
+    project<MP>(acc, a, sm.r_hi, sm.r_lo, lane);
     uint32_t fh[MP / 16][4], fl[MP / 16][4];
     features_frag<MP>(fh, fl, acc, sq_g, sq_g8, r0 + g < valid, r0 + g + 8 < valid, m, rsqrtf((float)m), t);
-    store_features<MP>(sm.ph_hi, sm.ph_lo, fh, fl, r0, g, t);
+    __syncthreads();  // every warp is done reading omega'; the region now takes phi(K)
+    store_features<MP>(sm.r_hi, sm.r_lo, fh, fl, r0, g, t);
   }
   __syncthreads();
 
@@ -234,8 +236,8 @@ favor_key_state_mma_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloa
       // A = phi^T: stored [k = row][m = feature] -> transposed load
       uint32_t ah[4], al[4];
       const int arow = 16 * ks + (lane & 7) + 8 * (lane >> 4), acol = 16 * mt + 8 * ((lane >> 3) & 1);
-      ldsm_x4_t(ah, sm.ph_hi + arow * LDP + acol);
-      ldsm_x4_t(al, sm.ph_lo + arow * LDP + acol);
+      ldsm_x4_t(ah, sm.r_hi + arow * LDP + acol);
+      ldsm_x4_t(al, sm.r_lo + arow * LDP + acol);
 #pragma unroll
       for (int np = 0; np < 4; ++np) {
         uint32_t b[4];  // V stored [k = row][n = dim]

@@ -40,7 +40,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
   }
   // k_hat-th largest key: the largest tau with |{key >= tau}| >= k_hat
   uint32_t tau = 0u;
-#pragma unroll 1
+#pragma unroll
   for (int bit = 31; bit >= 0; --bit) {
     const uint32_t cand = tau | (1u << bit);
     int c = 0;
