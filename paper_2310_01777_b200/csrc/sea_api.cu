@@ -47,6 +47,8 @@ WsLayout ws_layout(const sea_shape& s) {
   L.a_hat = take(rows * (size_t)s.Kc * sizeof(float));
   L.sel = take(rows * (size_t)s.k_hat * sizeof(int32_t));
   L.row_ptr = take((rows + 1) * sizeof(int32_t));
+  L.mask_bits = take(sparse_attn_tc_bits_bytes(s));
+  L.p_scratch = take(s.io == SEA_BF16 ? sparse_attn_tc_scratch_bytes(s) : 0);
   L.total = off;
   return L;
 }
@@ -117,10 +119,15 @@ sea_status sea_sparse_attn(const sea_shape* shape, const void* Q, const void* K,
     return SEA_ERR_INVALID_ARG;
   if (ws && !aligned16(ws)) return SEA_ERR_INVALID_ARG;
   if (ws && ws_bytes < (size_t)kStatusBytes) return SEA_ERR_WORKSPACE;
-  // the status word at the head of ws is all this stage needs; without ws it runs the kernels
-  // that have no device-side waits
-  return launch_sparse_attn(*shape, Q, K, V, row_ptr, col_idx, sel, O, P, static_cast<int32_t*>(ws),
-                            static_cast<cudaStream_t>(cuda_stream));
+  // With a full workspace every kernel is available; with only the status word at its head the
+  // per-row kernels run; without ws, those of them that have no device-side waits.
+  char* w = static_cast<char*>(ws);
+  const WsLayout L = ws_layout(*shape);
+  const bool full = ws && ws_bytes >= L.total;
+  return launch_sparse_attn(*shape, Q, K, V, row_ptr, col_idx, sel, O, P,
+                            full ? reinterpret_cast<uint32_t*>(w + L.mask_bits) : nullptr,
+                            full ? reinterpret_cast<float*>(w + L.p_scratch) : nullptr,
+                            static_cast<int32_t*>(ws), static_cast<cudaStream_t>(cuda_stream));
 }
 
 sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, const void* V,
@@ -161,7 +168,9 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
                         reinterpret_cast<int32_t*>(w + L.row_counts),
                         reinterpret_cast<int32_t*>(w + L.tile_sums), status, st);
   if (rc != SEA_OK) return rc;
-  return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P, status, st);
+  return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P,
+                            reinterpret_cast<uint32_t*>(w + L.mask_bits), reinterpret_cast<float*>(w + L.p_scratch),
+                            status, st);
 }
 
 sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes) {

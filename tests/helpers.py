@@ -52,9 +52,12 @@ class GpuRun:
     def topk_mask(self):
         sea.sea_topk_mask(self.shape, self.A_hat, self.sel, self.row_ptr, self.col_idx, self.ws)
 
-    def sparse_attn(self, use_sel=True):
+    def sparse_attn(self, use_sel=True, lean_ws=False):
+        """With the full workspace the stage may run its tensor-core tile kernel; with only the
+        status word (``lean_ws``) it runs the per-row kernels."""
         sea.sea_sparse_attn(self.shape, self.d["Q"], self.d["K"], self.d["V"], self.row_ptr, self.col_idx,
-                            self.sel if use_sel else None, self.O, self.P, self.ws)
+                            self.sel if use_sel else None, self.O, self.P,
+                            self.ws[:256] if lean_ws else self.ws)
 
     # the fused call ------------------------------------------------------------------
     def attention(self):

@@ -51,6 +51,32 @@ def test_stages_match_oracle_on_small_shapes(w):
     global_mask_properties(run)
 
 
+TILE_CASES = [w for w in SMALL_CASES if w.dtype == "bf16" and w.T % 128 == 0 and w.r >= 4 and w.r & (w.r - 1) == 0] + [
+    small("tiles_r4", dtype="bf16", T=384, Kc=96, k_hat=9, causal=True, H=3),            # 32 columns per key tile
+    small("tiles_r8_nc", dtype="bf16", T=256, Kc=32, k_hat=1, causal=False),             # a single run per row
+    small("tiles_r128", dtype="bf16", T=1024, Kc=8, k_hat=3, causal=True),               # a column spans one tile
+    small("tiles_r512", dtype="bf16", T=2048, Kc=4, k_hat=2, causal=True, H=1),          # a column spans four tiles
+    small("tiles_wide", dtype="bf16", T=2048, Kc=512, k_hat=40, causal=True, H=1, m=64), # 16 words of mask bits per row
+]
+
+
+@pytest.mark.parametrize("w", TILE_CASES, ids=lambda w: w.name)
+def test_tile_kernel_and_row_kernels_both_match_oracle(w):
+    """Shapes the tensor-core tile kernel accepts: it (full workspace) and the per-row kernels
+    (status word only) are each checked against the oracle."""
+    run = GpuRun(w)
+    run.estimate(); run.topk_mask(); run.sync()
+    for lean in (False, True):
+        run.O.fill_(float("nan")); run.P.fill_(float("nan"))
+        run.sparse_attn(lean_ws=lean)
+        run.sync()
+        assert run.status() == 0
+        for b in range(w.B):
+            for h in range(w.H):
+                check_head_against_oracle(run, b, h, check_estimate=False)
+        global_mask_properties(run)
+
+
 @pytest.mark.parametrize("w", SMALL_CASES[:6], ids=lambda w: w.name)
 def test_fused_call_equals_stage_calls_bitwise(w):
     a = GpuRun(w)
@@ -84,13 +110,20 @@ def test_fused_call_with_optional_outputs_omitted():
 def test_csr_path_equals_sel_path_and_generic_csr_matches_oracle():
     w = small("csr", causal=True, dtype="bf16", T=256, Kc=32, k_hat=6)
     run = GpuRun(w)
-    run.estimate(); run.topk_mask(); run.sparse_attn(use_sel=True); run.sync()
+    run.estimate(); run.topk_mask(); run.sparse_attn(use_sel=True, lean_ws=True); run.sync()
     O_sel, P_sel = run.O.clone(), run.P.clone()
     run.O.fill_(float("nan")); run.P.fill_(float("nan"))
     run.sparse_attn(use_sel=False); run.sync()
     nnz = int(run.row_ptr[-1])
-    assert torch.equal(O_sel, run.O)
+    assert torch.equal(O_sel, run.O)  # the per-row kernels share their arithmetic
     assert torch.equal(P_sel[:nnz].view(torch.int16), run.P[:nnz].view(torch.int16))
+    # the tensor-core tile kernel (full workspace) orders its sums differently: same tolerance as
+    # against the oracle
+    run.O.fill_(float("nan")); run.P.fill_(float("nan"))
+    run.sparse_attn(use_sel=True); run.sync()
+    assert run.status() == 0
+    check_float(np64(run.O), np64(O_sel), "bf16", "O tiles vs rows")
+    check_float(np64(run.P[:nnz]), np64(P_sel[:nnz]), "bf16", "P tiles vs rows")
 
     # an arbitrary CSR (unsorted columns, repeated keys, empty rows, one very long row)
     for dtype in ("f32", "bf16"):
