@@ -103,7 +103,7 @@ sea_status sea_topk_mask(const sea_shape* shape, const float* A_hat, int32_t* se
   int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
   return launch_topk_mask(*shape, A_hat, sel_buf, row_ptr, col_idx, nnz_cap,
                           reinterpret_cast<int32_t*>(w + L.row_counts),
-                          reinterpret_cast<int32_t*>(w + L.tile_sums),
+                          reinterpret_cast<int32_t*>(w + L.tile_sums), nullptr,
                           reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -125,7 +125,7 @@ sea_status sea_sparse_attn(const sea_shape* shape, const void* Q, const void* K,
   const WsLayout L = ws_layout(*shape);
   const bool full = ws && ws_bytes >= L.total;
   return launch_sparse_attn(*shape, Q, K, V, row_ptr, col_idx, sel, O, P,
-                            full ? reinterpret_cast<uint32_t*>(w + L.mask_bits) : nullptr,
+                            full ? reinterpret_cast<uint32_t*>(w + L.mask_bits) : nullptr, false,
                             full ? reinterpret_cast<float*>(w + L.p_scratch) : nullptr,
                             static_cast<int32_t*>(ws), static_cast<cudaStream_t>(cuda_stream));
 }
@@ -164,13 +164,13 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
   }
   int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
   int32_t* rp_buf = row_ptr ? row_ptr : reinterpret_cast<int32_t*>(w + L.row_ptr);
+  uint32_t* bits = reinterpret_cast<uint32_t*>(w + L.mask_bits);
   rc = launch_topk_mask(*shape, a_use, sel_buf, rp_buf, col_idx, nnz_cap,
                         reinterpret_cast<int32_t*>(w + L.row_counts),
-                        reinterpret_cast<int32_t*>(w + L.tile_sums), status, st);
+                        reinterpret_cast<int32_t*>(w + L.tile_sums), bits, status, st);
   if (rc != SEA_OK) return rc;
-  return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P,
-                            reinterpret_cast<uint32_t*>(w + L.mask_bits), reinterpret_cast<float*>(w + L.p_scratch),
-                            status, st);
+  return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P, bits, true,
+                            reinterpret_cast<float*>(w + L.p_scratch), status, st);
 }
 
 sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes) {

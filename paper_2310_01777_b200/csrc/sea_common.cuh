@@ -53,21 +53,23 @@ sea_status launch_estimate_bf16(const sea_shape& s, const void* Q, const void* K
 size_t estimate_split_bytes(const sea_shape& s);
 sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel,
                             int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
-                            int32_t* row_counts, int32_t* tile_sums, int32_t* status,
-                            cudaStream_t st);
+                            int32_t* row_counts, int32_t* tile_sums, uint32_t* mask_bits,
+                            int32_t* status, cudaStream_t st);
 // mask_bits and p_scratch (workspace areas of the tensor-core kernel) may be null: the per-row
-// kernels are used then.
+// kernels are used then.  bits_valid: mask_bits already holds the bit strings of `sel`
+// (launch_topk_mask wrote them); otherwise they are derived from `sel` first.
 sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, const void* V,
                               const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
-                              void* O, void* P, uint32_t* mask_bits, float* p_scratch, int32_t* status,
-                              cudaStream_t st);
+                              void* O, void* P, uint32_t* mask_bits, bool bits_valid, float* p_scratch,
+                              int32_t* status, cudaStream_t st);
 size_t sparse_attn_tc_bits_bytes(const sea_shape& s);
 size_t sparse_attn_tc_scratch_bytes(const sea_shape& s);
 bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, const int32_t* status,
                                const void* mask_bits, const void* p_scratch);
 sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* K, const void* V,
                                  const int32_t* row_ptr, const int32_t* sel, void* O, void* P,
-                                 uint32_t* mask_bits, float* p_scratch, int32_t* status, cudaStream_t st);
+                                 uint32_t* mask_bits, bool bits_valid, float* p_scratch, int32_t* status,
+                                 cudaStream_t st);
 bool sparse_attn_tma_applicable(const sea_shape& s, const int32_t* sel, const int32_t* status);
 sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void* K, const void* V,
                                   const int32_t* row_ptr, const int32_t* sel, void* O, void* P,

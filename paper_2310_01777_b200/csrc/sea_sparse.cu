@@ -369,10 +369,10 @@ sea_status launch_typed(const sea_shape& s, const T* Q, const T* K, const T* V,
 
 sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, const void* V,
                               const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
-                              void* O, void* P, uint32_t* mask_bits, float* p_scratch, int32_t* status,
-                              cudaStream_t st) {
+                              void* O, void* P, uint32_t* mask_bits, bool bits_valid, float* p_scratch,
+                              int32_t* status, cudaStream_t st) {
   if (sparse_attn_tc_applicable(s, sel, status, mask_bits, p_scratch))
-    return launch_sparse_attn_tc(s, Q, K, V, row_ptr, sel, O, P, mask_bits, p_scratch, status, st);
+    return launch_sparse_attn_tc(s, Q, K, V, row_ptr, sel, O, P, mask_bits, bits_valid, p_scratch, status, st);
   if (sparse_attn_tma_applicable(s, sel, status))
     return launch_sparse_attn_tma(s, Q, K, V, row_ptr, sel, O, P, status, st);
   if (s.io == SEA_BF16) {

@@ -765,8 +765,8 @@ bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, const int
 }
 
 sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* K, const void* V, const int32_t* row_ptr,
-                                 const int32_t* sel, void* O, void* P, uint32_t* mask_bits, float* p_scratch,
-                                 int32_t* status, cudaStream_t st) {
+                                 const int32_t* sel, void* O, void* P, uint32_t* mask_bits, bool bits_valid,
+                                 float* p_scratch, int32_t* status, cudaStream_t st) {
   const unsigned long long rows = (unsigned long long)s.B * s.H * s.T;
   CUtensorMap mq, mk, mv;
   if (!make_tile_map(&mq, Q, rows) || !make_tile_map(&mk, K, rows) || !make_tile_map(&mv, V, rows)) return SEA_ERR_CUDA;
@@ -787,9 +787,11 @@ sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* 
   const float scale = s.scale != 0.f ? s.scale : 0.125f;
   prm.scale_log2 = scale * 1.4426950408889634f;
 
-  sel_to_bits_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sel, mask_bits, (int)rows, s.k_hat, prm.words);
-  sea_status rc = check_launch();
-  if (rc != SEA_OK) return rc;
+  if (!bits_valid) {
+    sel_to_bits_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(sel, mask_bits, (int)rows, s.k_hat, prm.words);
+    const sea_status rc = check_launch();
+    if (rc != SEA_OK) return rc;
+  }
   const int L = prm.log2r < 7 ? prm.log2r : 7;
 #define SEA_TC(LL)                                                                   \
   case LL:                                                                           \

@@ -15,6 +15,8 @@ constexpr int kWarpsPerCta = 8;
 constexpr int kScanThreads = 256;
 constexpr int kScanPerThread = 8;
 constexpr int kScanTile = kScanThreads * kScanPerThread;
+constexpr int kThreadMaxKc = 128;  // shapes handled with one thread per row: the sorted-list walk costs
+constexpr int kThreadMaxK = 32;    // Kc * k_hat min/max pairs per row, the bit search about 64 * Kc / 32 * 32
 
 __device__ __forceinline__ uint32_t order_key(float v) {
   uint32_t u = __float_as_uint(v);
@@ -26,8 +28,8 @@ __device__ __forceinline__ uint32_t order_key(float v) {
 template <int VPL>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
-                 int32_t* __restrict__ row_counts, int rows, int Kc, int k_hat, int seq_len, int r,
-                 int causal) {
+                 int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc, int k_hat,
+                 int seq_len, int r, int causal) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kWarpsPerCta + warp;
   if (row >= rows) return;
@@ -70,6 +72,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
       my_sel[out_base + __popc(sb & lt_mask)] = col;
       cnt += causal ? max(0, min(r, i + 1 - col * r)) : r;
     }
+    if (mask_bits != nullptr && lane == 0 && 32 * t < Kc) mask_bits[(size_t)row * ((Kc + 31) / 32) + t] = sb;
     tie_seen += __popc(tb);
     out_base += __popc(sb);
   }
@@ -77,6 +80,87 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
     cnt = __reduce_add_sync(0xffffffffu, cnt);
     if (lane == 0) row_counts[row] = cnt;
   }
+}
+
+// Selection with one thread per row, for short rows and small k_hat: no cross-lane traffic at
+// all.  Every thread streams its row (16-byte loads; a row is a few cache lines that the
+// thread walks front to back) through a sorted list of the KMAX largest keys seen so far - a
+// max/min pair per list slot, branch-free - which leaves the k_hat-th largest key tau in the
+// last slot; a second walk over the row emits, in ascending column order, the columns above
+// tau and the first k_hat - |{key > tau}| columns equal to it: the same set as the bit search
+// below, ties going to the lower column.
+constexpr int kThreadRows = 128;  // threads (= rows) per CTA
+
+template <int KMAX>
+__device__ __forceinline__ void list_insert(uint32_t (&top)[KMAX], uint32_t x) {
+#pragma unroll
+  for (int s = 0; s < KMAX; ++s) {
+    const uint32_t hi = max(top[s], x);
+    x = min(top[s], x);
+    top[s] = hi;
+  }
+}
+
+template <int KMAX, bool kVec>
+__global__ void __launch_bounds__(kThreadRows)
+topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
+                        int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc,
+                        int k_hat, int seq_len, int r, int causal) {
+  const int row = blockIdx.x * kThreadRows + threadIdx.x;
+  if (row >= rows) return;
+  const float* a = A_hat + (size_t)row * Kc;
+  // Descending list.  Its first KMAX - k_hat slots hold a sentinel above every real key, so the
+  // k_hat-th largest real key always ends up in the last slot; 0 sorts below every real key.
+  uint32_t top[KMAX];
+#pragma unroll
+  for (int s = 0; s < KMAX; ++s) top[s] = s < KMAX - k_hat ? 0xffffffffu : 0u;
+  if (kVec) {  // Kc % 4 == 0: rows start on 16-byte boundaries
+    for (int j = 0; j < Kc; j += 4) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(a + j));
+      list_insert<KMAX>(top, order_key(v.x));
+      list_insert<KMAX>(top, order_key(v.y));
+      list_insert<KMAX>(top, order_key(v.z));
+      list_insert<KMAX>(top, order_key(v.w));
+    }
+  } else {
+    for (int j = 0; j < Kc; ++j) list_insert<KMAX>(top, order_key(__ldg(a + j)));
+  }
+  const uint32_t tau = top[KMAX - 1];
+  int n_gt = 0;
+#pragma unroll
+  for (int s = 0; s < KMAX; ++s) n_gt += (top[s] != 0xffffffffu && top[s] > tau);
+  const int need = k_hat - n_gt;  // how many columns equal to tau are taken (lowest first)
+
+  const int i = row % seq_len;
+  const int words = (Kc + 31) / 32;
+  int32_t* my_sel = sel + (size_t)row * k_hat;
+  int out = 0, tie_seen = 0, cnt = 0;
+  uint32_t word = 0u;
+  auto visit = [&](int j, float v) {
+    const uint32_t x = order_key(v);
+    const bool tie = x == tau;
+    const bool take = x > tau || (tie && tie_seen < need);
+    tie_seen += tie;
+    if (take) {
+      my_sel[out++] = j;
+      cnt += causal ? max(0, min(r, i + 1 - j * r)) : r;
+      word |= 1u << (j & 31);
+    }
+  };
+  for (int j0 = 0; j0 < Kc; j0 += 32) {
+    const int j1 = min(Kc, j0 + 32);
+    if (kVec) {
+      for (int j = j0; j < j1; j += 4) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(a + j));
+        visit(j, v.x); visit(j + 1, v.y); visit(j + 2, v.z); visit(j + 3, v.w);
+      }
+    } else {
+      for (int j = j0; j < j1; ++j) visit(j, __ldg(a + j));
+    }
+    if (mask_bits != nullptr) mask_bits[(size_t)row * words + (j0 >> 5)] = word;
+    word = 0u;
+  }
+  if (row_counts != nullptr) row_counts[row] = cnt;
 }
 
 // ---- exclusive scan of row_counts -> row_ptr (three small kernels) -------------------
@@ -186,10 +270,10 @@ fill_col_idx_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__
 }
 
 template <int VPL>
-void launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, int rows, const sea_shape& s,
-                 cudaStream_t st) {
+void launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, uint32_t* mask_bits, int rows,
+                 const sea_shape& s, cudaStream_t st) {
   const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
-  topk_rows_kernel<VPL><<<grid, kWarpsPerCta * 32, 0, st>>>(A_hat, sel, counts, rows, s.Kc, s.k_hat,
+  topk_rows_kernel<VPL><<<grid, kWarpsPerCta * 32, 0, st>>>(A_hat, sel, counts, mask_bits, rows, s.Kc, s.k_hat,
                                                              s.T, s.T / s.Kc, s.causal);
 }
 
@@ -197,18 +281,35 @@ void launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, int rows, co
 
 sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel, int32_t* row_ptr,
                             int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts,
-                            int32_t* tile_sums, int32_t* status, cudaStream_t st) {
+                            int32_t* tile_sums, uint32_t* mask_bits, int32_t* status, cudaStream_t st) {
   const int rows = s.B * s.H * s.T;
   const int r = s.T / s.Kc;
   int32_t* counts = s.causal ? row_counts : nullptr;
   const int vpl = (s.Kc + 31) / 32;
-  if (vpl <= 1) launch_topk<1>(A_hat, sel, counts, rows, s, st);
-  else if (vpl <= 2) launch_topk<2>(A_hat, sel, counts, rows, s, st);
-  else if (vpl <= 4) launch_topk<4>(A_hat, sel, counts, rows, s, st);
-  else if (vpl <= 8) launch_topk<8>(A_hat, sel, counts, rows, s, st);
-  else if (vpl <= 16) launch_topk<16>(A_hat, sel, counts, rows, s, st);
-  else if (vpl <= 32) launch_topk<32>(A_hat, sel, counts, rows, s, st);
-  else if (vpl <= 64) launch_topk<64>(A_hat, sel, counts, rows, s, st);
+  if (s.Kc <= kThreadMaxKc && s.k_hat <= kThreadMaxK) {
+    // a short row and few columns to keep: one thread per row
+    const int grid = (rows + kThreadRows - 1) / kThreadRows;
+#define SEA_TOPK_THREAD(KM)                                                                                     \
+  do {                                                                                                          \
+    if (s.Kc % 4 == 0)                                                                                          \
+      topk_rows_thread_kernel<KM, true><<<grid, kThreadRows, 0, st>>>(A_hat, sel, counts, mask_bits, rows,     \
+                                                                      s.Kc, s.k_hat, s.T, r, s.causal);        \
+    else                                                                                                        \
+      topk_rows_thread_kernel<KM, false><<<grid, kThreadRows, 0, st>>>(A_hat, sel, counts, mask_bits, rows,    \
+                                                                       s.Kc, s.k_hat, s.T, r, s.causal);       \
+  } while (0)
+    if (s.k_hat <= 8) SEA_TOPK_THREAD(8);
+    else if (s.k_hat <= 16) SEA_TOPK_THREAD(16);
+    else SEA_TOPK_THREAD(32);
+#undef SEA_TOPK_THREAD
+  }
+  else if (vpl <= 1) launch_topk<1>(A_hat, sel, counts, mask_bits, rows, s, st);
+  else if (vpl <= 2) launch_topk<2>(A_hat, sel, counts, mask_bits, rows, s, st);
+  else if (vpl <= 4) launch_topk<4>(A_hat, sel, counts, mask_bits, rows, s, st);
+  else if (vpl <= 8) launch_topk<8>(A_hat, sel, counts, mask_bits, rows, s, st);
+  else if (vpl <= 16) launch_topk<16>(A_hat, sel, counts, mask_bits, rows, s, st);
+  else if (vpl <= 32) launch_topk<32>(A_hat, sel, counts, mask_bits, rows, s, st);
+  else if (vpl <= 64) launch_topk<64>(A_hat, sel, counts, mask_bits, rows, s, st);
   else return SEA_ERR_UNSUPPORTED;
   sea_status rc = check_launch();
   if (rc != SEA_OK) return rc;
@@ -302,5 +403,5 @@ extern "C" sea_status sea_topk_mask_static(const sea_shape* shape, const float* 
   // by the kernels, the status word is the one thing that has to start at zero
   if (cudaMemsetAsync(scratch, 0, sizeof(int32_t), st) != cudaSuccess) return SEA_ERR_CUDA;
   return launch_topk_mask(*shape, A_hat, sel, row_ptr, col_idx, nnz_cap, scratch + kStaticHead,
-                          scratch + kStaticHead + kStaticMaxRows, scratch, st);
+                          scratch + kStaticHead + kStaticMaxRows, nullptr, scratch, st);
 }
