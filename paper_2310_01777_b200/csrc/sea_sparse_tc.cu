@@ -17,10 +17,10 @@
 // unnormalised fp32 probabilities of kept keys are parked in a scratch array and written to P
 // (rounded once, after the division by the row sum) when the item ends.
 //
-// Warp roles (512 threads, four warpgroups that re-balance their registers): warp 0 issues the
-// TMA copies (the item's mask bits and Q tile, K and V tiles through rings of 16 KB stages),
-// warp 1 issues the MMAs; warps 4..11 own the query rows (a row and one half of every tile's
-// columns per thread); warps 12..15 turn the parked probabilities into P.  All hand-offs are
+// Warp roles (warpgroups that re-balance their registers): warp 0 issues the TMA copies (the
+// item's mask bits and Q tile, K and V tiles through rings of 16 KB stages), warp 1 issues the
+// Q K^T MMAs, warp 2 the P V MMAs; the row warpgroups own the query rows (per thread a row and 128 / kSplit of every
+// tile's columns); the last warpgroup turns the parked probabilities into P.  All hand-offs are
 // mbarriers; every wait is bounded by a clock and a wait that runs out sets SEA_DEV_TIMEOUT,
 // after which all roles drain and leave.
 #include <cuda.h>
@@ -34,13 +34,25 @@ constexpr int kTile = 128;                // queries per work item, keys per til
 constexpr int kTileBytes = kTile * 128;   // 128 rows x 64 bf16
 constexpr int kNK = 4;                    // K ring stages
 constexpr int kNV = 3;                    // V ring stages
-constexpr int kThreads = 512;             // 4 warpgroups: control, 2 x row warps, P writers
-constexpr int kRegsCtl = 40;              // registers per thread after the warpgroups re-balance
-constexpr int kRegsRow = 200;
-constexpr int kRegsFix = 72;
+constexpr int kSplit = 4;                 // row warpgroups: each takes 128 / kSplit columns of every tile
+constexpr int kRowWarps = 4 * kSplit;
+constexpr int kRowThreads = 32 * kRowWarps;
+constexpr int kThreads = 128 * (kSplit + 2);  // warpgroups: control, kSplit x row warps, P writers
+constexpr int kChunks = 4 / kSplit;       // 32-column chunks per row thread and tile
+// Registers per thread after the warpgroups re-balance.  A warpgroup can only grow by what the
+// others of this CTA have given back, so over the warpgroups they sum to no more than the launch
+// allocation (kSplit 2: 4 x 128, kSplit 4: 6 x 80), or the growing warps would wait for ever.
+constexpr int kRegsLaunch = kSplit == 2 ? 128 : 80;
+constexpr int kRegsCtl = kSplit == 2 ? 40 : 32;
+constexpr int kRegsRow = kSplit == 2 ? 200 : 96;
+constexpr int kRegsFix = kSplit == 2 ? 72 : 64;
+static_assert(kRegsCtl + kSplit * kRegsRow + kRegsFix <= kRegsLaunch * (kSplit + 2), "register re-balance exceeds the launch allocation");
+static_assert(kRegsLaunch * kThreads <= 65536, "launch allocation exceeds the register file");
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;             // two S / P buffers of 128 columns
-constexpr uint32_t kColO = 256;           // two O buffers of 64 columns
+constexpr int kNS = 3;                    // S / P buffers of 128 columns: the MMAs run up to two tiles ahead of the rows
+constexpr uint32_t kColS = 0;
+constexpr uint32_t kColO = 128 * kNS;     // two O buffers of 64 columns
+static_assert(kColO + 128 <= kTmemCols, "tensor memory budget");
 constexpr unsigned long long kWaitNs = 1000000000ull;  // limit of one wait
 
 // Barrier indices inside the shared-memory barrier block.
@@ -51,16 +63,18 @@ enum {
   kBarKEmpty = kBarKFull + kNK,  // [kNK]
   kBarVFull = kBarKEmpty + kNK,  // [kNV]
   kBarVEmpty = kBarVFull + kNV,  // [kNV]
-  kBarSFull = kBarVEmpty + kNV,  // [2]  S tile written by the MMA
-  kBarSDone = kBarSFull + 2,     // [2]  S tile read (first pass) / P written (second pass)
-  kBarOFull = kBarSDone + 2,     // [2]
+  kBarSFull = kBarVEmpty + kNV,  // [kNS]  S tile written by the MMA
+  kBarSDone = kBarSFull + kNS,   // [kNS]  S tile read (first pass) / P written (second pass)
+  kBarOFull = kBarSDone + kNS,   // [2]
   kBarOEmpty = kBarOFull + 2,    // [2]
   kBarBitsFull = kBarOEmpty + 2,      // [2]  the item's mask bits have landed
   kBarBitsEmpty = kBarBitsFull + 2,   // [2]
   kBarFixFull = kBarBitsEmpty + 2,    // [2]  row normalisers handed to the P writers
   kBarFixEmpty = kBarFixFull + 2,     // [2]
-  kBarDrain = kBarFixEmpty + 2,       // [1]
-  kNumBars = kBarDrain + 1
+  kBarPFree = kBarFixEmpty + 2,       // [kNS]  the P V product has consumed the buffer
+  kBarDrain = kBarPFree + kNS,        // [1]
+  kBarDrain2 = kBarDrain + 1,         // [1]
+  kNumBars = kBarDrain2 + 1
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -116,14 +130,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
   d |= (uint64_t)2 << 61;
   return d;
 }
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-               ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
-               ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
-}
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
 }
@@ -139,6 +145,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_n(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld32(taddr, r); }
+__device__ __forceinline__ void tmem_ld_n(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld16(taddr, r); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
@@ -157,6 +172,49 @@ __device__ __forceinline__ float ex2(float x) {  // 2^x; x = -inf gives 0
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 // B = V tile read MN-major (keys are its K index), N = 64.
 constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+
+// The four MMAs of S = Q K^T (contraction steps of 16 along d; a step moves both descriptors on by
+// 32 bytes).  All operands are formed before the block, so that the issuing thread, which shares
+// its scheduler with row warps, spends one instruction per MMA inside it.
+__device__ __forceinline__ void issue_qk_mmas(uint32_t d_tmem, uint64_t q_desc, uint64_t k_desc) {
+  const uint64_t q1 = q_desc + 2, q2 = q_desc + 4, q3 = q_desc + 6;
+  const uint64_t k1 = k_desc + 2, k2 = k_desc + 4, k3 = k_desc + 6;
+  asm volatile(
+      "{\n .reg .pred pz, pt;\n"
+      "setp.ne.b32 pz, %0, %0;\n setp.eq.b32 pt, %0, %0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %5, %9, pz;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %6, %9, pt;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %3, %7, %9, pt;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %4, %8, %9, pt;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(q_desc), "l"(q1), "l"(q2), "l"(q3), "l"(k_desc), "l"(k1), "l"(k2), "l"(k3), "r"(kIdescQK)
+      : "memory");
+}
+// Eight of the sixteen MMAs of O += P V for one key tile (contraction steps 4 h .. 4 h + 3): step
+// k takes the head of P from columns 32 (k / 2) + 8 (k % 2) of the buffer, the remainder from 16
+// columns further on, and keys 16 k .. 16 k + 15 of the V stage (2048 bytes per step).
+// `accumulate` is 0 only for the very first MMA of a work item.
+__device__ __forceinline__ void issue_pv_half(uint32_t d_tmem, uint32_t p_tmem, uint64_t v_desc, int h, uint32_t accumulate) {
+  const uint32_t pa = p_tmem + 64 * h;
+  const uint64_t vd = v_desc + 512 * h;
+  const uint32_t a1 = pa + 16, a2 = pa + 8, a3 = pa + 24, a4 = pa + 32, a5 = pa + 48, a6 = pa + 40, a7 = pa + 56;
+  const uint64_t v1 = vd + 128, v2 = vd + 256, v3 = vd + 384;
+  asm volatile(
+      "{\n .reg .pred pf, pt;\n"
+      "setp.ne.b32 pf, %14, 0;\n setp.eq.b32 pt, %0, %0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %9, %13, pf;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%2], %9, %13, pt;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%3], %10, %13, pt;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%4], %10, %13, pt;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%5], %11, %13, pt;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%6], %11, %13, pt;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%7], %12, %13, pt;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%8], %12, %13, pt;\n"
+      "}\n"
+      ::"r"(d_tmem), "r"(pa), "r"(a1), "r"(a2), "r"(a3), "r"(a4), "r"(a5), "r"(a6), "r"(a7), "l"(vd), "l"(v1), "l"(v2),
+        "l"(v3), "r"(kIdescPV), "r"(accumulate)
+      : "memory");
+}
 
 struct TcParams {
   const __nv_bfloat16* Q;       // unused by the kernel body (TMA reads it); kept for clarity
@@ -238,67 +296,56 @@ __device__ __forceinline__ float chunk_max(const uint32_t (&v)[32], uint32_t tb,
 
 // Probabilities of one 32-column chunk: p = 2^(s * cs + bias) with bias = -max * cs for kept
 // columns and -inf otherwise; the row sum grows by them; hi / lo receive the bf16 head
-// (truncated) and the bf16 remainder, two columns per word.
-template <int L, bool kDiag>
+// (truncated) and the bf16 remainder, two columns per word.  With kWriteP the kept
+// probabilities are parked as fp32: run `rank` of the row starts at rank * r.
+template <int L, bool kDiag, bool kWriteP>
 __device__ __forceinline__ void chunk_probs(const uint32_t (&v)[32], uint32_t tb, int cg, int lim, float cs,
-                                            float neg_mc, float2& la, float2& lb, float (&pr)[32], uint32_t (&hi)[16],
-                                            uint32_t (&lo)[16]) {
+                                            float neg_mc, float2& la, float2& lb, uint32_t (&hi)[16],
+                                            uint32_t (&lo)[16], float* my_scratch, int rank_base, int off0) {
+  constexpr int R = 1 << (L < 5 ? L : 5);  // columns of this chunk per group
   const float2 cs2 = make_float2(cs, cs);
   const float2 m1 = make_float2(-1.f, -1.f);
 #pragma unroll
-  for (int e2 = 0; e2 < 16; ++e2) {
-    int g;
-    if constexpr (L >= 5) g = L >= 7 ? 0 : (32 * cg) >> L;
-    else g = ((32 * cg) >> L) + ((2 * e2) >> L);
-    const float bias = ((tb >> g) & 1u) ? neg_mc : -INFINITY;
-    const float b0 = (!kDiag || 2 * e2 <= lim) ? bias : -INFINITY;
-    const float b1 = (!kDiag || 2 * e2 + 1 <= lim) ? bias : -INFINITY;
-    const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * e2]), __uint_as_float(v[2 * e2 + 1])), cs2, make_float2(b0, b1));
-    const float2 pp = make_float2(ex2(x.x), ex2(x.y));
-    pr[2 * e2] = pp.x;
-    pr[2 * e2 + 1] = pp.y;
-    if (e2 & 1) lb = __fadd2_rn(lb, pp); else la = __fadd2_rn(la, pp);
-    const uint32_t h0 = __float_as_uint(pp.x) & 0xffff0000u, h1 = __float_as_uint(pp.y) & 0xffff0000u;
-    hi[e2] = __byte_perm(h0, h1, 0x7632);
-    const float2 rem = __ffma2_rn(make_float2(__uint_as_float(h0), __uint_as_float(h1)), m1, pp);  // p - head, exact
-    const __nv_bfloat162 l2 = __floats2bfloat162_rn(rem.x, rem.y);
-    lo[e2] = *reinterpret_cast<const uint32_t*>(&l2);
-  }
-}
-
-// Parks the kept probabilities of a chunk: run `rank` of the row starts at rank * r.
-template <int L>
-__device__ __forceinline__ void chunk_park(const float (&pr)[32], uint32_t tb, int cg, float* my_scratch, int rank_base, int off0) {
-  if constexpr (L >= 5) {
-    const int g = L >= 7 ? 0 : (32 * cg) >> L;
-    if ((tb >> g) & 1u) {
-      const int off = L < 7 ? ((rank_base + __popc(tb & ((1u << g) - 1u))) << L) + (32 * cg - (g << L)) : off0 + 32 * cg;
-      float4* dst = reinterpret_cast<float4*>(my_scratch + off);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) dst[e] = make_float4(pr[4 * e], pr[4 * e + 1], pr[4 * e + 2], pr[4 * e + 3]);
+  for (int gi = 0; gi < 32 / R; ++gi) {
+    const int g = L >= 7 ? 0 : ((32 * cg) >> L) + (L < 5 ? gi : 0);
+    const bool live = (tb >> g) & 1u;
+    const float bias = live ? neg_mc : -INFINITY;
+    float4* dst = nullptr;
+    if (kWriteP) {
+      const int off = L >= 7 ? off0 + 32 * cg
+                             : ((rank_base + __popc(tb & ((1u << g) - 1u))) << L) + (32 * cg + gi * R - (g << L));
+      dst = reinterpret_cast<float4*>(my_scratch + off);
     }
-  } else {
-    constexpr int R = 1 << L;
-    const int g0 = (32 * cg) >> L;
+    float2 prev = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int gi = 0; gi < 32 / R; ++gi) {
-      const int g = g0 + gi;
-      if ((tb >> g) & 1u) {
-        float4* dst = reinterpret_cast<float4*>(my_scratch + ((rank_base + __popc(tb & ((1u << g) - 1u))) << L));
-#pragma unroll
-        for (int e = 0; e < R / 4; ++e)
-          dst[e] = make_float4(pr[gi * R + 4 * e], pr[gi * R + 4 * e + 1], pr[gi * R + 4 * e + 2], pr[gi * R + 4 * e + 3]);
+    for (int e2 = gi * R / 2; e2 < (gi + 1) * R / 2; ++e2) {
+      const float b0 = (!kDiag || 2 * e2 <= lim) ? bias : -INFINITY;
+      const float b1 = (!kDiag || 2 * e2 + 1 <= lim) ? bias : -INFINITY;
+      const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * e2]), __uint_as_float(v[2 * e2 + 1])), cs2, make_float2(b0, b1));
+      const float2 pp = make_float2(ex2(x.x), ex2(x.y));
+      if (e2 & 1) lb = __fadd2_rn(lb, pp); else la = __fadd2_rn(la, pp);
+      const uint32_t h0 = __float_as_uint(pp.x) & 0xffff0000u, h1 = __float_as_uint(pp.y) & 0xffff0000u;
+      hi[e2] = __byte_perm(h0, h1, 0x7632);
+      const float2 rem = __ffma2_rn(make_float2(__uint_as_float(h0), __uint_as_float(h1)), m1, pp);  // p - head, exact
+      const __nv_bfloat162 l2 = __floats2bfloat162_rn(rem.x, rem.y);
+      lo[e2] = *reinterpret_cast<const uint32_t*>(&l2);
+      if (kWriteP) {
+        if (e2 & 1) {
+          if (live) dst[(e2 - gi * R / 2) >> 1] = make_float4(prev.x, prev.y, pp.x, pp.y);
+        } else {
+          prev = pp;
+        }
       }
     }
   }
 }
 
-// AND of a predicate over the 256 row threads (named barrier 1); also orders their memory accesses.
+// AND of a predicate over the row threads (named barrier 1); also orders their memory accesses.
 __device__ __forceinline__ bool rows_all(bool ok) {
   uint32_t r;
   asm volatile(
-      "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.and.pred p, 1, 256, q;\n selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(r) : "r"((uint32_t)ok) : "memory");
+      "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.and.pred p, 1, %2, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(r) : "r"((uint32_t)ok), "n"(kRowThreads) : "memory");
   return r != 0;
 }
 
@@ -325,9 +372,9 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
   const uint32_t bars = smem_u32(tail);                      // kNumBars x 8 B
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8 * kNumBars + 4);
-  float* xch = reinterpret_cast<float*>(tail + 8 * kNumBars + 8);       // [2 halves][128] partial maxima
-  float* xch_l = xch + 2 * kTile;                                        // [2 halves][128] partial sums
-  float* fix_inv = xch_l + 2 * kTile;                                      // [2 slots][128]
+  float* xch = reinterpret_cast<float*>(tail + 8 * kNumBars + 8);       // [kSplit][128] partial maxima
+  float* xch_l = xch + kSplit * kTile;                                   // [kSplit][128] partial sums
+  float* fix_inv = xch_l + kSplit * kTile;                                      // [2 slots][128]
   int* fix_base = reinterpret_cast<int*>(fix_inv + 2 * kTile);           // [2][128]
   int* fix_cnt = fix_base + 2 * kTile;                                   // [2][128]
   uint32_t* bits = reinterpret_cast<uint32_t*>(fix_cnt + 2 * kTile);     // [2 slots][128 rows][words]
@@ -337,9 +384,9 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
   if (tid == 0) {
     for (int i = 0; i < kNumBars; ++i) {
       uint32_t count = 1;
-      if ((i >= kBarSDone && i < kBarSDone + 2) || (i >= kBarOEmpty && i < kBarOEmpty + 2) ||
+      if ((i >= kBarSDone && i < kBarSDone + kNS) || (i >= kBarOEmpty && i < kBarOEmpty + 2) ||
           (i >= kBarBitsEmpty && i < kBarBitsEmpty + 2))
-        count = 8;  // one arrival per row warp
+        count = kRowWarps;  // one arrival per row warp
       if ((i >= kBarFixFull && i < kBarFixFull + 2) || (i >= kBarFixEmpty && i < kBarFixEmpty + 2)) count = 4;
       mbar_init(bar(i), count);
     }
@@ -402,78 +449,93 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         mbar_wait(bar(kBarBitsFull + (i & 1)), (i >> 1) & 1, abort_flag);
       }
     } else if (warp == 1 && lane == 0) {
-      // ---------------------------------------------------------------- MMA issuer
-      uint32_t q_it = 0, k_it = 0, v_it = 0, s_it = 0, s_waited = 0, o_it = 0;
+      // ---------------------------------------------------------------- issuer of S = Q K^T
+      // S/P buffer u % kNS serves use u (the tiles of the first pass, then of the second pass, item
+      // after item).  Before a buffer is written again its previous use must be over: the rows have
+      // read S (first-pass use, barrier SDone) or the P V product has consumed P (second-pass use,
+      // barrier PFree, committed by the other issuer).
+      uint32_t q_it = 0, k_it = 0, s_it = 0;
+      uint32_t prev_second = 0;  // bit b: the last use of buffer b belonged to a second pass
+      uint32_t pfree_par = 0;    // bit b: parity of the PFree phase that ends that use
+      uint32_t pfree_cnt = 0;    // bit b: parity of the number of second-pass uses of buffer b so far
       bool ok = true;
-      // waits until the row warps are done with S/P uses 0 .. upto-1
-      auto rows_done_upto = [&](uint32_t upto) {
-        while (ok && (int)s_waited < (int)upto) {
-          ok = mbar_wait(bar(kBarSDone + (s_waited & 1)), (s_waited >> 1) & 1, abort_flag);
-          ++s_waited;
-        }
-        tc_fence_after();
-      };
-      auto issue_qk = [&](uint32_t qb, bool last) {
-        const uint32_t u = s_it;
-        if (u >= 2) rows_done_upto(u - 1);
-        const uint32_t ks = k_it % kNK;
-        if (ok) ok = mbar_wait(bar(kBarKFull + ks), (k_it / kNK) & 1, abort_flag);
-        if (!ok) return;
-        tc_fence_after();
-        const uint32_t d = tmem + kColS + 128 * (u & 1);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          mma_ss(d, smem_desc(sQ + qb * kTileBytes + 32 * k, 16, 1024), smem_desc(sK + ks * kTileBytes + 32 * k, 16, 1024),
-                 kIdescQK, k > 0);
-        mma_commit(bar(kBarKEmpty + ks));
-        mma_commit(bar(kBarSFull + (u & 1)));
-        if (last) mma_commit(bar(kBarQEmpty + qb));
-        ++s_it;
-        ++k_it;
-      };
-      auto issue_pv = [&](uint32_t u, uint32_t ob, bool first, bool last) {
-        rows_done_upto(u + 1);
-        if (ok && first) ok = mbar_wait(bar(kBarOEmpty + ob), ((o_it >> 1) & 1) ^ 1, abort_flag);
-        const uint32_t vs = v_it % kNV;
-        if (ok) ok = mbar_wait(bar(kBarVFull + vs), (v_it / kNV) & 1, abort_flag);
-        if (!ok) return;
-        tc_fence_after();
-        const uint32_t d = tmem + kColO + 64 * ob;
-        const uint32_t a0 = tmem + kColS + 128 * (u & 1);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t a_hi = a0 + 32 * (k >> 1) + 8 * (k & 1);
-          const uint64_t bd = smem_desc(sV + vs * kTileBytes + 2048 * k, 8192, 1024);
-          mma_ts(d, a_hi, bd, kIdescPV, !(first && k == 0));
-          mma_ts(d, a_hi + 16, bd, kIdescPV, 1);
-        }
-        mma_commit(bar(kBarVEmpty + vs));
-        if (last) mma_commit(bar(kBarOFull + ob));
-        ++v_it;
-      };
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const Item it = decode_item(item, p);
-        const uint32_t qb = q_it & 1, ob = o_it & 1;
+        const uint32_t qb = q_it & 1;
         ok = mbar_wait(bar(kBarQFull + qb), (q_it >> 1) & 1, abort_flag);
-        for (int t = 0; t < it.nt && ok; ++t) issue_qk(qb, false);               // first pass: scores only
-        for (int t = 0; t < it.nt && ok; ++t) {                                    // second pass
-          issue_qk(qb, t == it.nt - 1);
-          if (t >= 1 && ok) issue_pv(s_it - 2, ob, t == 1, false);
+        const uint64_t q_desc = smem_desc(sQ + qb * kTileBytes, 16, 1024);
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+          for (int t = 0; t < it.nt && ok; ++t) {
+            const uint32_t u = s_it, b = u % kNS;
+            if (u >= (uint32_t)kNS) {
+              if ((prev_second >> b) & 1u) ok = mbar_wait(bar(kBarPFree + b), (pfree_par >> b) & 1u, abort_flag);
+              else ok = mbar_wait(bar(kBarSDone + b), ((u - kNS) / kNS) & 1, abort_flag);
+            }
+            const uint32_t ks = k_it % kNK;
+            if (ok) ok = mbar_wait(bar(kBarKFull + ks), (k_it / kNK) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            issue_qk_mmas(tmem + kColS + 128 * b, q_desc, smem_desc(sK + ks * kTileBytes, 16, 1024));
+            mma_commit(bar(kBarKEmpty + ks));
+            mma_commit(bar(kBarSFull + b));
+            if (pass == 1 && t == it.nt - 1) mma_commit(bar(kBarQEmpty + qb));
+            if (pass == 1) {
+              prev_second |= 1u << b;
+              pfree_par = (pfree_par & ~(1u << b)) | (pfree_cnt & (1u << b));
+              pfree_cnt ^= 1u << b;
+            } else {
+              prev_second &= ~(1u << b);
+            }
+            ++s_it;
+            ++k_it;
+          }
         }
-        if (ok) issue_pv(s_it - 1, ob, it.nt == 1, true);
         ++q_it;
-        ++o_it;
       }
-      // every MMA issued so far must have finished before tensor memory is released
+      // every MMA issued by this thread must have finished before tensor memory is released
       mma_commit(bar(kBarDrain));
       mbar_wait(bar(kBarDrain), 0, abort_flag);
+    } else if (warp == 2 && lane == 0) {
+      // ---------------------------------------------------------------- issuer of O += P V
+      uint32_t v_it = 0, o_it = 0, use0 = 0, s_waited = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const Item it = decode_item(item, p);
+        const uint32_t ob = o_it & 1;
+        const uint32_t d = tmem + kColO + 64 * ob;
+        for (int t = 0; t < it.nt && ok; ++t) {
+          const uint32_t u = use0 + it.nt + t, b = u % kNS;  // the second pass follows the item's first
+          // the rows have written P.  A parity wait only tells the current phase from the one before
+          // it, so this thread follows SDone through every use, the first-pass ones included.
+          while (ok && s_waited <= u) {
+            ok = mbar_wait(bar(kBarSDone + s_waited % kNS), (s_waited / kNS) & 1, abort_flag);
+            ++s_waited;
+          }
+          if (ok && t == 0) ok = mbar_wait(bar(kBarOEmpty + ob), ((o_it >> 1) & 1) ^ 1, abort_flag);
+          const uint32_t vs = v_it % kNV;
+          if (ok) ok = mbar_wait(bar(kBarVFull + vs), (v_it / kNV) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t vd = smem_desc(sV + vs * kTileBytes, 8192, 1024);
+          issue_pv_half(d, tmem + kColS + 128 * b, vd, 0, t == 0 ? 0u : 1u);
+          issue_pv_half(d, tmem + kColS + 128 * b, vd, 1, 1u);
+          mma_commit(bar(kBarVEmpty + vs));
+          mma_commit(bar(kBarPFree + b));
+          if (t == it.nt - 1) mma_commit(bar(kBarOFull + ob));
+          ++v_it;
+        }
+        use0 += 2 * it.nt;
+        ++o_it;
+      }
+      mma_commit(bar(kBarDrain2));
+      mbar_wait(bar(kBarDrain2), 0, abort_flag);
     }
-  } else if (warp < 12) {
+  } else if (warp < 4 + kRowWarps) {
     // ---------------------------------------------------------------- row warps: a query row and
-    // one half of every tile's columns per thread
+    // 128 / kSplit of every tile's columns per thread
     reg_inc<kRegsRow>();
     const int quarter = warp & 3;          // tensor-memory lanes 32*quarter .. +31
-    const int half = (warp - 4) >> 2;      // columns 64*half .. +63 of every tile
+    const int part = (warp - 4) >> 2;      // columns (128 / kSplit) * part .. of every tile
     const int rt = quarter * 32 + lane;    // row inside the work item
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     const int log2r = p.log2r;
@@ -486,7 +548,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       const int row = it.row0 + rt;
       const uint32_t slot = it_cnt & 1;
       int p_base = 0, p_cnt = 0;
-      if (kWriteP && half == 0) {
+      if (kWriteP && part == 0) {
         p_base = __ldg(p.row_ptr + row);
         p_cnt = __ldg(p.row_ptr + row + 1) - p_base;
       }
@@ -495,33 +557,34 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       // ---- first pass: the row's maximum over its kept scores
       float mx = -INFINITY;
       for (int t = 0; t < it.nt && ok; ++t) {
-        const uint32_t b = s_it & 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + b), (s_it >> 1) & 1, abort_flag));
+        const uint32_t b = s_it % kNS;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + b), (s_it / kNS) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
         int off0;
         const uint32_t tb = tile_bits<L>(my_bits, t, log2r, 0, off0);
-        const uint32_t src = lane_addr + kColS + 128 * b + 64 * half;
-        uint32_t v0[32], v1[32];
-        tmem_ld32(src, v0);
-        tmem_ld32(src + 32, v1);
+        const uint32_t src = lane_addr + kColS + 128 * b + 32 * kChunks * part;
+        uint32_t v[kChunks][32];
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) tmem_ld32(src + 32 * c, v[c]);
         tmem_ld_wait();
-        if (p.causal && t == it.qt) {
-          mx = chunk_max<L, true>(v0, tb, 2 * half, rt - 64 * half, mx);
-          mx = chunk_max<L, true>(v1, tb, 2 * half + 1, rt - 64 * half - 32, mx);
-        } else {
-          mx = chunk_max<L, false>(v0, tb, 2 * half, 0, mx);
-          mx = chunk_max<L, false>(v1, tb, 2 * half + 1, 0, mx);
+        const bool diag = p.causal && t == it.qt;
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          const int cg = kChunks * part + c;
+          if (diag) mx = chunk_max<L, true>(v[c], tb, cg, rt - 32 * cg, mx);
+          else mx = chunk_max<L, false>(v[c], tb, cg, 0, mx);
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kBarSDone + b));
         ++s_it;
       }
-      xch[half * kTile + rt] = mx;
+      xch[part * kTile + rt] = mx;
       ok = rows_all(ok);
       if (!ok) break;
-      mx = fmaxf(xch[rt], xch[kTile + rt]);
+#pragma unroll
+      for (int q = 0; q < kSplit; ++q) mx = fmaxf(mx, xch[q * kTile + rt]);
       if (mx == -INFINITY) mx = 0.f;  // a row that keeps no key: every probability is zero below
       const float neg_mc = -mx * cs;
       float* my_scratch = kWriteP ? p.p_scratch + (size_t)row * KR : nullptr;
@@ -529,28 +592,26 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
       int rank_base = 0;
       for (int t = 0; t < it.nt && ok; ++t) {
-        const uint32_t b = s_it & 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + b), (s_it >> 1) & 1, abort_flag));
+        const uint32_t b = s_it % kNS;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + b), (s_it / kNS) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
         int off0;
         const uint32_t tb = tile_bits<L>(my_bits, t, log2r, rank_base, off0);
-        const uint32_t src = lane_addr + kColS + 128 * b + 64 * half;
-        uint32_t v0[32], v1[32];
-        tmem_ld32(src, v0);
-        tmem_ld32(src + 32, v1);
+        const uint32_t src = lane_addr + kColS + 128 * b + 32 * kChunks * part;
+        uint32_t v[kChunks][32];
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) tmem_ld32(src + 32 * c, v[c]);
         tmem_ld_wait();
         const bool diag = p.causal && t == it.qt;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          float pr[32];
+        for (int c = 0; c < kChunks; ++c) {
           uint32_t hi[16], lo[16];
-          const int cg = 2 * half + c;
-          if (diag) chunk_probs<L, true>(c ? v1 : v0, tb, cg, rt - 32 * cg, cs, neg_mc, la, lb, pr, hi, lo);
-          else chunk_probs<L, false>(c ? v1 : v0, tb, cg, 0, cs, neg_mc, la, lb, pr, hi, lo);
+          const int cg = kChunks * part + c;
+          if (diag) chunk_probs<L, true, kWriteP>(v[c], tb, cg, rt - 32 * cg, cs, neg_mc, la, lb, hi, lo, my_scratch, rank_base, off0);
+          else chunk_probs<L, false, kWriteP>(v[c], tb, cg, 0, cs, neg_mc, la, lb, hi, lo, my_scratch, rank_base, off0);
           tmem_st16(src + 32 * c, hi);
           tmem_st16(src + 32 * c + 16, lo);
-          if (kWriteP) chunk_park<L>(pr, tb, cg, my_scratch, rank_base, off0);
         }
         rank_base = next_rank<L>(rank_base, tb, t, log2r);
         tmem_st_wait();
@@ -561,25 +622,28 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kBarBitsEmpty + slot));
-      xch_l[half * kTile + rt] = (la.x + la.y) + (lb.x + lb.y);
+      xch_l[part * kTile + rt] = (la.x + la.y) + (lb.x + lb.y);
       ok = rows_all(ok);
       if (!ok) break;
-      const float l = xch_l[rt] + xch_l[kTile + rt];
+      float l = 0.f;
+#pragma unroll
+      for (int q = 0; q < kSplit; ++q) l += xch_l[q * kTile + rt];
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      // ---- the item's output row (this thread: 32 of its 64 columns)
+      // ---- the item's output row (this thread: 64 / kSplit of its columns)
       const uint32_t ob = it_cnt & 1;
       ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull + ob), (it_cnt >> 1) & 1, abort_flag));
       if (ok) {
         tc_fence_after();
-        uint32_t o[32];
-        tmem_ld32(lane_addr + kColO + 64 * ob + 32 * half, o);
+        constexpr int kOC = 64 / kSplit;
+        uint32_t o[kOC];
+        tmem_ld_n(lane_addr + kColO + 64 * ob + kOC * part, o);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kBarOEmpty + ob));
-        uint4* out = reinterpret_cast<uint4*>(p.O + (size_t)row * kHeadDim + 32 * half);
+        uint4* out = reinterpret_cast<uint4*>(p.O + (size_t)row * kHeadDim + kOC * part);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < kOC / 8; ++e) {
           uint32_t w[4];
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
@@ -588,7 +652,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
           }
           out[e] = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        if (kWriteP && half == 0) {
+        if (kWriteP && part == 0) {
           // hand the rows' normalisers to the warps that write P
           ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarFixEmpty + slot), ((it_cnt >> 1) & 1) ^ 1, abort_flag));
           if (ok) {
@@ -605,7 +669,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     // ---------------------------------------------------------------- P writers: 32 rows per warp
     reg_dec<kRegsFix>();
     if (kWriteP) {
-      const int w4 = warp - 12;
+      const int w4 = warp - (4 + kRowWarps);
       const int KR = p.k_hat << p.log2r;
       uint32_t it_cnt = 0;
       bool ok = true;
@@ -614,43 +678,33 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         const uint32_t slot = it_cnt & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarFixFull + slot), (it_cnt >> 1) & 1, abort_flag));
         if (!ok) break;
-        // P = parked probability / row sum, rounded once; four rows in flight per step
-        for (int r0 = 0; r0 < 32; r0 += 4) {
-          float4 val[4][2];
-          int n[4], base[4];
-          float inv[4];
+        // P = parked probability / row sum, rounded once.  Rows are taken eight at a time, in
+        // slices of 128 keys (one 16-byte load per lane and row), so that eight loads are in flight.
+        const int* cnt_s = fix_cnt + slot * kTile + 32 * w4;
+        const int* base_s = fix_base + slot * kTile + 32 * w4;
+        const float* inv_s = fix_inv + slot * kTile + 32 * w4;
+        const float* src0 = p.p_scratch + (size_t)(it.row0 + 32 * w4) * KR;
+        for (int u0 = 0; u0 < KR; u0 += 128) {
+          const int u = u0 + 4 * lane;
+          for (int r0 = 0; r0 < 32; r0 += 8) {
+            int longest = 0;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int rr = slot * kTile + 32 * w4 + r0 + j;
-            n[j] = fix_cnt[rr];
-            base[j] = fix_base[rr];
-            inv[j] = fix_inv[rr];
-            const float4* src = reinterpret_cast<const float4*>(p.p_scratch + (size_t)(it.row0 + 32 * w4 + r0 + j) * KR);
+            for (int j = 0; j < 8; ++j) longest = max(longest, cnt_s[r0 + j]);
+            if (longest <= u0) continue;  // none of these rows reaches this slice
+            float4 val[8];
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-              const int u4 = lane + 32 * k;
-              val[j][k] = 4 * u4 < n[j] ? __ldcg(src + u4) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-          }
+            for (int j = 0; j < 8; ++j)
+              val[j] = u < cnt_s[r0 + j] ? __ldcg(reinterpret_cast<const float4*>(src0 + (size_t)(r0 + j) * KR + u))
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            __nv_bfloat16* dst = p.P + (size_t)base[j];
-#pragma unroll
-            for (int k = 0; k < 2; ++k) {
-              const int u = 4 * (lane + 32 * k);
-              const float f[4] = {val[j][k].x * inv[j], val[j][k].y * inv[j], val[j][k].z * inv[j], val[j][k].w * inv[j]};
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                if (u + e < n[j]) dst[u + e] = __float2bfloat16_rn(f[e]);
-            }
-            // rows longer than 256 keys: the rest, one float4 per lane and step
-            const float4* src = reinterpret_cast<const float4*>(p.p_scratch + (size_t)(it.row0 + 32 * w4 + r0 + j) * KR);
-            for (int u4 = lane + 64; 4 * u4 < n[j]; u4 += 32) {
-              const float4 x = __ldcg(src + u4);
-              const float f[4] = {x.x * inv[j], x.y * inv[j], x.z * inv[j], x.w * inv[j]};
+            for (int j = 0; j < 8; ++j) {
+              const int n = cnt_s[r0 + j];
+              const float inv = inv_s[r0 + j];
+              __nv_bfloat16* dst = p.P + (size_t)base_s[r0 + j] + u;
+              const float f[4] = {val[j].x * inv, val[j].y * inv, val[j].z * inv, val[j].w * inv};
 #pragma unroll
               for (int e = 0; e < 4; ++e)
-                if (4 * u4 + e < n[j]) dst[4 * u4 + e] = __float2bfloat16_rn(f[e]);
+                if (u + e < n) dst[e] = __float2bfloat16_rn(f[e]);
             }
           }
         }
@@ -732,7 +786,7 @@ int log2_exact(int x) {
 template <int L, bool kWriteP>
 sea_status launch_tc(const sea_shape& s, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                      const TcParams& prm, cudaStream_t st) {
-  const size_t smem = 1024 + (size_t)(2 + kNK + kNV) * kTileBytes + 8 * kNumBars + 8 + (size_t)10 * kTile * 4 +
+  const size_t smem = 1024 + (size_t)(2 + kNK + kNV) * kTileBytes + 8 * kNumBars + 8 + (size_t)(2 * kSplit + 6) * kTile * 4 +
                       2 * (size_t)prm.words * kTile * 4;
   auto kern = sparse_attn_tiles_tc_kernel<L, kWriteP>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SEA_ERR_CUDA;
