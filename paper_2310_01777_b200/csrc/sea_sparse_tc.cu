@@ -34,7 +34,7 @@ constexpr int kTile = 128;                // queries per work item, keys per til
 constexpr int kTileBytes = kTile * 128;   // 128 rows x 64 bf16
 constexpr int kNK = 4;                    // K ring stages
 constexpr int kNV = 3;                    // V ring stages
-constexpr int kSplit = 4;                 // row warpgroups: each takes 128 / kSplit columns of every tile
+constexpr int kSplit = 2;                 // row warpgroups: each takes 128 / kSplit columns of every tile
 constexpr int kRowWarps = 4 * kSplit;
 constexpr int kRowThreads = 32 * kRowWarps;
 constexpr int kThreads = 128 * (kSplit + 2);  // warpgroups: control, kSplit x row warps, P writers
@@ -100,20 +100,35 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 // Waits for the phase with the given parity; gives up (and raises the CTA's abort flag) after
-// kWaitNs, or as soon as another role has raised the flag.
+// kWaitNs, or as soon as another role has raised the flag.  kSleepNs > 0 backs off between
+// polls: for roles whose hand-offs happen once per work item, so that their polling does not
+// take issue slots from the warps that compute.
+template <int kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 32; ++i)
+    for (int i = 0; i < 32; ++i) {
       if (mbar_try(bar, parity)) return true;
+      if (kSleepNs > 0) __nanosleep(kSleepNs);
+    }
     if (*abort_flag) return false;
     if (global_ns() - t0 > kWaitNs) {
       *abort_flag = 1;
       return false;
     }
   }
+}
+// Waits for two barriers; the first polls of both are issued together so that their latencies
+// overlap (the issuing threads are single threads whose every instruction is on the critical path).
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
+                                           volatile int* abort_flag) {
+  const uint32_t ra = mbar_try(bar_a, par_a), rb = mbar_try(bar_b, par_b);
+  if (ra & rb) return true;
+  if (!ra && !mbar_wait(bar_a, par_a, abort_flag)) return false;
+  if (!rb && !mbar_wait(bar_b, par_b, abort_flag)) return false;
+  return true;
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
@@ -413,11 +428,11 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const Item it = decode_item(item, p);
         const uint32_t qb = q_it & 1;
-        ok = mbar_wait(bar(kBarBitsEmpty + qb), ((q_it >> 1) & 1) ^ 1, abort_flag);
+        ok = mbar_wait<100>(bar(kBarBitsEmpty + qb), ((q_it >> 1) & 1) ^ 1, abort_flag);
         if (!ok) break;
         mbar_expect_tx(bar(kBarBitsFull + qb), bits_bytes);
         bulk_load(smem_u32(bits) + qb * bits_bytes, p.mask_bits + (size_t)it.row0 * p.words, bits_bytes, bar(kBarBitsFull + qb));
-        ok = mbar_wait(bar(kBarQEmpty + qb), ((q_it >> 1) & 1) ^ 1, abort_flag);
+        ok = mbar_wait<100>(bar(kBarQEmpty + qb), ((q_it >> 1) & 1) ^ 1, abort_flag);
         if (!ok) break;
         mbar_expect_tx(bar(kBarQFull + qb), kTileBytes);
         tma_load_2d(sQ + qb * kTileBytes, &map_q, 0, it.row0, bar(kBarQFull + qb));
@@ -425,14 +440,14 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         for (int pass = 0; pass < 2 && ok; ++pass) {
           for (int t = 0; t < it.nt; ++t) {
             const uint32_t ks = k_it % kNK;
-            ok = mbar_wait(bar(kBarKEmpty + ks), ((k_it / kNK) & 1) ^ 1, abort_flag);
+            ok = mbar_wait<100>(bar(kBarKEmpty + ks), ((k_it / kNK) & 1) ^ 1, abort_flag);
             if (!ok) break;
             mbar_expect_tx(bar(kBarKFull + ks), kTileBytes);
             tma_load_2d(sK + ks * kTileBytes, &map_k, 0, it.bh * p.T + t * kTile, bar(kBarKFull + ks));
             ++k_it;
             if (pass == 1) {
               const uint32_t vs = v_it % kNV;
-              ok = mbar_wait(bar(kBarVEmpty + vs), ((v_it / kNV) & 1) ^ 1, abort_flag);
+              ok = mbar_wait<100>(bar(kBarVEmpty + vs), ((v_it / kNV) & 1) ^ 1, abort_flag);
               if (!ok) break;
               mbar_expect_tx(bar(kBarVFull + vs), kTileBytes);
               tma_load_2d(sV + vs * kTileBytes, &map_v, 0, it.bh * p.T + t * kTile, bar(kBarVFull + vs));
@@ -455,6 +470,8 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       // read S (first-pass use, barrier SDone) or the P V product has consumed P (second-pass use,
       // barrier PFree, committed by the other issuer).
       uint32_t q_it = 0, k_it = 0, s_it = 0;
+      uint32_t b = 0, round = 0;  // use s_it = round * kNS + b occupies buffer b
+      const uint64_t k_desc0 = smem_desc(sK, 16, 1024);  // a stage further on: + 16 KB / 16
       uint32_t prev_second = 0;  // bit b: the last use of buffer b belonged to a second pass
       uint32_t pfree_par = 0;    // bit b: parity of the PFree phase that ends that use
       uint32_t pfree_cnt = 0;    // bit b: parity of the number of second-pass uses of buffer b so far
@@ -466,16 +483,19 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         const uint64_t q_desc = smem_desc(sQ + qb * kTileBytes, 16, 1024);
         for (int pass = 0; pass < 2 && ok; ++pass) {
           for (int t = 0; t < it.nt && ok; ++t) {
-            const uint32_t u = s_it, b = u % kNS;
-            if (u >= (uint32_t)kNS) {
-              if ((prev_second >> b) & 1u) ok = mbar_wait(bar(kBarPFree + b), (pfree_par >> b) & 1u, abort_flag);
-              else ok = mbar_wait(bar(kBarSDone + b), ((u - kNS) / kNS) & 1, abort_flag);
-            }
+            const uint32_t u = s_it;
             const uint32_t ks = k_it % kNK;
-            if (ok) ok = mbar_wait(bar(kBarKFull + ks), (k_it / kNK) & 1, abort_flag);
+            const uint32_t kbar = bar(kBarKFull + ks), kpar = (k_it / kNK) & 1;
+            if (u >= (uint32_t)kNS) {
+              // the buffer's previous use is over (its round number is one less than this use's)
+              if ((prev_second >> b) & 1u) ok = mbar_wait2(bar(kBarPFree + b), (pfree_par >> b) & 1u, kbar, kpar, abort_flag);
+              else ok = mbar_wait2(bar(kBarSDone + b), (round & 1u) ^ 1u, kbar, kpar, abort_flag);
+            } else {
+              ok = mbar_wait(kbar, kpar, abort_flag);
+            }
             if (!ok) break;
             tc_fence_after();
-            issue_qk_mmas(tmem + kColS + 128 * b, q_desc, smem_desc(sK + ks * kTileBytes, 16, 1024));
+            issue_qk_mmas(tmem + kColS + 128 * b, q_desc, k_desc0 + 1024ull * ks);
             mma_commit(bar(kBarKEmpty + ks));
             mma_commit(bar(kBarSFull + b));
             if (pass == 1 && t == it.nt - 1) mma_commit(bar(kBarQEmpty + qb));
@@ -488,6 +508,10 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
             }
             ++s_it;
             ++k_it;
+            if (++b == (uint32_t)kNS) {
+              b = 0;
+              ++round;
+            }
           }
         }
         ++q_it;
@@ -498,6 +522,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     } else if (warp == 2 && lane == 0) {
       // ---------------------------------------------------------------- issuer of O += P V
       uint32_t v_it = 0, o_it = 0, use0 = 0, s_waited = 0;
+      const uint64_t v_desc0 = smem_desc(sV, 8192, 1024);  // a stage further on: + 16 KB / 16
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const Item it = decode_item(item, p);
@@ -507,16 +532,17 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
           const uint32_t u = use0 + it.nt + t, b = u % kNS;  // the second pass follows the item's first
           // the rows have written P.  A parity wait only tells the current phase from the one before
           // it, so this thread follows SDone through every use, the first-pass ones included.
-          while (ok && s_waited <= u) {
+          while (ok && s_waited < u) {
             ok = mbar_wait(bar(kBarSDone + s_waited % kNS), (s_waited / kNS) & 1, abort_flag);
             ++s_waited;
           }
           if (ok && t == 0) ok = mbar_wait(bar(kBarOEmpty + ob), ((o_it >> 1) & 1) ^ 1, abort_flag);
           const uint32_t vs = v_it % kNV;
-          if (ok) ok = mbar_wait(bar(kBarVFull + vs), (v_it / kNV) & 1, abort_flag);
+          if (ok) ok = mbar_wait2(bar(kBarSDone + b), (u / kNS) & 1, bar(kBarVFull + vs), (v_it / kNV) & 1, abort_flag);
+          ++s_waited;
           if (!ok) break;
           tc_fence_after();
-          const uint64_t vd = smem_desc(sV + vs * kTileBytes, 8192, 1024);
+          const uint64_t vd = v_desc0 + 1024ull * vs;
           issue_pv_half(d, tmem + kColS + 128 * b, vd, 0, t == 0 ? 0u : 1u);
           issue_pv_half(d, tmem + kColS + 128 * b, vd, 1, 1u);
           mma_commit(bar(kBarVEmpty + vs));
@@ -676,7 +702,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it_cnt) {
         const Item it = decode_item(item, p);
         const uint32_t slot = it_cnt & 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarFixFull + slot), (it_cnt >> 1) & 1, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait<500>(bar(kBarFixFull + slot), (it_cnt >> 1) & 1, abort_flag));
         if (!ok) break;
         // P = parked probability / row sum, rounded once.  Rows are taken eight at a time, in
         // slices of 128 keys (one 16-byte load per lane and row), so that eight loads are in flight.
