@@ -11,7 +11,11 @@ metric is quoted.  One JSON line is printed by rank 0.
              L2 flushed between steps, max over ranks.
   e2e        the same through sea_attention_host: pinned host Q, K, V, omega, W_dec in, O out.
   roofline   the sparse-attention kernel: algorithmic bytes (Q + O + every row's gathered K/V)
-             over its CUDA-event time, against the measured HBM copy bandwidth.
+             over its CUDA-event time, against the measured HBM copy bandwidth.  The kernel forms
+             the masked products as dense tiles on the tensor cores and gathers nothing, so this
+             figure exceeds 1; `tensor` inside it gives the FLOPs the kernel really executes
+             (every key tile a query tile may see, Q K^T twice and P V as head + remainder)
+             against the measured dense bf16 peak.
   stages     per-stage milliseconds from a second pass that calls the three stage entry points
              with events between them (same kernels as the fused call).
   cpu_baseline  the fp64 oracle on a bounded sample of heads, on this machine's host cores.
@@ -35,18 +39,21 @@ if ROOT not in sys.path:
 
 METRIC = "SEA attention-layer tokens/s on 1 B200 (all stages)"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparse-attention launch, from the ncu capture
-# summarised in profiles/sparse_attn_tma_opt_1p3b.md (one launch covers the whole workload).
-NCU_TRAFFIC_BYTES = {"opt_1p3b": 183.9e6}
+# summarised in profiles/sparse_attn_tiles_tc_opt_1p3b.md (one launch covers the whole workload).
+NCU_TRAFFIC_BYTES = {"opt_1p3b": 450.5e6}
 
 
 def measured_peaks():
+    """(HBM GB/s, dense bf16 TFLOP/s for a kernel timed alone, 'measured' | 'fallback')."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
+            j = json.load(f)
+        return float(j["hbm_gbs"]), float(j["bf16_tflops"]), "measured"
     except Exception:
-        return FALLBACK_HBM_GBS, "fallback"
+        return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
 
 
 class ClockSampler:
@@ -293,8 +300,15 @@ def main():
     d2h = O.numel() * O.element_size()
 
     if rank == 0:
-        peak, peak_kind = measured_peaks()
+        peak, tc_peak, peak_kind = measured_peaks()
         alg_bytes = 2 * w.rows * w.d * elem + 2 * nnz * w.d * elem  # Q + O + gathered K and V
+        # what the tile kernel executes: per (query tile, key tile) pair S = Q K^T in both passes and
+        # P V with P as bf16 head + remainder, 2 * 128 * 128 * 64 FLOPs each
+        r = w.T // w.Kc
+        tiled = w.dtype == "bf16" and w.T % 128 == 0 and r >= 4 and r & (r - 1) == 0 and w.k_hat * 96 >= w.Kc
+        nq = w.T // 128
+        pairs = w.B * w.H * (nq * (nq + 1) // 2 if w.causal else nq * nq)
+        exec_flops = pairs * 4 * (2 * 128 * 128 * w.d) if tiled else None
         sparse_s = stage_ms[2] / 1e3
         unique_bytes = 4 * w.rows * w.d * elem + nnz * elem + w.rows * w.k_hat * 4 + (w.rows + 1) * 4
         achieved = alg_bytes / sparse_s / 1e9
@@ -309,10 +323,15 @@ def main():
             "clocks": clocks,
             "stages_ms": {"estimate": stage_ms[0], "topk_mask": stage_ms[1], "sparse_attn": stage_ms[2]},
             "nnz": nnz,
-            "roofline": {"kernel": "sparse_attn_blocks_tma_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+            "roofline": {"kernel": "sparse_attn_tiles_tc_kernel" if tiled else "sparse_attn_blocks_tma_kernel",
+                         "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_source": f"{peak_kind} HBM copy bandwidth",
-                         "algorithmic_bytes": alg_bytes, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                         "algorithmic_bytes": alg_bytes, "traffic": NCU_TRAFFIC_BYTES.get(w.name) if tiled else None,
                          "ms": stage_ms[2], "sparse_stage_tokens_per_s": w.B * w.T / sparse_s,
+                         "tensor": None if not tiled else {
+                             "executed_flops": exec_flops, "achieved": exec_flops / sparse_s / 1e12, "peak": tc_peak,
+                             "unit": "TFLOP/s", "frac": exec_flops / sparse_s / 1e12 / tc_peak,
+                             "peak_source": f"{peak_kind} dense bf16 (burst)"},
                          # K and V of every head fit the L2 together, so the bytes that must cross HBM are
                          # far fewer than the algorithmic ones: Q, K, V once, O and P once, sel and row_ptr
                          "compulsory_hbm_bytes": unique_bytes,
