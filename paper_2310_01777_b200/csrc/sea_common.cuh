@@ -51,6 +51,13 @@ sea_status launch_estimate_bf16(const sea_shape& s, const void* Q, const void* K
                                 const float* omega, const float* W_dec, float* A_hat,
                                 float* est_state, void* est_split, int32_t* status, cudaStream_t st);
 size_t estimate_split_bytes(const sea_shape& s);
+// tcgen05 form of the bf16 estimator (sea_estimate_tc.cu)
+bool estimate_tc_applicable(const sea_shape& s);
+size_t estimate_tc_state_bytes(const sea_shape& s);
+size_t estimate_tc_split_bytes(const sea_shape& s);
+sea_status launch_estimate_tc(const sea_shape& s, const void* Q, const void* K, const void* V,
+                              const float* omega, const float* W_dec, float* A_hat, float* est_state,
+                              void* est_split, int32_t* status, cudaStream_t st);
 sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel,
                             int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
                             int32_t* row_counts, int32_t* tile_sums, uint32_t* mask_bits,

@@ -324,6 +324,8 @@ sea_status launch_estimate_f32(const sea_shape& s, const void* Q, const void* K,
 sea_status launch_estimate(const sea_shape& s, const void* Q, const void* K, const void* V,
                            const float* omega, const float* W_dec, float* A_hat, float* est_state,
                            void* est_split, int32_t* status, cudaStream_t st) {
+  if (estimate_tc_applicable(s))
+    return launch_estimate_tc(s, Q, K, V, omega, W_dec, A_hat, est_state, est_split, status, st);
   if (s.io == SEA_BF16)
     return launch_estimate_bf16(s, Q, K, V, omega, W_dec, A_hat, est_state, est_split, status, st);
   return launch_estimate_f32(s, Q, K, V, omega, W_dec, A_hat, est_state, status, st);

@@ -1,0 +1,740 @@
+// Attention estimation for bf16 inputs on the 5th-generation tensor cores (tcgen05, accumulators
+// in tensor memory, operands staged by TMA).
+//
+//   x = u d^(-1/4);  phi_f(u) = exp(omega_f.x - |x|^2/2) / sqrt(m)          (Sec. 3 "Performer (FAVOR+)")
+//   C_i = sum_j phi(q_i).phi(k_j) v_j / sum_j phi(q_i).phi(k_j);  A_hat = C W_dec   (Sec. 3.1, one
+//   linear head in place of the trained decoder)
+//
+// The sequence is cut into chunks of 128 rows, one CTA per (chunk, head):
+//   1. favor_state_tc_kernel:  S_c = phi(K_c)^T V_c  [m x 64]  and  z_c = phi(K_c)^T 1  [m]
+//   2. favor_scan_tc_kernel:   exclusive prefix over the chunks of a head (causal) or the total,
+//                              in a fixed order, written as bf16 head / remainder MMA operands
+//   3. favor_output_tc_kernel: num = phi(Q_c) S + (phi(Q_c) phi(K_c)^T . tril) V_c, den likewise,
+//                              C = num / den, A_hat = C W_dec
+// Precision: the estimate has to agree with fp64 to 1e-3 and the feature map exponentiates a
+// projection of magnitude ~10, so every fp32 operand is carried as a bf16 head plus a bf16
+// remainder (2^-17 relative) and a product A B is evaluated as A_hi B_hi + A_hi B_lo + A_lo B_hi;
+// Q, K and V are exact in bf16.  d^(-1/4) is folded into omega beforehand.
+//
+// Inside a CTA eight row warps own the 128 rows (a row and half of a tile's columns per thread:
+// exponentials, masks, normalisers, splits) and one thread of a ninth warp issues the copies and
+// the MMAs; the phases of a chunk follow one another through single-use mbarriers.  Every wait is
+// bounded; a wait that runs out sets SEA_DEV_TIMEOUT and the CTA drains and leaves.
+#include "sea_common.cuh"
+#include "sea_tc.cuh"
+
+namespace sea {
+namespace {
+
+using namespace tc;
+
+constexpr int kRows = 128;                 // rows per chunk
+constexpr int kTileBytes = kRows * 128;    // 128 rows x 64 bf16
+constexpr int kRowWarps = 8;
+constexpr int kThreads = 32 * (kRowWarps + 1);
+constexpr int kWTile = 128;                // decoder columns per pass
+
+// ---- operand preparation -----------------------------------------------------------------
+// omega * d^(-1/4) as bf16 head / remainder [2][MP][64] (rows >= m zero) and W_dec as
+// [2][64][KcP] (columns >= Kc zero).
+__global__ void favor_prep_tc_kernel(const float* __restrict__ omega, const float* __restrict__ W_dec,
+                                     __nv_bfloat16* __restrict__ om, __nv_bfloat16* __restrict__ wd, int m, int MP,
+                                     int Kc, int KcP, float in_scale) {
+  const int n_om = MP * kHeadDim, n_w = kHeadDim * KcP;
+  for (int v = blockIdx.x * blockDim.x + threadIdx.x; v < n_om + n_w; v += gridDim.x * blockDim.x) {
+    float x;
+    __nv_bfloat16 *hi, *lo;
+    if (v < n_om) {
+      x = (v / kHeadDim) < m ? omega[v] * in_scale : 0.f;
+      hi = om + v;
+      lo = om + n_om + v;
+    } else {
+      const int u = v - n_om, e = u / KcP, c = u - e * KcP;
+      x = c < Kc ? W_dec[(size_t)e * Kc + c] : 0.f;
+      hi = wd + u;
+      lo = wd + n_w + u;
+    }
+    const __nv_bfloat16 h = __float2bfloat16_rn(x);
+    *hi = h;
+    *lo = __float2bfloat16_rn(x - __bfloat162float(h));
+  }
+}
+
+// ---- pieces shared by the two chunk kernels ----------------------------------------------------
+// |u|^2 / 16 = |x|^2 / 2 of one row of a bf16 [.][64] matrix.
+__device__ __forceinline__ float half_sq_norm(const __nv_bfloat16* row) {
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint4 t = __ldg(reinterpret_cast<const uint4*>(row) + i);
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xffff0000u);
+      s = fmaf(lo, lo, fmaf(hi, hi, s));
+    }
+  }
+  return s * (1.f / 16.f);
+}
+
+// Features of 32 projections (columns 32c .. 32c+31 of the row's projection tile): zero for
+// padded features and for rows outside the sequence.
+__device__ __forceinline__ void features32(const uint32_t (&e)[32], float (&phi)[32], float sq, bool row_ok, int c, int m,
+                                           float inv_sqrt_m) {
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const float v = __expf(__uint_as_float(e[i]) - sq) * inv_sqrt_m;
+    phi[i] = (row_ok && 32 * c + i < m) ? v : 0.f;
+  }
+}
+__device__ __forceinline__ void split32(const float (&x)[32], uint32_t (&hi)[16], uint32_t (&lo)[16]) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) split_pair(x[2 * i], x[2 * i + 1], hi[i], lo[i]);
+}
+// Writes 32 values of row `r` (columns 32c ..) of a [128][MP] operand kept as 64-column atoms of
+// 128-byte rows with the 128-byte swizzle (atom stride 16 KB).
+__device__ __forceinline__ void store_row32_swizzled(unsigned char* base, int r, int c, const uint32_t (&w)[16]) {
+  unsigned char* row = base + (c >> 1) * kTileBytes + r * 128;
+  const int q0 = (c & 1) * 4;
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    *reinterpret_cast<uint4*>(row + (((q0 + j) ^ (r & 7)) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+}
+// Column offset (32-bit tensor-memory columns) of contraction step ks inside an operand written
+// as [16 head words | 16 remainder words] per 32 values; the remainder sits 16 columns further on.
+__device__ __forceinline__ uint32_t a_col(int ks) { return 32u * (ks >> 1) + 8u * (ks & 1); }
+
+// AND of a predicate over the row threads (named barrier 1); also orders their memory accesses.
+__device__ __forceinline__ bool rows_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.and.pred p, 1, %2, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(r) : "r"((uint32_t)ok), "n"(32 * kRowWarps) : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
+  fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+}
+
+struct EstParams {
+  const __nv_bfloat16 *Q, *K;   // for the rows' norms
+  float* state_s;               // [BH][nchunk][MP][64]
+  float* state_z;               // [BH][nchunk][MP]
+  const float* z_prefix;        // [BH][nchunk][MP]
+  float* A_hat;
+  int32_t* status;
+  int T, m, Kc, nchunk, causal;
+};
+
+// ---- kernel 1: chunk key states ---------------------------------------------------------------
+enum { kS_Load = 0, kS_E, kS_Phi, kS_S, kS_Drain, kS_NumBars };
+
+template <int MP>
+__global__ void __launch_bounds__(kThreads, 1)
+favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                      const __grid_constant__ CUtensorMap map_om, const EstParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* sm = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
+  unsigned char* sK = sm;                              // 16 KB
+  unsigned char* sV = sK + kTileBytes;                 // 16 KB
+  unsigned char* sOm = sV + kTileBytes;                // head 16 KB, remainder 16 KB ([MP][64])
+  unsigned char* sPhi = sOm + 2 * kTileBytes;          // head 32 KB, remainder 32 KB ([2 atoms][128 keys][64 f])
+  unsigned char* sOnes = sPhi + 4 * kTileBytes;        // 16 rows x 128 B of 1.0
+  unsigned char* tail = sOnes + 2048;
+  const uint32_t bars = smem_u32(tail);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * kS_NumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8 * kS_NumBars + 4);
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+  constexpr uint32_t kColE = 0, kColS = 128, kColZ = 192, kCols = 256;
+
+  const int chunk = blockIdx.x, bh = blockIdx.y;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    mbar_init(bar(kS_Load), 1);
+    mbar_init(bar(kS_E), 1);
+    mbar_init(bar(kS_Phi), kRowWarps);
+    mbar_init(bar(kS_S), 1);
+    mbar_init(bar(kS_Drain), 1);
+    *abort_flag = 0;
+    mbar_init_fence();
+  }
+  for (int i = tid; i < 2048 / 4; i += kThreads) reinterpret_cast<uint32_t*>(sOnes)[i] = 0x3f803f80u;
+  fence_async_smem();
+  if (warp == kRowWarps) tmem_alloc(smem_u32(tmem_slot), kCols);
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == kRowWarps) {
+    if (lane == 0) {
+      // ------------------------------------------------------------ copies and MMAs
+      bool ok = true;
+      mbar_expect_tx(bar(kS_Load), 2 * kTileBytes + 2 * MP * 128);
+      tma_load_3d(smem_u32(sK), &map_k, 0, chunk * kRows, bh, bar(kS_Load));
+      tma_load_3d(smem_u32(sV), &map_v, 0, chunk * kRows, bh, bar(kS_Load));
+      tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kS_Load));
+      tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kS_Load));
+      ok = mbar_wait(bar(kS_Load), 0, abort_flag);
+      if (ok) {
+        fence_after();
+        // E = K omega'^T (head, then remainder of omega'), contraction over d in four steps
+        const uint64_t dk = smem_desc(smem_u32(sK), 16, 1024);
+        const uint64_t doh = smem_desc(smem_u32(sOm), 16, 1024), dol = smem_desc(smem_u32(sOm) + kTileBytes, 16, 1024);
+        constexpr uint32_t idE = idesc_bf16(MP, false, false);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mma_ss(tmem + kColE, dk + 2 * k, doh + 2 * k, idE, k > 0);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mma_ss(tmem + kColE, dk + 2 * k, dol + 2 * k, idE, 1);
+        mma_commit(bar(kS_E));
+        ok = mbar_wait(bar(kS_Phi), 0, abort_flag);
+      }
+      if (ok) {
+        fence_after();
+        // S = phi^T V and z = phi^T 1: A = phi read MN-major (features are its M index), B = V and a
+        // tile of ones read MN-major; contraction over the 128 keys in eight steps
+        constexpr uint32_t idS = idesc_bf16(64, true, true), idZ = idesc_bf16(16, true, true);
+        const uint64_t dones = smem_desc(smem_u32(sOnes), 2048, 1024);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint64_t ah = smem_desc(smem_u32(sPhi) + 2048 * k, kTileBytes, 1024);
+          const uint64_t al = smem_desc(smem_u32(sPhi) + 2 * kTileBytes + 2048 * k, kTileBytes, 1024);
+          const uint64_t bv = smem_desc(smem_u32(sV) + 2048 * k, kTileBytes, 1024);
+          mma_ss(tmem + kColS, ah, bv, idS, k > 0);
+          mma_ss(tmem + kColS, al, bv, idS, 1);
+          mma_ss(tmem + kColZ, ah, dones, idZ, k > 0);
+          mma_ss(tmem + kColZ, al, dones, idZ, 1);
+        }
+        mma_commit(bar(kS_S));
+      }
+      mma_commit(bar(kS_Drain));
+      mbar_wait(bar(kS_Drain), 0, abort_flag);
+      mbar_wait_drain(bar(kS_Load), 0);  // the copies have landed before the CTA may leave
+    }
+  } else {
+    // -------------------------------------------------------------- row warps
+    const int quarter = warp & 3, half = warp >> 2, rt = quarter * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const int row = chunk * kRows + rt;
+    const bool row_ok = row < p.T;
+    const float sq = row_ok ? half_sq_norm(p.K + ((size_t)bh * p.T + row) * kHeadDim) : 0.f;
+    const float inv_sqrt_m = rsqrtf((float)p.m);
+    bool ok = __all_sync(0xffffffffu, mbar_wait(bar(kS_E), 0, abort_flag));
+    if (ok) {
+      fence_after();
+      for (int c = half; c < MP / 32; c += 2) {
+        uint32_t e[32];
+        tmem_ld32(lane_addr + kColE + 32 * c, e);
+        tmem_ld_wait();
+        float phi[32];
+        features32(e, phi, sq, row_ok, c, p.m, inv_sqrt_m);
+        uint32_t hi[16], lo[16];
+        split32(phi, hi, lo);
+        store_row32_swizzled(sPhi, rt, c, hi);
+        store_row32_swizzled(sPhi + 2 * kTileBytes, rt, c, lo);
+      }
+      fence_async_smem();
+      warp_arrive(bar(kS_Phi), lane);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(kS_S), 0, abort_flag));
+    }
+    if (ok) {
+      fence_after();
+      // tensor-memory lane = feature; this thread stores 32 of its feature's 64 state columns
+      uint32_t s[32], z[32];
+      tmem_ld32(lane_addr + kColS + 32 * half, s);
+      if (half == 0) tmem_ld32(lane_addr + kColZ, z);
+      tmem_ld_wait();
+      if (rt < MP) {
+        const size_t base = ((size_t)bh * p.nchunk + chunk) * MP + rt;
+        float4* dst = reinterpret_cast<float4*>(p.state_s + base * kHeadDim + 32 * half);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          dst[i] = make_float4(__uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1]), __uint_as_float(s[4 * i + 2]),
+                               __uint_as_float(s[4 * i + 3]));
+        if (half == 0) p.state_z[base] = __uint_as_float(z[0]);
+      }
+    }
+  }
+  fence_before();
+  __syncthreads();
+  if (warp == kRowWarps) {
+    __syncwarp();
+    fence_after();
+    tmem_dealloc(tmem, kCols);
+  }
+  if (tid == 0 && *abort_flag) atomicOr(p.status, SEA_DEV_TIMEOUT);
+}
+
+// ---- kernel 2: combination of the chunk states along the sequence ------------------------------
+// One thread per (head, feature, pair of columns) - and per (head, feature) for z - walks the
+// chunks in order: exclusive prefix when causal, the total (written for chunk 0 only) otherwise.
+// Output per (head, chunk): bf16 head [MP][64], bf16 remainder [MP][64], and z as fp32 [MP].
+__global__ void favor_scan_tc_kernel(const float* __restrict__ state_s, const float* __restrict__ state_z,
+                                     __nv_bfloat16* __restrict__ s_split, float* __restrict__ z_prefix, int nchunk, int MP,
+                                     long long total_threads, int causal) {
+  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= total_threads) return;
+  const int per_head = MP * 33;  // 32 column pairs and one z slot per feature
+  const long long bh = gid / per_head;
+  const int v = (int)(gid - bh * per_head);
+  const int f = v / 33, slot = v - f * 33;
+  if (slot == 32) {
+    const float* src = state_z + (size_t)bh * nchunk * MP + f;
+    float* dst = z_prefix + (size_t)bh * nchunk * MP + f;
+    float r = 0.f;
+    for (int ch = 0; ch < nchunk; ++ch) {
+      if (causal) dst[(size_t)ch * MP] = r;
+      r += src[(size_t)ch * MP];
+    }
+    if (!causal) dst[0] = r;
+    return;
+  }
+  const size_t per_chunk = (size_t)MP * kHeadDim;
+  const float* src = state_s + (size_t)bh * nchunk * per_chunk + (size_t)f * kHeadDim + 2 * slot;
+  __nv_bfloat16* dst = s_split + (size_t)bh * nchunk * 2 * per_chunk + (size_t)f * kHeadDim + 2 * slot;
+  float r0 = 0.f, r1 = 0.f;
+#pragma unroll 4
+  for (int ch = 0; ch < nchunk; ++ch) {
+    const float2 x = *reinterpret_cast<const float2*>(src + ch * per_chunk);
+    if (causal) {
+      uint32_t hi, lo;
+      split_pair(r0, r1, hi, lo);
+      *reinterpret_cast<uint32_t*>(dst + ch * 2 * per_chunk) = hi;
+      *reinterpret_cast<uint32_t*>(dst + ch * 2 * per_chunk + per_chunk) = lo;
+    }
+    r0 += x.x;
+    r1 += x.y;
+  }
+  if (!causal) {
+    uint32_t hi, lo;
+    split_pair(r0, r1, hi, lo);
+    *reinterpret_cast<uint32_t*>(dst) = hi;
+    *reinterpret_cast<uint32_t*>(dst + per_chunk) = lo;
+  }
+}
+
+// ---- kernel 3: per-chunk output and decoder -----------------------------------------------------
+enum {
+  kO_Load = 0, kO_E, kO_Phi, kO_A, kO_P, kO_Num, kO_C,
+  kO_W,                    // [2] decoder columns staged
+  kO_WDone = kO_W + 2,     // [2] the MMAs that read them are complete
+  kO_Ahat = kO_WDone + 2,  // [2] A_hat tile in tensor memory
+  kO_AFree = kO_Ahat + 2,  // [2] rows have read it
+  kO_Drain = kO_AFree + 2,
+  kO_NumBars
+};
+
+template <int MP>
+__global__ void __launch_bounds__(kThreads, 1)
+favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                       const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_om,
+                       const __grid_constant__ CUtensorMap map_s, const __grid_constant__ CUtensorMap map_w,
+                       const EstParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* sm = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
+  unsigned char* sQ = sm;                              // 16 KB
+  unsigned char* sK = sQ + kTileBytes;                 // 16 KB
+  unsigned char* sV = sK + kTileBytes;                 // 16 KB
+  unsigned char* sOm = sV + kTileBytes;                // head, remainder: 32 KB
+  unsigned char* sS = sOm + 2 * kTileBytes;            // prefix state head, remainder [MP][64]: 32 KB
+  unsigned char* sPhi = sS + 2 * kTileBytes;           // phi(K) head 32 KB, remainder 32 KB; later the decoder columns
+  unsigned char* tail = sPhi + 4 * kTileBytes;
+  const uint32_t bars = smem_u32(tail);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * kO_NumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8 * kO_NumBars + 4);
+  float* z_s = reinterpret_cast<float*>(tail + 8 * kO_NumBars + 16);  // [128]
+  float* den_x = z_s + 128;                                            // [2][128]
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+  // tensor memory: projections of Q -> phi(Q); projections of K -> in-chunk kernel matrix -> its
+  // masked head / remainder; numerator; C; the first two regions later hold the A_hat tiles
+  constexpr uint32_t kColQ = 0, kColA = 128, kColNum = 256, kColC = 320, kCols = 512;
+
+  const int chunk = blockIdx.x, bh = blockIdx.y;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool causal = p.causal != 0;
+  const bool has_prefix = !causal || chunk > 0;
+  const int n_ct = (p.Kc + kWTile - 1) / kWTile;
+  if (tid == 0) {
+    for (int i = 0; i < kO_NumBars; ++i) {
+      const bool from_rows = i == kO_Phi || i == kO_P || i == kO_C || (i >= kO_AFree && i < kO_AFree + 2);
+      mbar_init(bar(i), from_rows ? kRowWarps : 1);
+    }
+    *abort_flag = 0;
+    mbar_init_fence();
+  }
+  if (warp == kRowWarps) tmem_alloc(smem_u32(tmem_slot), kCols);
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == kRowWarps) {
+    if (lane == 0) {
+      // ------------------------------------------------------------ copies and MMAs
+      bool ok = true;
+      const int state_idx = (bh * p.nchunk + (causal ? chunk : 0)) * 2;
+      uint32_t bytes = kTileBytes + 2 * MP * 128;
+      if (causal) bytes += 2 * kTileBytes;
+      if (has_prefix) bytes += 2 * MP * 128 + MP * 4;
+      mbar_expect_tx(bar(kO_Load), bytes);
+      tma_load_3d(smem_u32(sQ), &map_q, 0, chunk * kRows, bh, bar(kO_Load));
+      if (causal) {
+        tma_load_3d(smem_u32(sK), &map_k, 0, chunk * kRows, bh, bar(kO_Load));
+        tma_load_3d(smem_u32(sV), &map_v, 0, chunk * kRows, bh, bar(kO_Load));
+      }
+      tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kO_Load));
+      tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kO_Load));
+      if (has_prefix) {
+        tma_load_3d(smem_u32(sS), &map_s, 0, 0, state_idx, bar(kO_Load));
+        tma_load_3d(smem_u32(sS) + kTileBytes, &map_s, 0, 0, state_idx + 1, bar(kO_Load));
+        bulk_load(smem_u32(z_s), p.z_prefix + (size_t)(state_idx / 2) * MP, MP * 4, bar(kO_Load));
+      }
+      uint32_t w_loads[2] = {0, 0};  // copies armed per buffer
+      auto load_w = [&](int ct) {  // decoder columns 128 ct ..: head atoms, remainder atoms (64 columns each)
+        const int b = ct & 1;
+        const uint32_t dst = smem_u32(sPhi) + b * 2 * kTileBytes;
+        mbar_expect_tx(bar(kO_W + b), 4 * 8192);
+        for (int part = 0; part < 2; ++part)
+          for (int atom = 0; atom < 2; ++atom)
+            tma_load_3d(dst + part * kTileBytes + atom * 8192, &map_w, ct * kWTile + 64 * atom, 0, part, bar(kO_W + b));
+        ++w_loads[b];
+      };
+      ok = mbar_wait(bar(kO_Load), 0, abort_flag);
+      if (ok) {
+        fence_after();
+        const uint64_t doh = smem_desc(smem_u32(sOm), 16, 1024), dol = smem_desc(smem_u32(sOm) + kTileBytes, 16, 1024);
+        constexpr uint32_t idE = idesc_bf16(MP, false, false);
+        const uint64_t dq = smem_desc(smem_u32(sQ), 16, 1024);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, doh + 2 * k, idE, k > 0);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, dol + 2 * k, idE, 1);
+        if (causal) {
+          const uint64_t dk = smem_desc(smem_u32(sK), 16, 1024);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColA, dk + 2 * k, doh + 2 * k, idE, k > 0);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColA, dk + 2 * k, dol + 2 * k, idE, 1);
+        }
+        mma_commit(bar(kO_E));
+        ok = mbar_wait(bar(kO_Phi), 0, abort_flag);
+      }
+      if (ok) {
+        fence_after();
+        if (causal) {
+          // in-chunk kernel matrix phi(Q) phi(K)^T: A = phi(Q) in tensor memory, B = phi(K) K-major
+          constexpr uint32_t idA = idesc_bf16(128, false, false);
+#pragma unroll
+          for (int k = 0; k < MP / 16; ++k) {
+            const uint32_t off = (k >> 2) * kTileBytes + (k & 3) * 32;
+            const uint64_t bh_ = smem_desc(smem_u32(sPhi) + off, 16, 1024);
+            const uint64_t bl_ = smem_desc(smem_u32(sPhi) + 2 * kTileBytes + off, 16, 1024);
+            const uint32_t a = tmem + kColQ + a_col(k);
+            mma_ts(tmem + kColA, a, bh_, idA, k > 0);
+            mma_ts(tmem + kColA, a, bl_, idA, 1);
+            mma_ts(tmem + kColA, a + 16, bh_, idA, 1);
+          }
+          mma_commit(bar(kO_A));
+        }
+        if (has_prefix) {
+          // phi(Q) S: B = the state read MN-major (16 features = 2048 bytes per step)
+          constexpr uint32_t idN = idesc_bf16(64, false, true);
+#pragma unroll
+          for (int k = 0; k < MP / 16; ++k) {
+            const uint64_t bh_ = smem_desc(smem_u32(sS) + 2048 * k, kTileBytes, 1024);
+            const uint64_t bl_ = smem_desc(smem_u32(sS) + kTileBytes + 2048 * k, kTileBytes, 1024);
+            const uint32_t a = tmem + kColQ + a_col(k);
+            mma_ts(tmem + kColNum, a, bh_, idN, k > 0);
+            mma_ts(tmem + kColNum, a, bl_, idN, 1);
+            mma_ts(tmem + kColNum, a + 16, bh_, idN, 1);
+          }
+        }
+        if (causal) ok = mbar_wait(bar(kO_P), 0, abort_flag);
+      }
+      if (ok) {
+        fence_after();
+        if (causal) {
+          // phi(K) is no longer read (the rows waited for the kernel matrix): its place takes the decoder columns
+          load_w(0);
+          if (n_ct > 1) load_w(1);
+          constexpr uint32_t idN = idesc_bf16(64, false, true);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint64_t bv = smem_desc(smem_u32(sV) + 2048 * k, kTileBytes, 1024);
+            const uint32_t a = tmem + kColA + a_col(k);
+            mma_ts(tmem + kColNum, a, bv, idN, (has_prefix || k > 0) ? 1u : 0u);
+            mma_ts(tmem + kColNum, a + 16, bv, idN, 1);
+          }
+        } else {
+          load_w(0);
+          if (n_ct > 1) load_w(1);
+        }
+        mma_commit(bar(kO_Num));
+        ok = mbar_wait(bar(kO_C), 0, abort_flag);
+      }
+      if (ok) {
+        fence_after();
+        // A_hat tile = C W: A = C in tensor memory (64 values: four steps), B = decoder columns MN-major
+        constexpr uint32_t idW = idesc_bf16(kWTile, false, true);
+        for (int ct = 0; ct < n_ct && ok; ++ct) {
+          const int b = ct & 1;
+          ok = mbar_wait(bar(kO_W + b), (ct >> 1) & 1, abort_flag);
+          if (ok && ct >= 2) ok = mbar_wait(bar(kO_AFree + b), ((ct >> 1) - 1) & 1, abort_flag);
+          if (!ok) break;
+          fence_after();
+          const uint32_t wbase = smem_u32(sPhi) + b * 2 * kTileBytes;
+          const uint32_t d = tmem + (b ? kColA : kColQ);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const uint64_t wh = smem_desc(wbase + 2048 * k, 8192, 1024);
+            const uint64_t wl = smem_desc(wbase + kTileBytes + 2048 * k, 8192, 1024);
+            const uint32_t a = tmem + kColC + a_col(k);
+            mma_ts(d, a, wh, idW, k > 0);
+            mma_ts(d, a, wl, idW, 1);
+            mma_ts(d, a + 16, wh, idW, 1);
+          }
+          mma_commit(bar(kO_Ahat + b));
+          mma_commit(bar(kO_WDone + b));
+          if (ct >= 1 && ct + 1 < n_ct) {
+            // columns of pass ct + 1 go where pass ct - 1 read from
+            ok = mbar_wait(bar(kO_WDone + (b ^ 1)), ((ct - 1) >> 1) & 1, abort_flag);
+            if (ok) load_w(ct + 1);
+          }
+        }
+      }
+      mma_commit(bar(kO_Drain));
+      mbar_wait(bar(kO_Drain), 0, abort_flag);
+      // copies still in flight must land before the CTA may leave
+      mbar_wait_drain(bar(kO_Load), 0);
+      for (int b = 0; b < 2; ++b)
+        if (w_loads[b]) mbar_wait_drain(bar(kO_W + b), (w_loads[b] - 1) & 1);
+    }
+  } else {
+    // -------------------------------------------------------------- row warps
+    const int quarter = warp & 3, half = warp >> 2, rt = quarter * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const int row = chunk * kRows + rt;
+    const bool row_ok = row < p.T;
+    const size_t grow = (size_t)bh * p.T + row;
+    const float sq_q = row_ok ? half_sq_norm(p.Q + grow * kHeadDim) : 0.f;
+    const float sq_k = (row_ok && causal) ? half_sq_norm(p.K + grow * kHeadDim) : 0.f;
+    const float inv_sqrt_m = rsqrtf((float)p.m);
+    float den = 0.f;
+    bool ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_E), 0, abort_flag));
+    if (ok && has_prefix) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Load), 0, abort_flag));  // z has landed
+    if (ok) {
+      fence_after();
+      for (int c = half; c < MP / 32; c += 2) {
+        uint32_t e[32];
+        float phi[32];
+        uint32_t hi[16], lo[16];
+        tmem_ld32(lane_addr + kColQ + 32 * c, e);
+        tmem_ld_wait();
+        features32(e, phi, sq_q, row_ok, c, p.m, inv_sqrt_m);
+        if (has_prefix) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) den = fmaf(phi[i], z_s[32 * c + i], den);
+        }
+        split32(phi, hi, lo);
+        tmem_st16(lane_addr + kColQ + 32 * c, hi);
+        tmem_st16(lane_addr + kColQ + 32 * c + 16, lo);
+        if (causal) {
+          tmem_ld32(lane_addr + kColA + 32 * c, e);
+          tmem_ld_wait();
+          features32(e, phi, sq_k, row_ok, c, p.m, inv_sqrt_m);
+          split32(phi, hi, lo);
+          store_row32_swizzled(sPhi, rt, c, hi);
+          store_row32_swizzled(sPhi + 2 * kTileBytes, rt, c, lo);
+        }
+      }
+      tmem_st_wait();
+      fence_async_smem();
+      warp_arrive(bar(kO_Phi), lane);
+      if (causal) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_A), 0, abort_flag));
+    }
+    if (ok && causal) {
+      fence_after();
+      // keep keys j <= i of the chunk; rows of the normaliser; head / remainder in place
+      for (int c = half; c < 4; c += 2) {
+        uint32_t e[32];
+        float a[32];
+        uint32_t hi[16], lo[16];
+        tmem_ld32(lane_addr + kColA + 32 * c, e);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          a[i] = (32 * c + i <= rt) ? __uint_as_float(e[i]) : 0.f;
+          den += a[i];
+        }
+        split32(a, hi, lo);
+        tmem_st16(lane_addr + kColA + 32 * c, hi);
+        tmem_st16(lane_addr + kColA + 32 * c + 16, lo);
+      }
+      tmem_st_wait();
+      warp_arrive(bar(kO_P), lane);
+    }
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Num), 0, abort_flag));
+    den_x[half * kRows + rt] = den;
+    ok = rows_all(ok);
+    if (ok) {
+      fence_after();
+      den = den_x[rt] + den_x[kRows + rt];
+      if (row_ok && !(den > 0.f && den < INFINITY)) atomicOr(p.status, SEA_DEV_NONFINITE);
+      const float inv = 1.f / den;
+      uint32_t e[32];
+      float cv[32];
+      uint32_t hi[16], lo[16];
+      tmem_ld32(lane_addr + kColNum + 32 * half, e);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) cv[i] = row_ok ? __uint_as_float(e[i]) * inv : 0.f;
+      split32(cv, hi, lo);
+      tmem_st16(lane_addr + kColC + 32 * half, hi);
+      tmem_st16(lane_addr + kColC + 32 * half + 16, lo);
+      tmem_st_wait();
+      warp_arrive(bar(kO_C), lane);
+      float* out = p.A_hat + grow * p.Kc;
+      const bool vec = (p.Kc & 3) == 0;
+      for (int ct = 0; ct < n_ct && ok; ++ct) {
+        const int b = ct & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Ahat + b), (ct >> 1) & 1, abort_flag));
+        if (!ok) break;
+        fence_after();
+        for (int c = half; c < 4; c += 2) {
+          tmem_ld32(lane_addr + (b ? kColA : kColQ) + 32 * c, e);
+          tmem_ld_wait();
+          const int col0 = ct * kWTile + 32 * c;
+          if (row_ok) {
+            if (vec) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                if (col0 + 4 * i < p.Kc)
+                  *reinterpret_cast<float4*>(out + col0 + 4 * i) =
+                      make_float4(__uint_as_float(e[4 * i]), __uint_as_float(e[4 * i + 1]), __uint_as_float(e[4 * i + 2]),
+                                  __uint_as_float(e[4 * i + 3]));
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (col0 + i < p.Kc) out[col0 + i] = __uint_as_float(e[i]);
+            }
+          }
+        }
+        warp_arrive(bar(kO_AFree + b), lane);
+      }
+    }
+  }
+  fence_before();
+  __syncthreads();
+  if (warp == kRowWarps) {
+    __syncwarp();
+    fence_after();
+    tmem_dealloc(tmem, kCols);
+  }
+  if (tid == 0 && *abort_flag) atomicOr(p.status, SEA_DEV_TIMEOUT);
+}
+
+int padded_features(int m) { return m <= 32 ? 32 : (m <= 64 ? 64 : 128); }
+size_t padded_kc(const sea_shape& s) { return ((size_t)s.Kc + 63) / 64 * 64; }  // whole 64-column copy boxes
+
+template <int MP>
+sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bfloat16* K, const __nv_bfloat16* V,
+                     const float* omega, const float* W_dec, float* A_hat, float* state, unsigned char* scratch,
+                     int32_t* status, cudaStream_t st) {
+  const int BH = s.B * s.H;
+  const int nchunk = (s.T + kRows - 1) / kRows;
+  const size_t KcP = padded_kc(s);
+  // carve-up of the scratch area (estimate_tc_split_bytes)
+  __nv_bfloat16* om = reinterpret_cast<__nv_bfloat16*>(scratch);                       // [2][MP][64]
+  __nv_bfloat16* wd = om + 2 * 128 * kHeadDim;                                         // [2][64][KcP]
+  __nv_bfloat16* s_split = wd + 2 * kHeadDim * KcP;                                    // [BH][nchunk][2][MP][64]
+  float* z_prefix = reinterpret_cast<float*>(s_split + (size_t)BH * nchunk * 2 * MP * kHeadDim);  // [BH][nchunk][MP]
+  float* state_s = state;                                                              // [BH][nchunk][MP][64]
+  float* state_z = state + (size_t)BH * nchunk * MP * kHeadDim;                        // [BH][nchunk][MP]
+
+  CUtensorMap mq, mk, mv, mom, ms, mw;
+  if (!make_map_bf16_3d(&mq, Q, kHeadDim, s.T, BH, kHeadDim, kRows) ||
+      !make_map_bf16_3d(&mk, K, kHeadDim, s.T, BH, kHeadDim, kRows) ||
+      !make_map_bf16_3d(&mv, V, kHeadDim, s.T, BH, kHeadDim, kRows) ||
+      !make_map_bf16_3d(&mom, om, kHeadDim, MP, 2, kHeadDim, MP) ||
+      !make_map_bf16_3d(&ms, s_split, kHeadDim, MP, (unsigned long long)BH * nchunk * 2, kHeadDim, MP) ||
+      !make_map_bf16_3d(&mw, wd, KcP, kHeadDim, 2, 64, kHeadDim))
+    return SEA_ERR_CUDA;
+
+  const int n_prep = MP * kHeadDim + kHeadDim * (int)KcP;
+  favor_prep_tc_kernel<<<(n_prep + 255) / 256, 256, 0, st>>>(omega, W_dec, om, wd, s.m, MP, s.Kc, (int)KcP,
+                                                             0.35355339059327373f);
+  sea_status rc = check_launch();
+  if (rc != SEA_OK) return rc;
+
+  EstParams prm{};
+  prm.Q = Q;
+  prm.K = K;
+  prm.state_s = state_s;
+  prm.state_z = state_z;
+  prm.z_prefix = z_prefix;
+  prm.A_hat = A_hat;
+  prm.status = status;
+  prm.T = s.T;
+  prm.m = s.m;
+  prm.Kc = s.Kc;
+  prm.nchunk = nchunk;
+  prm.causal = s.causal;
+
+  const size_t smem1 = 1024 + 8 * kTileBytes + 2048 + 8 * kS_NumBars + 16;
+  const size_t smem3 = 1024 + 11 * kTileBytes + 8 * kO_NumBars + 16 + 3 * 128 * 4;
+  if (cudaFuncSetAttribute(favor_state_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
+      cudaFuncSetAttribute(favor_output_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem3) != cudaSuccess)
+    return SEA_ERR_CUDA;
+  const dim3 grid(nchunk, BH);
+  // a causal sequence of one chunk has no prefix to form
+  if (!(s.causal && nchunk == 1)) {
+    favor_state_tc_kernel<MP><<<grid, kThreads, smem1, st>>>(mk, mv, mom, prm);
+    if ((rc = check_launch()) != SEA_OK) return rc;
+    const long long total = (long long)BH * MP * 33;
+    favor_scan_tc_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(state_s, state_z, s_split, z_prefix, nchunk, MP,
+                                                                          total, s.causal);
+    if ((rc = check_launch()) != SEA_OK) return rc;
+  }
+  favor_output_tc_kernel<MP><<<grid, kThreads, smem3, st>>>(mq, mk, mv, mom, ms, mw, prm);
+  return check_launch();
+}
+
+}  // namespace
+
+// fp32 chunk states [BH][nchunk][MP][65] of the tensor-core estimator.
+size_t estimate_tc_state_bytes(const sea_shape& s) {
+  if (s.m <= 0) return 0;
+  const size_t nchunk = ((size_t)s.T + kRows - 1) / kRows;
+  return (size_t)s.B * s.H * nchunk * padded_features(s.m) * (kHeadDim + 1) * sizeof(float);
+}
+// bf16 operands: omega' and W_dec (head / remainder) and the scanned states with their normalisers.
+size_t estimate_tc_split_bytes(const sea_shape& s) {
+  if (s.m <= 0) return 0;
+  const size_t nchunk = ((size_t)s.T + kRows - 1) / kRows;
+  const size_t MP = padded_features(s.m);
+  const size_t elems = 2 * (size_t)128 * kHeadDim + 2 * (size_t)kHeadDim * padded_kc(s) +
+                       (size_t)s.B * s.H * nchunk * (2 * MP * kHeadDim + 2 * MP);
+  return elems * sizeof(__nv_bfloat16) + 256;
+}
+bool estimate_tc_applicable(const sea_shape& s) {
+  return s.io == SEA_BF16 && s.m >= 16 && s.m <= 128 && encode_fn() != nullptr;
+}
+
+sea_status launch_estimate_tc(const sea_shape& s, const void* Q, const void* K, const void* V, const float* omega,
+                              const float* W_dec, float* A_hat, float* est_state, void* split_buf, int32_t* status,
+                              cudaStream_t st) {
+  using T = __nv_bfloat16;
+  unsigned char* scratch = static_cast<unsigned char*>(split_buf);
+  switch (padded_features(s.m)) {
+    case 32:
+      return launch_mp<32>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, scratch, status, st);
+    case 64:
+      return launch_mp<64>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, scratch, status, st);
+    default:
+      return launch_mp<128>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, scratch, status, st);
+  }
+}
+
+}  // namespace sea
