@@ -16,9 +16,9 @@
 // remainder (2^-17 relative) and a product A B is evaluated as A_hi B_hi + A_hi B_lo + A_lo B_hi;
 // Q, K and V are exact in bf16.  d^(-1/4) is folded into omega beforehand.
 //
-// Inside a CTA eight row warps own the 128 rows (a row and half of a tile's columns per thread:
-// exponentials, masks, normalisers, splits) and one thread of a ninth warp issues the copies and
-// the MMAs; the phases of a chunk follow one another through single-use mbarriers.  Every wait is
+// Inside a CTA sixteen row warps own the 128 rows (a row and a quarter of a tile's columns per
+// thread: exponentials, masks, normalisers, splits) and one thread of a further warp issues the
+// copies and the MMAs; the phases of a chunk follow one another through single-use mbarriers.  Every wait is
 // bounded; a wait that runs out sets SEA_DEV_TIMEOUT and the CTA drains and leaves.
 #include "sea_common.cuh"
 #include "sea_tc.cuh"
@@ -30,7 +30,8 @@ using namespace tc;
 
 constexpr int kRows = 128;                 // rows per chunk
 constexpr int kTileBytes = kRows * 128;    // 128 rows x 64 bf16
-constexpr int kRowWarps = 8;
+constexpr int kParts = 2;                  // row warpgroups: each takes every kParts-th 32-column chunk of a tile
+constexpr int kRowWarps = 4 * kParts;
 constexpr int kThreads = 32 * (kRowWarps + 1);
 constexpr int kWTile = 128;                // decoder columns per pass
 
@@ -215,7 +216,7 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     }
   } else {
     // -------------------------------------------------------------- row warps
-    const int quarter = warp & 3, half = warp >> 2, rt = quarter * 32 + lane;
+    const int quarter = warp & 3, part = warp >> 2, rt = quarter * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     const int row = chunk * kRows + rt;
     const bool row_ok = row < p.T;
@@ -224,7 +225,7 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     bool ok = __all_sync(0xffffffffu, mbar_wait(bar(kS_E), 0, abort_flag));
     if (ok) {
       fence_after();
-      for (int c = half; c < MP / 32; c += 2) {
+      for (int c = part; c < MP / 32; c += kParts) {
         uint32_t e[32];
         tmem_ld32(lane_addr + kColE + 32 * c, e);
         tmem_ld_wait();
@@ -241,19 +242,24 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     }
     if (ok) {
       fence_after();
-      // tensor-memory lane = feature; this thread stores 32 of its feature's 64 state columns
-      uint32_t s[32], z[32];
-      tmem_ld32(lane_addr + kColS + 32 * half, s);
-      if (half == 0) tmem_ld32(lane_addr + kColZ, z);
-      tmem_ld_wait();
-      if (rt < MP) {
-        const size_t base = ((size_t)bh * p.nchunk + chunk) * MP + rt;
-        float4* dst = reinterpret_cast<float4*>(p.state_s + base * kHeadDim + 32 * half);
+      // tensor-memory lane = feature; parts 0 and 1 store 32 of the feature's 64 state columns
+      // each, part 2 the normaliser
+      if (part < 3) {
+        uint32_t s[32];
+        tmem_ld32(lane_addr + (part < 2 ? kColS + 32 * part : kColZ), s);
+        tmem_ld_wait();
+        if (rt < MP) {
+          const size_t base = ((size_t)bh * p.nchunk + chunk) * MP + rt;
+          if (part < 2) {
+            float4* dst = reinterpret_cast<float4*>(p.state_s + base * kHeadDim + 32 * part);
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-          dst[i] = make_float4(__uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1]), __uint_as_float(s[4 * i + 2]),
-                               __uint_as_float(s[4 * i + 3]));
-        if (half == 0) p.state_z[base] = __uint_as_float(z[0]);
+            for (int i = 0; i < 8; ++i)
+              dst[i] = make_float4(__uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1]), __uint_as_float(s[4 * i + 2]),
+                                   __uint_as_float(s[4 * i + 3]));
+          } else {
+            p.state_z[base] = __uint_as_float(s[0]);
+          }
+        }
       }
     }
   }
@@ -345,7 +351,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * kO_NumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8 * kO_NumBars + 4);
   float* z_s = reinterpret_cast<float*>(tail + 8 * kO_NumBars + 16);  // [128]
-  float* den_x = z_s + 128;                                            // [2][128]
+  float* den_x = z_s + 128;                                            // [kParts][128]
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   // tensor memory: projections of Q -> phi(Q); projections of K -> in-chunk kernel matrix -> its
   // masked head / remainder; numerator; C; the first two regions later hold the A_hat tiles
@@ -513,7 +519,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     }
   } else {
     // -------------------------------------------------------------- row warps
-    const int quarter = warp & 3, half = warp >> 2, rt = quarter * 32 + lane;
+    const int quarter = warp & 3, part = warp >> 2, rt = quarter * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     const int row = chunk * kRows + rt;
     const bool row_ok = row < p.T;
@@ -526,7 +532,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     if (ok && has_prefix) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Load), 0, abort_flag));  // z has landed
     if (ok) {
       fence_after();
-      for (int c = half; c < MP / 32; c += 2) {
+      for (int c = part; c < MP / 32; c += kParts) {
         uint32_t e[32];
         float phi[32];
         uint32_t hi[16], lo[16];
@@ -557,7 +563,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     if (ok && causal) {
       fence_after();
       // keep keys j <= i of the chunk; rows of the normaliser; head / remainder in place
-      for (int c = half; c < 4; c += 2) {
+      for (int c = part; c < 4; c += kParts) {
         uint32_t e[32];
         float a[32];
         uint32_t hi[16], lo[16];
@@ -576,24 +582,28 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       warp_arrive(bar(kO_P), lane);
     }
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Num), 0, abort_flag));
-    den_x[half * kRows + rt] = den;
+    den_x[part * kRows + rt] = den;
     ok = rows_all(ok);
     if (ok) {
       fence_after();
-      den = den_x[rt] + den_x[kRows + rt];
+      den = 0.f;
+#pragma unroll
+      for (int q = 0; q < kParts; ++q) den += den_x[q * kRows + rt];
       if (row_ok && !(den > 0.f && den < INFINITY)) atomicOr(p.status, SEA_DEV_NONFINITE);
       const float inv = 1.f / den;
       uint32_t e[32];
-      float cv[32];
-      uint32_t hi[16], lo[16];
-      tmem_ld32(lane_addr + kColNum + 32 * half, e);
-      tmem_ld_wait();
+      if (part < 2) {  // C has 64 columns: two chunks
+        float cv[32];
+        uint32_t hi[16], lo[16];
+        tmem_ld32(lane_addr + kColNum + 32 * part, e);
+        tmem_ld_wait();
 #pragma unroll
-      for (int i = 0; i < 32; ++i) cv[i] = row_ok ? __uint_as_float(e[i]) * inv : 0.f;
-      split32(cv, hi, lo);
-      tmem_st16(lane_addr + kColC + 32 * half, hi);
-      tmem_st16(lane_addr + kColC + 32 * half + 16, lo);
-      tmem_st_wait();
+        for (int i = 0; i < 32; ++i) cv[i] = row_ok ? __uint_as_float(e[i]) * inv : 0.f;
+        split32(cv, hi, lo);
+        tmem_st16(lane_addr + kColC + 32 * part, hi);
+        tmem_st16(lane_addr + kColC + 32 * part + 16, lo);
+        tmem_st_wait();
+      }
       warp_arrive(bar(kO_C), lane);
       float* out = p.A_hat + grow * p.Kc;
       const bool vec = (p.Kc & 3) == 0;
@@ -602,7 +612,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Ahat + b), (ct >> 1) & 1, abort_flag));
         if (!ok) break;
         fence_after();
-        for (int c = half; c < 4; c += 2) {
+        for (int c = part; c < 4; c += kParts) {
           tmem_ld32(lane_addr + (b ? kColA : kColQ) + 32 * c, e);
           tmem_ld_wait();
           const int col0 = ct * kWTile + 32 * c;
@@ -683,7 +693,7 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   prm.causal = s.causal;
 
   const size_t smem1 = 1024 + 8 * kTileBytes + 2048 + 8 * kS_NumBars + 16;
-  const size_t smem3 = 1024 + 11 * kTileBytes + 8 * kO_NumBars + 16 + 3 * 128 * 4;
+  const size_t smem3 = 1024 + 11 * kTileBytes + 8 * kO_NumBars + 16 + (1 + kParts) * 128 * 4;
   if (cudaFuncSetAttribute(favor_state_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
       cudaFuncSetAttribute(favor_output_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem3) != cudaSuccess)
     return SEA_ERR_CUDA;
