@@ -126,7 +126,8 @@ struct EstParams {
   const float* z_prefix;        // [BH][nchunk][MP]
   float* A_hat;
   int32_t* status;
-  int T, m, Kc, nchunk, causal;
+  int BH, T, m, Kc, nchunk, causal;
+  int tma_store;                // A_hat leaves through TMA stores (its rows are 16-byte multiples)
 };
 
 // ---- kernel 1: chunk key states ---------------------------------------------------------------
@@ -243,23 +244,22 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     if (ok) {
       fence_after();
       // tensor-memory lane = feature; parts 0 and 1 store 32 of the feature's 64 state columns
-      // each, part 2 the normaliser
-      if (part < 3) {
-        uint32_t s[32];
-        tmem_ld32(lane_addr + (part < 2 ? kColS + 32 * part : kColZ), s);
-        tmem_ld_wait();
-        if (rt < MP) {
-          const size_t base = ((size_t)bh * p.nchunk + chunk) * MP + rt;
-          if (part < 2) {
-            float4* dst = reinterpret_cast<float4*>(p.state_s + base * kHeadDim + 32 * part);
+      // each, the last part also the normaliser
+      constexpr int kZPart = kParts > 2 ? 2 : 0;
+      uint32_t s[32], z[32];
+      if (part < 2) tmem_ld32(lane_addr + kColS + 32 * part, s);
+      if (part == kZPart) tmem_ld32(lane_addr + kColZ, z);
+      tmem_ld_wait();
+      if (rt < MP) {
+        const size_t base = ((size_t)bh * p.nchunk + chunk) * MP + rt;
+        if (part < 2) {
+          float4* dst = reinterpret_cast<float4*>(p.state_s + base * kHeadDim + 32 * part);
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              dst[i] = make_float4(__uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1]), __uint_as_float(s[4 * i + 2]),
-                                   __uint_as_float(s[4 * i + 3]));
-          } else {
-            p.state_z[base] = __uint_as_float(s[0]);
-          }
+          for (int i = 0; i < 8; ++i)
+            dst[i] = make_float4(__uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1]), __uint_as_float(s[4 * i + 2]),
+                                 __uint_as_float(s[4 * i + 3]));
         }
+        if (part == kZPart) p.state_z[base] = __uint_as_float(z[0]);
       }
     }
   }
@@ -322,8 +322,14 @@ __global__ void favor_scan_tc_kernel(const float* __restrict__ state_s, const fl
 }
 
 // ---- kernel 3: per-chunk output and decoder -----------------------------------------------------
+// Persistent: a CTA walks the (head, chunk) items blockIdx.x, blockIdx.x + gridDim.x, ...; omega'
+// is staged once, the next item's tiles are copied in as soon as the current item has stopped
+// reading their places, and every barrier below completes once per item (or once per decoder pass).
 enum {
-  kO_Load = 0, kO_E, kO_Phi, kO_A, kO_P, kO_Num, kO_C,
+  kO_Om = 0,               // omega' staged (once)
+  kO_QK,                   // the item's Q (and K) tile
+  kO_VS,                   // the item's V tile, prefix state and its normaliser
+  kO_E, kO_Phi, kO_A, kO_P, kO_Num, kO_C,
   kO_W,                    // [2] decoder columns staged
   kO_WDone = kO_W + 2,     // [2] the MMAs that read them are complete
   kO_Ahat = kO_WDone + 2,  // [2] A_hat tile in tensor memory
@@ -332,12 +338,22 @@ enum {
   kO_NumBars
 };
 
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];\n"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory"); }
+// Named barrier `id` over the 128 threads of one column group of the row warps.
+__device__ __forceinline__ void part_sync(int id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
+
 template <int MP>
 __global__ void __launch_bounds__(kThreads, 1)
 favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_om,
                        const __grid_constant__ CUtensorMap map_s, const __grid_constant__ CUtensorMap map_w,
-                       const EstParams p) {
+                       const __grid_constant__ CUtensorMap map_a, const EstParams p) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* sm = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   unsigned char* sQ = sm;                              // 16 KB
@@ -346,7 +362,8 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   unsigned char* sOm = sV + kTileBytes;                // head, remainder: 32 KB
   unsigned char* sS = sOm + 2 * kTileBytes;            // prefix state head, remainder [MP][64]: 32 KB
   unsigned char* sPhi = sS + 2 * kTileBytes;           // phi(K) head 32 KB, remainder 32 KB; later the decoder columns
-  unsigned char* tail = sPhi + 4 * kTileBytes;
+  unsigned char* sOut = sPhi + 4 * kTileBytes;         // kParts boxes of 128 rows x 32 fp32 on their way to A_hat
+  unsigned char* tail = sOut + kParts * kTileBytes;
   const uint32_t bars = smem_u32(tail);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * kO_NumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8 * kO_NumBars + 4);
@@ -357,11 +374,10 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   // masked head / remainder; numerator; C; the first two regions later hold the A_hat tiles
   constexpr uint32_t kColQ = 0, kColA = 128, kColNum = 256, kColC = 320, kCols = 512;
 
-  const int chunk = blockIdx.x, bh = blockIdx.y;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool causal = p.causal != 0;
-  const bool has_prefix = !causal || chunk > 0;
   const int n_ct = (p.Kc + kWTile - 1) / kWTile;
+  const int n_items = p.BH * p.nchunk;
   if (tid == 0) {
     for (int i = 0; i < kO_NumBars; ++i) {
       const bool from_rows = i == kO_Phi || i == kO_P || i == kO_C || (i >= kO_AFree && i < kO_AFree + 2);
@@ -380,55 +396,85 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     if (lane == 0) {
       // ------------------------------------------------------------ copies and MMAs
       bool ok = true;
-      const int state_idx = (bh * p.nchunk + (causal ? chunk : 0)) * 2;
-      uint32_t bytes = kTileBytes + 2 * MP * 128;
-      if (causal) bytes += 2 * kTileBytes;
-      if (has_prefix) bytes += 2 * MP * 128 + MP * 4;
-      mbar_expect_tx(bar(kO_Load), bytes);
-      tma_load_3d(smem_u32(sQ), &map_q, 0, chunk * kRows, bh, bar(kO_Load));
-      if (causal) {
-        tma_load_3d(smem_u32(sK), &map_k, 0, chunk * kRows, bh, bar(kO_Load));
-        tma_load_3d(smem_u32(sV), &map_v, 0, chunk * kRows, bh, bar(kO_Load));
-      }
-      tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kO_Load));
-      tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kO_Load));
-      if (has_prefix) {
-        tma_load_3d(smem_u32(sS), &map_s, 0, 0, state_idx, bar(kO_Load));
-        tma_load_3d(smem_u32(sS) + kTileBytes, &map_s, 0, 0, state_idx + 1, bar(kO_Load));
-        bulk_load(smem_u32(z_s), p.z_prefix + (size_t)(state_idx / 2) * MP, MP * 4, bar(kO_Load));
-      }
-      uint32_t w_loads[2] = {0, 0};  // copies armed per buffer
-      auto load_w = [&](int ct) {  // decoder columns 128 ct ..: head atoms, remainder atoms (64 columns each)
-        const int b = ct & 1;
+      uint32_t it = 0;          // items done: parity of the per-item barriers
+      uint32_t g = 0;           // decoder passes issued so far: pass g uses buffers g & 1
+      uint32_t w_next = 0;      // decoder passes whose columns have been requested
+      uint32_t afree_next = 0;  // decoder passes whose tile the rows are known to have read
+      auto load_qk = [&](int item) {
+        const int bh = item / p.nchunk, chunk = item - bh * p.nchunk;
+        mbar_expect_tx(bar(kO_QK), causal ? 2 * kTileBytes : kTileBytes);
+        tma_load_3d(smem_u32(sQ), &map_q, 0, chunk * kRows, bh, bar(kO_QK));
+        if (causal) tma_load_3d(smem_u32(sK), &map_k, 0, chunk * kRows, bh, bar(kO_QK));
+      };
+      auto load_vs = [&](int item) {
+        const int bh = item / p.nchunk, chunk = item - bh * p.nchunk;
+        const bool prefix = !causal || chunk > 0;
+        const int state_idx = (bh * p.nchunk + (causal ? chunk : 0)) * 2;
+        mbar_expect_tx(bar(kO_VS), (causal ? kTileBytes : 0) + (prefix ? 2 * MP * 128 + MP * 4 : 0));
+        if (causal) tma_load_3d(smem_u32(sV), &map_v, 0, chunk * kRows, bh, bar(kO_VS));
+        if (prefix) {
+          tma_load_3d(smem_u32(sS), &map_s, 0, 0, state_idx, bar(kO_VS));
+          tma_load_3d(smem_u32(sS) + kTileBytes, &map_s, 0, 0, state_idx + 1, bar(kO_VS));
+          bulk_load(smem_u32(z_s), p.z_prefix + (size_t)(state_idx / 2) * MP, MP * 4, bar(kO_VS));
+        }
+      };
+      // decoder columns of pass number w_next (column tile ct of its item) into buffer w_next & 1
+      auto load_w = [&](int ct) {
+        const int b = w_next & 1;
         const uint32_t dst = smem_u32(sPhi) + b * 2 * kTileBytes;
         mbar_expect_tx(bar(kO_W + b), 4 * 8192);
         for (int part = 0; part < 2; ++part)
           for (int atom = 0; atom < 2; ++atom)
             tma_load_3d(dst + part * kTileBytes + atom * 8192, &map_w, ct * kWTile + 64 * atom, 0, part, bar(kO_W + b));
-        ++w_loads[b];
+        ++w_next;
       };
-      ok = mbar_wait(bar(kO_Load), 0, abort_flag);
-      if (ok) {
-        fence_after();
-        const uint64_t doh = smem_desc(smem_u32(sOm), 16, 1024), dol = smem_desc(smem_u32(sOm) + kTileBytes, 16, 1024);
-        constexpr uint32_t idE = idesc_bf16(MP, false, false);
-        const uint64_t dq = smem_desc(smem_u32(sQ), 16, 1024);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, doh + 2 * k, idE, k > 0);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, dol + 2 * k, idE, 1);
-        if (causal) {
-          const uint64_t dk = smem_desc(smem_u32(sK), 16, 1024);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColA, dk + 2 * k, doh + 2 * k, idE, k > 0);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColA, dk + 2 * k, dol + 2 * k, idE, 1);
+      auto wait_afree_upto = [&](uint32_t upto) {  // the rows have read the tiles of passes 0 .. upto-1
+        while (ok && afree_next < upto) {
+          ok = mbar_wait(bar(kO_AFree + (afree_next & 1)), (afree_next >> 1) & 1, abort_flag);
+          ++afree_next;
         }
-        mma_commit(bar(kO_E));
-        ok = mbar_wait(bar(kO_Phi), 0, abort_flag);
+      };
+      const int first = blockIdx.x;
+      if (first < n_items) {
+        mbar_expect_tx(bar(kO_Om), 2 * MP * 128);
+        tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kO_Om));
+        tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kO_Om));
+        load_qk(first);
+        load_vs(first);
+        ok = mbar_wait(bar(kO_Om), 0, abort_flag);
       }
-      if (ok) {
+      const uint64_t doh = smem_desc(smem_u32(sOm), 16, 1024), dol = smem_desc(smem_u32(sOm) + kTileBytes, 16, 1024);
+      for (int item = first; item < n_items && ok; item += gridDim.x, ++it) {
+        const int chunk = item % p.nchunk;
+        const bool has_prefix = !causal || chunk > 0;
+        const int next = item + gridDim.x;
+        const uint32_t par = it & 1;
+        ok = mbar_wait(bar(kO_QK), par, abort_flag);
+        wait_afree_upto(g);  // the projections go where the previous item's A_hat tiles were
+        if (!ok) break;
         fence_after();
+        {
+          constexpr uint32_t idE = idesc_bf16(MP, false, false);
+          const uint64_t dq = smem_desc(smem_u32(sQ), 16, 1024);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, doh + 2 * k, idE, k > 0);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, dol + 2 * k, idE, 1);
+          if (causal) {
+            const uint64_t dk = smem_desc(smem_u32(sK), 16, 1024);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) mma_ss(tmem + kColA, dk + 2 * k, doh + 2 * k, idE, k > 0);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) mma_ss(tmem + kColA, dk + 2 * k, dol + 2 * k, idE, 1);
+          }
+          mma_commit(bar(kO_E));
+        }
+        ok = mbar_wait(bar(kO_Phi), par, abort_flag);
+        if (ok) ok = mbar_wait(bar(kO_VS), par, abort_flag);
+        if (!ok) break;
+        fence_after();
+        // the rows have read the projections, so the Q and K tiles are free for the next item
+        if (next < n_items) load_qk(next);
         if (causal) {
           // in-chunk kernel matrix phi(Q) phi(K)^T: A = phi(Q) in tensor memory, B = phi(K) K-major
           constexpr uint32_t idA = idesc_bf16(128, false, false);
@@ -457,14 +503,16 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             mma_ts(tmem + kColNum, a + 16, bh_, idN, 1);
           }
         }
-        if (causal) ok = mbar_wait(bar(kO_P), 0, abort_flag);
-      }
-      if (ok) {
-        fence_after();
         if (causal) {
-          // phi(K) is no longer read (the rows waited for the kernel matrix): its place takes the decoder columns
-          load_w(0);
-          if (n_ct > 1) load_w(1);
+          ok = mbar_wait(bar(kO_P), par, abort_flag);
+          if (!ok) break;
+          fence_after();
+        }
+        // phi(K) is no longer read (the rows waited for the kernel matrix): its place takes the
+        // decoder columns of this item's first passes
+        load_w(0);
+        if (n_ct > 1) load_w(1);
+        if (causal) {
           constexpr uint32_t idN = idesc_bf16(64, false, true);
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
@@ -473,21 +521,19 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             mma_ts(tmem + kColNum, a, bv, idN, (has_prefix || k > 0) ? 1u : 0u);
             mma_ts(tmem + kColNum, a + 16, bv, idN, 1);
           }
-        } else {
-          load_w(0);
-          if (n_ct > 1) load_w(1);
         }
         mma_commit(bar(kO_Num));
-        ok = mbar_wait(bar(kO_C), 0, abort_flag);
-      }
-      if (ok) {
+        ok = mbar_wait(bar(kO_C), par, abort_flag);
+        if (!ok) break;
         fence_after();
+        // numerator complete and read: V, the state and its normaliser are free for the next item
+        if (next < n_items) load_vs(next);
         // A_hat tile = C W: A = C in tensor memory (64 values: four steps), B = decoder columns MN-major
         constexpr uint32_t idW = idesc_bf16(kWTile, false, true);
-        for (int ct = 0; ct < n_ct && ok; ++ct) {
-          const int b = ct & 1;
-          ok = mbar_wait(bar(kO_W + b), (ct >> 1) & 1, abort_flag);
-          if (ok && ct >= 2) ok = mbar_wait(bar(kO_AFree + b), ((ct >> 1) - 1) & 1, abort_flag);
+        for (int ct = 0; ct < n_ct && ok; ++ct, ++g) {
+          const uint32_t b = g & 1;
+          ok = mbar_wait(bar(kO_W + b), (g >> 1) & 1, abort_flag);
+          if (g >= 2) wait_afree_upto(g - 1);  // the rows have read the tile that was in this buffer
           if (!ok) break;
           fence_after();
           const uint32_t wbase = smem_u32(sPhi) + b * 2 * kTileBytes;
@@ -504,136 +550,167 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           mma_commit(bar(kO_Ahat + b));
           mma_commit(bar(kO_WDone + b));
           if (ct >= 1 && ct + 1 < n_ct) {
-            // columns of pass ct + 1 go where pass ct - 1 read from
-            ok = mbar_wait(bar(kO_WDone + (b ^ 1)), ((ct - 1) >> 1) & 1, abort_flag);
+            // columns of the next pass go where the previous pass read from
+            ok = mbar_wait(bar(kO_WDone + (b ^ 1)), ((g - 1) >> 1) & 1, abort_flag);
             if (ok) load_w(ct + 1);
           }
         }
       }
       mma_commit(bar(kO_Drain));
       mbar_wait(bar(kO_Drain), 0, abort_flag);
-      // copies still in flight must land before the CTA may leave
-      mbar_wait_drain(bar(kO_Load), 0);
-      for (int b = 0; b < 2; ++b)
-        if (w_loads[b]) mbar_wait_drain(bar(kO_W + b), (w_loads[b] - 1) & 1);
+      // copies still in flight must land before the CTA may leave (only after a wait ran out can
+      // any be outstanding here: every armed phase is waited for in the loop above)
+      if (!ok) {
+        mbar_wait_drain(bar(kO_Om), 0);
+        mbar_wait_drain(bar(kO_QK), it & 1);
+        mbar_wait_drain(bar(kO_VS), it & 1);
+        for (uint32_t w = (w_next >= 2 ? w_next - 2 : 0); w < w_next; ++w) mbar_wait_drain(bar(kO_W + (w & 1)), (w >> 1) & 1);
+      }
     }
   } else {
     // -------------------------------------------------------------- row warps
     const int quarter = warp & 3, part = warp >> 2, rt = quarter * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
-    const int row = chunk * kRows + rt;
-    const bool row_ok = row < p.T;
-    const size_t grow = (size_t)bh * p.T + row;
-    const float sq_q = row_ok ? half_sq_norm(p.Q + grow * kHeadDim) : 0.f;
-    const float sq_k = (row_ok && causal) ? half_sq_norm(p.K + grow * kHeadDim) : 0.f;
     const float inv_sqrt_m = rsqrtf((float)p.m);
-    float den = 0.f;
-    bool ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_E), 0, abort_flag));
-    if (ok && has_prefix) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Load), 0, abort_flag));  // z has landed
-    if (ok) {
-      fence_after();
-      for (int c = part; c < MP / 32; c += kParts) {
-        uint32_t e[32];
-        float phi[32];
-        uint32_t hi[16], lo[16];
-        tmem_ld32(lane_addr + kColQ + 32 * c, e);
-        tmem_ld_wait();
-        features32(e, phi, sq_q, row_ok, c, p.m, inv_sqrt_m);
-        if (has_prefix) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) den = fmaf(phi[i], z_s[32 * c + i], den);
-        }
-        split32(phi, hi, lo);
-        tmem_st16(lane_addr + kColQ + 32 * c, hi);
-        tmem_st16(lane_addr + kColQ + 32 * c + 16, lo);
-        if (causal) {
-          tmem_ld32(lane_addr + kColA + 32 * c, e);
-          tmem_ld_wait();
-          features32(e, phi, sq_k, row_ok, c, p.m, inv_sqrt_m);
-          split32(phi, hi, lo);
-          store_row32_swizzled(sPhi, rt, c, hi);
-          store_row32_swizzled(sPhi + 2 * kTileBytes, rt, c, lo);
-        }
-      }
-      tmem_st_wait();
-      fence_async_smem();
-      warp_arrive(bar(kO_Phi), lane);
-      if (causal) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_A), 0, abort_flag));
-    }
-    if (ok && causal) {
-      fence_after();
-      // keep keys j <= i of the chunk; rows of the normaliser; head / remainder in place
-      for (int c = part; c < 4; c += kParts) {
-        uint32_t e[32];
-        float a[32];
-        uint32_t hi[16], lo[16];
-        tmem_ld32(lane_addr + kColA + 32 * c, e);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          a[i] = (32 * c + i <= rt) ? __uint_as_float(e[i]) : 0.f;
-          den += a[i];
-        }
-        split32(a, hi, lo);
-        tmem_st16(lane_addr + kColA + 32 * c, hi);
-        tmem_st16(lane_addr + kColA + 32 * c + 16, lo);
-      }
-      tmem_st_wait();
-      warp_arrive(bar(kO_P), lane);
-    }
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Num), 0, abort_flag));
-    den_x[part * kRows + rt] = den;
-    ok = rows_all(ok);
-    if (ok) {
-      fence_after();
-      den = 0.f;
-#pragma unroll
-      for (int q = 0; q < kParts; ++q) den += den_x[q * kRows + rt];
-      if (row_ok && !(den > 0.f && den < INFINITY)) atomicOr(p.status, SEA_DEV_NONFINITE);
-      const float inv = 1.f / den;
-      uint32_t e[32];
-      if (part < 2) {  // C has 64 columns: two chunks
-        float cv[32];
-        uint32_t hi[16], lo[16];
-        tmem_ld32(lane_addr + kColNum + 32 * part, e);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) cv[i] = row_ok ? __uint_as_float(e[i]) * inv : 0.f;
-        split32(cv, hi, lo);
-        tmem_st16(lane_addr + kColC + 32 * part, hi);
-        tmem_st16(lane_addr + kColC + 32 * part + 16, lo);
-        tmem_st_wait();
-      }
-      warp_arrive(bar(kO_C), lane);
-      float* out = p.A_hat + grow * p.Kc;
-      const bool vec = (p.Kc & 3) == 0;
-      for (int ct = 0; ct < n_ct && ok; ++ct) {
-        const int b = ct & 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Ahat + b), (ct >> 1) & 1, abort_flag));
-        if (!ok) break;
+    const bool elected = quarter == 0 && lane == 0;  // issues this column group's stores
+    unsigned char* my_box = sOut + part * kTileBytes;
+    uint32_t it = 0, g = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
+      const int bh = item / p.nchunk, chunk = item - bh * p.nchunk;
+      const bool has_prefix = !causal || chunk > 0;
+      const uint32_t par = it & 1;
+      const int row = chunk * kRows + rt;
+      const bool row_ok = row < p.T;
+      const size_t grow = (size_t)bh * p.T + row;
+      const float sq_q = row_ok ? half_sq_norm(p.Q + grow * kHeadDim) : 0.f;
+      const float sq_k = (row_ok && causal) ? half_sq_norm(p.K + grow * kHeadDim) : 0.f;
+      float den = 0.f;
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_E), par, abort_flag));
+      if (ok && has_prefix) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_VS), par, abort_flag));  // z has landed
+      if (ok) {
         fence_after();
-        for (int c = part; c < 4; c += kParts) {
-          tmem_ld32(lane_addr + (b ? kColA : kColQ) + 32 * c, e);
+        for (int c = part; c < MP / 32; c += kParts) {
+          uint32_t e[32];
+          float phi[32];
+          uint32_t hi[16], lo[16];
+          tmem_ld32(lane_addr + kColQ + 32 * c, e);
           tmem_ld_wait();
-          const int col0 = ct * kWTile + 32 * c;
-          if (row_ok) {
-            if (vec) {
+          features32(e, phi, sq_q, row_ok, c, p.m, inv_sqrt_m);
+          if (has_prefix) {
+            float d4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-              for (int i = 0; i < 8; ++i)
-                if (col0 + 4 * i < p.Kc)
-                  *reinterpret_cast<float4*>(out + col0 + 4 * i) =
-                      make_float4(__uint_as_float(e[4 * i]), __uint_as_float(e[4 * i + 1]), __uint_as_float(e[4 * i + 2]),
-                                  __uint_as_float(e[4 * i + 3]));
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (col0 + i < p.Kc) out[col0 + i] = __uint_as_float(e[i]);
-            }
+            for (int i = 0; i < 32; ++i) d4[i & 3] = fmaf(phi[i], z_s[32 * c + i], d4[i & 3]);
+            den += (d4[0] + d4[1]) + (d4[2] + d4[3]);
+          }
+          split32(phi, hi, lo);
+          tmem_st16(lane_addr + kColQ + 32 * c, hi);
+          tmem_st16(lane_addr + kColQ + 32 * c + 16, lo);
+          if (causal) {
+            tmem_ld32(lane_addr + kColA + 32 * c, e);
+            tmem_ld_wait();
+            features32(e, phi, sq_k, row_ok, c, p.m, inv_sqrt_m);
+            split32(phi, hi, lo);
+            store_row32_swizzled(sPhi, rt, c, hi);
+            store_row32_swizzled(sPhi + 2 * kTileBytes, rt, c, lo);
           }
         }
-        warp_arrive(bar(kO_AFree + b), lane);
+        tmem_st_wait();
+        fence_async_smem();
+        warp_arrive(bar(kO_Phi), lane);
+        if (causal) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_A), par, abort_flag));
+      }
+      if (ok && causal) {
+        fence_after();
+        // keep keys j <= i of the chunk; rows of the normaliser; head / remainder in place
+        for (int c = part; c < 4; c += kParts) {
+          uint32_t e[32];
+          float a[32];
+          uint32_t hi[16], lo[16];
+          tmem_ld32(lane_addr + kColA + 32 * c, e);
+          tmem_ld_wait();
+          float d4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            a[i] = (32 * c + i <= rt) ? __uint_as_float(e[i]) : 0.f;
+            d4[i & 3] += a[i];
+          }
+          den += (d4[0] + d4[1]) + (d4[2] + d4[3]);
+          split32(a, hi, lo);
+          tmem_st16(lane_addr + kColA + 32 * c, hi);
+          tmem_st16(lane_addr + kColA + 32 * c + 16, lo);
+        }
+        tmem_st_wait();
+        warp_arrive(bar(kO_P), lane);
+      }
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Num), par, abort_flag));
+      den_x[part * kRows + rt] = den;
+      ok = rows_all(ok);
+      if (ok) {
+        fence_after();
+        den = 0.f;
+#pragma unroll
+        for (int q = 0; q < kParts; ++q) den += den_x[q * kRows + rt];
+        if (row_ok && !(den > 0.f && den < INFINITY)) atomicOr(p.status, SEA_DEV_NONFINITE);
+        const float inv = 1.f / den;
+        if (part < 2) {  // C has 64 columns: two chunks
+          uint32_t e[32];
+          float cv[32];
+          uint32_t hi[16], lo[16];
+          tmem_ld32(lane_addr + kColNum + 32 * part, e);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) cv[i] = row_ok ? __uint_as_float(e[i]) * inv : 0.f;
+          split32(cv, hi, lo);
+          tmem_st16(lane_addr + kColC + 32 * part, hi);
+          tmem_st16(lane_addr + kColC + 32 * part + 16, lo);
+          tmem_st_wait();
+        }
+        warp_arrive(bar(kO_C), lane);
+      }
+      // ---- decoder passes: tile out of tensor memory, then to A_hat
+      float* out = p.A_hat + grow * p.Kc;
+      for (int ct = 0; ct < n_ct; ++ct, ++g) {
+        const uint32_t b = g & 1;
+        constexpr int kMine = 4 / kParts;  // chunks of the 128-column tile per thread
+        uint32_t e[kMine][32];
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Ahat + b), (g >> 1) & 1, abort_flag));
+        if (ok) {
+          fence_after();
+#pragma unroll
+          for (int cc = 0; cc < kMine; ++cc) tmem_ld32(lane_addr + (b ? kColA : kColQ) + 32 * (part + kParts * cc), e[cc]);
+          tmem_ld_wait();
+          warp_arrive(bar(kO_AFree + b), lane);
+        }
+#pragma unroll
+        for (int cc = 0; cc < kMine; ++cc) {
+          const int col0 = ct * kWTile + 32 * (part + kParts * cc);
+          if (p.tma_store) {
+            // the column group's box: wait until its previous store has been read out, fill it
+            // (128-byte rows, swizzled like the copy expects), hand it to the copy engine
+            if (elected) bulk_wait_read();
+            part_sync(2 + part);
+            if (ok) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4*>(my_box + rt * 128 + ((j ^ (rt & 7)) << 4)) =
+                    make_uint4(e[cc][4 * j], e[cc][4 * j + 1], e[cc][4 * j + 2], e[cc][4 * j + 3]);
+            }
+            fence_async_smem();
+            part_sync(2 + part);
+            if (elected && ok && col0 < p.Kc) {
+              tma_store_3d(&map_a, smem_u32(my_box), col0, chunk * kRows, bh);
+              bulk_commit();
+            }
+          } else if (ok && row_ok) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (col0 + i < p.Kc) out[col0 + i] = __uint_as_float(e[cc][i]);
+          }
+        }
       }
     }
+    if (elected) bulk_wait_all();
   }
   fence_before();
   __syncthreads();
@@ -663,7 +740,7 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   float* state_s = state;                                                              // [BH][nchunk][MP][64]
   float* state_z = state + (size_t)BH * nchunk * MP * kHeadDim;                        // [BH][nchunk][MP]
 
-  CUtensorMap mq, mk, mv, mom, ms, mw;
+  CUtensorMap mq, mk, mv, mom, ms, mw, ma;
   if (!make_map_bf16_3d(&mq, Q, kHeadDim, s.T, BH, kHeadDim, kRows) ||
       !make_map_bf16_3d(&mk, K, kHeadDim, s.T, BH, kHeadDim, kRows) ||
       !make_map_bf16_3d(&mv, V, kHeadDim, s.T, BH, kHeadDim, kRows) ||
@@ -686,14 +763,19 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   prm.z_prefix = z_prefix;
   prm.A_hat = A_hat;
   prm.status = status;
+  prm.BH = BH;
   prm.T = s.T;
   prm.m = s.m;
   prm.Kc = s.Kc;
   prm.nchunk = nchunk;
   prm.causal = s.causal;
+  // A_hat [BH][T][Kc] fp32 in boxes of 128 rows x 32 columns; without a map (rows that are no
+  // multiple of 16 bytes) the rows store their values themselves
+  prm.tma_store = (s.Kc % 4 == 0 && make_map_3d(&ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, A_hat, s.Kc, s.T, BH, 32, kRows)) ? 1 : 0;
+  if (!prm.tma_store) ma = mq;  // a valid map that is never used
 
   const size_t smem1 = 1024 + 8 * kTileBytes + 2048 + 8 * kS_NumBars + 16;
-  const size_t smem3 = 1024 + 11 * kTileBytes + 8 * kO_NumBars + 16 + (1 + kParts) * 128 * 4;
+  const size_t smem3 = 1024 + (11 + kParts) * kTileBytes + 8 * kO_NumBars + 16 + (1 + kParts) * 128 * 4;
   if (cudaFuncSetAttribute(favor_state_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
       cudaFuncSetAttribute(favor_output_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem3) != cudaSuccess)
     return SEA_ERR_CUDA;
@@ -707,7 +789,11 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
                                                                           total, s.causal);
     if ((rc = check_launch()) != SEA_OK) return rc;
   }
-  favor_output_tc_kernel<MP><<<grid, kThreads, smem3, st>>>(mq, mk, mv, mom, ms, mw, prm);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return SEA_ERR_CUDA;
+  const int n_items = BH * nchunk;
+  favor_output_tc_kernel<MP><<<n_items < sms ? n_items : sms, kThreads, smem3, st>>>(mq, mk, mv, mom, ms, mw, ma, prm);
   return check_launch();
 }
 

@@ -159,19 +159,24 @@ inline EncodeTiledFn encode_fn() {
   }();
   return fn;
 }
-// bf16 [d2][d1][d0] (d0 fastest, dense), boxes of b1 x b0 elements of one d2 slice, 128-byte
-// swizzle (b0 * 2 bytes must be 128); out-of-range rows read as zero.
-inline bool make_map_bf16_3d(CUtensorMap* map, const void* ptr, unsigned long long d0, unsigned long long d1,
-                             unsigned long long d2, unsigned b0, unsigned b1) {
+// Dense [d2][d1][d0] tensor (d0 fastest) of `elem_bytes`-byte elements, boxes of b1 x b0 elements
+// of one d2 slice, 128-byte swizzle (b0 * elem_bytes must be 128); out-of-range elements read as
+// zero and are not written.
+inline bool make_map_3d(CUtensorMap* map, CUtensorMapDataType type, unsigned elem_bytes, const void* ptr,
+                        unsigned long long d0, unsigned long long d1, unsigned long long d2, unsigned b0, unsigned b1) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[3] = {d0, d1, d2};
-  const cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
+  const cuuint64_t strides[2] = {d0 * elem_bytes, d0 * d1 * elem_bytes};
   const cuuint32_t box[3] = {b0, b1, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+  return fn(map, type, 3, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+inline bool make_map_bf16_3d(CUtensorMap* map, const void* ptr, unsigned long long d0, unsigned long long d1,
+                             unsigned long long d2, unsigned b0, unsigned b1) {
+  return make_map_3d(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, d0, d1, d2, b0, b1);
 }
 
 }  // namespace tc
