@@ -78,14 +78,30 @@ __device__ __forceinline__ float half_sq_norm(const __nv_bfloat16* row) {
   return s * (1.f / 16.f);
 }
 
-// Features of 32 projections (columns 32c .. 32c+31 of the row's projection tile): zero for
-// padded features and for rows outside the sequence.
-__device__ __forceinline__ void features32(const uint32_t (&e)[32], float (&phi)[32], float sq, bool row_ok, int c, int m,
-                                           float inv_sqrt_m) {
+// Features of 32 projections (columns 32c .. 32c+31 of the row's projection tile):
+// exp(e - |x|^2/2) / sqrt(m) = 2^(e log2(e) + bias) with the row's bias = -(|x|^2/2) log2(e) -
+// log2(m)/2, or -inf for a row outside the sequence (2^-inf = 0); padded features give zero.
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float feature_bias(float half_sq, bool row_ok, int m) {
+  return row_ok ? -half_sq * 1.4426950408889634f - 0.5f * log2f((float)m) : -INFINITY;
+}
+__device__ __forceinline__ void features32(const uint32_t (&e)[32], float (&phi)[32], float bias, int c, int m) {
+  const float2 l2e = make_float2(1.4426950408889634f, 1.4426950408889634f), b2 = make_float2(bias, bias);
+  if (32 * c + 32 <= m) {
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const float v = __expf(__uint_as_float(e[i]) - sq) * inv_sqrt_m;
-    phi[i] = (row_ok && 32 * c + i < m) ? v : 0.f;
+    for (int i = 0; i < 16; ++i) {
+      const float2 x = __ffma2_rn(make_float2(__uint_as_float(e[2 * i]), __uint_as_float(e[2 * i + 1])), l2e, b2);
+      phi[2 * i] = ex2f(x.x);
+      phi[2 * i + 1] = ex2f(x.y);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      phi[i] = 32 * c + i < m ? ex2f(fmaf(__uint_as_float(e[i]), 1.4426950408889634f, bias)) : 0.f;
   }
 }
 __device__ __forceinline__ void split32(const float (&x)[32], uint32_t (&hi)[16], uint32_t (&lo)[16]) {
@@ -221,8 +237,7 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     const int row = chunk * kRows + rt;
     const bool row_ok = row < p.T;
-    const float sq = row_ok ? half_sq_norm(p.K + ((size_t)bh * p.T + row) * kHeadDim) : 0.f;
-    const float inv_sqrt_m = rsqrtf((float)p.m);
+    const float bias = feature_bias(row_ok ? half_sq_norm(p.K + ((size_t)bh * p.T + row) * kHeadDim) : 0.f, row_ok, p.m);
     bool ok = __all_sync(0xffffffffu, mbar_wait(bar(kS_E), 0, abort_flag));
     if (ok) {
       fence_after();
@@ -231,7 +246,7 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
         tmem_ld32(lane_addr + kColE + 32 * c, e);
         tmem_ld_wait();
         float phi[32];
-        features32(e, phi, sq, row_ok, c, p.m, inv_sqrt_m);
+        features32(e, phi, bias, c, p.m);
         uint32_t hi[16], lo[16];
         split32(phi, hi, lo);
         store_row32_swizzled(sPhi, rt, c, hi);
@@ -571,7 +586,6 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     // -------------------------------------------------------------- row warps
     const int quarter = warp & 3, part = warp >> 2, rt = quarter * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
-    const float inv_sqrt_m = rsqrtf((float)p.m);
     const bool elected = quarter == 0 && lane == 0;  // issues this column group's stores
     unsigned char* my_box = sOut + part * kTileBytes;
     uint32_t it = 0, g = 0;
@@ -583,8 +597,8 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       const int row = chunk * kRows + rt;
       const bool row_ok = row < p.T;
       const size_t grow = (size_t)bh * p.T + row;
-      const float sq_q = row_ok ? half_sq_norm(p.Q + grow * kHeadDim) : 0.f;
-      const float sq_k = (row_ok && causal) ? half_sq_norm(p.K + grow * kHeadDim) : 0.f;
+      const float bias_q = feature_bias(row_ok ? half_sq_norm(p.Q + grow * kHeadDim) : 0.f, row_ok, p.m);
+      const float bias_k = feature_bias((row_ok && causal) ? half_sq_norm(p.K + grow * kHeadDim) : 0.f, row_ok, p.m);
       float den = 0.f;
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_E), par, abort_flag));
       if (ok && has_prefix) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_VS), par, abort_flag));  // z has landed
@@ -596,7 +610,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           uint32_t hi[16], lo[16];
           tmem_ld32(lane_addr + kColQ + 32 * c, e);
           tmem_ld_wait();
-          features32(e, phi, sq_q, row_ok, c, p.m, inv_sqrt_m);
+          features32(e, phi, bias_q, c, p.m);
           if (has_prefix) {
             float d4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -609,7 +623,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           if (causal) {
             tmem_ld32(lane_addr + kColA + 32 * c, e);
             tmem_ld_wait();
-            features32(e, phi, sq_k, row_ok, c, p.m, inv_sqrt_m);
+            features32(e, phi, bias_k, c, p.m);
             split32(phi, hi, lo);
             store_row32_swizzled(sPhi, rt, c, hi);
             store_row32_swizzled(sPhi + 2 * kTileBytes, rt, c, lo);

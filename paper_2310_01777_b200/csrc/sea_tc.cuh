@@ -140,7 +140,8 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t tmem, uint32_t cols) {
 __device__ __forceinline__ void split_pair(float x, float y, uint32_t& hi, uint32_t& lo) {
   const uint32_t hx = __float_as_uint(x) & 0xffff0000u, hy = __float_as_uint(y) & 0xffff0000u;
   hi = __byte_perm(hx, hy, 0x7632);
-  const __nv_bfloat162 l = __floats2bfloat162_rn(x - __uint_as_float(hx), y - __uint_as_float(hy));
+  const float2 rem = __ffma2_rn(make_float2(__uint_as_float(hx), __uint_as_float(hy)), make_float2(-1.f, -1.f), make_float2(x, y));
+  const __nv_bfloat162 l = __floats2bfloat162_rn(rem.x, rem.y);
   lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
