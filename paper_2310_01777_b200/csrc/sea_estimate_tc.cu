@@ -135,6 +135,13 @@ __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
   if (lane == 0) mbar_arrive(bar);
 }
 
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];\n"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory"); }
 struct EstParams {
   const __nv_bfloat16 *Q, *K;   // for the rows' norms
   float* state_s;               // [BH][nchunk][MP][64]
@@ -152,7 +159,8 @@ enum { kS_Load = 0, kS_E, kS_Phi, kS_S, kS_Drain, kS_NumBars };
 template <int MP>
 __global__ void __launch_bounds__(kThreads, 1)
 favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                      const __grid_constant__ CUtensorMap map_om, const EstParams p) {
+                      const __grid_constant__ CUtensorMap map_om, const __grid_constant__ CUtensorMap map_phi,
+                      const EstParams p) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* sm = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   unsigned char* sK = sm;                              // 16 KB
@@ -211,6 +219,15 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
       }
       if (ok) {
         fence_after();
+        if (p.causal) {
+          // the output kernel needs phi(K) of its own chunk again: keep the tiles (head atoms, remainder atoms)
+          constexpr int kAtoms = MP > 64 ? 2 : 1;
+          const int slice0 = (bh * p.nchunk + chunk) * 2 * kAtoms;
+          for (int part = 0; part < 2; ++part)
+            for (int a = 0; a < kAtoms; ++a)
+              tma_store_3d(&map_phi, smem_u32(sPhi) + part * 2 * kTileBytes + a * kTileBytes, 0, 0, slice0 + part * kAtoms + a);
+          bulk_commit();
+        }
         // S = phi^T V and z = phi^T 1: A = phi read MN-major (features are its M index), B = V and a
         // tile of ones read MN-major; contraction over the 128 keys in eight steps
         constexpr uint32_t idS = idesc_bf16(64, true, true), idZ = idesc_bf16(16, true, true);
@@ -230,6 +247,7 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
       mma_commit(bar(kS_Drain));
       mbar_wait(bar(kS_Drain), 0, abort_flag);
       mbar_wait_drain(bar(kS_Load), 0);  // the copies have landed before the CTA may leave
+      bulk_wait_all();                   // and the stored tiles have left shared memory
     }
   } else {
     // -------------------------------------------------------------- row warps
@@ -342,7 +360,8 @@ __global__ void favor_scan_tc_kernel(const float* __restrict__ state_s, const fl
 // reading their places, and every barrier below completes once per item (or once per decoder pass).
 enum {
   kO_Om = 0,               // omega' staged (once)
-  kO_QK,                   // the item's Q (and K) tile
+  kO_QK,                   // the item's Q tile
+  kO_PhiK,                 // the item's phi(K) tiles (causal)
   kO_VS,                   // the item's V tile, prefix state and its normaliser
   kO_E, kO_Phi, kO_A, kO_P, kO_Num, kO_C,
   kO_W,                    // [2] decoder columns staged
@@ -353,13 +372,6 @@ enum {
   kO_NumBars
 };
 
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
-  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];\n"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory"); }
 // Named barrier `id` over the 128 threads of one column group of the row warps.
 __device__ __forceinline__ void part_sync(int id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
 
@@ -368,7 +380,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_om,
                        const __grid_constant__ CUtensorMap map_s, const __grid_constant__ CUtensorMap map_w,
-                       const __grid_constant__ CUtensorMap map_a, const EstParams p) {
+                       const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_phi,
+                       const EstParams p) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* sm = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   unsigned char* sQ = sm;                              // 16 KB
@@ -382,7 +395,8 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   const uint32_t bars = smem_u32(tail);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * kO_NumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8 * kO_NumBars + 4);
-  float* z_s = reinterpret_cast<float*>(tail + 8 * kO_NumBars + 16);  // [128]
+  constexpr int kTailHead = (8 * kO_NumBars + 8 + 127) / 128 * 128;  // barriers, slot, flag; z_s is a bulk-copy target (16-byte rule)
+  float* z_s = reinterpret_cast<float*>(tail + kTailHead);           // [128]
   float* den_x = z_s + 128;                                            // [kParts][128]
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   // tensor memory: projections of Q -> phi(Q); projections of K -> in-chunk kernel matrix -> its
@@ -417,9 +431,17 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       uint32_t afree_next = 0;  // decoder passes whose tile the rows are known to have read
       auto load_qk = [&](int item) {
         const int bh = item / p.nchunk, chunk = item - bh * p.nchunk;
-        mbar_expect_tx(bar(kO_QK), causal ? 2 * kTileBytes : kTileBytes);
+        mbar_expect_tx(bar(kO_QK), kTileBytes);
         tma_load_3d(smem_u32(sQ), &map_q, 0, chunk * kRows, bh, bar(kO_QK));
-        if (causal) tma_load_3d(smem_u32(sK), &map_k, 0, chunk * kRows, bh, bar(kO_QK));
+      };
+      // phi(K) of the item's chunk, as the state kernel left it: head atoms, remainder atoms
+      constexpr int kAtoms = MP > 64 ? 2 : 1;
+      auto load_phik = [&](int item) {
+        mbar_expect_tx(bar(kO_PhiK), 2 * kAtoms * kTileBytes);
+        for (int part = 0; part < 2; ++part)
+          for (int a = 0; a < kAtoms; ++a)
+            tma_load_3d(smem_u32(sPhi) + part * 2 * kTileBytes + a * kTileBytes, &map_phi, 0, 0,
+                        item * 2 * kAtoms + part * kAtoms + a, bar(kO_PhiK));
       };
       auto load_vs = [&](int item) {
         const int bh = item / p.nchunk, chunk = item - bh * p.nchunk;
@@ -468,6 +490,8 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         wait_afree_upto(g);  // the projections go where the previous item's A_hat tiles were
         if (!ok) break;
         fence_after();
+        // ... and the decoder columns of the previous item are no longer read: their place takes phi(K)
+        if (causal) load_phik(item);
         {
           constexpr uint32_t idE = idesc_bf16(MP, false, false);
           const uint64_t dq = smem_desc(smem_u32(sQ), 16, 1024);
@@ -475,22 +499,17 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, doh + 2 * k, idE, k > 0);
 #pragma unroll
           for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, dol + 2 * k, idE, 1);
-          if (causal) {
-            const uint64_t dk = smem_desc(smem_u32(sK), 16, 1024);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) mma_ss(tmem + kColA, dk + 2 * k, doh + 2 * k, idE, k > 0);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) mma_ss(tmem + kColA, dk + 2 * k, dol + 2 * k, idE, 1);
-          }
           mma_commit(bar(kO_E));
         }
         ok = mbar_wait(bar(kO_Phi), par, abort_flag);
         if (ok) ok = mbar_wait(bar(kO_VS), par, abort_flag);
         if (!ok) break;
         fence_after();
-        // the rows have read the projections, so the Q and K tiles are free for the next item
+        // the rows have read the projections, so the Q tile is free for the next item
         if (next < n_items) load_qk(next);
         if (causal) {
+          ok = mbar_wait(bar(kO_PhiK), par, abort_flag);
+          if (!ok) break;
           // in-chunk kernel matrix phi(Q) phi(K)^T: A = phi(Q) in tensor memory, B = phi(K) K-major
           constexpr uint32_t idA = idesc_bf16(128, false, false);
 #pragma unroll
@@ -579,6 +598,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         mbar_wait_drain(bar(kO_Om), 0);
         mbar_wait_drain(bar(kO_QK), it & 1);
         mbar_wait_drain(bar(kO_VS), it & 1);
+        if (causal) mbar_wait_drain(bar(kO_PhiK), it & 1);
         for (uint32_t w = (w_next >= 2 ? w_next - 2 : 0); w < w_next; ++w) mbar_wait_drain(bar(kO_W + (w & 1)), (w >> 1) & 1);
       }
     }
@@ -598,7 +618,6 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       const bool row_ok = row < p.T;
       const size_t grow = (size_t)bh * p.T + row;
       const float bias_q = feature_bias(row_ok ? half_sq_norm(p.Q + grow * kHeadDim) : 0.f, row_ok, p.m);
-      const float bias_k = feature_bias((row_ok && causal) ? half_sq_norm(p.K + grow * kHeadDim) : 0.f, row_ok, p.m);
       float den = 0.f;
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_E), par, abort_flag));
       if (ok && has_prefix) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_VS), par, abort_flag));  // z has landed
@@ -620,17 +639,8 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           split32(phi, hi, lo);
           tmem_st16(lane_addr + kColQ + 32 * c, hi);
           tmem_st16(lane_addr + kColQ + 32 * c + 16, lo);
-          if (causal) {
-            tmem_ld32(lane_addr + kColA + 32 * c, e);
-            tmem_ld_wait();
-            features32(e, phi, bias_k, c, p.m);
-            split32(phi, hi, lo);
-            store_row32_swizzled(sPhi, rt, c, hi);
-            store_row32_swizzled(sPhi + 2 * kTileBytes, rt, c, lo);
-          }
         }
         tmem_st_wait();
-        fence_async_smem();
         warp_arrive(bar(kO_Phi), lane);
         if (causal) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_A), par, abort_flag));
       }
@@ -751,16 +761,18 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   __nv_bfloat16* wd = om + 2 * 128 * kHeadDim;                                         // [2][64][KcP]
   __nv_bfloat16* s_split = wd + 2 * kHeadDim * KcP;                                    // [BH][nchunk][2][MP][64]
   float* z_prefix = reinterpret_cast<float*>(s_split + (size_t)BH * nchunk * 2 * MP * kHeadDim);  // [BH][nchunk][MP]
+  __nv_bfloat16* phik = reinterpret_cast<__nv_bfloat16*>(z_prefix + (size_t)BH * nchunk * MP);  // [BH][nchunk][2][atoms][128][64]
   float* state_s = state;                                                              // [BH][nchunk][MP][64]
   float* state_z = state + (size_t)BH * nchunk * MP * kHeadDim;                        // [BH][nchunk][MP]
 
-  CUtensorMap mq, mk, mv, mom, ms, mw, ma;
+  CUtensorMap mq, mk, mv, mom, ms, mw, ma, mphi;
   if (!make_map_bf16_3d(&mq, Q, kHeadDim, s.T, BH, kHeadDim, kRows) ||
       !make_map_bf16_3d(&mk, K, kHeadDim, s.T, BH, kHeadDim, kRows) ||
       !make_map_bf16_3d(&mv, V, kHeadDim, s.T, BH, kHeadDim, kRows) ||
       !make_map_bf16_3d(&mom, om, kHeadDim, MP, 2, kHeadDim, MP) ||
       !make_map_bf16_3d(&ms, s_split, kHeadDim, MP, (unsigned long long)BH * nchunk * 2, kHeadDim, MP) ||
-      !make_map_bf16_3d(&mw, wd, KcP, kHeadDim, 2, 64, kHeadDim))
+      !make_map_bf16_3d(&mw, wd, KcP, kHeadDim, 2, 64, kHeadDim) ||
+      !make_map_bf16_3d(&mphi, phik, kHeadDim, kRows, (unsigned long long)BH * nchunk * 2 * (MP > 64 ? 2 : 1), kHeadDim, kRows))
     return SEA_ERR_CUDA;
 
   const int n_prep = MP * kHeadDim + kHeadDim * (int)KcP;
@@ -789,15 +801,15 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   if (!prm.tma_store) ma = mq;  // a valid map that is never used
 
   const size_t smem1 = 1024 + 8 * kTileBytes + 2048 + 8 * kS_NumBars + 16;
-  const size_t smem3 = 1024 + (11 + kParts) * kTileBytes + 8 * kO_NumBars + 16 + (1 + kParts) * 128 * 4;
+  const size_t smem3 = 1024 + (11 + kParts) * kTileBytes + (8 * kO_NumBars + 8 + 127) / 128 * 128 + (1 + kParts) * 128 * 4;
   if (cudaFuncSetAttribute(favor_state_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
       cudaFuncSetAttribute(favor_output_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem3) != cudaSuccess)
     return SEA_ERR_CUDA;
   const dim3 grid(nchunk, BH);
+  favor_state_tc_kernel<MP><<<grid, kThreads, smem1, st>>>(mk, mv, mom, mphi, prm);
+  if ((rc = check_launch()) != SEA_OK) return rc;
   // a causal sequence of one chunk has no prefix to form
   if (!(s.causal && nchunk == 1)) {
-    favor_state_tc_kernel<MP><<<grid, kThreads, smem1, st>>>(mk, mv, mom, prm);
-    if ((rc = check_launch()) != SEA_OK) return rc;
     const long long total = (long long)BH * MP * 33;
     favor_scan_tc_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(state_s, state_z, s_split, z_prefix, nchunk, MP,
                                                                           total, s.causal);
@@ -807,7 +819,7 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return SEA_ERR_CUDA;
   const int n_items = BH * nchunk;
-  favor_output_tc_kernel<MP><<<n_items < sms ? n_items : sms, kThreads, smem3, st>>>(mq, mk, mv, mom, ms, mw, ma, prm);
+  favor_output_tc_kernel<MP><<<n_items < sms ? n_items : sms, kThreads, smem3, st>>>(mq, mk, mv, mom, ms, mw, ma, mphi, prm);
   return check_launch();
 }
 
@@ -825,7 +837,8 @@ size_t estimate_tc_split_bytes(const sea_shape& s) {
   const size_t nchunk = ((size_t)s.T + kRows - 1) / kRows;
   const size_t MP = padded_features(s.m);
   const size_t elems = 2 * (size_t)128 * kHeadDim + 2 * (size_t)kHeadDim * padded_kc(s) +
-                       (size_t)s.B * s.H * nchunk * (2 * MP * kHeadDim + 2 * MP);
+                       (size_t)s.B * s.H * nchunk * (2 * MP * kHeadDim + 2 * MP) +
+                       (size_t)s.B * s.H * nchunk * 2 * (MP > 64 ? 2 : 1) * kRows * kHeadDim;  // phi(K) tiles
   return elems * sizeof(__nv_bfloat16) + 256;
 }
 bool estimate_tc_applicable(const sea_shape& s) {
