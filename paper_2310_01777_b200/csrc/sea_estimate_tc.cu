@@ -157,17 +157,19 @@ struct EstParams {
 enum { kS_Load = 0, kS_E, kS_Phi, kS_S, kS_Drain, kS_NumBars };
 
 template <int MP>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                       const __grid_constant__ CUtensorMap map_om, const __grid_constant__ CUtensorMap map_phi,
                       const EstParams p) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* sm = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
+  // phi(K) (head 32 KB, remainder 32 KB: [2 atoms][128 keys][64 f]) is written only after the
+  // projections are complete, over the K tile and omega' that fed them: two CTAs fit an SM
+  unsigned char* sPhi = sm;                            // 64 KB
   unsigned char* sK = sm;                              // 16 KB
-  unsigned char* sV = sK + kTileBytes;                 // 16 KB
-  unsigned char* sOm = sV + kTileBytes;                // head 16 KB, remainder 16 KB ([MP][64])
-  unsigned char* sPhi = sOm + 2 * kTileBytes;          // head 32 KB, remainder 32 KB ([2 atoms][128 keys][64 f])
-  unsigned char* sOnes = sPhi + 4 * kTileBytes;        // 16 rows x 128 B of 1.0
+  unsigned char* sOm = sK + kTileBytes;                // head 16 KB, remainder 16 KB ([MP][64])
+  unsigned char* sV = sPhi + 4 * kTileBytes;           // 16 KB
+  unsigned char* sOnes = sV + kTileBytes;              // 16 rows x 128 B of 1.0
   unsigned char* tail = sOnes + 2048;
   const uint32_t bars = smem_u32(tail);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * kS_NumBars);
@@ -800,7 +802,7 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   prm.tma_store = (s.Kc % 4 == 0 && make_map_3d(&ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, A_hat, s.Kc, s.T, BH, 32, kRows)) ? 1 : 0;
   if (!prm.tma_store) ma = mq;  // a valid map that is never used
 
-  const size_t smem1 = 1024 + 8 * kTileBytes + 2048 + 8 * kS_NumBars + 16;
+  const size_t smem1 = 1024 + 5 * kTileBytes + 2048 + 8 * kS_NumBars + 16;
   const size_t smem3 = 1024 + (11 + kParts) * kTileBytes + (8 * kO_NumBars + 8 + 127) / 128 * 128 + (1 + kParts) * 128 * 4;
   if (cudaFuncSetAttribute(favor_state_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
       cudaFuncSetAttribute(favor_output_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem3) != cudaSuccess)
