@@ -42,7 +42,7 @@ WsLayout ws_layout(const sea_shape& s) {
   L.status = take(kStatusBytes);
   auto larger = [](size_t a, size_t b) { return a > b ? a : b; };
   L.est_state = take(s.m > 0 ? larger(BH * nchunk * (size_t)s.m * (kHeadDim + 1) * sizeof(float), estimate_tc_state_bytes(s)) : 0);
-  L.est_split = take(s.m > 0 ? larger(estimate_split_bytes(s), estimate_tc_split_bytes(s)) : 0);
+  L.est_split = take(s.m > 0 ? estimate_tc_split_bytes(s) : 0);
   L.row_counts = take(rows * sizeof(int32_t));
   L.tile_sums = take(((rows + kScanTileRows - 1) / kScanTileRows + 1) * sizeof(int32_t));
   L.a_hat = take(rows * (size_t)s.Kc * sizeof(float));

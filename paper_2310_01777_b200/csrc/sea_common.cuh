@@ -47,11 +47,7 @@ sea_status launch_estimate(const sea_shape& s, const void* Q, const void* K, con
 sea_status launch_estimate_f32(const sea_shape& s, const void* Q, const void* K, const void* V,
                                const float* omega, const float* W_dec, float* A_hat,
                                float* est_state, int32_t* status, cudaStream_t st);
-sea_status launch_estimate_bf16(const sea_shape& s, const void* Q, const void* K, const void* V,
-                                const float* omega, const float* W_dec, float* A_hat,
-                                float* est_state, void* est_split, int32_t* status, cudaStream_t st);
-size_t estimate_split_bytes(const sea_shape& s);
-// tcgen05 form of the bf16 estimator (sea_estimate_tc.cu)
+// bf16 estimator on tcgen05 (sea_estimate_tc.cu)
 bool estimate_tc_applicable(const sea_shape& s);
 size_t estimate_tc_state_bytes(const sea_shape& s);
 size_t estimate_tc_split_bytes(const sea_shape& s);

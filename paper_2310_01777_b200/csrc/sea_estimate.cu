@@ -9,8 +9,8 @@
 // in a fixed order: an exclusive prefix for causal attention, the total otherwise.
 // Kernel 3 computes, per chunk, phi(Q_c) S + (phi(Q_c) phi(K_c)^T . tril) [V_c | 1]
 // (the second term only when causal), divides, applies W_dec and writes A_hat.
-// This file is the plain fp32 FMA form used for fp32 inputs; bf16 inputs take the tensor-core
-// form in sea_estimate_mma.cu.
+// This file is the plain fp32 FMA form used for fp32 inputs (chunks of 64 rows); bf16 inputs
+// take the tensor-core form in sea_estimate_tc.cu (chunks of 128 rows).
 #include "sea_common.cuh"
 
 namespace sea {
@@ -324,10 +324,11 @@ sea_status launch_estimate_f32(const sea_shape& s, const void* Q, const void* K,
 sea_status launch_estimate(const sea_shape& s, const void* Q, const void* K, const void* V,
                            const float* omega, const float* W_dec, float* A_hat, float* est_state,
                            void* est_split, int32_t* status, cudaStream_t st) {
-  if (estimate_tc_applicable(s))
+  if (s.io == SEA_BF16) {
+    // the tensor-core form needs the driver's tensor-map encoder; there is no other bf16 path
+    if (!estimate_tc_applicable(s)) return SEA_ERR_CUDA;
     return launch_estimate_tc(s, Q, K, V, omega, W_dec, A_hat, est_state, est_split, status, st);
-  if (s.io == SEA_BF16)
-    return launch_estimate_bf16(s, Q, K, V, omega, W_dec, A_hat, est_state, est_split, status, st);
+  }
   return launch_estimate_f32(s, Q, K, V, omega, W_dec, A_hat, est_state, status, st);
 }
 

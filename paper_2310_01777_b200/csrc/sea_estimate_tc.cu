@@ -5,21 +5,25 @@
 //   C_i = sum_j phi(q_i).phi(k_j) v_j / sum_j phi(q_i).phi(k_j);  A_hat = C W_dec   (Sec. 3.1, one
 //   linear head in place of the trained decoder)
 //
-// The sequence is cut into chunks of 128 rows, one CTA per (chunk, head):
-//   1. favor_state_tc_kernel:  S_c = phi(K_c)^T V_c  [m x 64]  and  z_c = phi(K_c)^T 1  [m]
+// The sequence is cut into chunks of 128 rows:
+//   1. favor_state_tc_kernel:  S_c = phi(K_c)^T V_c  [m x 64]  and  z_c = phi(K_c)^T 1  [m], one CTA
+//                              per (chunk, head), two CTAs per SM; causal: phi(K_c) is kept as
+//                              ready-made operand tiles for kernel 3
 //   2. favor_scan_tc_kernel:   exclusive prefix over the chunks of a head (causal) or the total,
 //                              in a fixed order, written as bf16 head / remainder MMA operands
 //   3. favor_output_tc_kernel: num = phi(Q_c) S + (phi(Q_c) phi(K_c)^T . tril) V_c, den likewise,
-//                              C = num / den, A_hat = C W_dec
+//                              C = num / den, A_hat = C W_dec; persistent CTAs that copy the next
+//                              chunk's tiles in while the current one is computed, A_hat leaves
+//                              through TMA stores
 // Precision: the estimate has to agree with fp64 to 1e-3 and the feature map exponentiates a
 // projection of magnitude ~10, so every fp32 operand is carried as a bf16 head plus a bf16
 // remainder (2^-17 relative) and a product A B is evaluated as A_hi B_hi + A_hi B_lo + A_lo B_hi;
 // Q, K and V are exact in bf16.  d^(-1/4) is folded into omega beforehand.
 //
-// Inside a CTA sixteen row warps own the 128 rows (a row and a quarter of a tile's columns per
-// thread: exponentials, masks, normalisers, splits) and one thread of a further warp issues the
-// copies and the MMAs; the phases of a chunk follow one another through single-use mbarriers.  Every wait is
-// bounded; a wait that runs out sets SEA_DEV_TIMEOUT and the CTA drains and leaves.
+// Inside a CTA eight row warps own the 128 rows (a row and half of a tile's columns per thread:
+// exponentials, masks, normalisers, splits) and one thread of a ninth warp issues the copies and
+// the MMAs; the phases of a chunk follow one another through mbarriers.  Every wait is bounded; a
+// wait that runs out sets SEA_DEV_TIMEOUT and the CTA drains and leaves.
 #include "sea_common.cuh"
 #include "sea_tc.cuh"
 
@@ -379,16 +383,14 @@ __device__ __forceinline__ void part_sync(int id) { asm volatile("bar.sync %0, 1
 
 template <int MP>
 __global__ void __launch_bounds__(kThreads, 1)
-favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                       const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_om,
+favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_om,
                        const __grid_constant__ CUtensorMap map_s, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_phi,
                        const EstParams p) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* sm = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   unsigned char* sQ = sm;                              // 16 KB
-  unsigned char* sK = sQ + kTileBytes;                 // 16 KB
-  unsigned char* sV = sK + kTileBytes;                 // 16 KB
+  unsigned char* sV = sQ + kTileBytes;                 // 16 KB
   unsigned char* sOm = sV + kTileBytes;                // head, remainder: 32 KB
   unsigned char* sS = sOm + 2 * kTileBytes;            // prefix state head, remainder [MP][64]: 32 KB
   unsigned char* sPhi = sS + 2 * kTileBytes;           // phi(K) head 32 KB, remainder 32 KB; later the decoder columns
@@ -803,7 +805,7 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   if (!prm.tma_store) ma = mq;  // a valid map that is never used
 
   const size_t smem1 = 1024 + 5 * kTileBytes + 2048 + 8 * kS_NumBars + 16;
-  const size_t smem3 = 1024 + (11 + kParts) * kTileBytes + (8 * kO_NumBars + 8 + 127) / 128 * 128 + (1 + kParts) * 128 * 4;
+  const size_t smem3 = 1024 + (10 + kParts) * kTileBytes + (8 * kO_NumBars + 8 + 127) / 128 * 128 + (1 + kParts) * 128 * 4;
   if (cudaFuncSetAttribute(favor_state_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
       cudaFuncSetAttribute(favor_output_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem3) != cudaSuccess)
     return SEA_ERR_CUDA;
@@ -821,7 +823,7 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return SEA_ERR_CUDA;
   const int n_items = BH * nchunk;
-  favor_output_tc_kernel<MP><<<n_items < sms ? n_items : sms, kThreads, smem3, st>>>(mq, mk, mv, mom, ms, mw, ma, mphi, prm);
+  favor_output_tc_kernel<MP><<<n_items < sms ? n_items : sms, kThreads, smem3, st>>>(mq, mv, mom, ms, mw, ma, mphi, prm);
   return check_launch();
 }
 

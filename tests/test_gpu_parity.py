@@ -77,6 +77,35 @@ def test_tile_kernel_and_row_kernels_both_match_oracle(w):
         global_mask_properties(run)
 
 
+EST_CASES = [
+    small("est_m16", dtype="bf16", causal=True, T=256, Kc=32, m=16),
+    small("est_m48", dtype="bf16", T=384, Kc=32, m=48),                              # features padded to 64
+    small("est_kc8", dtype="bf16", causal=True, T=256, Kc=8, k_hat=2, m=64),          # A_hat narrower than a store box
+    small("est_kc30", dtype="bf16", causal=True, T=120, Kc=30, k_hat=5, m=32),        # rows of A_hat no multiple of 16 bytes
+    small("est_kc512", dtype="bf16", causal=True, T=512, Kc=512, k_hat=20, m=64, H=1),   # four decoder passes per chunk
+    small("est_T64", dtype="bf16", causal=True, T=64, Kc=16, m=128),                  # one partial chunk
+    small("est_many", dtype="bf16", causal=True, B=4, H=10, T=640, Kc=64, m=128),     # 200 chunks: persistent CTAs wrap
+    small("est_nc_many", dtype="bf16", B=3, H=20, T=384, Kc=96, k_hat=7, m=64),       # 180 chunks, non-causal
+]
+
+
+@pytest.mark.parametrize("w", EST_CASES, ids=lambda w: w.name)
+def test_tensor_core_estimator_shapes(w):
+    """Shapes that exercise the chunked estimator's paths: feature padding, partial chunks,
+    several decoder passes, both ways of storing A_hat, more chunks than CTAs."""
+    run = GpuRun(w)
+    run.A_hat.fill_(float("nan"))
+    run.estimate()
+    run.sync()
+    assert run.status() == 0
+    assert bool(torch.isfinite(run.A_hat).all())
+    heads = [(0, 0), (w.B - 1, w.H - 1), (w.B // 2, w.H // 2)]
+    for b, h in sorted(set(heads)):
+        ref = orc.estimate_head(np64(run.host["Q"][b, h]), np64(run.host["K"][b, h]), np64(run.host["V"][b, h]),
+                                np64(run.host["omega"]), np64(run.host["W_dec"]), w.causal)
+        check_a_hat(run.A_hat[b, h].cpu().numpy(), ref)
+
+
 @pytest.mark.parametrize("w", SMALL_CASES[:6], ids=lambda w: w.name)
 def test_fused_call_equals_stage_calls_bitwise(w):
     a = GpuRun(w)
