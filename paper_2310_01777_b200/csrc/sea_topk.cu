@@ -83,22 +83,56 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
 }
 
 // Selection with one thread per row, for short rows and small k_hat: no cross-lane traffic at
-// all.  Every thread streams its row (16-byte loads; a row is a few cache lines that the
-// thread walks front to back) through a sorted list of the KMAX largest keys seen so far - a
-// max/min pair per list slot, branch-free - which leaves the k_hat-th largest key tau in the
-// last slot; a second walk over the row emits, in ascending column order, the columns above
-// tau and the first k_hat - |{key > tau}| columns equal to it: the same set as the bit search
-// below, ties going to the lower column.
+// all.  Every thread walks its row (16-byte loads; a row is a few cache lines that the thread
+// reads front to back) in groups of KMAX keys and keeps the KMAX largest keys seen so far as a
+// descending list in registers: a group is sorted ascending by a bitonic network, the
+// element-wise maximum with the list is then a bitonic sequence holding the KMAX largest of
+// both, and a bitonic merge sorts it again - all compare-exchanges on fixed registers, no
+// branches.  That leaves the k_hat-th largest key tau in the last slot; a second walk over the
+// row emits, in ascending column order, the columns above tau and the first
+// k_hat - |{key > tau}| columns equal to it: the same set as the bit search below, ties going to
+// the lower column.
 constexpr int kThreadRows = 128;  // threads (= rows) per CTA
 
-template <int KMAX>
-__device__ __forceinline__ void list_insert(uint32_t (&top)[KMAX], uint32_t x) {
+// a[i] >= a[l] afterwards when kDescending, a[i] <= a[l] otherwise
+template <bool kDescending>
+__device__ __forceinline__ void cmp_exchange(uint32_t& x, uint32_t& y) {
+  const uint32_t hi = max(x, y), lo = min(x, y);
+  x = kDescending ? hi : lo;
+  y = kDescending ? lo : hi;
+}
+template <int N>
+__device__ __forceinline__ void bitonic_sort_ascending(uint32_t (&a)[N]) {
 #pragma unroll
-  for (int s = 0; s < KMAX; ++s) {
-    const uint32_t hi = max(top[s], x);
-    x = min(top[s], x);
-    top[s] = hi;
-  }
+  for (int k = 2; k <= N; k <<= 1)
+#pragma unroll
+    for (int j = k >> 1; j > 0; j >>= 1)
+#pragma unroll
+      for (int i = 0; i < N; ++i) {
+        const int l = i ^ j;
+        if (l > i) {
+          if ((i & k) == 0) cmp_exchange<false>(a[i], a[l]);
+          else cmp_exchange<true>(a[i], a[l]);
+        }
+      }
+}
+template <int N>
+__device__ __forceinline__ void bitonic_merge_descending(uint32_t (&a)[N]) {
+#pragma unroll
+  for (int j = N >> 1; j > 0; j >>= 1)
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      const int l = i ^ j;
+      if (l > i) cmp_exchange<true>(a[i], a[l]);
+    }
+}
+// top (descending) <- the KMAX largest of top and grp (any order; destroyed)
+template <int KMAX>
+__device__ __forceinline__ void merge_group(uint32_t (&top)[KMAX], uint32_t (&grp)[KMAX]) {
+  bitonic_sort_ascending<KMAX>(grp);
+#pragma unroll
+  for (int s = 0; s < KMAX; ++s) top[s] = max(top[s], grp[s]);
+  bitonic_merge_descending<KMAX>(top);
 }
 
 template <int KMAX, bool kVec>
@@ -114,16 +148,24 @@ topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ s
   uint32_t top[KMAX];
 #pragma unroll
   for (int s = 0; s < KMAX; ++s) top[s] = s < KMAX - k_hat ? 0xffffffffu : 0u;
-  if (kVec) {  // Kc % 4 == 0: rows start on 16-byte boundaries
-    for (int j = 0; j < Kc; j += 4) {
-      const float4 v = __ldg(reinterpret_cast<const float4*>(a + j));
-      list_insert<KMAX>(top, order_key(v.x));
-      list_insert<KMAX>(top, order_key(v.y));
-      list_insert<KMAX>(top, order_key(v.z));
-      list_insert<KMAX>(top, order_key(v.w));
+  for (int j0 = 0; j0 < Kc; j0 += KMAX) {
+    uint32_t grp[KMAX];  // keys j0 .. j0 + KMAX - 1; beyond the row: 0
+    if (kVec) {  // Kc % 4 == 0: rows start on 16-byte boundaries
+#pragma unroll
+      for (int j = 0; j < KMAX; j += 4) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        const bool in = j0 + j < Kc;
+        if (in) v = __ldg(reinterpret_cast<const float4*>(a + j0 + j));
+        grp[j] = in ? order_key(v.x) : 0u;
+        grp[j + 1] = in ? order_key(v.y) : 0u;
+        grp[j + 2] = in ? order_key(v.z) : 0u;
+        grp[j + 3] = in ? order_key(v.w) : 0u;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < KMAX; ++j) grp[j] = j0 + j < Kc ? order_key(__ldg(a + j0 + j)) : 0u;
     }
-  } else {
-    for (int j = 0; j < Kc; ++j) list_insert<KMAX>(top, order_key(__ldg(a + j)));
+    merge_group<KMAX>(top, grp);
   }
   const uint32_t tau = top[KMAX - 1];
   int n_gt = 0;
@@ -251,7 +293,7 @@ __global__ void uniform_row_ptr_kernel(int32_t* __restrict__ row_ptr, int rows, 
 // contains the diagonal is cut.
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 fill_col_idx_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__ row_ptr,
-                    int32_t* __restrict__ col_idx, long long nnz_cap, int rows, int k_hat, int r,
+                    int32_t* __restrict__ col_idx, long long nnz_cap, int rows, int k_hat, int r, int log2r,
                     int32_t* __restrict__ status) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kWarpsPerCta + warp;
@@ -263,9 +305,14 @@ fill_col_idx_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__
     n = (int)max(0ll, min((long long)n, nnz_cap - base));
   }
   const int32_t* my_sel = sel + (size_t)row * k_hat;
-  for (int pos = lane; pos < n; pos += 32) {
-    const int b = pos / r;
-    col_idx[(size_t)base + pos] = __ldg(my_sel + b) * r + (pos - b * r);
+  if (log2r >= 0) {  // r a power of two: the run and the offset inside it are a shift and a mask
+    for (int pos = lane; pos < n; pos += 32)
+      col_idx[(size_t)base + pos] = (__ldg(my_sel + (pos >> log2r)) << log2r) + (pos & (r - 1));
+  } else {
+    for (int pos = lane; pos < n; pos += 32) {
+      const int b = pos / r;
+      col_idx[(size_t)base + pos] = __ldg(my_sel + b) * r + (pos - b * r);
+    }
   }
 }
 
@@ -328,8 +375,11 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
   }
   if (col_idx != nullptr) {
     const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+    int log2r = -1;
+    for (int l = 0; l < 31; ++l)
+      if ((1 << l) == r) log2r = l;
     fill_col_idx_kernel<<<grid, kWarpsPerCta * 32, 0, st>>>(sel, row_ptr, col_idx, (long long)nnz_cap,
-                                                            rows, s.k_hat, r, status);
+                                                            rows, s.k_hat, r, log2r, status);
     if ((rc = check_launch()) != SEA_OK) return rc;
   }
   return SEA_OK;
