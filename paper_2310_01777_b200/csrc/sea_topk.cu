@@ -84,25 +84,27 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
 
 // Selection with one thread per row, for short rows and small k_hat: no cross-lane traffic at
 // all.  Every thread walks its row (16-byte loads; a row is a few cache lines that the thread
-// reads front to back) in groups of KMAX keys and keeps the KMAX largest keys seen so far as a
-// descending list in registers: a group is sorted ascending by a bitonic network, the
+// reads front to back) in groups of KMAX values and keeps the KMAX largest values seen so far as
+// a descending list in registers: a group is sorted ascending by a bitonic network, the
 // element-wise maximum with the list is then a bitonic sequence holding the KMAX largest of
 // both, and a bitonic merge sorts it again - all compare-exchanges on fixed registers, no
-// branches.  That leaves the k_hat-th largest key tau in the last slot; a second walk over the
-// row emits, in ascending column order, the columns above tau and the first
-// k_hat - |{key > tau}| columns equal to it: the same set as the bit search below, ties going to
-// the lower column.
+// branches.  That leaves the k_hat-th largest value tau in the last slot; a second walk over
+// the row builds, 32 columns at a time, the bit masks of the columns above tau and equal to it,
+// keeps the first k_hat - |{value > tau}| of the equal ones, and emits the set bits in ascending
+// column order: the same set as the bit search below, ties going to the lower column.  The walk
+// works on the floats themselves: inputs are finite, and the float comparisons treat -0 and +0
+// as equal exactly as the bit search's keys do.
 constexpr int kThreadRows = 128;  // threads (= rows) per CTA
 
-// a[i] >= a[l] afterwards when kDescending, a[i] <= a[l] otherwise
+// x >= y afterwards when kDescending, x <= y otherwise
 template <bool kDescending>
-__device__ __forceinline__ void cmp_exchange(uint32_t& x, uint32_t& y) {
-  const uint32_t hi = max(x, y), lo = min(x, y);
+__device__ __forceinline__ void cmp_exchange(float& x, float& y) {
+  const float hi = fmaxf(x, y), lo = fminf(x, y);
   x = kDescending ? hi : lo;
   y = kDescending ? lo : hi;
 }
 template <int N>
-__device__ __forceinline__ void bitonic_sort_ascending(uint32_t (&a)[N]) {
+__device__ __forceinline__ void bitonic_sort_ascending(float (&a)[N]) {
 #pragma unroll
   for (int k = 2; k <= N; k <<= 1)
 #pragma unroll
@@ -117,7 +119,7 @@ __device__ __forceinline__ void bitonic_sort_ascending(uint32_t (&a)[N]) {
       }
 }
 template <int N>
-__device__ __forceinline__ void bitonic_merge_descending(uint32_t (&a)[N]) {
+__device__ __forceinline__ void bitonic_merge_descending(float (&a)[N]) {
 #pragma unroll
   for (int j = N >> 1; j > 0; j >>= 1)
 #pragma unroll
@@ -128,10 +130,10 @@ __device__ __forceinline__ void bitonic_merge_descending(uint32_t (&a)[N]) {
 }
 // top (descending) <- the KMAX largest of top and grp (any order; destroyed)
 template <int KMAX>
-__device__ __forceinline__ void merge_group(uint32_t (&top)[KMAX], uint32_t (&grp)[KMAX]) {
+__device__ __forceinline__ void merge_group(float (&top)[KMAX], float (&grp)[KMAX]) {
   bitonic_sort_ascending<KMAX>(grp);
 #pragma unroll
-  for (int s = 0; s < KMAX; ++s) top[s] = max(top[s], grp[s]);
+  for (int s = 0; s < KMAX; ++s) top[s] = fmaxf(top[s], grp[s]);
   bitonic_merge_descending<KMAX>(top);
 }
 
@@ -143,64 +145,78 @@ topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ s
   const int row = blockIdx.x * kThreadRows + threadIdx.x;
   if (row >= rows) return;
   const float* a = A_hat + (size_t)row * Kc;
-  // Descending list.  Its first KMAX - k_hat slots hold a sentinel above every real key, so the
-  // k_hat-th largest real key always ends up in the last slot; 0 sorts below every real key.
-  uint32_t top[KMAX];
+  // Descending list.  Its first KMAX - k_hat slots hold +inf, above every (finite) value, so the
+  // k_hat-th largest value of the row always ends up in the last slot; -inf stands for columns
+  // beyond the row.
+  float top[KMAX];
 #pragma unroll
-  for (int s = 0; s < KMAX; ++s) top[s] = s < KMAX - k_hat ? 0xffffffffu : 0u;
+  for (int s = 0; s < KMAX; ++s) top[s] = s < KMAX - k_hat ? INFINITY : -INFINITY;
   for (int j0 = 0; j0 < Kc; j0 += KMAX) {
-    uint32_t grp[KMAX];  // keys j0 .. j0 + KMAX - 1; beyond the row: 0
+    float grp[KMAX];
     if (kVec) {  // Kc % 4 == 0: rows start on 16-byte boundaries
 #pragma unroll
       for (int j = 0; j < KMAX; j += 4) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        const bool in = j0 + j < Kc;
-        if (in) v = __ldg(reinterpret_cast<const float4*>(a + j0 + j));
-        grp[j] = in ? order_key(v.x) : 0u;
-        grp[j + 1] = in ? order_key(v.y) : 0u;
-        grp[j + 2] = in ? order_key(v.z) : 0u;
-        grp[j + 3] = in ? order_key(v.w) : 0u;
+        float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (j0 + j < Kc) v = __ldg(reinterpret_cast<const float4*>(a + j0 + j));
+        grp[j] = v.x; grp[j + 1] = v.y; grp[j + 2] = v.z; grp[j + 3] = v.w;
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < KMAX; ++j) grp[j] = j0 + j < Kc ? order_key(__ldg(a + j0 + j)) : 0u;
+      for (int j = 0; j < KMAX; ++j) grp[j] = j0 + j < Kc ? __ldg(a + j0 + j) : -INFINITY;
     }
     merge_group<KMAX>(top, grp);
   }
-  const uint32_t tau = top[KMAX - 1];
+  const float tau = top[KMAX - 1];
   int n_gt = 0;
 #pragma unroll
-  for (int s = 0; s < KMAX; ++s) n_gt += (top[s] != 0xffffffffu && top[s] > tau);
-  const int need = k_hat - n_gt;  // how many columns equal to tau are taken (lowest first)
+  for (int s = 0; s < KMAX; ++s) n_gt += (top[s] != INFINITY && top[s] > tau);
+  int ties_left = k_hat - n_gt;  // how many columns equal to tau are still to be taken (lowest first)
 
   const int i = row % seq_len;
   const int words = (Kc + 31) / 32;
   int32_t* my_sel = sel + (size_t)row * k_hat;
-  int out = 0, tie_seen = 0, cnt = 0;
-  uint32_t word = 0u;
-  auto visit = [&](int j, float v) {
-    const uint32_t x = order_key(v);
-    const bool tie = x == tau;
-    const bool take = x > tau || (tie && tie_seen < need);
-    tie_seen += tie;
-    if (take) {
-      my_sel[out++] = j;
-      cnt += causal ? max(0, min(r, i + 1 - j * r)) : r;
-      word |= 1u << (j & 31);
-    }
-  };
+  int out = 0, cnt = 0;
   for (int j0 = 0; j0 < Kc; j0 += 32) {
-    const int j1 = min(Kc, j0 + 32);
+    uint32_t gt = 0u, eq = 0u;
     if (kVec) {
-      for (int j = j0; j < j1; j += 4) {
-        const float4 v = __ldg(reinterpret_cast<const float4*>(a + j));
-        visit(j, v.x); visit(j + 1, v.y); visit(j + 2, v.z); visit(j + 3, v.w);
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (j0 + j < Kc) v = __ldg(reinterpret_cast<const float4*>(a + j0 + j));
+        const float x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          gt |= (x[e] > tau ? 1u : 0u) << (j + e);
+          eq |= (x[e] == tau ? 1u : 0u) << (j + e);
+        }
       }
     } else {
-      for (int j = j0; j < j1; ++j) visit(j, __ldg(a + j));
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float x = j0 + j < Kc ? __ldg(a + j0 + j) : -INFINITY;
+        gt |= (x > tau ? 1u : 0u) << j;
+        eq |= (x == tau ? 1u : 0u) << j;
+      }
     }
+    // the lowest ties_left columns among the equal ones
+    uint32_t eq_taken = eq;
+    if (__popc(eq) > ties_left) {
+      eq_taken = 0u;
+      for (int t = 0; t < ties_left; ++t) {
+        const uint32_t low = eq & (0u - eq);
+        eq_taken |= low;
+        eq ^= low;
+      }
+    }
+    ties_left -= __popc(eq_taken);
+    uint32_t word = gt | eq_taken;
     if (mask_bits != nullptr) mask_bits[(size_t)row * words + (j0 >> 5)] = word;
-    word = 0u;
+    while (word) {
+      const int j = j0 + __ffs(word) - 1;
+      word &= word - 1u;
+      my_sel[out++] = j;
+      cnt += causal ? max(0, min(r, i + 1 - j * r)) : r;
+    }
   }
   if (row_counts != nullptr) row_counts[row] = cnt;
 }
