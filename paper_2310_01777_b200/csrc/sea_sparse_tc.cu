@@ -167,8 +167,12 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
 }
-__device__ __forceinline__ void tmem_ld_n(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld32(taddr, r); }
-__device__ __forceinline__ void tmem_ld_n(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld16(taddr, r); }
+template <int N>
+__device__ __forceinline__ void tmem_ld_n(uint32_t taddr, uint32_t (&r)[N]) {
+  static_assert(N == 16 || N == 32, "tensor-memory loads of 16 or 32 columns");
+  if constexpr (N == 32) tmem_ld32(taddr, r);
+  else tmem_ld16(taddr, r);
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
@@ -569,6 +573,51 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     const float cs = p.scale_log2;
     uint32_t s_it = 0, it_cnt = 0;
     bool ok = true;
+    struct {
+      bool active;
+      float inv;
+      int row, p_base, p_cnt;
+      uint32_t it_cnt;
+    } pend = {false, 0.f, 0, 0, 0, 0u};
+    // Output row of the pending item (this thread: 64 / kSplit of its columns), and the hand-over
+    // of the rows' normalisers to the warps that write P.
+    auto epilogue = [&]() -> bool {
+      if (!pend.active) return true;
+      pend.active = false;
+      const uint32_t ob = pend.it_cnt & 1, pslot = pend.it_cnt & 1;
+      bool good = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull + ob), (pend.it_cnt >> 1) & 1, abort_flag));
+      if (!good) return false;
+      tc_fence_after();
+      constexpr int kOC = 64 / kSplit;
+      uint32_t o[kOC];
+      tmem_ld_n(lane_addr + kColO + 64 * ob + kOC * part, o);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kBarOEmpty + ob));
+      uint4* out = reinterpret_cast<uint4*>(p.O + (size_t)pend.row * kHeadDim + kOC * part);
+#pragma unroll
+      for (int e = 0; e < kOC / 8; ++e) {
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(o[8 * e + 2 * k]) * pend.inv,
+                                                         __uint_as_float(o[8 * e + 2 * k + 1]) * pend.inv);
+          w[k] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        out[e] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      if (kWriteP && part == 0) {
+        good = __all_sync(0xffffffffu, mbar_wait(bar(kBarFixEmpty + pslot), ((pend.it_cnt >> 1) & 1) ^ 1, abort_flag));
+        if (!good) return false;
+        fix_inv[pslot * kTile + rt] = pend.inv;
+        fix_base[pslot * kTile + rt] = pend.p_base;
+        fix_cnt[pslot * kTile + rt] = pend.p_cnt;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kBarFixFull + pslot));
+      }
+      return true;
+    };
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it_cnt) {
       const Item it = decode_item(item, p);
       const int row = it.row0 + rt;
@@ -606,6 +655,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         if (lane == 0) mbar_arrive(bar(kBarSDone + b));
         ++s_it;
       }
+      if (ok) ok = epilogue();  // the previous item's output row
       xch[part * kTile + rt] = mx;
       ok = rows_all(ok);
       if (!ok) break;
@@ -655,42 +705,16 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
 #pragma unroll
       for (int q = 0; q < kSplit; ++q) l += xch_l[q * kTile + rt];
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      // ---- the item's output row (this thread: 64 / kSplit of its columns)
-      const uint32_t ob = it_cnt & 1;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull + ob), (it_cnt >> 1) & 1, abort_flag));
-      if (ok) {
-        tc_fence_after();
-        constexpr int kOC = 64 / kSplit;
-        uint32_t o[kOC];
-        tmem_ld_n(lane_addr + kColO + 64 * ob + kOC * part, o);
-        tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(kBarOEmpty + ob));
-        uint4* out = reinterpret_cast<uint4*>(p.O + (size_t)row * kHeadDim + kOC * part);
-#pragma unroll
-        for (int e = 0; e < kOC / 8; ++e) {
-          uint32_t w[4];
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(o[8 * e + 2 * k]) * inv, __uint_as_float(o[8 * e + 2 * k + 1]) * inv);
-            w[k] = *reinterpret_cast<const uint32_t*>(&h);
-          }
-          out[e] = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-        if (kWriteP && part == 0) {
-          // hand the rows' normalisers to the warps that write P
-          ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarFixEmpty + slot), ((it_cnt >> 1) & 1) ^ 1, abort_flag));
-          if (ok) {
-            fix_inv[slot * kTile + rt] = inv;
-            fix_base[slot * kTile + rt] = p_base;
-            fix_cnt[slot * kTile + rt] = p_cnt;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarFixFull + slot));
-          }
-        }
-      }
+      // the item's output row is written while the next item's first pass runs (by then the last
+      // P V product has long finished); remember what that needs
+      pend.active = true;
+      pend.inv = inv;
+      pend.row = row;
+      pend.it_cnt = it_cnt;
+      pend.p_base = p_base;
+      pend.p_cnt = p_cnt;
     }
+    if (ok) ok = epilogue();
   } else {
     // ---------------------------------------------------------------- P writers: 32 rows per warp
     reg_dec<kRegsFix>();
