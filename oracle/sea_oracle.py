@@ -20,6 +20,12 @@ the paper's steps in the paper's order:
     topk_select         Sec. 3.1 "Grouped Top-k Selection", per-query grouping:
                         the k_hat largest entries of each row of A_hat; equal
                         values go to the lower column.
+    topk_select_grouped Sec. 3.1 "Grouped Top-k Selection", causal-per-batch
+                        grouping: A_hat of one batch element is viewed as
+                        [T, H, Kc]; for every query position the H * k_hat
+                        largest of its H * Kc entries are kept (no exchange along
+                        T); equal values go to the lower flattened index
+                        h * Kc + c.  Heads then hold different numbers of columns.
     expand_mask         Sec. 3.1 "Linear Sparse Attention Mask Generation" and
                         App. "Sparse Interpolation": nearest-neighbour
                         up-sampling of the compressed mask done on indices; a
@@ -29,10 +35,14 @@ the paper's steps in the paper's order:
                         mask positions), sigma (softmax over a row's non-zeros),
                         then C = A* V.
     sea_attention_head  the four steps chained.
+    sea_attention_grouped_batch
+                        the same chain for one batch element with the
+                        causal-per-batch selection in place of the per-query one.
 
 Pins (tests/test_oracle_*.py): k_hat = Kc reproduces dense (causal) softmax
-attention from a library routine; top-k equals a brute-force ordering;
-expansion equals a library nearest-neighbour resize; the feature form equals
+attention from a library routine; top-k equals a brute-force ordering (the
+grouped form too: brute force over the flattened slab, H = 1 reduces to the
+per-query form, a head that dominates takes every slot); expansion equals a library nearest-neighbour resize; the feature form equals
 the normalised T x T kernel-matrix product and its expectation equals
 exp(q.k / sqrt(d)); rows of A* sum to one; causal outputs do not depend on
 later tokens.
@@ -51,6 +61,8 @@ __all__ = [
     "decode_estimate",
     "estimate_head",
     "topk_select",
+    "topk_select_grouped",
+    "sea_attention_grouped_batch",
     "expand_mask",
     "sparse_attention",
     "sea_attention_head",
@@ -123,16 +135,38 @@ def topk_select(A_hat, k_hat: int) -> np.ndarray:
     return sel
 
 
+def topk_select_grouped(A_hat, k_hat: int):
+    """Causal-per-batch selection over A_hat [H, T, Kc] of one batch element.
+
+    Returns ``cols[h][t]``: the ascending selected columns of head h at query t.
+    Over the heads every query keeps exactly H * k_hat columns.
+    """
+    A_hat = _f64(A_hat)
+    H, T, Kc = A_hat.shape
+    if not 1 <= k_hat <= Kc:
+        raise ValueError("k_hat out of range")
+    cols = [[None] * T for _ in range(H)]
+    for t in range(T):
+        slab = A_hat[:, t, :].reshape(H * Kc)  # flattened index h * Kc + c
+        order = np.argsort(-slab, kind="stable")[: H * k_hat]
+        taken = np.zeros(H * Kc, dtype=bool)
+        taken[order] = True
+        taken = taken.reshape(H, Kc)
+        for h in range(H):
+            cols[h][t] = np.flatnonzero(taken[h])
+    return cols
+
+
 def expand_mask(sel, T: int, Kc: int, causal: bool, query_index=None):
     """Flat CSR (row_ptr [n+1], col_idx [nnz]) of the up-sampled mask of one head.
 
-    Row t of ``sel`` belongs to query ``query_index[t]`` (default: t, all T queries).
+    Row t of ``sel`` (an array [n, k_hat], or a list of n column arrays of any
+    lengths) belongs to query ``query_index[t]`` (default: t, all T queries).
     """
-    sel = np.asarray(sel)
     if T % Kc != 0:
         raise ValueError("T must be a multiple of Kc")
     r = T // Kc
-    n = sel.shape[0]
+    n = len(sel)
     if query_index is None:
         query_index = np.arange(n)
     row_ptr = np.zeros(n + 1, dtype=np.int64)
@@ -181,6 +215,25 @@ def sea_attention_head(Q, K, V, k_hat: int, Kc: int, causal: bool, scale: float,
     return dict(A_hat=_f64(A_hat), sel=sel, row_ptr=row_ptr, col_idx=col_idx, O=O, P=P)
 
 
+def sea_attention_grouped_batch(Q, K, V, k_hat: int, Kc: int, causal: bool, scale: float,
+                                A_hat=None, omega=None, W_dec=None):
+    """All stages for one batch element (arrays [H, T, .]) with the causal-per-batch selection.
+
+    Returns the list over heads of dicts with A_hat, cols, row_ptr, col_idx, O, P.
+    """
+    Q, K, V = np.asarray(Q), np.asarray(K), np.asarray(V)
+    H, T = Q.shape[0], Q.shape[1]
+    if A_hat is None:
+        A_hat = np.stack([estimate_head(Q[h], K[h], V[h], omega, W_dec, causal) for h in range(H)])
+    cols = topk_select_grouped(A_hat, k_hat)
+    out = []
+    for h in range(H):
+        row_ptr, col_idx = expand_mask(cols[h], T, Kc, causal)
+        O, P = sparse_attention(Q[h], K[h], V[h], row_ptr, col_idx, scale)
+        out.append(dict(A_hat=_f64(A_hat[h]), cols=cols[h], row_ptr=row_ptr, col_idx=col_idx, O=O, P=P))
+    return out
+
+
 def flatten_heads(per_head, T: int):
     """Join per-head results in flat row order ((b*H + h)*T + i).
 
@@ -196,7 +249,7 @@ def flatten_heads(per_head, T: int):
         row_ptr=np.concatenate(row_ptr),
         col_idx=np.concatenate([r["col_idx"] for r in per_head]),
         P=np.concatenate([r["P"] for r in per_head]),
-        sel=np.concatenate([r["sel"] for r in per_head], axis=0),
+        sel=np.concatenate([r["sel"] for r in per_head], axis=0) if "sel" in per_head[0] else None,
         O=np.concatenate([r["O"] for r in per_head], axis=0),
         A_hat=np.concatenate([r["A_hat"] for r in per_head], axis=0),
     )
