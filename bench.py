@@ -18,6 +18,8 @@ metric is quoted.  One JSON line is printed by rank 0.
              against the measured dense bf16 peak.
   stages     per-stage milliseconds from a second pass that calls the three stage entry points
              with events between them (same kernels as the fused call).
+  grouped    the same step with the causal-per-batch grouping (sea_attention_grouped) on this
+             rank, and its selection and sparse stages; per-rank, not part of `value`.
   cpu_baseline  the fp64 oracle on a bounded sample of heads, on this machine's host cores.
 
 With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no
@@ -290,6 +292,45 @@ def main():
     if not torch.equal(hO, O.cpu()):
         raise SystemExit("host entry point and device entry point disagree")
 
+    # ---- timed region 4: the causal-per-batch grouping (fused call, then its stages) ----
+    grouped = None
+    if w.Kc % 4 == 0 and w.H * w.Kc <= 32768:
+        bits = torch.empty((w.rows, (w.Kc + 31) // 32), dtype=torch.int32, device=dev)
+
+        def gstep():
+            sea.sea_attention_grouped(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O, ws, A_hat=A_hat,
+                                      mask_bits=bits, row_ptr=row_ptr, col_idx=col_idx, P=P)
+
+        for _ in range(3):
+            flush.zero_()
+            gstep()
+        g_launches = sea.sea_last_launch_count()
+        gev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        torch.cuda.synchronize(dev)
+        for a, b in gev:
+            flush.zero_()
+            a.record()
+            gstep()
+            b.record()
+        torch.cuda.synchronize(dev)
+        g_ms = sum(a.elapsed_time(b) for a, b in gev) / args.steps
+        gsev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        for e in gsev:
+            flush.zero_()
+            e[0].record()
+            sea.sea_topk_mask_grouped(shape, A_hat, bits, row_ptr, col_idx, ws)
+            e[1].record()
+            sea.sea_sparse_attn_masked(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, bits, O, P, ws)
+            e[2].record()
+        torch.cuda.synchronize(dev)
+        if sea.sea_device_status(ws) != 0:
+            raise SystemExit("device status word set by the grouped path")
+        grouped = {"grouping": "causal-per-batch", "ms_per_step": g_ms, "value": w.B * w.T / (g_ms / 1e3),
+                   "unit": "tokens/s", "gpu_launches_per_step": g_launches,
+                   "stages_ms": {"topk_mask_grouped": sum(e[0].elapsed_time(e[1]) for e in gsev) / args.steps,
+                                 "sparse_attn_masked": sum(e[1].elapsed_time(e[2]) for e in gsev) / args.steps},
+                   "nnz": int(row_ptr[-1])}
+
     ms_per_step = total_ms / args.steps
     if world > 1:
         t = torch.tensor([ms_per_step, e2e_ms], device=dev, dtype=torch.float64)
@@ -324,6 +365,7 @@ def main():
             "clocks": clocks,
             "stages_ms": {"estimate": stage_ms[0], "topk_mask": stage_ms[1], "sparse_attn": stage_ms[2]},
             "nnz": nnz,
+            "grouped": grouped,
             "roofline": {"kernel": "sparse_attn_tiles_tc_kernel" if tiled else "sparse_attn_blocks_tma_kernel",
                          "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_source": f"{peak_kind} HBM copy bandwidth",

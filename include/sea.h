@@ -162,6 +162,51 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
                          void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Causal-per-batch grouping, Sec. 3.1 "Grouped Top-k Selection" (the grouping the
+ * paper recommends and measures with, App. "FlatCSR").  A_hat of a batch element is
+ * viewed as [T, H, Kc]; for every query position t the H*k_hat largest of the H*Kc
+ * entries A_hat[b, :, t, :] are selected, with no exchange along T.  Equal values
+ * (including -0 and +0) go to the lower flattened index h*Kc + c.  A row (b, h, t)
+ * therefore keeps between 0 and min(Kc, H*k_hat) columns, and every (b, t) keeps
+ * exactly H*k_hat over its heads.  Requires Kc % 4 == 0 and H*Kc <= 32768.
+ *
+ * mask_bits [rows, ceil(Kc/32)] uint32 receives the selection (bit c%32 of word
+ * c/32 of a row is set when column c is kept; may be NULL).  The up-sampling and the
+ * CSR are those of sea_topk_mask, with rows in the same flat order (b*H + h)*T + t:
+ * where the paper stores one row per (b, t) over the flattened (head, key) axis and
+ * transposes inside its kernels, the rows here are already per head.  nnz_cap
+ * rows*k_hat*r always suffices.  col_idx may be NULL.
+ */
+sea_status sea_topk_mask_grouped(const sea_shape* shape, const float* A_hat, uint32_t* mask_bits,
+                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                                 void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * sea_sparse_attn for a mask given as bits (the output of sea_topk_mask_grouped, or
+ * any selection of compressed columns in that layout) together with its row_ptr.
+ * col_idx may be NULL when the shape allows the tile kernel (bf16, T % 128 == 0,
+ * r = T/Kc a power of two >= 4, full workspace); otherwise it is required and
+ * SEA_ERR_INVALID_ARG is returned without it.  When P is requested, no (b, t) may
+ * keep more than H*k_hat columns over its heads: rows beyond that budget are
+ * reported through SEA_DEV_ROW_OVERFLOW and their P entries are not written.
+ */
+sea_status sea_sparse_attn_masked(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                                  const int32_t* row_ptr, const int32_t* col_idx,
+                                  const uint32_t* mask_bits, void* O, void* P,
+                                  void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * The whole layer with the causal-per-batch grouping:
+ * sea_estimate -> sea_topk_mask_grouped -> sea_sparse_attn_masked on one stream.
+ * Optional outputs and A_hat_in as for sea_attention.
+ */
+sea_status sea_attention_grouped(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                                 const float* omega, const float* W_dec, const float* A_hat_in,
+                                 void* O, float* A_hat, uint32_t* mask_bits, int32_t* row_ptr,
+                                 int32_t* col_idx, int64_t nnz_cap, void* P,
+                                 void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * sea_attention for callers whose tensors live in HOST memory (pinned memory
  * gives asynchronous copies).  hQ, hK, hV, homega, hW_dec are copied to staging
  * areas inside `ws` on the stream, the layer runs, and O is copied back to hO.

@@ -50,6 +50,7 @@ WsLayout ws_layout(const sea_shape& s) {
   L.row_ptr = take((rows + 1) * sizeof(int32_t));
   L.mask_bits = take(sparse_attn_tc_bits_bytes(s));
   L.p_scratch = take(s.io == SEA_BF16 ? sparse_attn_tc_scratch_bytes(s) : 0);
+  L.park_off = take(s.io == SEA_BF16 ? rows * sizeof(int32_t) : 0);
   L.total = off;
   return L;
 }
@@ -172,6 +173,97 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
   if (rc != SEA_OK) return rc;
   return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P, bits, true,
                             reinterpret_cast<float*>(w + L.p_scratch), status, st);
+}
+
+sea_status sea_topk_mask_grouped(const sea_shape* shape, const float* A_hat, uint32_t* mask_bits,
+                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* ws,
+                                 size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  const sea_status rc = validate_shape(shape, false);
+  if (rc != SEA_OK) return rc;
+  if (!topk_grouped_supported(*shape)) return SEA_ERR_UNSUPPORTED;
+  if (!A_hat || !row_ptr || !ws) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(A_hat) || !aligned16(row_ptr) || !aligned16(ws) || (mask_bits && !aligned16(mask_bits)) ||
+      (col_idx && !aligned16(col_idx)))
+    return SEA_ERR_INVALID_ARG;
+  if (col_idx && nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
+  if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  const WsLayout L = ws_layout(*shape);
+  if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  uint32_t* bits = mask_bits ? mask_bits : reinterpret_cast<uint32_t*>(w + L.mask_bits);
+  return launch_topk_mask_grouped(*shape, A_hat, bits, row_ptr, col_idx, nnz_cap,
+                                  reinterpret_cast<int32_t*>(w + L.row_counts),
+                                  reinterpret_cast<int32_t*>(w + L.tile_sums),
+                                  reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
+}
+
+sea_status sea_sparse_attn_masked(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                                  const int32_t* row_ptr, const int32_t* col_idx, const uint32_t* mask_bits,
+                                  void* O, void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  const sea_status rc = validate_shape(shape, false);
+  if (rc != SEA_OK) return rc;
+  if (!Q || !K || !V || !row_ptr || !O || !mask_bits) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(row_ptr) ||
+      !aligned16(mask_bits) || (P && !aligned16(P)) || (col_idx && !aligned16(col_idx)))
+    return SEA_ERR_INVALID_ARG;
+  if (ws && !aligned16(ws)) return SEA_ERR_INVALID_ARG;
+  if (ws && ws_bytes < (size_t)kStatusBytes) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  const WsLayout L = ws_layout(*shape);
+  const bool full = ws && ws_bytes >= L.total && shape->io == SEA_BF16;
+  return launch_sparse_attn_masked(*shape, Q, K, V, row_ptr, col_idx, mask_bits, O, P,
+                                   full ? reinterpret_cast<int32_t*>(w + L.park_off) : nullptr,
+                                   full ? reinterpret_cast<float*>(w + L.p_scratch) : nullptr,
+                                   static_cast<int32_t*>(ws), static_cast<cudaStream_t>(cuda_stream));
+}
+
+sea_status sea_attention_grouped(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                                 const float* omega, const float* W_dec, const float* A_hat_in, void* O,
+                                 float* A_hat, uint32_t* mask_bits, int32_t* row_ptr, int32_t* col_idx,
+                                 int64_t nnz_cap, void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  const bool estimate = A_hat_in == nullptr;
+  sea_status rc = validate_shape(shape, estimate);
+  if (rc != SEA_OK) return rc;
+  if (!topk_grouped_supported(*shape)) return SEA_ERR_UNSUPPORTED;
+  if (!Q || !K || !V || !O || !ws) return SEA_ERR_INVALID_ARG;
+  if (estimate && (!omega || !W_dec)) return SEA_ERR_INVALID_ARG;
+  if (P && !col_idx) return SEA_ERR_INVALID_ARG;  // probabilities are only meaningful beside their indices
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(ws) ||
+      (omega && !aligned16(omega)) || (W_dec && !aligned16(W_dec)) || (A_hat_in && !aligned16(A_hat_in)) ||
+      (A_hat && !aligned16(A_hat)) || (mask_bits && !aligned16(mask_bits)) || (row_ptr && !aligned16(row_ptr)) ||
+      (col_idx && !aligned16(col_idx)) || (P && !aligned16(P)))
+    return SEA_ERR_INVALID_ARG;
+  if (col_idx && nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
+  if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  const WsLayout L = ws_layout(*shape);
+  if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
+  // without col_idx the sparse stage must be able to work from the bits alone
+  uint32_t* bits = mask_bits ? mask_bits : reinterpret_cast<uint32_t*>(w + L.mask_bits);
+  float* scratch = shape->io == SEA_BF16 ? reinterpret_cast<float*>(w + L.p_scratch) : nullptr;
+  int32_t* park = shape->io == SEA_BF16 ? reinterpret_cast<int32_t*>(w + L.park_off) : nullptr;
+  if (!col_idx && !(park && sparse_attn_tc_applicable(*shape, nullptr, true, status, bits, scratch)))
+    return SEA_ERR_INVALID_ARG;
+
+  const float* a_use = A_hat_in;
+  if (estimate) {
+    float* a_out = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
+    rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state),
+                         w + L.est_split, status, st);
+    if (rc != SEA_OK) return rc;
+    a_use = a_out;
+  }
+  int32_t* rp_buf = row_ptr ? row_ptr : reinterpret_cast<int32_t*>(w + L.row_ptr);
+  rc = launch_topk_mask_grouped(*shape, a_use, bits, rp_buf, col_idx, nnz_cap,
+                                reinterpret_cast<int32_t*>(w + L.row_counts),
+                                reinterpret_cast<int32_t*>(w + L.tile_sums), status, st);
+  if (rc != SEA_OK) return rc;
+  return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, scratch, status, st);
 }
 
 sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes) {

@@ -34,6 +34,7 @@ struct WsLayout {
   size_t row_ptr;     // int32 [rows+1]
   size_t mask_bits;   // uint32 [rows][ceil(Kc/32)]   selected columns as bits (tensor-core sparse stage)
   size_t p_scratch;   // float [rows][k_hat*r]        unnormalised probabilities (tensor-core sparse stage)
+  size_t park_off;    // int32 [rows]                 offsets into p_scratch (masks with rows of differing lengths)
   size_t total;
 };
 
@@ -58,6 +59,24 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
                             int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
                             int32_t* row_counts, int32_t* tile_sums, uint32_t* mask_bits,
                             int32_t* status, cudaStream_t st);
+sea_status launch_row_ptr_scan(const int32_t* row_counts, int32_t* tile_sums, int32_t* row_ptr, int rows,
+                               cudaStream_t st);
+// Causal-per-batch grouping (sea_topk_grouped.cu).  mask_bits is written in full.
+bool topk_grouped_supported(const sea_shape& s);
+sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint32_t* mask_bits,
+                                    int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                                    int32_t* row_counts, int32_t* tile_sums, int32_t* status,
+                                    cudaStream_t st);
+// Where each row parks its unnormalised probabilities when rows keep differing numbers of columns:
+// the (b, t) slabs of H*k_hat*r floats follow one another, the heads inside a slab.  Rows of a slab
+// that keeps more than H*k_hat columns get -1 and SEA_DEV_ROW_OVERFLOW is raised.
+sea_status launch_park_offsets(const sea_shape& s, const uint32_t* mask_bits, int32_t* park_off,
+                               int32_t* status, cudaStream_t st);
+// Sparse stage for a mask given as bits with its row_ptr (rows of any length).
+sea_status launch_sparse_attn_masked(const sea_shape& s, const void* Q, const void* K, const void* V,
+                                     const int32_t* row_ptr, const int32_t* col_idx,
+                                     const uint32_t* mask_bits, void* O, void* P, int32_t* park_off,
+                                     float* p_scratch, int32_t* status, cudaStream_t st);
 // mask_bits and p_scratch (workspace areas of the tensor-core kernel) may be null: the per-row
 // kernels are used then.  bits_valid: mask_bits already holds the bit strings of `sel`
 // (launch_topk_mask wrote them); otherwise they are derived from `sel` first.
@@ -65,14 +84,19 @@ sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, 
                               const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
                               void* O, void* P, uint32_t* mask_bits, bool bits_valid, float* p_scratch,
                               int32_t* status, cudaStream_t st);
+sea_status launch_sparse_attn_rows(const sea_shape& s, const void* Q, const void* K, const void* V,
+                                   const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
+                                   void* O, void* P, cudaStream_t st);
 size_t sparse_attn_tc_bits_bytes(const sea_shape& s);
 size_t sparse_attn_tc_scratch_bytes(const sea_shape& s);
-bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, const int32_t* status,
+// have_bits: mask_bits already holds the mask (sel may then be null)
+bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, bool have_bits, const int32_t* status,
                                const void* mask_bits, const void* p_scratch);
+// park_off: per-row offsets into p_scratch (null: row * k_hat * r, the per-query layout)
 sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* K, const void* V,
                                  const int32_t* row_ptr, const int32_t* sel, void* O, void* P,
-                                 uint32_t* mask_bits, bool bits_valid, float* p_scratch, int32_t* status,
-                                 cudaStream_t st);
+                                 uint32_t* mask_bits, bool bits_valid, float* p_scratch,
+                                 const int32_t* park_off, int32_t* status, cudaStream_t st);
 bool sparse_attn_tma_applicable(const sea_shape& s, const int32_t* sel, const int32_t* status);
 sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void* K, const void* V,
                                   const int32_t* row_ptr, const int32_t* sel, void* O, void* P,
@@ -129,6 +153,13 @@ struct Io<__nv_bfloat16> {
   __device__ static __nv_bfloat16 to_io(float x) { return __float2bfloat16_rn(x); }
   __device__ static float from_io(__nv_bfloat16 x) { return __bfloat162float(x); }
 };
+
+// 32-bit key whose unsigned order is the float order, with -0 folded onto +0.
+__device__ __forceinline__ uint32_t order_key(float v) {
+  uint32_t u = __float_as_uint(v);
+  if (u == 0x80000000u) u = 0u;  // -0 ties with +0
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll

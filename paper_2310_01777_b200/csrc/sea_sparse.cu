@@ -371,10 +371,34 @@ sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, 
                               const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
                               void* O, void* P, uint32_t* mask_bits, bool bits_valid, float* p_scratch,
                               int32_t* status, cudaStream_t st) {
-  if (sparse_attn_tc_applicable(s, sel, status, mask_bits, p_scratch))
-    return launch_sparse_attn_tc(s, Q, K, V, row_ptr, sel, O, P, mask_bits, bits_valid, p_scratch, status, st);
+  if (sparse_attn_tc_applicable(s, sel, false, status, mask_bits, p_scratch))
+    return launch_sparse_attn_tc(s, Q, K, V, row_ptr, sel, O, P, mask_bits, bits_valid, p_scratch, nullptr, status, st);
   if (sparse_attn_tma_applicable(s, sel, status))
     return launch_sparse_attn_tma(s, Q, K, V, row_ptr, sel, O, P, status, st);
+  return launch_sparse_attn_rows(s, Q, K, V, row_ptr, col_idx, sel, O, P, st);
+}
+
+sea_status launch_sparse_attn_masked(const sea_shape& s, const void* Q, const void* K, const void* V,
+                                     const int32_t* row_ptr, const int32_t* col_idx, const uint32_t* mask_bits,
+                                     void* O, void* P, int32_t* park_off, float* p_scratch, int32_t* status,
+                                     cudaStream_t st) {
+  if (park_off != nullptr && sparse_attn_tc_applicable(s, nullptr, true, status, mask_bits, p_scratch)) {
+    if (P != nullptr) {
+      const sea_status rc = launch_park_offsets(s, mask_bits, park_off, status, st);
+      if (rc != SEA_OK) return rc;
+    }
+    // the bits are only read: bits_valid keeps the launcher from deriving them from a selection list
+    return launch_sparse_attn_tc(s, Q, K, V, row_ptr, nullptr, O, P, const_cast<uint32_t*>(mask_bits), true, p_scratch,
+                                 P != nullptr ? park_off : nullptr, status, st);
+  }
+  if (col_idx == nullptr) return SEA_ERR_INVALID_ARG;
+  return launch_sparse_attn_rows(s, Q, K, V, row_ptr, col_idx, nullptr, O, P, st);
+}
+
+// The per-row kernels: any CSR, rows of any length.
+sea_status launch_sparse_attn_rows(const sea_shape& s, const void* Q, const void* K, const void* V,
+                                   const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel, void* O,
+                                   void* P, cudaStream_t st) {
   if (s.io == SEA_BF16) {
     using T = __nv_bfloat16;
     const int rows = s.B * s.H * s.T;

@@ -241,7 +241,8 @@ struct TcParams {
   const uint32_t* mask_bits;    // [rows][words] one bit per compressed column
   __nv_bfloat16* O;
   __nv_bfloat16* P;
-  float* p_scratch;             // [rows][k_hat * r] unnormalised probabilities of kept keys
+  float* p_scratch;             // unnormalised probabilities of kept keys: row `row` parks its runs at
+  const int32_t* park_off;      // park_off[row] (negative: nowhere), or at row * k_hat * r when this is null
   int32_t* status;
   int BH, T, words, log2r, k_hat, causal;
   float scale_log2;
@@ -320,7 +321,7 @@ __device__ __forceinline__ float chunk_max(const uint32_t (&v)[32], uint32_t tb,
 template <int L, bool kDiag, bool kWriteP>
 __device__ __forceinline__ void chunk_probs(const uint32_t (&v)[32], uint32_t tb, int cg, int lim, float cs,
                                             float neg_mc, float2& la, float2& lb, uint32_t (&hi)[16],
-                                            uint32_t (&lo)[16], float* my_scratch, int rank_base, int off0) {
+                                            uint32_t (&lo)[16], float* my_scratch, bool park, int rank_base, int off0) {
   constexpr int R = 1 << (L < 5 ? L : 5);  // columns of this chunk per group
   const float2 cs2 = make_float2(cs, cs);
   const float2 m1 = make_float2(-1.f, -1.f);
@@ -350,7 +351,7 @@ __device__ __forceinline__ void chunk_probs(const uint32_t (&v)[32], uint32_t tb
       lo[e2] = *reinterpret_cast<const uint32_t*>(&l2);
       if (kWriteP) {
         if (e2 & 1) {
-          if (live) dst[(e2 - gi * R / 2) >> 1] = make_float4(prev.x, prev.y, pp.x, pp.y);
+          if (live && park) dst[(e2 - gi * R / 2) >> 1] = make_float4(prev.x, prev.y, pp.x, pp.y);
         } else {
           prev = pp;
         }
@@ -396,7 +397,8 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
   float* fix_inv = xch_l + kSplit * kTile;                                      // [2 slots][128]
   int* fix_base = reinterpret_cast<int*>(fix_inv + 2 * kTile);           // [2][128]
   int* fix_cnt = fix_base + 2 * kTile;                                   // [2][128]
-  uint32_t* bits = reinterpret_cast<uint32_t*>(fix_cnt + 2 * kTile);     // [2 slots][128 rows][words]
+  int* fix_off = fix_cnt + 2 * kTile;                                    // [2][128]
+  uint32_t* bits = reinterpret_cast<uint32_t*>(fix_off + 2 * kTile);     // [2 slots][128 rows][words]
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -576,9 +578,9 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     struct {
       bool active;
       float inv;
-      int row, p_base, p_cnt;
+      int row, p_base, p_cnt, p_off;
       uint32_t it_cnt;
-    } pend = {false, 0.f, 0, 0, 0, 0u};
+    } pend = {false, 0.f, 0, 0, 0, 0, 0u};
     // Output row of the pending item (this thread: 64 / kSplit of its columns), and the hand-over
     // of the rows' normalisers to the warps that write P.
     auto epilogue = [&]() -> bool {
@@ -613,6 +615,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         fix_inv[pslot * kTile + rt] = pend.inv;
         fix_base[pslot * kTile + rt] = pend.p_base;
         fix_cnt[pslot * kTile + rt] = pend.p_cnt;
+        fix_off[pslot * kTile + rt] = pend.p_off;
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kBarFixFull + pslot));
       }
@@ -622,10 +625,18 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       const Item it = decode_item(item, p);
       const int row = it.row0 + rt;
       const uint32_t slot = it_cnt & 1;
-      int p_base = 0, p_cnt = 0;
-      if (kWriteP && part == 0) {
-        p_base = __ldg(p.row_ptr + row);
-        p_cnt = __ldg(p.row_ptr + row + 1) - p_base;
+      int p_base = 0, p_cnt = 0, p_off = 0;
+      bool park = kWriteP;
+      if (kWriteP) {
+        p_off = p.park_off != nullptr ? __ldg(p.park_off + row) : row * KR;
+        if (p_off < 0) {  // the row has no place in the parking area: its P entries are not produced
+          park = false;
+          p_off = 0;
+        }
+        if (part == 0 && park) {
+          p_base = __ldg(p.row_ptr + row);
+          p_cnt = __ldg(p.row_ptr + row + 1) - p_base;
+        }
       }
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarBitsFull + slot), (it_cnt >> 1) & 1, abort_flag));
       const uint32_t* my_bits = bits + slot * (kTile * p.words) + rt * p.words;
@@ -663,7 +674,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       for (int q = 0; q < kSplit; ++q) mx = fmaxf(mx, xch[q * kTile + rt]);
       if (mx == -INFINITY) mx = 0.f;  // a row that keeps no key: every probability is zero below
       const float neg_mc = -mx * cs;
-      float* my_scratch = kWriteP ? p.p_scratch + (size_t)row * KR : nullptr;
+      float* my_scratch = kWriteP ? p.p_scratch + p_off : nullptr;
       // ---- second pass: probabilities, row sum, P into tensor memory
       float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
       int rank_base = 0;
@@ -684,8 +695,8 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         for (int c = 0; c < kChunks; ++c) {
           uint32_t hi[16], lo[16];
           const int cg = kChunks * part + c;
-          if (diag) chunk_probs<L, true, kWriteP>(v[c], tb, cg, rt - 32 * cg, cs, neg_mc, la, lb, hi, lo, my_scratch, rank_base, off0);
-          else chunk_probs<L, false, kWriteP>(v[c], tb, cg, 0, cs, neg_mc, la, lb, hi, lo, my_scratch, rank_base, off0);
+          if (diag) chunk_probs<L, true, kWriteP>(v[c], tb, cg, rt - 32 * cg, cs, neg_mc, la, lb, hi, lo, my_scratch, park, rank_base, off0);
+          else chunk_probs<L, false, kWriteP>(v[c], tb, cg, 0, cs, neg_mc, la, lb, hi, lo, my_scratch, park, rank_base, off0);
           tmem_st16(src + 32 * c, hi);
           tmem_st16(src + 32 * c + 16, lo);
         }
@@ -713,6 +724,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       pend.it_cnt = it_cnt;
       pend.p_base = p_base;
       pend.p_cnt = p_cnt;
+      pend.p_off = p_off;
     }
     if (ok) ok = epilogue();
   } else {
@@ -720,11 +732,9 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     reg_dec<kRegsFix>();
     if (kWriteP) {
       const int w4 = warp - (4 + kRowWarps);
-      const int KR = p.k_hat << p.log2r;
       uint32_t it_cnt = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it_cnt) {
-        const Item it = decode_item(item, p);
         const uint32_t slot = it_cnt & 1;
         ok = __all_sync(0xffffffffu, mbar_wait<500>(bar(kBarFixFull + slot), (it_cnt >> 1) & 1, abort_flag));
         if (!ok) break;
@@ -733,8 +743,9 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         const int* cnt_s = fix_cnt + slot * kTile + 32 * w4;
         const int* base_s = fix_base + slot * kTile + 32 * w4;
         const float* inv_s = fix_inv + slot * kTile + 32 * w4;
-        const float* src0 = p.p_scratch + (size_t)(it.row0 + 32 * w4) * KR;
-        for (int u0 = 0; u0 < KR; u0 += 128) {
+        const int* off_s = fix_off + slot * kTile + 32 * w4;
+        const int longest_all = __reduce_max_sync(0xffffffffu, cnt_s[lane]);
+        for (int u0 = 0; u0 < longest_all; u0 += 128) {
           const int u = u0 + 4 * lane;
           for (int r0 = 0; r0 < 32; r0 += 8) {
             int longest = 0;
@@ -744,7 +755,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
             float4 val[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-              val[j] = u < cnt_s[r0 + j] ? __ldcg(reinterpret_cast<const float4*>(src0 + (size_t)(r0 + j) * KR + u))
+              val[j] = u < cnt_s[r0 + j] ? __ldcg(reinterpret_cast<const float4*>(p.p_scratch + off_s[r0 + j] + u))
                                          : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -836,7 +847,7 @@ int log2_exact(int x) {
 template <int L, bool kWriteP>
 sea_status launch_tc(const sea_shape& s, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                      const TcParams& prm, cudaStream_t st) {
-  const size_t smem = 1024 + (size_t)(2 + kNK + kNV) * kTileBytes + 8 * kNumBars + 8 + (size_t)(2 * kSplit + 6) * kTile * 4 +
+  const size_t smem = 1024 + (size_t)(2 + kNK + kNV) * kTileBytes + 8 * kNumBars + 8 + (size_t)(2 * kSplit + 8) * kTile * 4 +
                       2 * (size_t)prm.words * kTile * 4;
   auto kern = sparse_attn_tiles_tc_kernel<L, kWriteP>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SEA_ERR_CUDA;
@@ -858,9 +869,10 @@ size_t sparse_attn_tc_scratch_bytes(const sea_shape& s) {
   return (size_t)s.B * s.H * s.T * (size_t)s.k_hat * (size_t)(s.T / s.Kc) * sizeof(float);
 }
 
-bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, const int32_t* status, const void* mask_bits,
-                               const void* p_scratch) {
-  if (s.io != SEA_BF16 || sel == nullptr || status == nullptr || mask_bits == nullptr || p_scratch == nullptr) return false;
+bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, bool have_bits, const int32_t* status,
+                               const void* mask_bits, const void* p_scratch) {
+  if (s.io != SEA_BF16 || (sel == nullptr && !have_bits) || status == nullptr || mask_bits == nullptr || p_scratch == nullptr)
+    return false;
   const int r = s.T / s.Kc;
   if (s.T % kTile != 0 || log2_exact(r) < 2) return false;
   // dense tiles pay off while a row keeps at least about 1 % of the keys it may see
@@ -870,7 +882,7 @@ bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, const int
 
 sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* K, const void* V, const int32_t* row_ptr,
                                  const int32_t* sel, void* O, void* P, uint32_t* mask_bits, bool bits_valid,
-                                 float* p_scratch, int32_t* status, cudaStream_t st) {
+                                 float* p_scratch, const int32_t* park_off, int32_t* status, cudaStream_t st) {
   const unsigned long long rows = (unsigned long long)s.B * s.H * s.T;
   CUtensorMap mq, mk, mv;
   if (!make_tile_map(&mq, Q, rows) || !make_tile_map(&mk, K, rows) || !make_tile_map(&mv, V, rows)) return SEA_ERR_CUDA;
@@ -881,6 +893,7 @@ sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* 
   prm.O = static_cast<__nv_bfloat16*>(O);
   prm.P = static_cast<__nv_bfloat16*>(P);
   prm.p_scratch = p_scratch;
+  prm.park_off = park_off;
   prm.status = status;
   prm.BH = s.B * s.H;
   prm.T = s.T;

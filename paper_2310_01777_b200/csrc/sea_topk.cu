@@ -18,12 +18,6 @@ constexpr int kScanTile = kScanThreads * kScanPerThread;
 constexpr int kThreadMaxKc = 128;  // shapes handled with one thread per row: the sorted-list walk costs
 constexpr int kThreadMaxK = 32;    // Kc * k_hat min/max pairs per row, the bit search about 64 * Kc / 32 * 32
 
-__device__ __forceinline__ uint32_t order_key(float v) {
-  uint32_t u = __float_as_uint(v);
-  if (u == 0x80000000u) u = 0u;  // -0 ties with +0
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
 // One warp per row; lane l holds columns l, l+32, ... (VPL of them).
 template <int VPL>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
@@ -342,6 +336,19 @@ void launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, uint32_t* ma
 
 }  // namespace
 
+// row_ptr = exclusive prefix sums of the per-row counts, row_ptr[rows] = their total.
+sea_status launch_row_ptr_scan(const int32_t* row_counts, int32_t* tile_sums, int32_t* row_ptr, int rows,
+                               cudaStream_t st) {
+  sea_status rc;
+  const int ntiles = (rows + kScanTile - 1) / kScanTile;
+  scan_tile_sums_kernel<<<ntiles, kScanThreads, 0, st>>>(row_counts, tile_sums, rows);
+  if ((rc = check_launch()) != SEA_OK) return rc;
+  scan_tile_offsets_kernel<<<1, 1024, 0, st>>>(tile_sums, ntiles);
+  if ((rc = check_launch()) != SEA_OK) return rc;
+  scan_write_row_ptr_kernel<<<ntiles, kScanThreads, 0, st>>>(row_counts, tile_sums, row_ptr, rows);
+  return check_launch();
+}
+
 sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel, int32_t* row_ptr,
                             int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts,
                             int32_t* tile_sums, uint32_t* mask_bits, int32_t* status, cudaStream_t st) {
@@ -378,13 +385,7 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
   if (rc != SEA_OK) return rc;
 
   if (s.causal) {
-    const int ntiles = (rows + kScanTile - 1) / kScanTile;
-    scan_tile_sums_kernel<<<ntiles, kScanThreads, 0, st>>>(row_counts, tile_sums, rows);
-    if ((rc = check_launch()) != SEA_OK) return rc;
-    scan_tile_offsets_kernel<<<1, 1024, 0, st>>>(tile_sums, ntiles);
-    if ((rc = check_launch()) != SEA_OK) return rc;
-    scan_write_row_ptr_kernel<<<ntiles, kScanThreads, 0, st>>>(row_counts, tile_sums, row_ptr, rows);
-    if ((rc = check_launch()) != SEA_OK) return rc;
+    if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
   } else {
     uniform_row_ptr_kernel<<<(rows + 1 + 255) / 256, 256, 0, st>>>(row_ptr, rows, s.k_hat * r);
     if ((rc = check_launch()) != SEA_OK) return rc;

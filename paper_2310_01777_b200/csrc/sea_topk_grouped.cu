@@ -1,0 +1,275 @@
+// Mask generation with the causal-per-batch grouping (Sec. 3.1 "Grouped Top-k Selection"):
+// the estimate of a batch element is viewed as [T, H, Kc] and, for every query position, the
+// H * k_hat largest of its H * Kc entries are kept - the heads of a position compete for one
+// budget, positions never exchange anything.  Rows (b, h, t) then keep differing numbers of
+// columns; the selection leaves as one bit per compressed column, and the up-sampled mask as the
+// same flat CSR the per-query grouping produces (App. "FlatCSR" keeps one row per (b, t) over the
+// flattened (head, key) axis instead and transposes inside its kernels).
+//
+// One CTA per (b, t): its H * Kc values stay in registers as order-preserving 32-bit keys, the
+// (H * k_hat)-th largest key is found bit by bit with CTA-wide counts, and keys equal to it are
+// taken in ascending flattened index h * Kc + c until the budget is used up.
+#include "sea_common.cuh"
+
+namespace sea {
+namespace {
+
+constexpr int kMaxThreads = 1024;
+constexpr int kMaxVI = 8;           // 16-byte groups per thread
+constexpr int kWarpsPerCta = 8;     // row-per-warp kernels
+
+// Sum of v over the CTA.  `red` is one of two alternating 32-word buffers, so a single barrier
+// per call is enough.
+__device__ __forceinline__ int block_sum(int v, int* red, int nwarps) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = __reduce_add_sync(0xffffffffu, v);
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  const int t = lane < nwarps ? red[lane] : 0;
+  return __reduce_add_sync(0xffffffffu, t);
+}
+
+// Exclusive prefix of v over the threads of the CTA in thread order, and the CTA's total.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* tot, int nwarps, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();  // the previous call's readers are done with tot[]
+  if (lane == 31) tot[warp] = inc;
+  __syncthreads();
+  int w = lane < nwarps ? tot[lane] : 0;
+  int winc = w;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, winc, o);
+    if (lane >= o) winc += t;
+  }
+  total = __shfl_sync(0xffffffffu, winc, 31);
+  const int warp_off = __shfl_sync(0xffffffffu, winc - w, warp);
+  return inc - v + warp_off;
+}
+
+// Thread `tid` holds the 16-byte groups q = i * blockDim.x + tid (i < VI) of the position's
+// H * Kc / 4 groups; group q covers flattened indices 4 q .. 4 q + 3, all of one head because
+// Kc % 4 == 0.
+template <int VI>
+__global__ void __launch_bounds__(kMaxThreads)
+topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask_bits,
+                    int32_t* __restrict__ row_counts, int H, int T, int Kc, int k_sel, int r, int causal) {
+  extern __shared__ uint32_t sh_bits[];  // [H][words]
+  __shared__ int red[2][32];
+  __shared__ int scan_tot[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nthreads = blockDim.x, nwarps = nthreads >> 5;
+  const int bt = blockIdx.x;
+  const int b = bt / T, t = bt - b * T;
+  const int words = (Kc + 31) >> 5;
+  const int n4 = (H * Kc) >> 2;
+
+  uint32_t key[VI][4];
+#pragma unroll
+  for (int i = 0; i < VI; ++i) {
+    const int q = i * nthreads + tid;
+    key[i][0] = key[i][1] = key[i][2] = key[i][3] = 0u;  // below the key of every finite value
+    if (q < n4) {
+      const int f = 4 * q;
+      const int h = f / Kc, c = f - h * Kc;
+      const float4 v = __ldg(reinterpret_cast<const float4*>(A_hat + ((size_t)(b * H + h) * T + t) * Kc + c));
+      key[i][0] = order_key(v.x);
+      key[i][1] = order_key(v.y);
+      key[i][2] = order_key(v.z);
+      key[i][3] = order_key(v.w);
+    }
+  }
+  for (int w = tid; w < H * words; w += nthreads) sh_bits[w] = 0u;
+
+  // the k_sel-th largest key: the largest tau with |{key >= tau}| >= k_sel
+  uint32_t tau = 0u;
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t cand = tau | (1u << bit);
+    int c = 0;
+#pragma unroll
+    for (int i = 0; i < VI; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) c += key[i][e] >= cand;
+    if (block_sum(c, red[bit & 1], nwarps) >= k_sel) tau = cand;
+  }
+  int n_gt = 0, n_eq = 0;
+#pragma unroll
+  for (int i = 0; i < VI; ++i)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      n_gt += key[i][e] > tau;
+      n_eq += key[i][e] == tau;
+    }
+  n_gt = block_sum(n_gt, red[1], nwarps);
+  n_eq = block_sum(n_eq, red[0], nwarps);
+  const int need = k_sel - n_gt;  // how many keys equal to tau are taken (lowest flattened index first)
+
+  uint32_t taken = 0u;  // bit 4 i + e: element e of group i is selected
+  if (n_eq == need) {
+#pragma unroll
+    for (int i = 0; i < VI; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) taken |= (key[i][e] >= tau ? 1u : 0u) << (4 * i + e);
+  } else {
+    // more equal keys than places: rank them in flattened order (group index i-major, then thread)
+    int seen = 0;
+#pragma unroll
+    for (int i = 0; i < VI; ++i) {
+      int mine = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) mine += key[i][e] == tau;
+      int total;
+      int rank = seen + block_exclusive_scan(mine, scan_tot, nwarps, total);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool eq = key[i][e] == tau;
+        const bool take = key[i][e] > tau || (eq && rank < need);
+        rank += eq;
+        taken |= (take ? 1u : 0u) << (4 * i + e);
+      }
+      seen += total;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < VI; ++i) {
+    const uint32_t nib = (taken >> (4 * i)) & 15u;
+    const int q = i * nthreads + tid;
+    if (nib != 0u && q < n4) {
+      const int f = 4 * q;
+      const int h = f / Kc, c = f - h * Kc;
+      atomicOr(&sh_bits[h * words + (c >> 5)], nib << (c & 31));
+    }
+  }
+  __syncthreads();
+
+  // a warp per head: the row's bit string and its number of keys after up-sampling.  Column c
+  // covers keys c r .. c r + r - 1; a causal row keeps those <= t: the columns below
+  // (t + 1) / r in full and (t + 1) % r keys of the column at (t + 1) / r.
+  const int c_full = causal ? (t + 1) / r : Kc;
+  const int rem = causal ? (t + 1) - c_full * r : 0;
+  for (int h = warp; h < H; h += nwarps) {
+    const size_t row = (size_t)(b * H + h) * T + t;
+    int cnt = 0;
+    for (int w = lane; w < words; w += 32) {
+      const uint32_t word = sh_bits[h * words + w];
+      if (mask_bits != nullptr) mask_bits[row * words + w] = word;
+      const int lo = 32 * w;
+      const uint32_t full = c_full >= lo + 32 ? 0xffffffffu : (c_full <= lo ? 0u : (1u << (c_full - lo)) - 1u);
+      cnt += r * __popc(word & full);
+      if (c_full >= lo && c_full < lo + 32 && ((word >> (c_full - lo)) & 1u)) cnt += rem;
+    }
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if (lane == 0) row_counts[row] = cnt;
+  }
+}
+
+// One warp per row: the set bits in ascending order, r keys each, cut at the row's length (for a
+// causal row the kept keys are a prefix of that sequence).
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+fill_col_idx_bits_kernel(const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ row_ptr,
+                         int32_t* __restrict__ col_idx, long long nnz_cap, int rows, int words, int r, int log2r,
+                         int32_t* __restrict__ status) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kWarpsPerCta + warp;
+  if (row >= rows) return;
+  const int base = row_ptr[row];
+  int n = row_ptr[row + 1] - base;
+  if ((long long)base + n > nnz_cap) {
+    if (lane == 0) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
+    n = (int)max(0ll, min((long long)n, nnz_cap - base));
+  }
+  const uint32_t* my_bits = mask_bits + (size_t)row * words;
+  int done = 0;
+  for (int w = 0; w < words && done < n; ++w) {
+    const uint32_t word = __ldg(my_bits + w);
+    const int lim = min(__popc(word) * r, n - done);
+    for (int pos = lane; pos < lim; pos += 32) {
+      const int j = log2r >= 0 ? pos >> log2r : pos / r;
+      const int bit = __fns(word, 0, j + 1);  // position of the (j+1)-th set bit
+      col_idx[(size_t)base + done + pos] = (32 * w + bit) * r + (pos - j * r);
+    }
+    done += lim;
+  }
+}
+
+// One thread per (b, t): running offsets of its heads inside the position's slab of the parking
+// area.
+__global__ void park_offsets_kernel(const uint32_t* __restrict__ mask_bits, int32_t* __restrict__ park_off, int B,
+                                    int H, int T, int words, int r, int per_slab, int32_t* __restrict__ status) {
+  const int bt = blockIdx.x * blockDim.x + threadIdx.x;
+  if (bt >= B * T) return;
+  const int b = bt / T, t = bt - b * T;
+  int used = 0;
+  bool over = false;
+  for (int h = 0; h < H; ++h) {
+    const size_t row = (size_t)(b * H + h) * T + t;
+    int pc = 0;
+    for (int w = 0; w < words; ++w) pc += __popc(__ldg(mask_bits + row * words + w));
+    const int next = used + pc * r;
+    if (next > per_slab) over = true;
+    park_off[row] = over ? -1 : bt * per_slab + used;
+    used = next;
+  }
+  if (over) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
+}
+
+template <int VI>
+void launch_grouped(const float* A_hat, uint32_t* mask_bits, int32_t* counts, const sea_shape& s, int threads,
+                    cudaStream_t st) {
+  const size_t smem = (size_t)s.H * ((s.Kc + 31) / 32) * sizeof(uint32_t);
+  topk_grouped_kernel<VI><<<s.B * s.T, threads, smem, st>>>(A_hat, mask_bits, counts, s.H, s.T, s.Kc,
+                                                            s.H * s.k_hat, s.T / s.Kc, s.causal);
+}
+
+}  // namespace
+
+bool topk_grouped_supported(const sea_shape& s) {
+  return s.Kc % 4 == 0 && (long long)s.H * s.Kc <= 4ll * kMaxVI * kMaxThreads;
+}
+
+sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint32_t* mask_bits, int32_t* row_ptr,
+                                    int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts, int32_t* tile_sums,
+                                    int32_t* status, cudaStream_t st) {
+  if (!topk_grouped_supported(s)) return SEA_ERR_UNSUPPORTED;
+  const int rows = s.B * s.H * s.T;
+  const int r = s.T / s.Kc;
+  const int n4 = s.H * s.Kc / 4;
+  // four groups per thread while the CTA stays within its size limit
+  int threads = ((n4 + 3) / 4 + 31) / 32 * 32;
+  if (threads < 128) threads = 128;
+  if (threads > kMaxThreads) threads = kMaxThreads;
+  const int vi = (n4 + threads - 1) / threads;
+  if (vi <= 1) launch_grouped<1>(A_hat, mask_bits, row_counts, s, threads, st);
+  else if (vi <= 2) launch_grouped<2>(A_hat, mask_bits, row_counts, s, threads, st);
+  else if (vi <= 4) launch_grouped<4>(A_hat, mask_bits, row_counts, s, threads, st);
+  else launch_grouped<8>(A_hat, mask_bits, row_counts, s, threads, st);
+  sea_status rc = check_launch();
+  if (rc != SEA_OK) return rc;
+  if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
+  if (col_idx != nullptr) {
+    int log2r = -1;
+    for (int l = 0; l < 31; ++l)
+      if ((1 << l) == r) log2r = l;
+    const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+    fill_col_idx_bits_kernel<<<grid, kWarpsPerCta * 32, 0, st>>>(mask_bits, row_ptr, col_idx, (long long)nnz_cap, rows,
+                                                                 (s.Kc + 31) / 32, r, log2r, status);
+    if ((rc = check_launch()) != SEA_OK) return rc;
+  }
+  return SEA_OK;
+}
+
+sea_status launch_park_offsets(const sea_shape& s, const uint32_t* mask_bits, int32_t* park_off, int32_t* status,
+                               cudaStream_t st) {
+  const int n = s.B * s.T;
+  park_offsets_kernel<<<(n + 127) / 128, 128, 0, st>>>(mask_bits, park_off, s.B, s.H, s.T, (s.Kc + 31) / 32,
+                                                       s.T / s.Kc, s.H * s.k_hat * (s.T / s.Kc), status);
+  return check_launch();
+}
+
+}  // namespace sea

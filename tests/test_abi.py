@@ -90,6 +90,33 @@ def test_null_and_misaligned_pointers_are_rejected_before_launch(lib):
     assert rc == binding.SEA_ERR_INVALID_ARG  # P without col_idx
 
 
+def test_grouped_entry_points_reject_bad_arguments_before_launch(lib):
+    vp = ctypes.c_void_p
+    fake = vp(0x7F0000000000)
+    odd = vp(0x7F0000000004)
+    shp = sea.make_shape(WORKLOADS["opt_1p3b"])
+    rc = lib.sea_topk_mask_grouped(ctypes.byref(shp), fake, None, None, None, 0, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # row_ptr is required
+    rc = lib.sea_topk_mask_grouped(ctypes.byref(shp), fake, odd, fake, None, 0, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # misaligned mask_bits
+    rc = lib.sea_topk_mask_grouped(ctypes.byref(shp), fake, None, fake, None, 0, fake, 1024, None)
+    assert rc == binding.SEA_ERR_WORKSPACE
+    big = sea.make_shape(WORKLOADS["long_32k"])  # H * Kc = 65536 values per position
+    rc = lib.sea_topk_mask_grouped(ctypes.byref(big), fake, None, fake, None, 0, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_UNSUPPORTED
+    rc = lib.sea_sparse_attn_masked(ctypes.byref(shp), fake, fake, fake, fake, None, None, fake, None, None, 0, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # no mask
+    rc = lib.sea_sparse_attn_masked(ctypes.byref(shp), fake, fake, fake, fake, None, fake, fake, None, None, 0, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # no workspace, hence per-row kernels, and no col_idx
+    rc = lib.sea_attention_grouped(ctypes.byref(shp), fake, fake, fake, fake, fake, None, fake, None, None, None,
+                                   None, 0, fake, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # P without col_idx
+    f32 = sea.make_shape(WORKLOADS["tiny_f32"])
+    rc = lib.sea_attention_grouped(ctypes.byref(f32), fake, fake, fake, None, None, fake, fake, None, None, None,
+                                   None, 0, None, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # fp32 runs the per-row kernels, which need col_idx
+
+
 def test_status_strings(lib):
     assert binding.status_string(0) == "ok"
     assert "workspace" in binding.status_string(binding.SEA_ERR_WORKSPACE)
