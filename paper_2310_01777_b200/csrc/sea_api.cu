@@ -194,7 +194,7 @@ sea_status sea_topk_mask_grouped(const sea_shape* shape, const float* A_hat, uin
   uint32_t* bits = mask_bits ? mask_bits : reinterpret_cast<uint32_t*>(w + L.mask_bits);
   return launch_topk_mask_grouped(*shape, A_hat, bits, row_ptr, col_idx, nnz_cap,
                                   reinterpret_cast<int32_t*>(w + L.row_counts),
-                                  reinterpret_cast<int32_t*>(w + L.tile_sums),
+                                  reinterpret_cast<int32_t*>(w + L.tile_sums), nullptr,
                                   reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -214,7 +214,7 @@ sea_status sea_sparse_attn_masked(const sea_shape* shape, const void* Q, const v
   const WsLayout L = ws_layout(*shape);
   const bool full = ws && ws_bytes >= L.total && shape->io == SEA_BF16;
   return launch_sparse_attn_masked(*shape, Q, K, V, row_ptr, col_idx, mask_bits, O, P,
-                                   full ? reinterpret_cast<int32_t*>(w + L.park_off) : nullptr,
+                                   full ? reinterpret_cast<int32_t*>(w + L.park_off) : nullptr, false,
                                    full ? reinterpret_cast<float*>(w + L.p_scratch) : nullptr,
                                    static_cast<int32_t*>(ws), static_cast<cudaStream_t>(cuda_stream));
 }
@@ -259,11 +259,13 @@ sea_status sea_attention_grouped(const sea_shape* shape, const void* Q, const vo
     a_use = a_out;
   }
   int32_t* rp_buf = row_ptr ? row_ptr : reinterpret_cast<int32_t*>(w + L.row_ptr);
+  // the selection also lays out the parking area of the tile kernel when P is wanted
+  const bool tiles = park && sparse_attn_tc_applicable(*shape, nullptr, true, status, bits, scratch);
   rc = launch_topk_mask_grouped(*shape, a_use, bits, rp_buf, col_idx, nnz_cap,
                                 reinterpret_cast<int32_t*>(w + L.row_counts),
-                                reinterpret_cast<int32_t*>(w + L.tile_sums), status, st);
+                                reinterpret_cast<int32_t*>(w + L.tile_sums), tiles && P ? park : nullptr, status, st);
   if (rc != SEA_OK) return rc;
-  return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, scratch, status, st);
+  return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, true, scratch, status, st);
 }
 
 sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes) {

@@ -61,22 +61,24 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
                             int32_t* status, cudaStream_t st);
 sea_status launch_row_ptr_scan(const int32_t* row_counts, int32_t* tile_sums, int32_t* row_ptr, int rows,
                                cudaStream_t st);
-// Causal-per-batch grouping (sea_topk_grouped.cu).  mask_bits is written in full.
+// Causal-per-batch grouping (sea_topk_grouped.cu).  mask_bits is written in full; park_off, when
+// not null, receives the rows' offsets into the parking area of the tile kernel (see below).
 bool topk_grouped_supported(const sea_shape& s);
 sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint32_t* mask_bits,
                                     int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
-                                    int32_t* row_counts, int32_t* tile_sums, int32_t* status,
-                                    cudaStream_t st);
+                                    int32_t* row_counts, int32_t* tile_sums, int32_t* park_off,
+                                    int32_t* status, cudaStream_t st);
 // Where each row parks its unnormalised probabilities when rows keep differing numbers of columns:
 // the (b, t) slabs of H*k_hat*r floats follow one another, the heads inside a slab.  Rows of a slab
 // that keeps more than H*k_hat columns get -1 and SEA_DEV_ROW_OVERFLOW is raised.
 sea_status launch_park_offsets(const sea_shape& s, const uint32_t* mask_bits, int32_t* park_off,
                                int32_t* status, cudaStream_t st);
-// Sparse stage for a mask given as bits with its row_ptr (rows of any length).
+// Sparse stage for a mask given as bits with its row_ptr (rows of any length).  park_valid:
+// park_off already holds the offsets that belong to mask_bits.
 sea_status launch_sparse_attn_masked(const sea_shape& s, const void* Q, const void* K, const void* V,
                                      const int32_t* row_ptr, const int32_t* col_idx,
                                      const uint32_t* mask_bits, void* O, void* P, int32_t* park_off,
-                                     float* p_scratch, int32_t* status, cudaStream_t st);
+                                     bool park_valid, float* p_scratch, int32_t* status, cudaStream_t st);
 // mask_bits and p_scratch (workspace areas of the tensor-core kernel) may be null: the per-row
 // kernels are used then.  bits_valid: mask_bits already holds the bit strings of `sel`
 // (launch_topk_mask wrote them); otherwise they are derived from `sel` first.

@@ -7,8 +7,8 @@
 // flattened (head, key) axis instead and transposes inside its kernels).
 //
 // One CTA per (b, t): its H * Kc values stay in registers as order-preserving 32-bit keys, the
-// (H * k_hat)-th largest key is found bit by bit with CTA-wide counts, and keys equal to it are
-// taken in ascending flattened index h * Kc + c until the budget is used up.
+// (H * k_hat)-th largest key is found bit by bit, and keys equal to it are taken in ascending
+// flattened index h * Kc + c until the budget is used up.
 #include "sea_common.cuh"
 
 namespace sea {
@@ -56,19 +56,36 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* tot, int nwarps,
 // Thread `tid` holds the 16-byte groups q = i * blockDim.x + tid (i < VI) of the position's
 // H * Kc / 4 groups; group q covers flattened indices 4 q .. 4 q + 3, all of one head because
 // Kc % 4 == 0.
+//
+// The search for the k_sel-th largest key tau runs in two phases.  The first kPhase1Bits bits are
+// found with CTA-wide counts over all keys.  That fixes a bucket of keys sharing those bits: keys
+// above the bucket count towards every later candidate, keys below towards none, so the keys
+// inside it (a few per cent of the position's values for spread-out data) are copied to a list in
+// shared memory and one warp finds the remaining bits over the list alone, without CTA-wide
+// barriers.  A bucket that does not fit the list (many equal values) is searched like the first
+// phase.
+constexpr int kPhase1Bits = 12;
+constexpr int kListCap = 1024;
+
 template <int VI>
 __global__ void __launch_bounds__(kMaxThreads)
 topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask_bits,
-                    int32_t* __restrict__ row_counts, int H, int T, int Kc, int k_sel, int r, int causal) {
-  extern __shared__ uint32_t sh_bits[];  // [H][words]
+                    int32_t* __restrict__ row_counts, int32_t* __restrict__ park_off, int H, int T, int Kc, int k_sel,
+                    int r, int causal) {
+  extern __shared__ uint32_t sh_dyn[];  // [H][words] bits, then [H] selected columns per head
+  __shared__ uint32_t list[kListCap];
   __shared__ int red[2][32];
   __shared__ int scan_tot[32];
+  __shared__ int list_n;
+  __shared__ uint32_t found[3];  // tau, |{key > tau}|, |{key == tau}|
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nthreads = blockDim.x, nwarps = nthreads >> 5;
   const int bt = blockIdx.x;
   const int b = bt / T, t = bt - b * T;
   const int words = (Kc + 31) >> 5;
   const int n4 = (H * Kc) >> 2;
+  uint32_t* sh_bits = sh_dyn;
+  int* head_pc = reinterpret_cast<int*>(sh_dyn + H * words);
 
   uint32_t key[VI][4];
 #pragma unroll
@@ -86,28 +103,94 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
     }
   }
   for (int w = tid; w < H * words; w += nthreads) sh_bits[w] = 0u;
+  if (tid == 0) list_n = 0;
 
   // the k_sel-th largest key: the largest tau with |{key >= tau}| >= k_sel
   uint32_t tau = 0u;
-  for (int bit = 31; bit >= 0; --bit) {
+  int rb = 0;  // which of the two reduction buffers the next CTA-wide sum uses
+  for (int bit = 31; bit > 31 - kPhase1Bits; --bit) {
     const uint32_t cand = tau | (1u << bit);
     int c = 0;
 #pragma unroll
     for (int i = 0; i < VI; ++i)
 #pragma unroll
       for (int e = 0; e < 4; ++e) c += key[i][e] >= cand;
-    if (block_sum(c, red[bit & 1], nwarps) >= k_sel) tau = cand;
+    if (block_sum(c, red[rb], nwarps) >= k_sel) tau = cand;
+    rb ^= 1;
   }
-  int n_gt = 0, n_eq = 0;
+  // the bucket: keys whose first kPhase1Bits bits are tau's
+  constexpr uint32_t kSpan = 1u << (32 - kPhase1Bits);
+  const uint32_t bucket_top = tau | (kSpan - 1u);
+  int above = 0, inside = 0;
 #pragma unroll
   for (int i = 0; i < VI; ++i)
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      n_gt += key[i][e] > tau;
-      n_eq += key[i][e] == tau;
+      above += key[i][e] > bucket_top;
+      inside += (key[i][e] ^ tau) < kSpan;
     }
-  n_gt = block_sum(n_gt, red[1], nwarps);
-  n_eq = block_sum(n_eq, red[0], nwarps);
+  if (inside > 0) {
+    int at = atomicAdd(&list_n, inside);
+    if (at + inside <= kListCap) {
+#pragma unroll
+      for (int i = 0; i < VI; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if ((key[i][e] ^ tau) < kSpan) list[at++] = key[i][e];
+    }
+  }
+  above = block_sum(above, red[rb], nwarps);  // its barrier also publishes the list
+  rb ^= 1;
+  const int n_list = list_n;
+  int n_gt, n_eq;
+  if (n_list <= kListCap) {
+    if (warp == 0) {
+      for (int bit = 31 - kPhase1Bits; bit >= 0; --bit) {
+        const uint32_t cand = tau | (1u << bit);
+        int c = 0;
+        for (int idx = lane; idx < n_list; idx += 32) c += list[idx] >= cand;
+        if (__reduce_add_sync(0xffffffffu, c) + above >= k_sel) tau = cand;
+      }
+      int g = 0, e = 0;
+      for (int idx = lane; idx < n_list; idx += 32) {
+        g += list[idx] > tau;
+        e += list[idx] == tau;
+      }
+      g = __reduce_add_sync(0xffffffffu, g);
+      e = __reduce_add_sync(0xffffffffu, e);
+      if (lane == 0) {
+        found[0] = tau;
+        found[1] = (uint32_t)(above + g);
+        found[2] = (uint32_t)e;
+      }
+    }
+    __syncthreads();
+    tau = found[0];
+    n_gt = (int)found[1];
+    n_eq = (int)found[2];
+  } else {
+    for (int bit = 31 - kPhase1Bits; bit >= 0; --bit) {
+      const uint32_t cand = tau | (1u << bit);
+      int c = 0;
+#pragma unroll
+      for (int i = 0; i < VI; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) c += key[i][e] >= cand;
+      if (block_sum(c, red[rb], nwarps) >= k_sel) tau = cand;
+      rb ^= 1;
+    }
+    n_gt = 0;
+    n_eq = 0;
+#pragma unroll
+    for (int i = 0; i < VI; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        n_gt += key[i][e] > tau;
+        n_eq += key[i][e] == tau;
+      }
+    n_gt = block_sum(n_gt, red[rb], nwarps);
+    n_eq = block_sum(n_eq, red[rb ^ 1], nwarps);
+  }
   const int need = k_sel - n_gt;  // how many keys equal to tau are taken (lowest flattened index first)
 
   uint32_t taken = 0u;  // bit 4 i + e: element e of group i is selected
@@ -155,26 +238,43 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
   const int rem = causal ? (t + 1) - c_full * r : 0;
   for (int h = warp; h < H; h += nwarps) {
     const size_t row = (size_t)(b * H + h) * T + t;
-    int cnt = 0;
+    int cnt = 0, pc = 0;
     for (int w = lane; w < words; w += 32) {
       const uint32_t word = sh_bits[h * words + w];
       if (mask_bits != nullptr) mask_bits[row * words + w] = word;
       const int lo = 32 * w;
       const uint32_t full = c_full >= lo + 32 ? 0xffffffffu : (c_full <= lo ? 0u : (1u << (c_full - lo)) - 1u);
+      pc += __popc(word);
       cnt += r * __popc(word & full);
       if (c_full >= lo && c_full < lo + 32 && ((word >> (c_full - lo)) & 1u)) cnt += rem;
     }
     cnt = __reduce_add_sync(0xffffffffu, cnt);
-    if (lane == 0) row_counts[row] = cnt;
+    pc = __reduce_add_sync(0xffffffffu, pc);
+    if (lane == 0) {
+      row_counts[row] = cnt;
+      head_pc[h] = pc;
+    }
+  }
+  if (park_off != nullptr) {
+    // where each row parks its unnormalised probabilities: the heads of this position one after
+    // the other inside the position's slab of k_sel * r values
+    __syncthreads();
+    for (int h = tid; h < H; h += nthreads) {
+      int before = 0;
+      for (int g = 0; g < h; ++g) before += head_pc[g];
+      park_off[(size_t)(b * H + h) * T + t] = (bt * k_sel + before) * r;
+    }
   }
 }
 
 // One warp per row: the set bits in ascending order, r keys each, cut at the row's length (for a
-// causal row the kept keys are a prefix of that sequence).
+// causal row the kept keys are a prefix of that sequence).  Word by word, the lanes whose bit is
+// set note their position under their rank, which turns "the j-th selected column" into a lookup.
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 fill_col_idx_bits_kernel(const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ row_ptr,
                          int32_t* __restrict__ col_idx, long long nnz_cap, int rows, int words, int r, int log2r,
                          int32_t* __restrict__ status) {
+  __shared__ int col_of[kWarpsPerCta][32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kWarpsPerCta + warp;
   if (row >= rows) return;
@@ -185,16 +285,20 @@ fill_col_idx_bits_kernel(const uint32_t* __restrict__ mask_bits, const int32_t* 
     n = (int)max(0ll, min((long long)n, nnz_cap - base));
   }
   const uint32_t* my_bits = mask_bits + (size_t)row * words;
+  int32_t* out = col_idx + base;
   int done = 0;
   for (int w = 0; w < words && done < n; ++w) {
     const uint32_t word = __ldg(my_bits + w);
+    if (word == 0u) continue;
+    if ((word >> lane) & 1u) col_of[warp][__popc(word & ((1u << lane) - 1u))] = 32 * w + lane;
+    __syncwarp();
     const int lim = min(__popc(word) * r, n - done);
     for (int pos = lane; pos < lim; pos += 32) {
       const int j = log2r >= 0 ? pos >> log2r : pos / r;
-      const int bit = __fns(word, 0, j + 1);  // position of the (j+1)-th set bit
-      col_idx[(size_t)base + done + pos] = (32 * w + bit) * r + (pos - j * r);
+      out[done + pos] = col_of[warp][j] * r + (pos - j * r);
     }
     done += lim;
+    __syncwarp();
   }
 }
 
@@ -210,7 +314,14 @@ __global__ void park_offsets_kernel(const uint32_t* __restrict__ mask_bits, int3
   for (int h = 0; h < H; ++h) {
     const size_t row = (size_t)(b * H + h) * T + t;
     int pc = 0;
-    for (int w = 0; w < words; ++w) pc += __popc(__ldg(mask_bits + row * words + w));
+    if ((words & 3) == 0) {  // rows of whole 16-byte pieces (the caller's array is 16-byte aligned)
+      for (int w = 0; w < words; w += 4) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(mask_bits + row * words + w));
+        pc += __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
+      }
+    } else {
+      for (int w = 0; w < words; ++w) pc += __popc(__ldg(mask_bits + row * words + w));
+    }
     const int next = used + pc * r;
     if (next > per_slab) over = true;
     park_off[row] = over ? -1 : bt * per_slab + used;
@@ -220,10 +331,10 @@ __global__ void park_offsets_kernel(const uint32_t* __restrict__ mask_bits, int3
 }
 
 template <int VI>
-void launch_grouped(const float* A_hat, uint32_t* mask_bits, int32_t* counts, const sea_shape& s, int threads,
-                    cudaStream_t st) {
-  const size_t smem = (size_t)s.H * ((s.Kc + 31) / 32) * sizeof(uint32_t);
-  topk_grouped_kernel<VI><<<s.B * s.T, threads, smem, st>>>(A_hat, mask_bits, counts, s.H, s.T, s.Kc,
+void launch_grouped(const float* A_hat, uint32_t* mask_bits, int32_t* counts, int32_t* park_off, const sea_shape& s,
+                    int threads, cudaStream_t st) {
+  const size_t smem = ((size_t)s.H * ((s.Kc + 31) / 32) + s.H) * sizeof(uint32_t);
+  topk_grouped_kernel<VI><<<s.B * s.T, threads, smem, st>>>(A_hat, mask_bits, counts, park_off, s.H, s.T, s.Kc,
                                                             s.H * s.k_hat, s.T / s.Kc, s.causal);
 }
 
@@ -235,7 +346,7 @@ bool topk_grouped_supported(const sea_shape& s) {
 
 sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint32_t* mask_bits, int32_t* row_ptr,
                                     int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts, int32_t* tile_sums,
-                                    int32_t* status, cudaStream_t st) {
+                                    int32_t* park_off, int32_t* status, cudaStream_t st) {
   if (!topk_grouped_supported(s)) return SEA_ERR_UNSUPPORTED;
   const int rows = s.B * s.H * s.T;
   const int r = s.T / s.Kc;
@@ -245,10 +356,10 @@ sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint
   if (threads < 128) threads = 128;
   if (threads > kMaxThreads) threads = kMaxThreads;
   const int vi = (n4 + threads - 1) / threads;
-  if (vi <= 1) launch_grouped<1>(A_hat, mask_bits, row_counts, s, threads, st);
-  else if (vi <= 2) launch_grouped<2>(A_hat, mask_bits, row_counts, s, threads, st);
-  else if (vi <= 4) launch_grouped<4>(A_hat, mask_bits, row_counts, s, threads, st);
-  else launch_grouped<8>(A_hat, mask_bits, row_counts, s, threads, st);
+  if (vi <= 1) launch_grouped<1>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+  else if (vi <= 2) launch_grouped<2>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+  else if (vi <= 4) launch_grouped<4>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+  else launch_grouped<8>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
   sea_status rc = check_launch();
   if (rc != SEA_OK) return rc;
   if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
