@@ -57,27 +57,34 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* tot, int nwarps,
 // H * Kc / 4 groups; group q covers flattened indices 4 q .. 4 q + 3, all of one head because
 // Kc % 4 == 0.
 //
-// The search for the k_sel-th largest key tau runs in two phases.  The first kPhase1Bits bits are
-// found with CTA-wide counts over all keys.  That fixes a bucket of keys sharing those bits: keys
-// above the bucket count towards every later candidate, keys below towards none, so the keys
-// inside it (a few per cent of the position's values for spread-out data) are copied to a list in
-// shared memory and one warp finds the remaining bits over the list alone, without CTA-wide
-// barriers.  A bucket that does not fit the list (many equal values) is searched like the first
-// phase.
-constexpr int kPhase1Bits = 12;
+// The search for the k_sel-th largest key tau narrows a bucket of keys that share tau's leading
+// bits; keys above the bucket count towards every candidate inside it, keys below towards none.
+//   A  the first kBitsA bits (the sign and the upper exponent bits, which nearly all keys of a
+//      position share) bit by bit, with CTA-wide counts over all keys;
+//   B  the next kBitsB bits (lower exponent and upper mantissa bits, over which the keys spread
+//      widely, so that shared-memory counters rarely collide) by a histogram of the keys inside
+//      the bucket and a scan over it from the top;
+//   C  the remaining bits by one warp over a list of the keys still inside the bucket (a handful
+//      for spread-out data), without CTA-wide barriers.  A bucket that does not fit the list
+//      (many equal values) is searched as in A instead.
+constexpr int kBitsA = 5;
+constexpr int kBitsB = 12;
+constexpr int kBitsAB = kBitsA + kBitsB;
+constexpr int kBins = 1 << kBitsB;
 constexpr int kListCap = 1024;
 
-template <int VI>
-__global__ void __launch_bounds__(kMaxThreads)
+template <int VI, int kThreadsMax, int kMinCtas>
+__global__ void __launch_bounds__(kThreadsMax, kMinCtas)
 topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask_bits,
-                    int32_t* __restrict__ row_counts, int32_t* __restrict__ park_off, int H, int T, int Kc, int k_sel,
-                    int r, int causal) {
+                    int32_t* __restrict__ row_counts, int32_t* __restrict__ park_off, int H, int T, int Kc, int log2Kc,
+                    int k_sel, int r, int causal) {
   extern __shared__ uint32_t sh_dyn[];  // [H][words] bits, then [H] selected columns per head
+  __shared__ int hist[kBins];
   __shared__ uint32_t list[kListCap];
   __shared__ int red[2][32];
   __shared__ int scan_tot[32];
   __shared__ int list_n;
-  __shared__ uint32_t found[3];  // tau, |{key > tau}|, |{key == tau}|
+  __shared__ uint32_t found[3];  // after B: bin, |{key above it}|; after C: tau, |{key > tau}|, |{key == tau}|
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nthreads = blockDim.x, nwarps = nthreads >> 5;
   const int bt = blockIdx.x;
@@ -86,15 +93,28 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
   const int n4 = (H * Kc) >> 2;
   uint32_t* sh_bits = sh_dyn;
   int* head_pc = reinterpret_cast<int*>(sh_dyn + H * words);
+  // head and column of flattened index f
+  auto split = [&](int f, int& h, int& c) {
+    if (log2Kc >= 0) {
+      h = f >> log2Kc;
+      c = f & (Kc - 1);
+    } else {
+      h = f / Kc;
+      c = f - h * Kc;
+    }
+  };
 
+  for (int w = tid; w < kBins; w += nthreads) hist[w] = 0;
+  for (int w = tid; w < H * words; w += nthreads) sh_bits[w] = 0u;
+  if (tid == 0) list_n = 0;
   uint32_t key[VI][4];
 #pragma unroll
   for (int i = 0; i < VI; ++i) {
     const int q = i * nthreads + tid;
     key[i][0] = key[i][1] = key[i][2] = key[i][3] = 0u;  // below the key of every finite value
     if (q < n4) {
-      const int f = 4 * q;
-      const int h = f / Kc, c = f - h * Kc;
+      int h, c;
+      split(4 * q, h, c);
       const float4 v = __ldg(reinterpret_cast<const float4*>(A_hat + ((size_t)(b * H + h) * T + t) * Kc + c));
       key[i][0] = order_key(v.x);
       key[i][1] = order_key(v.y);
@@ -102,13 +122,11 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
       key[i][3] = order_key(v.w);
     }
   }
-  for (int w = tid; w < H * words; w += nthreads) sh_bits[w] = 0u;
-  if (tid == 0) list_n = 0;
 
-  // the k_sel-th largest key: the largest tau with |{key >= tau}| >= k_sel
+  // ---- A: the largest kBitsA-bit prefix with |{key >= prefix}| >= k_sel
   uint32_t tau = 0u;
   int rb = 0;  // which of the two reduction buffers the next CTA-wide sum uses
-  for (int bit = 31; bit > 31 - kPhase1Bits; --bit) {
+  for (int bit = 31; bit > 31 - kBitsA; --bit) {
     const uint32_t cand = tau | (1u << bit);
     int c = 0;
 #pragma unroll
@@ -118,17 +136,47 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
     if (block_sum(c, red[rb], nwarps) >= k_sel) tau = cand;
     rb ^= 1;
   }
-  // the bucket: keys whose first kPhase1Bits bits are tau's
-  constexpr uint32_t kSpan = 1u << (32 - kPhase1Bits);
-  const uint32_t bucket_top = tau | (kSpan - 1u);
-  int above = 0, inside = 0;
+  // ---- B: histogram of the next kBitsB bits of the keys inside A's bucket
+  constexpr uint32_t kSpanA = 1u << (32 - kBitsA);
+  int above = 0;
 #pragma unroll
   for (int i = 0; i < VI; ++i)
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      above += key[i][e] > bucket_top;
-      inside += (key[i][e] ^ tau) < kSpan;
+      const uint32_t d = key[i][e] ^ tau;  // below kSpanA: inside the bucket
+      above += key[i][e] > (tau | (kSpanA - 1u));
+      if (d < kSpanA && i * nthreads + tid < n4) atomicAdd(&hist[d >> (32 - kBitsAB)], 1);
     }
+  above = block_sum(above, red[rb], nwarps);  // its barrier also completes the histogram
+  rb ^= 1;
+  {
+    // the highest bin whose count, together with the keys above A's bucket and all bins above it,
+    // reaches k_sel.  Thread `tid` owns bins tid * per .. tid * per + per - 1.
+    const int per = (kBins + nthreads - 1) / nthreads;
+    const int first = tid * per;
+    int mine = 0;
+    for (int j = 0; j < per; ++j)
+      if (first + j < kBins) mine += hist[first + j];
+    int total;
+    const int below = block_exclusive_scan(mine, scan_tot, nwarps, total);
+    int over = above + total - below - mine;  // keys above this thread's bins
+    if (over < k_sel && over + mine >= k_sel) {
+      int bin = min(first + per, kBins) - 1;
+      while (over + hist[bin] < k_sel) over += hist[bin--];
+      found[0] = (uint32_t)bin;
+      found[1] = (uint32_t)over;
+    }
+    __syncthreads();
+  }
+  tau |= found[0] << (32 - kBitsAB);
+  above = (int)found[1];
+  // ---- C: the keys inside B's bucket
+  constexpr uint32_t kSpan = 1u << (32 - kBitsAB);
+  int inside = 0;
+#pragma unroll
+  for (int i = 0; i < VI; ++i)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) inside += (key[i][e] ^ tau) < kSpan;
   if (inside > 0) {
     int at = atomicAdd(&list_n, inside);
     if (at + inside <= kListCap) {
@@ -139,13 +187,12 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
           if ((key[i][e] ^ tau) < kSpan) list[at++] = key[i][e];
     }
   }
-  above = block_sum(above, red[rb], nwarps);  // its barrier also publishes the list
-  rb ^= 1;
+  __syncthreads();  // also: every thread has read found[] before it is written again
   const int n_list = list_n;
   int n_gt, n_eq;
   if (n_list <= kListCap) {
     if (warp == 0) {
-      for (int bit = 31 - kPhase1Bits; bit >= 0; --bit) {
+      for (int bit = 31 - kBitsAB; bit >= 0; --bit) {
         const uint32_t cand = tau | (1u << bit);
         int c = 0;
         for (int idx = lane; idx < n_list; idx += 32) c += list[idx] >= cand;
@@ -169,7 +216,7 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
     n_gt = (int)found[1];
     n_eq = (int)found[2];
   } else {
-    for (int bit = 31 - kPhase1Bits; bit >= 0; --bit) {
+    for (int bit = 31 - kBitsAB; bit >= 0; --bit) {
       const uint32_t cand = tau | (1u << bit);
       int c = 0;
 #pragma unroll
@@ -224,36 +271,41 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
     const uint32_t nib = (taken >> (4 * i)) & 15u;
     const int q = i * nthreads + tid;
     if (nib != 0u && q < n4) {
-      const int f = 4 * q;
-      const int h = f / Kc, c = f - h * Kc;
+      int h, c;
+      split(4 * q, h, c);
       atomicOr(&sh_bits[h * words + (c >> 5)], nib << (c & 31));
     }
   }
   __syncthreads();
 
-  // a warp per head: the row's bit string and its number of keys after up-sampling.  Column c
+  // a thread per head: the row's bit string and its number of keys after up-sampling.  Column c
   // covers keys c r .. c r + r - 1; a causal row keeps those <= t: the columns below
   // (t + 1) / r in full and (t + 1) % r keys of the column at (t + 1) / r.
   const int c_full = causal ? (t + 1) / r : Kc;
   const int rem = causal ? (t + 1) - c_full * r : 0;
-  for (int h = warp; h < H; h += nwarps) {
+  for (int h = tid; h < H; h += nthreads) {
     const size_t row = (size_t)(b * H + h) * T + t;
+    const uint32_t* src = sh_bits + h * words;
     int cnt = 0, pc = 0;
-    for (int w = lane; w < words; w += 32) {
-      const uint32_t word = sh_bits[h * words + w];
-      if (mask_bits != nullptr) mask_bits[row * words + w] = word;
+    for (int w = 0; w < words; ++w) {
+      const uint32_t word = src[w];
       const int lo = 32 * w;
       const uint32_t full = c_full >= lo + 32 ? 0xffffffffu : (c_full <= lo ? 0u : (1u << (c_full - lo)) - 1u);
       pc += __popc(word);
       cnt += r * __popc(word & full);
       if (c_full >= lo && c_full < lo + 32 && ((word >> (c_full - lo)) & 1u)) cnt += rem;
     }
-    cnt = __reduce_add_sync(0xffffffffu, cnt);
-    pc = __reduce_add_sync(0xffffffffu, pc);
-    if (lane == 0) {
-      row_counts[row] = cnt;
-      head_pc[h] = pc;
+    if (mask_bits != nullptr) {
+      uint32_t* dst = mask_bits + row * words;
+      if ((words & 3) == 0) {  // rows of whole 16-byte pieces
+        for (int w = 0; w < words; w += 4)
+          *reinterpret_cast<uint4*>(dst + w) = make_uint4(src[w], src[w + 1], src[w + 2], src[w + 3]);
+      } else {
+        for (int w = 0; w < words; ++w) dst[w] = src[w];
+      }
     }
+    row_counts[row] = cnt;
+    head_pc[h] = pc;
   }
   if (park_off != nullptr) {
     // where each row parks its unnormalised probabilities: the heads of this position one after
@@ -330,12 +382,15 @@ __global__ void park_offsets_kernel(const uint32_t* __restrict__ mask_bits, int3
   if (over) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
 }
 
-template <int VI>
+template <int VI, int kThreadsMax, int kMinCtas>
 void launch_grouped(const float* A_hat, uint32_t* mask_bits, int32_t* counts, int32_t* park_off, const sea_shape& s,
                     int threads, cudaStream_t st) {
   const size_t smem = ((size_t)s.H * ((s.Kc + 31) / 32) + s.H) * sizeof(uint32_t);
-  topk_grouped_kernel<VI><<<s.B * s.T, threads, smem, st>>>(A_hat, mask_bits, counts, park_off, s.H, s.T, s.Kc,
-                                                            s.H * s.k_hat, s.T / s.Kc, s.causal);
+  int log2Kc = -1;
+  for (int l = 0; l < 31; ++l)
+    if ((1 << l) == s.Kc) log2Kc = l;
+  topk_grouped_kernel<VI, kThreadsMax, kMinCtas><<<s.B * s.T, threads, smem, st>>>(
+      A_hat, mask_bits, counts, park_off, s.H, s.T, s.Kc, log2Kc, s.H * s.k_hat, s.T / s.Kc, s.causal);
 }
 
 }  // namespace
@@ -356,10 +411,15 @@ sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint
   if (threads < 128) threads = 128;
   if (threads > kMaxThreads) threads = kMaxThreads;
   const int vi = (n4 + threads - 1) / threads;
-  if (vi <= 1) launch_grouped<1>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
-  else if (vi <= 2) launch_grouped<2>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
-  else if (vi <= 4) launch_grouped<4>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
-  else launch_grouped<8>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+  if (threads <= 256) {  // small CTAs: several per SM
+    if (vi <= 1) launch_grouped<1, 256, 5>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+    else if (vi <= 2) launch_grouped<2, 256, 5>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+    else launch_grouped<4, 256, 5>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+  } else if (vi <= 4) {
+    launch_grouped<4, kMaxThreads, 1>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+  } else {
+    launch_grouped<8, kMaxThreads, 1>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+  }
   sea_status rc = check_launch();
   if (rc != SEA_OK) return rc;
   if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
