@@ -104,7 +104,13 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
     }
   };
 
-  for (int w = tid; w < kBins; w += nthreads) hist[w] = 0;
+  for (int w = 4 * tid; w < kBins; w += 4 * nthreads) *reinterpret_cast<int4*>(&hist[w]) = make_int4(0, 0, 0, 0);
+  // Bin x is owned by thread x >> log2per (a power of two of bins per thread, `owners` threads own
+  // some) and kept at word (x & (per - 1)) * owners + (x >> log2per): when the owners read their
+  // j-th bins, neighbouring lanes read neighbouring words.
+  int log2per = 0;
+  while ((nthreads << log2per) < kBins) ++log2per;
+  const int per = 1 << log2per, owners = kBins >> log2per;
   for (int w = tid; w < H * words; w += nthreads) sh_bits[w] = 0u;
   if (tid == 0) list_n = 0;
   uint32_t key[VI][4];
@@ -145,25 +151,26 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
     for (int e = 0; e < 4; ++e) {
       const uint32_t d = key[i][e] ^ tau;  // below kSpanA: inside the bucket
       above += key[i][e] > (tau | (kSpanA - 1u));
-      if (d < kSpanA && i * nthreads + tid < n4) atomicAdd(&hist[d >> (32 - kBitsAB)], 1);
+      if (d < kSpanA && i * nthreads + tid < n4) {
+        const int x = (int)(d >> (32 - kBitsAB));
+        atomicAdd(&hist[(x & (per - 1)) * owners + (x >> log2per)], 1);
+      }
     }
   above = block_sum(above, red[rb], nwarps);  // its barrier also completes the histogram
   rb ^= 1;
   {
     // the highest bin whose count, together with the keys above A's bucket and all bins above it,
-    // reaches k_sel.  Thread `tid` owns bins tid * per .. tid * per + per - 1.
-    const int per = (kBins + nthreads - 1) / nthreads;
-    const int first = tid * per;
+    // reaches k_sel.
     int mine = 0;
-    for (int j = 0; j < per; ++j)
-      if (first + j < kBins) mine += hist[first + j];
+    if (tid < owners)
+      for (int j = 0; j < per; ++j) mine += hist[j * owners + tid];
     int total;
     const int below = block_exclusive_scan(mine, scan_tot, nwarps, total);
     int over = above + total - below - mine;  // keys above this thread's bins
     if (over < k_sel && over + mine >= k_sel) {
-      int bin = min(first + per, kBins) - 1;
-      while (over + hist[bin] < k_sel) over += hist[bin--];
-      found[0] = (uint32_t)bin;
+      int j = per - 1;
+      while (over + hist[j * owners + tid] < k_sel) over += hist[j-- * owners + tid];
+      found[0] = (uint32_t)(tid * per + j);
       found[1] = (uint32_t)over;
     }
     __syncthreads();
