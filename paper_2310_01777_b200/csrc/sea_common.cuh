@@ -158,9 +158,8 @@ struct Io<__nv_bfloat16> {
 
 // 32-bit key whose unsigned order is the float order, with -0 folded onto +0.
 __device__ __forceinline__ uint32_t order_key(float v) {
-  uint32_t u = __float_as_uint(v);
-  if (u == 0x80000000u) u = 0u;  // -0 ties with +0
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  const uint32_t u = __float_as_uint(v + 0.f);  // -0 + 0 = +0: the two zeros tie; every other value is unchanged
+  return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);  // negative: all bits flip; else: the sign bit
 }
 
 __device__ __forceinline__ float warp_max(float v) {

@@ -57,20 +57,21 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* tot, int nwarps,
 // H * Kc / 4 groups; group q covers flattened indices 4 q .. 4 q + 3, all of one head because
 // Kc % 4 == 0.
 //
-// The search for the k_sel-th largest key tau narrows a bucket of keys that share tau's leading
-// bits; keys above the bucket count towards every candidate inside it, keys below towards none.
-//   A  the first kBitsA bits (the sign and the upper exponent bits, which nearly all keys of a
-//      position share) bit by bit, with CTA-wide counts over all keys;
-//   B  the next kBitsB bits (lower exponent and upper mantissa bits, over which the keys spread
-//      widely, so that shared-memory counters rarely collide) by a histogram of the keys inside
-//      the bucket and a scan over it from the top;
-//   C  the remaining bits by one warp over a list of the keys still inside the bucket (a handful
-//      for spread-out data), without CTA-wide barriers.  A bucket that does not fit the list
-//      (many equal values) is searched as in A instead.
-constexpr int kBitsA = 5;
-constexpr int kBitsB = 12;
-constexpr int kBitsAB = kBitsA + kBitsB;
-constexpr int kBins = 1 << kBitsB;
+// The search for the k_sel-th largest key tau:
+//   1  the position's largest key `top` (one CTA-wide maximum);
+//   2  a histogram of the distances top - key in steps of 2^kFineBits, over the kBins steps below
+//      `top` (for positive values that is every magnitude down to top / 65536; the keys spread
+//      widely over it, so the shared-memory counters rarely collide), and a scan over it that
+//      finds the step holding tau and the number of keys in the steps above it;
+//   3  the keys inside that step (a handful for spread-out data) go to a list and one warp finds
+//      tau among them, bit by bit, without CTA-wide barriers.
+// When fewer than k_sel keys lie inside the histogram's span (tau is negative while `top` is not)
+// or the step does not fit the list (many equal values), tau is found bit by bit with CTA-wide
+// counts over all keys instead.
+constexpr int kFineBits = 15;
+constexpr int kBinBits = 12;
+constexpr int kBins = 1 << kBinBits;
+constexpr uint32_t kFineMask = (1u << kFineBits) - 1u;
 constexpr int kListCap = 1024;
 
 template <int VI, int kThreadsMax, int kMinCtas>
@@ -84,7 +85,7 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
   __shared__ int red[2][32];
   __shared__ int scan_tot[32];
   __shared__ int list_n;
-  __shared__ uint32_t found[3];  // after B: bin, |{key above it}|; after C: tau, |{key > tau}|, |{key == tau}|
+  __shared__ uint32_t found[3];  // after 2: step, |{key above it}|; after 3: tau, |{key > tau}|, |{key == tau}|
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nthreads = blockDim.x, nwarps = nthreads >> 5;
   const int bt = blockIdx.x;
@@ -105,15 +106,17 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
   };
 
   for (int w = 4 * tid; w < kBins; w += 4 * nthreads) *reinterpret_cast<int4*>(&hist[w]) = make_int4(0, 0, 0, 0);
-  // Bin x is owned by thread x >> log2per (a power of two of bins per thread, `owners` threads own
-  // some) and kept at word (x & (per - 1)) * owners + (x >> log2per): when the owners read their
-  // j-th bins, neighbouring lanes read neighbouring words.
-  int log2per = 0;
-  while ((nthreads << log2per) < kBins) ++log2per;
-  const int per = 1 << log2per, owners = kBins >> log2per;
   for (int w = tid; w < H * words; w += nthreads) sh_bits[w] = 0u;
   if (tid == 0) list_n = 0;
+  // Step x of the histogram is owned by thread x >> log2per (a power of two of steps per thread,
+  // `owners` threads own some) and kept at word (x & (per - 1)) * owners + (x >> log2per): when the
+  // owners read their j-th steps, neighbouring lanes read neighbouring words.
+  int log2per = 0;
+  while ((nthreads << log2per) < kBins) ++log2per;
+  const int per = 1 << log2per, log2owners = kBinBits - log2per, owners = 1 << log2owners;
+
   uint32_t key[VI][4];
+  uint32_t top = 0u;
 #pragma unroll
   for (int i = 0; i < VI; ++i) {
     const int q = i * nthreads + tid;
@@ -127,103 +130,98 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
       key[i][2] = order_key(v.z);
       key[i][3] = order_key(v.w);
     }
+    top = max(max(top, key[i][0]), max(key[i][1], max(key[i][2], key[i][3])));
   }
-
-  // ---- A: the largest kBitsA-bit prefix with |{key >= prefix}| >= k_sel
-  uint32_t tau = 0u;
-  int rb = 0;  // which of the two reduction buffers the next CTA-wide sum uses
-  for (int bit = 31; bit > 31 - kBitsA; --bit) {
-    const uint32_t cand = tau | (1u << bit);
-    int c = 0;
-#pragma unroll
-    for (int i = 0; i < VI; ++i)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) c += key[i][e] >= cand;
-    if (block_sum(c, red[rb], nwarps) >= k_sel) tau = cand;
-    rb ^= 1;
-  }
-  // ---- B: histogram of the next kBitsB bits of the keys inside A's bucket
-  constexpr uint32_t kSpanA = 1u << (32 - kBitsA);
-  int above = 0;
+  // ---- 1: the largest key
+  top = __reduce_max_sync(0xffffffffu, top);
+  if (lane == 0) red[0][warp] = (int)top;
+  __syncthreads();  // also: the counters are zero
+  top = __reduce_max_sync(0xffffffffu, lane < nwarps ? (uint32_t)red[0][lane] : 0u);
+  // ---- 2: histogram of (top - key) >> kFineBits over the keys less than kBins steps below top
 #pragma unroll
   for (int i = 0; i < VI; ++i)
+    if (i * nthreads + tid < n4) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const uint32_t d = key[i][e] ^ tau;  // below kSpanA: inside the bucket
-      above += key[i][e] > (tau | (kSpanA - 1u));
-      if (d < kSpanA && i * nthreads + tid < n4) {
-        const int x = (int)(d >> (32 - kBitsAB));
-        atomicAdd(&hist[(x & (per - 1)) * owners + (x >> log2per)], 1);
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t x = (top - key[i][e]) >> kFineBits;
+        if (x < (uint32_t)kBins) atomicAdd(&hist[((x & (per - 1)) << log2owners) + (x >> log2per)], 1);
       }
     }
-  above = block_sum(above, red[rb], nwarps);  // its barrier also completes the histogram
-  rb ^= 1;
+  __syncthreads();
+  int n_gt = 0, n_eq = 0;
+  uint32_t tau = 0u;
+  bool searched = false;
   {
-    // the highest bin whose count, together with the keys above A's bucket and all bins above it,
-    // reaches k_sel.
+    // the first step (from the top) at which the running count reaches k_sel
     int mine = 0;
     if (tid < owners)
       for (int j = 0; j < per; ++j) mine += hist[j * owners + tid];
     int total;
-    const int below = block_exclusive_scan(mine, scan_tot, nwarps, total);
-    int over = above + total - below - mine;  // keys above this thread's bins
+    int over = block_exclusive_scan(mine, scan_tot, nwarps, total);  // keys in the steps above this thread's
     if (over < k_sel && over + mine >= k_sel) {
-      int j = per - 1;
-      while (over + hist[j * owners + tid] < k_sel) over += hist[j-- * owners + tid];
+      int j = 0;
+      while (over + hist[j * owners + tid] < k_sel) over += hist[j++ * owners + tid];
       found[0] = (uint32_t)(tid * per + j);
       found[1] = (uint32_t)over;
     }
     __syncthreads();
-  }
-  tau |= found[0] << (32 - kBitsAB);
-  above = (int)found[1];
-  // ---- C: the keys inside B's bucket
-  constexpr uint32_t kSpan = 1u << (32 - kBitsAB);
-  int inside = 0;
-#pragma unroll
-  for (int i = 0; i < VI; ++i)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) inside += (key[i][e] ^ tau) < kSpan;
-  if (inside > 0) {
-    int at = atomicAdd(&list_n, inside);
-    if (at + inside <= kListCap) {
+    if (total >= k_sel) {
+      // ---- 3: the keys inside the step
+      const uint32_t step = found[0];
+      const int above = (int)found[1];
+      int inside = 0;
 #pragma unroll
       for (int i = 0; i < VI; ++i)
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if ((key[i][e] ^ tau) < kSpan) list[at++] = key[i][e];
+        for (int e = 0; e < 4; ++e) inside += ((top - key[i][e]) >> kFineBits) == step;
+      if (inside > 0) {
+        int at = atomicAdd(&list_n, inside);
+        if (at + inside <= kListCap) {
+#pragma unroll
+          for (int i = 0; i < VI; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const uint32_t rel = top - key[i][e];
+              if ((rel >> kFineBits) == step) list[at++] = kFineMask - (rel & kFineMask);  // grows with the key
+            }
+        }
+      }
+      __syncthreads();  // also: every thread has read found[] before it is written again
+      const int n_list = list_n;
+      if (n_list <= kListCap) {
+        if (warp == 0) {
+          uint32_t fine = 0u;  // the k_sel-th largest key's position inside the step
+          for (int bit = kFineBits - 1; bit >= 0; --bit) {
+            const uint32_t cand = fine | (1u << bit);
+            int c = 0;
+            for (int idx = lane; idx < n_list; idx += 32) c += list[idx] >= cand;
+            if (__reduce_add_sync(0xffffffffu, c) + above >= k_sel) fine = cand;
+          }
+          int g = 0, e = 0;
+          for (int idx = lane; idx < n_list; idx += 32) {
+            g += list[idx] > fine;
+            e += list[idx] == fine;
+          }
+          g = __reduce_add_sync(0xffffffffu, g);
+          e = __reduce_add_sync(0xffffffffu, e);
+          if (lane == 0) {
+            found[0] = top - ((step << kFineBits) | (kFineMask - fine));
+            found[1] = (uint32_t)(above + g);
+            found[2] = (uint32_t)e;
+          }
+        }
+        __syncthreads();
+        tau = found[0];
+        n_gt = (int)found[1];
+        n_eq = (int)found[2];
+        searched = true;
+      }
     }
   }
-  __syncthreads();  // also: every thread has read found[] before it is written again
-  const int n_list = list_n;
-  int n_gt, n_eq;
-  if (n_list <= kListCap) {
-    if (warp == 0) {
-      for (int bit = 31 - kBitsAB; bit >= 0; --bit) {
-        const uint32_t cand = tau | (1u << bit);
-        int c = 0;
-        for (int idx = lane; idx < n_list; idx += 32) c += list[idx] >= cand;
-        if (__reduce_add_sync(0xffffffffu, c) + above >= k_sel) tau = cand;
-      }
-      int g = 0, e = 0;
-      for (int idx = lane; idx < n_list; idx += 32) {
-        g += list[idx] > tau;
-        e += list[idx] == tau;
-      }
-      g = __reduce_add_sync(0xffffffffu, g);
-      e = __reduce_add_sync(0xffffffffu, e);
-      if (lane == 0) {
-        found[0] = tau;
-        found[1] = (uint32_t)(above + g);
-        found[2] = (uint32_t)e;
-      }
-    }
-    __syncthreads();
-    tau = found[0];
-    n_gt = (int)found[1];
-    n_eq = (int)found[2];
-  } else {
-    for (int bit = 31 - kBitsAB; bit >= 0; --bit) {
+  if (!searched) {
+    // the largest tau with |{key >= tau}| >= k_sel, bit by bit over all keys
+    int rb = 0;  // which of the two reduction buffers the next CTA-wide sum uses
+    for (int bit = 31; bit >= 0; --bit) {
       const uint32_t cand = tau | (1u << bit);
       int c = 0;
 #pragma unroll
@@ -233,8 +231,6 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
       if (block_sum(c, red[rb], nwarps) >= k_sel) tau = cand;
       rb ^= 1;
     }
-    n_gt = 0;
-    n_eq = 0;
 #pragma unroll
     for (int i = 0; i < VI; ++i)
 #pragma unroll
