@@ -191,19 +191,31 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
       if (n_list <= kListCap) {
         if (warp == 0) {
           uint32_t fine = 0u;  // the k_sel-th largest key's position inside the step
-          for (int bit = kFineBits - 1; bit >= 0; --bit) {
-            const uint32_t cand = fine | (1u << bit);
-            int c = 0;
-            for (int idx = lane; idx < n_list; idx += 32) c += list[idx] >= cand;
-            if (__reduce_add_sync(0xffffffffu, c) + above >= k_sel) fine = cand;
-          }
           int g = 0, e = 0;
-          for (int idx = lane; idx < n_list; idx += 32) {
-            g += list[idx] > fine;
-            e += list[idx] == fine;
+          if (n_list <= 32) {
+            // an entry per lane: counts are ballots
+            const bool have = lane < n_list;
+            const uint32_t mine = have ? list[lane] : 0u;
+            for (int bit = kFineBits - 1; bit >= 0; --bit) {
+              const uint32_t cand = fine | (1u << bit);
+              if (__popc(__ballot_sync(0xffffffffu, have && mine >= cand)) + above >= k_sel) fine = cand;
+            }
+            g = __popc(__ballot_sync(0xffffffffu, have && mine > fine));
+            e = __popc(__ballot_sync(0xffffffffu, have && mine == fine));
+          } else {
+            for (int bit = kFineBits - 1; bit >= 0; --bit) {
+              const uint32_t cand = fine | (1u << bit);
+              int c = 0;
+              for (int idx = lane; idx < n_list; idx += 32) c += list[idx] >= cand;
+              if (__reduce_add_sync(0xffffffffu, c) + above >= k_sel) fine = cand;
+            }
+            for (int idx = lane; idx < n_list; idx += 32) {
+              g += list[idx] > fine;
+              e += list[idx] == fine;
+            }
+            g = __reduce_add_sync(0xffffffffu, g);
+            e = __reduce_add_sync(0xffffffffu, e);
           }
-          g = __reduce_add_sync(0xffffffffu, g);
-          e = __reduce_add_sync(0xffffffffu, e);
           if (lane == 0) {
             found[0] = top - ((step << kFineBits) | (kFineMask - fine));
             found[1] = (uint32_t)(above + g);
@@ -415,9 +427,9 @@ sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint
   if (threads > kMaxThreads) threads = kMaxThreads;
   const int vi = (n4 + threads - 1) / threads;
   if (threads <= 256) {  // small CTAs: several per SM
-    if (vi <= 1) launch_grouped<1, 256, 5>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
-    else if (vi <= 2) launch_grouped<2, 256, 5>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
-    else launch_grouped<4, 256, 5>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+    if (vi <= 1) launch_grouped<1, 256, 6>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+    else if (vi <= 2) launch_grouped<2, 256, 6>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+    else launch_grouped<4, 256, 6>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
   } else if (vi <= 4) {
     launch_grouped<4, kMaxThreads, 1>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
   } else {
