@@ -404,12 +404,15 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   float* den_x = z_s + 128;                                            // [kParts][128]
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   // tensor memory: projections of Q -> phi(Q); projections of K -> in-chunk kernel matrix -> its
-  // masked head / remainder; numerator; C; the first two regions later hold the A_hat tiles
-  constexpr uint32_t kColQ = 0, kColA = 128, kColNum = 256, kColC = 320, kCols = 512;
+  // masked head / remainder; numerator; C.  A_hat tiles: with a single decoder pass per item (Kc <=
+  // 128) the tile has columns of its own, so the next item's projections need not wait until the
+  // rows have read it; with several passes the tiles alternate between the first two regions.
+  constexpr uint32_t kColQ = 0, kColA = 128, kColNum = 256, kColC = 320, kColAh = 384, kCols = 512;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool causal = p.causal != 0;
   const int n_ct = (p.Kc + kWTile - 1) / kWTile;
+  const bool single = n_ct == 1;
   const int n_items = p.BH * p.nchunk;
   if (tid == 0) {
     for (int i = 0; i < kO_NumBars; ++i) {
@@ -491,10 +494,13 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         const int next = item + gridDim.x;
         const uint32_t par = it & 1;
         ok = mbar_wait(bar(kO_QK), par, abort_flag);
-        wait_afree_upto(g);  // the projections go where the previous item's A_hat tiles were
+        // the projections go where the previous item's A_hat tiles were, and phi(K) where its decoder
+        // columns were: the rows have read the former (which also means the MMAs that read the
+        // latter are complete); with a tile region of its own only the MMAs matter
+        if (!single) wait_afree_upto(g);
+        else if (ok && g > 0) ok = mbar_wait(bar(kO_WDone + ((g - 1) & 1)), ((g - 1) >> 1) & 1, abort_flag);
         if (!ok) break;
         fence_after();
-        // ... and the decoder columns of the previous item are no longer read: their place takes phi(K)
         if (causal) load_phik(item);
         {
           constexpr uint32_t idE = idesc_bf16(MP, false, false);
@@ -571,11 +577,13 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         for (int ct = 0; ct < n_ct && ok; ++ct, ++g) {
           const uint32_t b = g & 1;
           ok = mbar_wait(bar(kO_W + b), (g >> 1) & 1, abort_flag);
-          if (g >= 2) wait_afree_upto(g - 1);  // the rows have read the tile that was in this buffer
+          // the rows have read the tile that was in this buffer
+          if (single) wait_afree_upto(g);
+          else if (g >= 2) wait_afree_upto(g - 1);
           if (!ok) break;
           fence_after();
           const uint32_t wbase = smem_u32(sPhi) + b * 2 * kTileBytes;
-          const uint32_t d = tmem + (b ? kColA : kColQ);
+          const uint32_t d = tmem + (single ? kColAh : (b ? kColA : kColQ));
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const uint64_t wh = smem_desc(wbase + 2048 * k, 8192, 1024);
@@ -706,7 +714,8 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         if (ok) {
           fence_after();
 #pragma unroll
-          for (int cc = 0; cc < kMine; ++cc) tmem_ld32(lane_addr + (b ? kColA : kColQ) + 32 * (part + kParts * cc), e[cc]);
+          for (int cc = 0; cc < kMine; ++cc)
+            tmem_ld32(lane_addr + (single ? kColAh : (b ? kColA : kColQ)) + 32 * (part + kParts * cc), e[cc]);
           tmem_ld_wait();
           warp_arrive(bar(kO_AFree + b), lane);
         }
