@@ -83,7 +83,7 @@ sea_status sea_estimate(const sea_shape* shape, const void* Q, const void* K, co
   if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
   char* w = static_cast<char*>(ws);
   return launch_estimate(*shape, Q, K, V, omega, W_dec, A_hat, reinterpret_cast<float*>(w + L.est_state),
-                         w + L.est_split, reinterpret_cast<int32_t*>(w + L.status),
+                         w + L.est_split, nullptr, nullptr, reinterpret_cast<int32_t*>(w + L.status),
                          static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -105,7 +105,7 @@ sea_status sea_topk_mask(const sea_shape* shape, const float* A_hat, int32_t* se
   int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
   return launch_topk_mask(*shape, A_hat, sel_buf, row_ptr, col_idx, nnz_cap,
                           reinterpret_cast<int32_t*>(w + L.row_counts),
-                          reinterpret_cast<int32_t*>(w + L.tile_sums), nullptr,
+                          reinterpret_cast<int32_t*>(w + L.tile_sums), nullptr, false,
                           reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -156,20 +156,23 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
 
-  const float* a_use = A_hat_in;
-  if (estimate) {
-    float* a_out = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
-    rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state),
-                         w + L.est_split, status, st);
-    if (rc != SEA_OK) return rc;
-    a_use = a_out;
-  }
   int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
   int32_t* rp_buf = row_ptr ? row_ptr : reinterpret_cast<int32_t*>(w + L.row_ptr);
   uint32_t* bits = reinterpret_cast<uint32_t*>(w + L.mask_bits);
-  rc = launch_topk_mask(*shape, a_use, sel_buf, rp_buf, col_idx, nnz_cap,
-                        reinterpret_cast<int32_t*>(w + L.row_counts),
-                        reinterpret_cast<int32_t*>(w + L.tile_sums), bits, status, st);
+  int32_t* counts = reinterpret_cast<int32_t*>(w + L.row_counts);
+  const float* a_use = A_hat_in;
+  bool selected = false;
+  if (estimate) {
+    // where the estimator can, it selects each row's columns while the row is still on chip
+    float* a_out = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
+    const SelectOut so{sel_buf, shape->causal ? counts : nullptr, bits};
+    rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state),
+                         w + L.est_split, &so, &selected, status, st);
+    if (rc != SEA_OK) return rc;
+    a_use = a_out;
+  }
+  rc = launch_topk_mask(*shape, a_use, sel_buf, rp_buf, col_idx, nnz_cap, counts,
+                        reinterpret_cast<int32_t*>(w + L.tile_sums), bits, selected, status, st);
   if (rc != SEA_OK) return rc;
   return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P, bits, true,
                             reinterpret_cast<float*>(w + L.p_scratch), status, st);
@@ -254,7 +257,7 @@ sea_status sea_attention_grouped(const sea_shape* shape, const void* Q, const vo
   if (estimate) {
     float* a_out = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
     rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state),
-                         w + L.est_split, status, st);
+                         w + L.est_split, nullptr, nullptr, status, st);
     if (rc != SEA_OK) return rc;
     a_use = a_out;
   }

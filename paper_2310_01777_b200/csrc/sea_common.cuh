@@ -41,23 +41,36 @@ struct WsLayout {
 WsLayout ws_layout(const sea_shape& s);
 sea_status validate_shape(const sea_shape* s, bool need_estimator);
 
-// Stage launchers (defined one per .cu file).  All are asynchronous on `st`.
+// Where the per-query selection goes when the estimator's output kernel performs it (see
+// estimate_tc_selects): the same three arrays launch_topk_mask's selection kernel writes.
+struct SelectOut {
+  int32_t* sel;         // [rows][k_hat]
+  int32_t* row_counts;  // [rows], causal shapes only (null otherwise)
+  uint32_t* mask_bits;  // [rows][ceil(Kc/32)] or null
+};
+
+// Stage launchers (defined one per .cu file).  All are asynchronous on `st`.  select_out may be
+// null; *selected tells whether the selection was performed.
 sea_status launch_estimate(const sea_shape& s, const void* Q, const void* K, const void* V,
                            const float* omega, const float* W_dec, float* A_hat,
-                           float* est_state, void* est_split, int32_t* status, cudaStream_t st);
+                           float* est_state, void* est_split, const SelectOut* select_out, bool* selected,
+                           int32_t* status, cudaStream_t st);
 sea_status launch_estimate_f32(const sea_shape& s, const void* Q, const void* K, const void* V,
                                const float* omega, const float* W_dec, float* A_hat,
                                float* est_state, int32_t* status, cudaStream_t st);
 // bf16 estimator on tcgen05 (sea_estimate_tc.cu)
 bool estimate_tc_applicable(const sea_shape& s);
+bool estimate_tc_selects(const sea_shape& s);
 size_t estimate_tc_state_bytes(const sea_shape& s);
 size_t estimate_tc_split_bytes(const sea_shape& s);
 sea_status launch_estimate_tc(const sea_shape& s, const void* Q, const void* K, const void* V,
                               const float* omega, const float* W_dec, float* A_hat, float* est_state,
-                              void* est_split, int32_t* status, cudaStream_t st);
+                              void* est_split, const SelectOut* select_out, int32_t* status, cudaStream_t st);
+// selected: sel, row_counts and mask_bits already hold the selection (the estimator wrote them);
+// only the row pointers and the column indices are produced then.
 sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel,
                             int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
-                            int32_t* row_counts, int32_t* tile_sums, uint32_t* mask_bits,
+                            int32_t* row_counts, int32_t* tile_sums, uint32_t* mask_bits, bool selected,
                             int32_t* status, cudaStream_t st);
 sea_status launch_row_ptr_scan(const int32_t* row_counts, int32_t* tile_sums, int32_t* row_ptr, int rows,
                                cudaStream_t st);

@@ -323,11 +323,15 @@ sea_status launch_estimate_f32(const sea_shape& s, const void* Q, const void* K,
 
 sea_status launch_estimate(const sea_shape& s, const void* Q, const void* K, const void* V,
                            const float* omega, const float* W_dec, float* A_hat, float* est_state,
-                           void* est_split, int32_t* status, cudaStream_t st) {
+                           void* est_split, const SelectOut* select_out, bool* selected, int32_t* status,
+                           cudaStream_t st) {
+  if (selected != nullptr) *selected = false;
   if (s.io == SEA_BF16) {
     // the tensor-core form needs the driver's tensor-map encoder; there is no other bf16 path
     if (!estimate_tc_applicable(s)) return SEA_ERR_CUDA;
-    return launch_estimate_tc(s, Q, K, V, omega, W_dec, A_hat, est_state, est_split, status, st);
+    const bool sel = select_out != nullptr && select_out->sel != nullptr && estimate_tc_selects(s);
+    if (selected != nullptr) *selected = sel;
+    return launch_estimate_tc(s, Q, K, V, omega, W_dec, A_hat, est_state, est_split, sel ? select_out : nullptr, status, st);
   }
   return launch_estimate_f32(s, Q, K, V, omega, W_dec, A_hat, est_state, status, st);
 }

@@ -25,6 +25,7 @@
 // the MMAs; the phases of a chunk follow one another through mbarriers.  Every wait is bounded; a
 // wait that runs out sets SEA_DEV_TIMEOUT and the CTA drains and leaves.
 #include "sea_common.cuh"
+#include "sea_select.cuh"
 #include "sea_tc.cuh"
 
 namespace sea {
@@ -37,6 +38,15 @@ constexpr int kTileBytes = kRows * 128;    // 128 rows x 64 bf16
 constexpr int kParts = 2;                  // row warpgroups: each takes every kParts-th 32-column chunk of a tile
 constexpr int kRowWarps = 4 * kParts;
 constexpr int kThreads = 32 * (kRowWarps + 1);
+// The output kernel has two more warpgroups: the control warp's (copies and MMAs; three warps idle)
+// and one that selects the k_hat largest entries of every row of the A_hat tile while it is in
+// tensor memory.  Registers per thread after the warpgroups re-balance: a warpgroup can only grow
+// by what the others of the CTA have given back.
+constexpr int kThreadsOut = 128 * (kParts + 2);
+constexpr int kRegsOutLaunch = 65536 / kThreadsOut;
+constexpr int kRegsOutRow = 168, kRegsOutCtl = 72, kRegsOutSel = 104;
+static_assert(128 * (kParts * kRegsOutRow + kRegsOutCtl + kRegsOutSel) <= kRegsOutLaunch * kThreadsOut,
+              "register re-balance exceeds the launch allocation");
 constexpr int kWTile = 128;                // decoder columns per pass
 
 // ---- operand preparation -----------------------------------------------------------------
@@ -155,7 +165,17 @@ struct EstParams {
   int32_t* status;
   int BH, T, m, Kc, nchunk, causal;
   int tma_store;                // A_hat leaves through TMA stores (its rows are 16-byte multiples)
+  // selection inside the output kernel (Kc <= 128): null when the caller selects elsewhere
+  int32_t* sel;                 // [BH * T][k_hat] ascending columns
+  int32_t* row_counts;          // [BH * T] keys per row after up-sampling (null: not wanted)
+  uint32_t* mask_bits;          // [BH * T][ceil(Kc / 32)] (null: not wanted)
+  int k_hat, r;
 };
+
+template <int kRegs>
+__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegs)); }
+template <int kRegs>
+__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegs)); }
 
 // ---- kernel 1: chunk key states ---------------------------------------------------------------
 enum { kS_Load = 0, kS_E, kS_Phi, kS_S, kS_Drain, kS_NumBars };
@@ -381,8 +401,8 @@ enum {
 // Named barrier `id` over the 128 threads of one column group of the row warps.
 __device__ __forceinline__ void part_sync(int id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
 
-template <int MP>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int MP, int KSEL>
+__global__ void __launch_bounds__(kThreadsOut, 1)
 favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_om,
                        const __grid_constant__ CUtensorMap map_s, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_phi,
@@ -413,11 +433,13 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   const bool causal = p.causal != 0;
   const int n_ct = (p.Kc + kWTile - 1) / kWTile;
   const bool single = n_ct == 1;
+  const bool selecting = KSEL > 0 && p.sel != nullptr;  // the launcher only asks for it with a single pass
   const int n_items = p.BH * p.nchunk;
   if (tid == 0) {
     for (int i = 0; i < kO_NumBars; ++i) {
-      const bool from_rows = i == kO_Phi || i == kO_P || i == kO_C || (i >= kO_AFree && i < kO_AFree + 2);
-      mbar_init(bar(i), from_rows ? kRowWarps : 1);
+      const bool from_rows = i == kO_Phi || i == kO_P || i == kO_C;
+      const bool tile_read = i >= kO_AFree && i < kO_AFree + 2;  // the rows, and the selecting warps
+      mbar_init(bar(i), tile_read ? kRowWarps + (selecting ? 4 : 0) : (from_rows ? kRowWarps : 1));
     }
     *abort_flag = 0;
     mbar_init_fence();
@@ -428,8 +450,81 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == kRowWarps) {
-    if (lane == 0) {
+  if (warp >= kRowWarps + 4) {
+    // -------------------------------------------------------------- selection from the A_hat tile
+    reg_dec<kRegsOutSel>();
+    if constexpr (KSEL > 0) {
+      if (selecting) {
+        using namespace select;
+        const int quarter = warp & 3, rt = quarter * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+        const int words = (p.Kc + 31) >> 5;
+        uint32_t g = 0;
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++g) {
+          const int bh = item / p.nchunk, chunk = item - bh * p.nchunk;
+          const int row = chunk * kRows + rt;
+          const bool row_ok = row < p.T;
+          const size_t grow = (size_t)bh * p.T + row;
+          const uint32_t b = g & 1;
+          if (!__all_sync(0xffffffffu, mbar_wait(bar(kO_Ahat + b), (g >> 1) & 1, abort_flag))) break;
+          fence_after();
+          // descending list of the KSEL largest values seen; +inf in the slots beyond k_hat keeps the
+          // k_hat-th largest value of the row in the last slot, -inf stands for columns beyond Kc
+          float top[KSEL];
+#pragma unroll
+          for (int q = 0; q < KSEL; ++q) top[q] = q < KSEL - p.k_hat ? INFINITY : -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            if (32 * c < p.Kc) {
+              uint32_t e[32];
+              tmem_ld32(lane_addr + kColAh + 32 * c, e);
+              tmem_ld_wait();
+#pragma unroll
+              for (int h0 = 0; h0 < 32; h0 += KSEL) {
+                float grp[KSEL];
+#pragma unroll
+                for (int j = 0; j < KSEL; ++j) grp[j] = 32 * c + h0 + j < p.Kc ? __uint_as_float(e[h0 + j]) : -INFINITY;
+                merge_group<KSEL>(top, grp);
+              }
+            }
+          }
+          const float tau = top[KSEL - 1];
+          int n_gt = 0;
+#pragma unroll
+          for (int q = 0; q < KSEL; ++q) n_gt += (top[q] != INFINITY && top[q] > tau);
+          int ties_left = p.k_hat - n_gt;
+          uint32_t gt[4] = {0u, 0u, 0u, 0u}, eq[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            if (32 * c < p.Kc) {
+              uint32_t e[32];
+              tmem_ld32(lane_addr + kColAh + 32 * c, e);
+              tmem_ld_wait();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float x = 32 * c + j < p.Kc ? __uint_as_float(e[j]) : -INFINITY;
+                gt[c] |= (x > tau ? 1u : 0u) << j;
+                eq[c] |= (x == tau ? 1u : 0u) << j;
+              }
+            }
+          }
+          warp_arrive(bar(kO_AFree + b), lane);
+          if (row_ok) {
+            int32_t* my_sel = p.sel + grow * p.k_hat;
+            int out = 0, cnt = 0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              if (32 * c < p.Kc)
+                emit_columns(gt[c], eq[c], 32 * c, ties_left, my_sel, out, cnt,
+                             p.mask_bits != nullptr ? p.mask_bits + grow * words + c : nullptr, row, p.r, p.causal);
+            if (p.row_counts != nullptr) p.row_counts[grow] = cnt;
+          }
+        }
+      }
+    }
+  } else if (warp >= kRowWarps) {
+    reg_dec<kRegsOutCtl>();
+    if (warp == kRowWarps && lane == 0) {
       // ------------------------------------------------------------ copies and MMAs
       bool ok = true;
       uint32_t it = 0;          // items done: parity of the per-item barriers
@@ -616,6 +711,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     }
   } else {
     // -------------------------------------------------------------- row warps
+    reg_inc<kRegsOutRow>();
     const int quarter = warp & 3, part = warp >> 2, rt = quarter * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     const bool elected = quarter == 0 && lane == 0;  // issues this column group's stores
@@ -765,7 +861,7 @@ size_t padded_kc(const sea_shape& s) { return ((size_t)s.Kc + 63) / 64 * 64; }  
 template <int MP>
 sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bfloat16* K, const __nv_bfloat16* V,
                      const float* omega, const float* W_dec, float* A_hat, float* state, unsigned char* scratch,
-                     int32_t* status, cudaStream_t st) {
+                     const SelectOut* so, int32_t* status, cudaStream_t st) {
   const int BH = s.B * s.H;
   const int nchunk = (s.T + kRows - 1) / kRows;
   const size_t KcP = padded_kc(s);
@@ -812,11 +908,18 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   // multiple of 16 bytes) the rows store their values themselves
   prm.tma_store = (s.Kc % 4 == 0 && make_map_3d(&ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, A_hat, s.Kc, s.T, BH, 32, kRows)) ? 1 : 0;
   if (!prm.tma_store) ma = mq;  // a valid map that is never used
+  const bool selecting = so != nullptr && so->sel != nullptr && estimate_tc_selects(s);
+  if (selecting) {
+    prm.sel = so->sel;
+    prm.row_counts = so->row_counts;
+    prm.mask_bits = so->mask_bits;
+    prm.k_hat = s.k_hat;
+    prm.r = s.T / s.Kc;
+  }
 
   const size_t smem1 = 1024 + 5 * kTileBytes + 2048 + 8 * kS_NumBars + 16;
   const size_t smem3 = 1024 + (10 + kParts) * kTileBytes + (8 * kO_NumBars + 8 + 127) / 128 * 128 + (1 + kParts) * 128 * 4;
-  if (cudaFuncSetAttribute(favor_state_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
-      cudaFuncSetAttribute(favor_output_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem3) != cudaSuccess)
+  if (cudaFuncSetAttribute(favor_state_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess)
     return SEA_ERR_CUDA;
   const dim3 grid(nchunk, BH);
   favor_state_tc_kernel<MP><<<grid, kThreads, smem1, st>>>(mk, mv, mom, mphi, prm);
@@ -832,7 +935,18 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return SEA_ERR_CUDA;
   const int n_items = BH * nchunk;
-  favor_output_tc_kernel<MP><<<n_items < sms ? n_items : sms, kThreads, smem3, st>>>(mq, mv, mom, ms, mw, ma, mphi, prm);
+  const int grid3 = n_items < sms ? n_items : sms;
+#define SEA_OUT(KS)                                                                                                       \
+  do {                                                                                                                    \
+    if (cudaFuncSetAttribute(favor_output_tc_kernel<MP, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem3) != \
+        cudaSuccess)                                                                                                      \
+      return SEA_ERR_CUDA;                                                                                                \
+    favor_output_tc_kernel<MP, KS><<<grid3, kThreadsOut, smem3, st>>>(mq, mv, mom, ms, mw, ma, mphi, prm);               \
+  } while (0)
+  if (!selecting) SEA_OUT(0);
+  else if (s.k_hat <= 16) SEA_OUT(16);
+  else SEA_OUT(32);
+#undef SEA_OUT
   return check_launch();
 }
 
@@ -857,19 +971,22 @@ size_t estimate_tc_split_bytes(const sea_shape& s) {
 bool estimate_tc_applicable(const sea_shape& s) {
   return s.io == SEA_BF16 && s.m >= 16 && s.m <= 128 && encode_fn() != nullptr;
 }
+// The output kernel can select a row's k_hat largest entries itself while the row's whole A_hat is
+// one tile in tensor memory.
+bool estimate_tc_selects(const sea_shape& s) { return estimate_tc_applicable(s) && s.Kc <= kWTile && s.k_hat <= 32; }
 
 sea_status launch_estimate_tc(const sea_shape& s, const void* Q, const void* K, const void* V, const float* omega,
-                              const float* W_dec, float* A_hat, float* est_state, void* split_buf, int32_t* status,
-                              cudaStream_t st) {
+                              const float* W_dec, float* A_hat, float* est_state, void* split_buf, const SelectOut* so,
+                              int32_t* status, cudaStream_t st) {
   using T = __nv_bfloat16;
   unsigned char* scratch = static_cast<unsigned char*>(split_buf);
   switch (padded_features(s.m)) {
     case 32:
-      return launch_mp<32>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, scratch, status, st);
+      return launch_mp<32>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, scratch, so, status, st);
     case 64:
-      return launch_mp<64>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, scratch, status, st);
+      return launch_mp<64>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, scratch, so, status, st);
     default:
-      return launch_mp<128>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, scratch, status, st);
+      return launch_mp<128>(s, (const T*)Q, (const T*)K, (const T*)V, omega, W_dec, A_hat, est_state, scratch, so, status, st);
   }
 }
 

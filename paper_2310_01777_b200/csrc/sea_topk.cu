@@ -7,9 +7,12 @@
 // bit-by-bit search with warp-wide counts, and columns holding exactly that key are taken
 // in ascending column order until k_hat are chosen.
 #include "sea_common.cuh"
+#include "sea_select.cuh"
 
 namespace sea {
 namespace {
+
+using namespace select;
 
 constexpr int kWarpsPerCta = 8;
 constexpr int kScanThreads = 256;
@@ -90,47 +93,6 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
 // as equal exactly as the bit search's keys do.
 constexpr int kThreadRows = 128;  // threads (= rows) per CTA
 
-// x >= y afterwards when kDescending, x <= y otherwise
-template <bool kDescending>
-__device__ __forceinline__ void cmp_exchange(float& x, float& y) {
-  const float hi = fmaxf(x, y), lo = fminf(x, y);
-  x = kDescending ? hi : lo;
-  y = kDescending ? lo : hi;
-}
-template <int N>
-__device__ __forceinline__ void bitonic_sort_ascending(float (&a)[N]) {
-#pragma unroll
-  for (int k = 2; k <= N; k <<= 1)
-#pragma unroll
-    for (int j = k >> 1; j > 0; j >>= 1)
-#pragma unroll
-      for (int i = 0; i < N; ++i) {
-        const int l = i ^ j;
-        if (l > i) {
-          if ((i & k) == 0) cmp_exchange<false>(a[i], a[l]);
-          else cmp_exchange<true>(a[i], a[l]);
-        }
-      }
-}
-template <int N>
-__device__ __forceinline__ void bitonic_merge_descending(float (&a)[N]) {
-#pragma unroll
-  for (int j = N >> 1; j > 0; j >>= 1)
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-      const int l = i ^ j;
-      if (l > i) cmp_exchange<true>(a[i], a[l]);
-    }
-}
-// top (descending) <- the KMAX largest of top and grp (any order; destroyed)
-template <int KMAX>
-__device__ __forceinline__ void merge_group(float (&top)[KMAX], float (&grp)[KMAX]) {
-  bitonic_sort_ascending<KMAX>(grp);
-#pragma unroll
-  for (int s = 0; s < KMAX; ++s) top[s] = fmaxf(top[s], grp[s]);
-  bitonic_merge_descending<KMAX>(top);
-}
-
 template <int KMAX, bool kVec>
 __global__ void __launch_bounds__(kThreadRows)
 topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
@@ -192,25 +154,8 @@ topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ s
         eq |= (x == tau ? 1u : 0u) << j;
       }
     }
-    // the lowest ties_left columns among the equal ones
-    uint32_t eq_taken = eq;
-    if (__popc(eq) > ties_left) {
-      eq_taken = 0u;
-      for (int t = 0; t < ties_left; ++t) {
-        const uint32_t low = eq & (0u - eq);
-        eq_taken |= low;
-        eq ^= low;
-      }
-    }
-    ties_left -= __popc(eq_taken);
-    uint32_t word = gt | eq_taken;
-    if (mask_bits != nullptr) mask_bits[(size_t)row * words + (j0 >> 5)] = word;
-    while (word) {
-      const int j = j0 + __ffs(word) - 1;
-      word &= word - 1u;
-      my_sel[out++] = j;
-      cnt += causal ? max(0, min(r, i + 1 - j * r)) : r;
-    }
+    emit_columns(gt, eq, j0, ties_left, my_sel, out, cnt, mask_bits != nullptr ? mask_bits + (size_t)row * words + (j0 >> 5) : nullptr,
+                 i, r, causal);
   }
   if (row_counts != nullptr) row_counts[row] = cnt;
 }
@@ -351,12 +296,16 @@ sea_status launch_row_ptr_scan(const int32_t* row_counts, int32_t* tile_sums, in
 
 sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel, int32_t* row_ptr,
                             int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts,
-                            int32_t* tile_sums, uint32_t* mask_bits, int32_t* status, cudaStream_t st) {
+                            int32_t* tile_sums, uint32_t* mask_bits, bool selected, int32_t* status,
+                            cudaStream_t st) {
   const int rows = s.B * s.H * s.T;
   const int r = s.T / s.Kc;
   int32_t* counts = s.causal ? row_counts : nullptr;
   const int vpl = (s.Kc + 31) / 32;
-  if (s.Kc <= kThreadMaxKc && s.k_hat <= kThreadMaxK) {
+  sea_status rc = SEA_OK;
+  if (selected) {
+    // sel, the counts and the bits are in place already
+  } else if (s.Kc <= kThreadMaxKc && s.k_hat <= kThreadMaxK) {
     // a short row and few columns to keep: one thread per row
     const int grid = (rows + kThreadRows - 1) / kThreadRows;
 #define SEA_TOPK_THREAD(KM)                                                                                     \
@@ -381,8 +330,7 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
   else if (vpl <= 32) launch_topk<32>(A_hat, sel, counts, mask_bits, rows, s, st);
   else if (vpl <= 64) launch_topk<64>(A_hat, sel, counts, mask_bits, rows, s, st);
   else return SEA_ERR_UNSUPPORTED;
-  sea_status rc = check_launch();
-  if (rc != SEA_OK) return rc;
+  if (!selected && (rc = check_launch()) != SEA_OK) return rc;
 
   if (s.causal) {
     if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
@@ -470,5 +418,5 @@ extern "C" sea_status sea_topk_mask_static(const sea_shape* shape, const float* 
   // by the kernels, the status word is the one thing that has to start at zero
   if (cudaMemsetAsync(scratch, 0, sizeof(int32_t), st) != cudaSuccess) return SEA_ERR_CUDA;
   return launch_topk_mask(*shape, A_hat, sel, row_ptr, col_idx, nnz_cap, scratch + kStaticHead,
-                          scratch + kStaticHead + kStaticMaxRows, nullptr, scratch, st);
+                          scratch + kStaticHead + kStaticMaxRows, nullptr, false, scratch, st);
 }

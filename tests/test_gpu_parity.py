@@ -106,7 +106,15 @@ def test_tensor_core_estimator_shapes(w):
         check_a_hat(run.A_hat[b, h].cpu().numpy(), ref)
 
 
-@pytest.mark.parametrize("w", SMALL_CASES[:6], ids=lambda w: w.name)
+# every small shape once; among them bf16 shapes with Kc <= 128, where the fused call selects inside
+# the estimator's output kernel (k_hat up to 16, and 17 .. 32), and shapes where it does not
+FUSED_CASES = list({w.name: w for w in SMALL_CASES + TILE_CASES + [
+    small("sel32", dtype="bf16", T=256, Kc=128, k_hat=29, causal=True, m=64, B=2),   # the 32-slot list
+    small("sel_three_words", dtype="bf16", T=192, Kc=96, k_hat=16, causal=True, m=16),  # Kc of three words, T % 128 != 0
+]}.values())
+
+
+@pytest.mark.parametrize("w", FUSED_CASES, ids=lambda w: w.name)
 def test_fused_call_equals_stage_calls_bitwise(w):
     a = GpuRun(w)
     a.estimate(); a.topk_mask(); a.sparse_attn(); a.sync()
