@@ -44,7 +44,7 @@ constexpr int kThreads = 32 * (kRowWarps + 1);
 // by what the others of the CTA have given back.
 constexpr int kThreadsOut = 128 * (kParts + 2);
 constexpr int kRegsOutLaunch = 65536 / kThreadsOut;
-constexpr int kRegsOutRow = 168, kRegsOutCtl = 72, kRegsOutSel = 104;
+constexpr int kRegsOutRow = 168, kRegsOutCtl = 104, kRegsOutSel = 72;
 static_assert(128 * (kParts * kRegsOutRow + kRegsOutCtl + kRegsOutSel) <= kRegsOutLaunch * kThreadsOut,
               "register re-balance exceeds the launch allocation");
 constexpr int kWTile = 128;                // decoder columns per pass
