@@ -466,7 +466,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           const bool row_ok = row < p.T;
           const size_t grow = (size_t)bh * p.T + row;
           const uint32_t b = g & 1;
-          if (!__all_sync(0xffffffffu, mbar_wait(bar(kO_Ahat + b), (g >> 1) & 1, abort_flag))) break;
+          if (!__all_sync(0xffffffffu, mbar_wait_idle(bar(kO_Ahat + b), (g >> 1) & 1, abort_flag))) break;
           fence_after();
           // descending list of the KSEL largest values seen; +inf in the slots beyond k_hat keeps the
           // k_hat-th largest value of the row in the last slot, -inf stands for columns beyond Kc

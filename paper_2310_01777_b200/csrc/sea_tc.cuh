@@ -51,6 +51,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+// The same for a role whose hand-offs happen once per work item and that is off the critical path:
+// it sleeps between polls, so that its polling takes no issue slots from the warps that compute.
+__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i) {
+      if (mbar_try(bar, parity)) return true;
+      __nanosleep(200);
+    }
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitNs) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
 // For the way out: waits for an armed copy barrier whatever the abort flag says (a CTA must not
 // leave while copies into its shared memory are in flight), bounded by time alone.
 __device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity) {
