@@ -207,12 +207,16 @@ sea_status sea_attention_grouped(const sea_shape* shape, const void* Q, const vo
                                  void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
- * sea_attention for callers whose tensors live in HOST memory (pinned memory
- * gives asynchronous copies).  hQ, hK, hV, homega, hW_dec are copied to staging
- * areas inside `ws` on the stream, the layer runs, and O is copied back to hO.
- * Bytes needed: sea_workspace_host_bytes().  The call returns after the stream
- * has been synchronised, so hO is valid on return.  The paper has no
- * counterpart; this is the end-to-end form of the call above.
+ * sea_attention for callers whose tensors live in HOST memory.  hQ, hK, hV,
+ * homega, hW_dec are copied to staging areas inside `ws`, the layer runs, and O
+ * is copied back to hO.  The heads are independent, so the call is a pipeline
+ * over up to eight slices of them: a slice is computed on `cuda_stream` while
+ * the next slice's inputs arrive and the previous slice's O leaves on two
+ * streams that the call creates and destroys (with a few events); this overlap
+ * needs pinned host memory, pageable memory gives the same result serially.
+ * Bytes needed: sea_workspace_host_bytes().  The call returns after all its work
+ * has finished, so hO is valid on return.  Not for use during stream capture.
+ * The paper has no counterpart; this is the end-to-end form of the call above.
  */
 sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes);
 sea_status sea_attention_host(const sea_shape* shape, const void* hQ, const void* hK,

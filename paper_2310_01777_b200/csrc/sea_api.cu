@@ -304,21 +304,72 @@ sea_status sea_attention_host(const sea_shape* shape, const void* hQ, const void
   char* dO = dV + qkv;
   char* dOm = dO + qkv;
   char* dWd = dOm + align_up(om_b, 256);
-  if (cudaMemcpyAsync(dQ, hQ, qkv_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(dK, hK, qkv_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(dV, hV, qkv_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(dOm, homega, om_b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(dWd, hW_dec, wd_b, cudaMemcpyHostToDevice, st) != cudaSuccess)
-    return SEA_ERR_CUDA;
-  const int keep = Launch::count();
-  rc = sea_attention(shape, dQ, dK, dV, reinterpret_cast<const float*>(dOm),
-                     reinterpret_cast<const float*>(dWd), nullptr, dO, nullptr, nullptr, nullptr, nullptr,
-                     0, nullptr, ws, inner, cuda_stream);
-  (void)keep;
-  if (rc != SEA_OK) return rc;
-  if (cudaMemcpyAsync(hO, dO, qkv_b, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SEA_ERR_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return SEA_ERR_CUDA;
-  return SEA_OK;
+
+  // The heads are independent, so the call runs as a pipeline over slices of them: while one slice
+  // is computed on the caller's stream, the next one's Q, K, V come in on a second stream and the
+  // previous one's O goes out on a third (the link carries both directions at once).  The streams
+  // and events live for this call only.
+  const int BH = shape->B * shape->H;
+  int nslice = 1;
+  for (int c = 8; c >= 2; c >>= 1)
+    if (BH % c == 0 && BH / c >= 8) {
+      nslice = c;
+      break;
+    }
+  sea_shape sub = *shape;
+  sub.B = 1;
+  sub.H = BH / nslice;
+  const size_t slice_b = qkv_b / nslice;
+
+  constexpr int kMaxSlices = 8;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t ev_begin = nullptr, ev_in[kMaxSlices] = {}, ev_done[kMaxSlices] = {};
+  bool good = cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ev_begin, cudaEventDisableTiming) == cudaSuccess;
+  for (int c = 0; c < nslice && good; ++c)
+    good = cudaEventCreateWithFlags(&ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ev_done[c], cudaEventDisableTiming) == cudaSuccess;
+  rc = good ? SEA_OK : SEA_ERR_CUDA;
+  int launches = 0;
+  // the staging areas may still be read by work the caller enqueued earlier on `st`
+  if (rc == SEA_OK && (cudaEventRecord(ev_begin, st) != cudaSuccess || cudaStreamWaitEvent(s_in, ev_begin, 0) != cudaSuccess ||
+                       cudaStreamWaitEvent(s_out, ev_begin, 0) != cudaSuccess))
+    rc = SEA_ERR_CUDA;
+  if (rc == SEA_OK && (cudaMemcpyAsync(dOm, homega, om_b, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+                       cudaMemcpyAsync(dWd, hW_dec, wd_b, cudaMemcpyHostToDevice, s_in) != cudaSuccess))
+    rc = SEA_ERR_CUDA;
+  for (int c = 0; c < nslice && rc == SEA_OK; ++c) {
+    const size_t off = (size_t)c * slice_b;
+    if (cudaMemcpyAsync(dQ + off, static_cast<const char*>(hQ) + off, slice_b, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+        cudaMemcpyAsync(dK + off, static_cast<const char*>(hK) + off, slice_b, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+        cudaMemcpyAsync(dV + off, static_cast<const char*>(hV) + off, slice_b, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+        cudaEventRecord(ev_in[c], s_in) != cudaSuccess || cudaStreamWaitEvent(st, ev_in[c], 0) != cudaSuccess) {
+      rc = SEA_ERR_CUDA;
+      break;
+    }
+    rc = sea_attention(&sub, dQ + off, dK + off, dV + off, reinterpret_cast<const float*>(dOm),
+                       reinterpret_cast<const float*>(dWd), nullptr, dO + off, nullptr, nullptr, nullptr, nullptr, 0,
+                       nullptr, ws, inner, cuda_stream);
+    launches += Launch::count();
+    if (rc != SEA_OK) break;
+    if (cudaEventRecord(ev_done[c], st) != cudaSuccess || cudaStreamWaitEvent(s_out, ev_done[c], 0) != cudaSuccess ||
+        cudaMemcpyAsync(static_cast<char*>(hO) + off, dO + off, slice_b, cudaMemcpyDeviceToHost, s_out) != cudaSuccess)
+      rc = SEA_ERR_CUDA;
+  }
+  // everything enqueued has to finish before the streams and events go away, success or not
+  if (s_in && cudaStreamSynchronize(s_in) != cudaSuccess && rc == SEA_OK) rc = SEA_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess && rc == SEA_OK) rc = SEA_ERR_CUDA;
+  if (s_out && cudaStreamSynchronize(s_out) != cudaSuccess && rc == SEA_OK) rc = SEA_ERR_CUDA;
+  for (int c = 0; c < kMaxSlices; ++c) {
+    if (ev_in[c]) cudaEventDestroy(ev_in[c]);
+    if (ev_done[c]) cudaEventDestroy(ev_done[c]);
+  }
+  if (ev_begin) cudaEventDestroy(ev_begin);
+  if (s_in) cudaStreamDestroy(s_in);
+  if (s_out) cudaStreamDestroy(s_out);
+  Launch::count() = launches;
+  return rc;
 }
 
 sea_status sea_device_status(void* ws, int32_t* out, int32_t clear, void* cuda_stream) {
