@@ -347,7 +347,7 @@ def main():
         # what the tile kernel executes: per (query tile, key tile) pair S = Q K^T in both passes and
         # P V with P as bf16 head + remainder, 2 * 128 * 128 * 64 FLOPs each
         r = w.T // w.Kc
-        tiled = w.dtype == "bf16" and w.T % 128 == 0 and r >= 4 and r & (r - 1) == 0 and w.k_hat * 96 >= w.Kc
+        tiled = w.dtype == "bf16" and w.T % 128 == 0 and r >= 4 and r & (r - 1) == 0 and w.k_hat * 40 >= w.Kc
         nq = w.T // 128
         pairs = w.B * w.H * (nq * (nq + 1) // 2 if w.causal else nq * nq)
         exec_flops = pairs * 4 * (2 * 128 * 128 * w.d) if tiled else None

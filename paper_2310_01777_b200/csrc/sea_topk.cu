@@ -21,12 +21,16 @@ constexpr int kScanTile = kScanThreads * kScanPerThread;
 constexpr int kThreadMaxKc = 128;  // shapes handled with one thread per row: the sorted-list walk costs
 constexpr int kThreadMaxK = 32;    // Kc * k_hat min/max pairs per row, the bit search about 64 * Kc / 32 * 32
 
+constexpr int kHistBins = 256;
+constexpr int kHistShift = 17;
+
 // One warp per row; lane l holds columns l, l+32, ... (VPL of them).
 template <int VPL>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
                  int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc, int k_hat,
                  int seq_len, int r, int causal) {
+  __shared__ int hist_all[kWarpsPerCta][kHistBins];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kWarpsPerCta + warp;
   if (row >= rows) return;
@@ -37,16 +41,104 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
     const int col = lane + 32 * t;
     key[t] = col < Kc ? order_key(__ldg(a + col)) : 0u;  // padding sorts below every real value
   }
-  // k_hat-th largest key: the largest tau with |{key >= tau}| >= k_hat
+  // k_hat-th largest key: the largest tau with |{key >= tau}| >= k_hat.  First try: the row's
+  // largest key `top`, a histogram of (top - key) >> kHistShift over the kHistBins steps below it
+  // (1/64 of an octave each: four octaves of magnitudes), a scan for the step that holds tau, and a
+  // search by ballots among the keys inside that step (one per lane).
   uint32_t tau = 0u;
+  bool found = false;
+  {
+    int* hist = hist_all[warp];
+    uint32_t top = 0u;
 #pragma unroll
-  for (int bit = 31; bit >= 0; --bit) {
-    const uint32_t cand = tau | (1u << bit);
-    int c = 0;
+    for (int t = 0; t < VPL; ++t) top = max(top, key[t]);
+    top = __reduce_max_sync(0xffffffffu, top);
+    // step x is kept at word (x & 7) * 32 + (x >> 3): lane x >> 3 owns it and reads it without conflicts
 #pragma unroll
-    for (int t = 0; t < VPL; ++t) c += key[t] >= cand;
-    c = __reduce_add_sync(0xffffffffu, c);
-    if (c >= k_hat) tau = cand;
+    for (int j = 0; j < kHistBins / 32; ++j) hist[j * 32 + lane] = 0;
+    __syncwarp();
+#pragma unroll
+    for (int t = 0; t < VPL; ++t) {
+      const uint32_t x = (top - key[t]) >> kHistShift;
+      if (x < (uint32_t)kHistBins && lane + 32 * t < Kc) atomicAdd(&hist[(x & 7u) * 32u + (x >> 3)], 1);
+    }
+    __syncwarp();
+    int bins[kHistBins / 32], mine = 0;
+#pragma unroll
+    for (int j = 0; j < kHistBins / 32; ++j) {
+      bins[j] = hist[j * 32 + lane];
+      mine += bins[j];
+    }
+    int inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
+    }
+    const int total = __shfl_sync(0xffffffffu, inc, 31);
+    if (total >= k_hat) {
+      int over = inc - mine;  // keys in the steps above this lane's
+      const bool owner = over < k_hat && over + mine >= k_hat;
+      int step = 0;
+      if (owner) {
+#pragma unroll
+        for (int j = 0; j < kHistBins / 32; ++j)
+          if (over + bins[j] < k_hat && step == j) {
+            over += bins[j];
+            ++step;
+          }
+        step += lane * (kHistBins / 32);
+      }
+      const int src = __ffs(__ballot_sync(0xffffffffu, owner)) - 1;
+      step = __shfl_sync(0xffffffffu, step, src);
+      const int above = __shfl_sync(0xffffffffu, over, src);
+      // the keys inside the step, one per lane when there are at most 32
+      int inside = 0;
+#pragma unroll
+      for (int t = 0; t < VPL; ++t) inside += ((top - key[t]) >> kHistShift) == (uint32_t)step;
+      int pos = inside;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, pos, o);
+        if (lane >= o) pos += v;
+      }
+      const int n_in = __shfl_sync(0xffffffffu, pos, 31);
+      if (n_in <= 32) {
+        uint32_t* list = reinterpret_cast<uint32_t*>(hist);  // the counters are no longer needed
+        __syncwarp();
+        pos -= inside;
+        constexpr uint32_t kFine = (1u << kHistShift) - 1u;
+#pragma unroll
+        for (int t = 0; t < VPL; ++t) {
+          const uint32_t rel = top - key[t];
+          if ((rel >> kHistShift) == (uint32_t)step) list[pos++] = kFine - (rel & kFine);  // grows with the key
+        }
+        __syncwarp();
+        const bool have = lane < n_in;
+        const uint32_t fine_mine = have ? list[lane] : 0u;
+        uint32_t fine = 0u;
+#pragma unroll
+        for (int bit = kHistShift - 1; bit >= 0; --bit) {
+          const uint32_t cand = fine | (1u << bit);
+          if (__popc(__ballot_sync(0xffffffffu, have && fine_mine >= cand)) + above >= k_hat) fine = cand;
+        }
+        tau = top - (((uint32_t)step << kHistShift) | (kFine - fine));
+        found = true;
+      }
+    }
+    __syncwarp();
+  }
+  if (!found) {
+    // bit by bit with warp-wide counts over all keys
+#pragma unroll
+    for (int bit = 31; bit >= 0; --bit) {
+      const uint32_t cand = tau | (1u << bit);
+      int c = 0;
+#pragma unroll
+      for (int t = 0; t < VPL; ++t) c += key[t] >= cand;
+      c = __reduce_add_sync(0xffffffffu, c);
+      if (c >= k_hat) tau = cand;
+    }
   }
   int n_gt = 0;
 #pragma unroll
