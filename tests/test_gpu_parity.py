@@ -203,6 +203,30 @@ def test_topk_ties_and_signed_zeros_are_bit_exact():
     check_head_against_oracle(run, 0, 0, check_estimate=False)
 
 
+@pytest.mark.parametrize("Kc,k_hat", [(256, 16), (512, 200), (1024, 33)])
+def test_wide_row_selection_paths_are_bit_exact(Kc, k_hat):
+    """Rows wider than 128 columns are selected by a warp per row: a histogram below the row's
+    largest value, or, when the threshold lies outside the histogram's span or too many values
+    share its step, a bit search.  Rows built to take each way, checked against the oracle."""
+    w = small("wide_paths", T=2 * Kc, Kc=Kc, k_hat=k_hat, m=0, H=1)
+    host = make_inputs(w)
+    a = host["A_hat"]
+    a[0, 0, 0, :] = 0.25                       # all equal: every value shares the threshold's step
+    a[0, 0, 1, :] = -torch.rand(Kc) - 1.0      # one large value, the rest negative: the threshold
+    a[0, 0, 1, 7] = 3.0                        #   is far below the histogram's span
+    a[0, 0, 2, ::2] = -0.0                     # signed zeros tie
+    a[0, 0, 2, 1::2] = 0.0
+    a[0, 0, 3, :] = torch.round(a[0, 0, 3, :] * 4) / 4     # heavy duplication
+    a[0, 0, 4, :] = 1.0 + torch.arange(Kc) * 2.0 ** -20     # many distinct values inside one step
+    a[0, 0, 5, :] = a[0, 0, 5, :] * 1e-30                   # tiny magnitudes
+    a[0, 0, 6, :] = a[0, 0, 6, :].abs() * 1e30              # huge magnitudes
+    a[0, 0, 7, :] = -a[0, 0, 7, :].abs() - 0.5              # all negative
+    run = GpuRun(w, inputs=host)
+    run.topk_mask(); run.sparse_attn(); run.sync()
+    assert run.status() == 0
+    check_head_against_oracle(run, 0, 0, check_estimate=False)
+
+
 def test_small_nnz_cap_sets_status_and_stays_in_bounds():
     w = small("cap", causal=False, T=128, Kc=32, k_hat=4, H=1, m=0)
     run = GpuRun(w)
