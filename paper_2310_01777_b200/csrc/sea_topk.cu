@@ -352,7 +352,18 @@ fill_col_idx_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__
     n = (int)max(0ll, min((long long)n, nnz_cap - base));
   }
   const int32_t* my_sel = sel + (size_t)row * k_hat;
-  if (log2r >= 0) {  // r a power of two: the run and the offset inside it are a shift and a mask
+  if (log2r >= 0 && k_hat <= 32) {
+    // r a power of two: the run and the offset inside it are a shift and a mask; the row's
+    // selected columns sit one per lane and are fetched by shuffles
+    const int mine = lane < k_hat ? __ldg(my_sel + lane) << log2r : 0;
+    int32_t* out = col_idx + base;
+    const int n_up = (n + 31) & ~31;  // every lane takes part in the shuffles
+#pragma unroll 4
+    for (int pos = lane; pos < n_up; pos += 32) {
+      const int start = __shfl_sync(0xffffffffu, mine, (pos >> log2r) & 31);
+      if (pos < n) out[pos] = start + (pos & (r - 1));
+    }
+  } else if (log2r >= 0) {
     for (int pos = lane; pos < n; pos += 32)
       col_idx[(size_t)base + pos] = (__ldg(my_sel + (pos >> log2r)) << log2r) + (pos & (r - 1));
   } else {
