@@ -26,6 +26,15 @@ the paper's steps in the paper's order:
                         largest of its H * Kc entries are kept (no exchange along
                         T); equal values go to the lower flattened index
                         h * Kc + c.  Heads then hold different numbers of columns.
+    topk_select_causal_aware
+                        the per-query selection restricted, for a causal row i,
+                        to the compressed columns that hold at least one key
+                        j <= i (columns 0 .. floor(i / r)); a row keeps
+                        min(k_hat, floor(i / r) + 1) columns, so no row is left
+                        without keys.  (The paper resizes every causal row of the
+                        estimate to its own width, App. "Visualization of
+                        intermediate buffers"; this is the part of that which the
+                        fixed-ratio interpolation used here can express.)
     expand_mask         Sec. 3.1 "Linear Sparse Attention Mask Generation" and
                         App. "Sparse Interpolation": nearest-neighbour
                         up-sampling of the compressed mask done on indices; a
@@ -62,6 +71,7 @@ __all__ = [
     "estimate_head",
     "topk_select",
     "topk_select_grouped",
+    "topk_select_causal_aware",
     "sea_attention_grouped_batch",
     "expand_mask",
     "sparse_attention",
@@ -154,6 +164,24 @@ def topk_select_grouped(A_hat, k_hat: int):
         taken = taken.reshape(H, Kc)
         for h in range(H):
             cols[h][t] = np.flatnonzero(taken[h])
+    return cols
+
+
+def topk_select_causal_aware(A_hat, k_hat: int, T: int):
+    """Rows of A_hat [T, Kc] are queries 0 .. T-1 of a causal head.  Returns the list of ascending
+    column arrays: row i chooses among columns 0 .. floor(i / r), r = T / Kc."""
+    A_hat = _f64(A_hat)
+    n, Kc = A_hat.shape
+    if n != T or T % Kc != 0:
+        raise ValueError("one row per query, T a multiple of Kc")
+    if not 1 <= k_hat <= Kc:
+        raise ValueError("k_hat out of range")
+    r = T // Kc
+    cols = []
+    for i in range(T):
+        visible = i // r + 1  # columns that start at or before key i
+        order = np.argsort(-A_hat[i, :visible], kind="stable")
+        cols.append(np.sort(order[: min(k_hat, visible)]))
     return cols
 
 

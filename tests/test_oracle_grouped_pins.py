@@ -168,3 +168,51 @@ def test_grouped_pins_catch_planted_mistakes():
 
     for bad in (grouped_along_T, per_query, smallest):
         assert bad(A, k_hat) != want
+
+
+# ---------------------------------------------------------------------------
+# Causal-aware per-query selection: only columns that hold a visible key compete.
+# ---------------------------------------------------------------------------
+def test_causal_aware_selection_bruteforce_and_invariants():
+    g = rng(31)
+    T, Kc, k_hat = 48, 12, 5
+    r = T // Kc
+    A = np.round(g.standard_normal((T, Kc)) * 2) / 2  # duplicates: ties go to the lower column
+    cols = orc.topk_select_causal_aware(A, k_hat, T)
+    for i in range(T):
+        visible = i // r + 1
+        order = sorted(range(visible), key=lambda c: (-float(A[i, c]), c))
+        assert list(cols[i]) == sorted(order[: min(k_hat, visible)])
+        assert len(cols[i]) == min(k_hat, visible)
+    row_ptr, col_idx = orc.expand_mask(cols, T, Kc, True)
+    counts = np.diff(row_ptr)
+    assert np.all(counts >= 1), "no causal row is left without keys"
+    for i in range(T):
+        js = col_idx[row_ptr[i]:row_ptr[i + 1]]
+        assert np.all(js <= i) and np.all(np.diff(js) > 0)
+    # once every column is visible and the row's k_hat best lie among them, it is the per-query selection
+    plain = orc.topk_select(A, k_hat)
+    for i in range(T - r, T):
+        assert list(cols[i]) == list(plain[i])
+    # where the plain selection already avoids invisible columns the two agree, elsewhere they differ
+    differ = sum(list(cols[i]) != [c for c in plain[i]] for i in range(T))
+    assert differ > 0
+
+
+def test_causal_aware_first_rows_are_dense_causal_attention():
+    """While floor(i / r) + 1 <= k_hat every visible column is kept: rows 0 .. k_hat * r - 1 see
+    every key j <= i, i.e. dense causal attention there."""
+    g = rng(32)
+    T, Kc, k_hat, d = 64, 16, 4, 8
+    r = T // Kc
+    Q, K, V = (g.standard_normal((T, d)) for _ in range(3))
+    A = g.standard_normal((T, Kc))
+    cols = orc.topk_select_causal_aware(A, k_hat, T)
+    row_ptr, col_idx = orc.expand_mask(cols, T, Kc, True)
+    O, P = orc.sparse_attention(Q, K, V, row_ptr, col_idx, 0.3)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q)[None], torch.from_numpy(K)[None], torch.from_numpy(V)[None], is_causal=True,
+        scale=0.3)[0].numpy()
+    n_dense = k_hat * r
+    np.testing.assert_allclose(O[:n_dense], ref[:n_dense], atol=1e-12)
+    assert np.array_equal(np.diff(row_ptr)[:n_dense], np.arange(1, n_dense + 1))
