@@ -18,8 +18,10 @@ metric is quoted.  One JSON line is printed by rank 0.
              against the measured dense bf16 peak.
   stages     per-stage milliseconds from a second pass that calls the three stage entry points
              with events between them (same kernels as the fused call).
-  grouped    the same step with the causal-per-batch grouping (sea_attention_grouped) on this
-             rank, and its selection and sparse stages; per-rank, not part of `value`.
+  grouped, causal_aware
+             the same step with the causal-per-batch grouping (sea_attention_grouped) and with the
+             causal-aware per-query selection (sea_attention_causal_aware) on this rank, and their
+             selection and sparse stages; per-rank, not part of `value`.
   cpu_baseline  the fp64 oracle on a bounded sample of heads, on this machine's host cores.
 
 With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no
@@ -292,14 +294,13 @@ def main():
     if not torch.equal(hO, O.cpu()):
         raise SystemExit("host entry point and device entry point disagree")
 
-    # ---- timed region 4: the causal-per-batch grouping (fused call, then its stages) ----
-    grouped = None
-    if w.Kc % 4 == 0 and w.H * w.Kc <= 32768:
+    # ---- timed region 4: the selections that leave as bit masks (fused call, then the stages) ----
+    def time_bits_mode(label, fused_fn, topk_fn):
         bits = torch.empty((w.rows, (w.Kc + 31) // 32), dtype=torch.int32, device=dev)
 
         def gstep():
-            sea.sea_attention_grouped(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O, ws, A_hat=A_hat,
-                                      mask_bits=bits, row_ptr=row_ptr, col_idx=col_idx, P=P)
+            fused_fn(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O, ws, A_hat=A_hat, mask_bits=bits,
+                     row_ptr=row_ptr, col_idx=col_idx, P=P)
 
         for _ in range(3):
             flush.zero_()
@@ -318,18 +319,26 @@ def main():
         for e in gsev:
             flush.zero_()
             e[0].record()
-            sea.sea_topk_mask_grouped(shape, A_hat, bits, row_ptr, col_idx, ws)
+            topk_fn(shape, A_hat, bits, row_ptr, col_idx, ws)
             e[1].record()
             sea.sea_sparse_attn_masked(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, bits, O, P, ws)
             e[2].record()
         torch.cuda.synchronize(dev)
         if sea.sea_device_status(ws) != 0:
-            raise SystemExit("device status word set by the grouped path")
-        grouped = {"grouping": "causal-per-batch", "ms_per_step": g_ms, "value": w.B * w.T / (g_ms / 1e3),
-                   "unit": "tokens/s", "gpu_launches_per_step": g_launches,
-                   "stages_ms": {"topk_mask_grouped": sum(e[0].elapsed_time(e[1]) for e in gsev) / args.steps,
-                                 "sparse_attn_masked": sum(e[1].elapsed_time(e[2]) for e in gsev) / args.steps},
-                   "nnz": int(row_ptr[-1])}
+            raise SystemExit(f"device status word set by the {label} path")
+        return {"selection": label, "ms_per_step": g_ms, "value": w.B * w.T / (g_ms / 1e3), "unit": "tokens/s",
+                "gpu_launches_per_step": g_launches,
+                "stages_ms": {"topk_mask": sum(e[0].elapsed_time(e[1]) for e in gsev) / args.steps,
+                              "sparse_attn_masked": sum(e[1].elapsed_time(e[2]) for e in gsev) / args.steps},
+                "nnz": int(row_ptr[-1])}
+
+    grouped = None
+    if w.Kc % 4 == 0 and w.H * w.Kc <= 32768:
+        grouped = time_bits_mode("causal-per-batch", sea.sea_attention_grouped, sea.sea_topk_mask_grouped)
+    causal_aware = None
+    if w.causal:
+        causal_aware = time_bits_mode("causal-aware per-query", sea.sea_attention_causal_aware,
+                                      sea.sea_topk_mask_causal_aware)
 
     ms_per_step = total_ms / args.steps
     if world > 1:
@@ -366,6 +375,7 @@ def main():
             "stages_ms": {"estimate": stage_ms[0], "topk_mask": stage_ms[1], "sparse_attn": stage_ms[2]},
             "nnz": nnz,
             "grouped": grouped,
+            "causal_aware": causal_aware,
             "roofline": {"kernel": "sparse_attn_tiles_tc_kernel" if tiled else "sparse_attn_blocks_tma_kernel",
                          "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_source": f"{peak_kind} HBM copy bandwidth",

@@ -207,6 +207,27 @@ sea_status sea_attention_grouped(const sea_shape* shape, const void* Q, const vo
                                  void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Causal-aware per-query selection (causal shapes only; other shapes return
+ * SEA_ERR_UNSUPPORTED).  The paper resizes every causal row of the estimate to the
+ * row's own width (App. "Visualization of intermediate buffers"), so a row never
+ * spends its budget on keys it may not see.  With the fixed interpolation ratio
+ * used here that becomes: row i chooses its k_hat largest entries among the
+ * compressed columns that hold a key j <= i (columns 0 .. floor(i / r)) and keeps
+ * min(k_hat, floor(i / r) + 1) of them; no row is left without keys, and the first
+ * k_hat*r rows of a head see every key up to their own.  Ties as in sea_topk_mask.
+ * Outputs and the sparse stage as for sea_topk_mask_grouped / sea_sparse_attn_masked
+ * (a row keeps at most k_hat columns, so the budget rule of the latter holds).
+ */
+sea_status sea_topk_mask_causal_aware(const sea_shape* shape, const float* A_hat, uint32_t* mask_bits,
+                                      int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                                      void* ws, size_t ws_bytes, void* cuda_stream);
+sea_status sea_attention_causal_aware(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                                      const float* omega, const float* W_dec, const float* A_hat_in,
+                                      void* O, float* A_hat, uint32_t* mask_bits, int32_t* row_ptr,
+                                      int32_t* col_idx, int64_t nnz_cap, void* P,
+                                      void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * sea_attention for callers whose tensors live in HOST memory.  hQ, hK, hV,
  * homega, hW_dec are copied to staging areas inside `ws`, the layer runs, and O
  * is copied back to hO.  The heads are independent, so the call is a pipeline

@@ -178,13 +178,22 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
                             reinterpret_cast<float*>(w + L.p_scratch), status, st);
 }
 
-sea_status sea_topk_mask_grouped(const sea_shape* shape, const float* A_hat, uint32_t* mask_bits,
-                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* ws,
-                                 size_t ws_bytes, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+// The two selections whose rows keep differing numbers of columns (the result leaves as bits).
+enum class BitsMode { kPerBatch, kCausalAware };
+bool bits_mode_supported(const sea_shape& s, BitsMode mode) {
+  return mode == BitsMode::kPerBatch ? topk_grouped_supported(s) : s.causal == 1;
+}
+
+sea_status topk_mask_bits(BitsMode mode, const sea_shape* shape, const float* A_hat, uint32_t* mask_bits,
+                          int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* ws, size_t ws_bytes,
+                          void* cuda_stream) {
   Launch::count() = 0;
   const sea_status rc = validate_shape(shape, false);
   if (rc != SEA_OK) return rc;
-  if (!topk_grouped_supported(*shape)) return SEA_ERR_UNSUPPORTED;
+  if (!bits_mode_supported(*shape, mode)) return SEA_ERR_UNSUPPORTED;
   if (!A_hat || !row_ptr || !ws) return SEA_ERR_INVALID_ARG;
   if (!aligned16(A_hat) || !aligned16(row_ptr) || !aligned16(ws) || (mask_bits && !aligned16(mask_bits)) ||
       (col_idx && !aligned16(col_idx)))
@@ -195,10 +204,30 @@ sea_status sea_topk_mask_grouped(const sea_shape* shape, const float* A_hat, uin
   if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
   char* w = static_cast<char*>(ws);
   uint32_t* bits = mask_bits ? mask_bits : reinterpret_cast<uint32_t*>(w + L.mask_bits);
-  return launch_topk_mask_grouped(*shape, A_hat, bits, row_ptr, col_idx, nnz_cap,
-                                  reinterpret_cast<int32_t*>(w + L.row_counts),
-                                  reinterpret_cast<int32_t*>(w + L.tile_sums), nullptr,
-                                  reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
+  int32_t* counts = reinterpret_cast<int32_t*>(w + L.row_counts);
+  int32_t* sums = reinterpret_cast<int32_t*>(w + L.tile_sums);
+  int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (mode == BitsMode::kPerBatch)
+    return launch_topk_mask_grouped(*shape, A_hat, bits, row_ptr, col_idx, nnz_cap, counts, sums, nullptr, status, st);
+  return launch_topk_mask_aware(*shape, A_hat, bits, row_ptr, col_idx, nnz_cap, counts, sums, status, st);
+}
+}  // namespace
+
+extern "C" {
+
+sea_status sea_topk_mask_grouped(const sea_shape* shape, const float* A_hat, uint32_t* mask_bits,
+                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* ws,
+                                 size_t ws_bytes, void* cuda_stream) {
+  return topk_mask_bits(BitsMode::kPerBatch, shape, A_hat, mask_bits, row_ptr, col_idx, nnz_cap, ws, ws_bytes,
+                        cuda_stream);
+}
+
+sea_status sea_topk_mask_causal_aware(const sea_shape* shape, const float* A_hat, uint32_t* mask_bits,
+                                      int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* ws,
+                                      size_t ws_bytes, void* cuda_stream) {
+  return topk_mask_bits(BitsMode::kCausalAware, shape, A_hat, mask_bits, row_ptr, col_idx, nnz_cap, ws, ws_bytes,
+                        cuda_stream);
 }
 
 sea_status sea_sparse_attn_masked(const sea_shape* shape, const void* Q, const void* K, const void* V,
@@ -222,15 +251,18 @@ sea_status sea_sparse_attn_masked(const sea_shape* shape, const void* Q, const v
                                    static_cast<int32_t*>(ws), static_cast<cudaStream_t>(cuda_stream));
 }
 
-sea_status sea_attention_grouped(const sea_shape* shape, const void* Q, const void* K, const void* V,
-                                 const float* omega, const float* W_dec, const float* A_hat_in, void* O,
-                                 float* A_hat, uint32_t* mask_bits, int32_t* row_ptr, int32_t* col_idx,
-                                 int64_t nnz_cap, void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+sea_status attention_bits(BitsMode mode, const sea_shape* shape, const void* Q, const void* K, const void* V,
+                          const float* omega, const float* W_dec, const float* A_hat_in, void* O, float* A_hat,
+                          uint32_t* mask_bits, int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* P, void* ws,
+                          size_t ws_bytes, void* cuda_stream) {
   Launch::count() = 0;
   const bool estimate = A_hat_in == nullptr;
   sea_status rc = validate_shape(shape, estimate);
   if (rc != SEA_OK) return rc;
-  if (!topk_grouped_supported(*shape)) return SEA_ERR_UNSUPPORTED;
+  if (!bits_mode_supported(*shape, mode)) return SEA_ERR_UNSUPPORTED;
   if (!Q || !K || !V || !O || !ws) return SEA_ERR_INVALID_ARG;
   if (estimate && (!omega || !W_dec)) return SEA_ERR_INVALID_ARG;
   if (P && !col_idx) return SEA_ERR_INVALID_ARG;  // probabilities are only meaningful beside their indices
@@ -262,13 +294,38 @@ sea_status sea_attention_grouped(const sea_shape* shape, const void* Q, const vo
     a_use = a_out;
   }
   int32_t* rp_buf = row_ptr ? row_ptr : reinterpret_cast<int32_t*>(w + L.row_ptr);
-  // the selection also lays out the parking area of the tile kernel when P is wanted
-  const bool tiles = park && sparse_attn_tc_applicable(*shape, nullptr, true, status, bits, scratch);
-  rc = launch_topk_mask_grouped(*shape, a_use, bits, rp_buf, col_idx, nnz_cap,
-                                reinterpret_cast<int32_t*>(w + L.row_counts),
-                                reinterpret_cast<int32_t*>(w + L.tile_sums), tiles && P ? park : nullptr, status, st);
+  int32_t* counts = reinterpret_cast<int32_t*>(w + L.row_counts);
+  int32_t* sums = reinterpret_cast<int32_t*>(w + L.tile_sums);
+  if (mode == BitsMode::kPerBatch) {
+    // the selection also lays out the parking area of the tile kernel when P is wanted
+    const bool tiles = park && sparse_attn_tc_applicable(*shape, nullptr, true, status, bits, scratch);
+    rc = launch_topk_mask_grouped(*shape, a_use, bits, rp_buf, col_idx, nnz_cap, counts, sums, tiles && P ? park : nullptr,
+                                  status, st);
+    if (rc != SEA_OK) return rc;
+    return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, true, scratch, status, st);
+  }
+  rc = launch_topk_mask_aware(*shape, a_use, bits, rp_buf, col_idx, nnz_cap, counts, sums, status, st);
   if (rc != SEA_OK) return rc;
-  return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, true, scratch, status, st);
+  return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, false, scratch, status, st);
+}
+}  // namespace
+
+extern "C" {
+
+sea_status sea_attention_grouped(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                                 const float* omega, const float* W_dec, const float* A_hat_in, void* O,
+                                 float* A_hat, uint32_t* mask_bits, int32_t* row_ptr, int32_t* col_idx,
+                                 int64_t nnz_cap, void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return attention_bits(BitsMode::kPerBatch, shape, Q, K, V, omega, W_dec, A_hat_in, O, A_hat, mask_bits, row_ptr,
+                        col_idx, nnz_cap, P, ws, ws_bytes, cuda_stream);
+}
+
+sea_status sea_attention_causal_aware(const sea_shape* shape, const void* Q, const void* K, const void* V,
+                                      const float* omega, const float* W_dec, const float* A_hat_in, void* O,
+                                      float* A_hat, uint32_t* mask_bits, int32_t* row_ptr, int32_t* col_idx,
+                                      int64_t nnz_cap, void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return attention_bits(BitsMode::kCausalAware, shape, Q, K, V, omega, W_dec, A_hat_in, O, A_hat, mask_bits, row_ptr,
+                        col_idx, nnz_cap, P, ws, ws_bytes, cuda_stream);
 }
 
 sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes) {

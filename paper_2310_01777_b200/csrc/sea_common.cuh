@@ -81,6 +81,15 @@ sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint
                                     int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
                                     int32_t* row_counts, int32_t* tile_sums, int32_t* park_off,
                                     int32_t* status, cudaStream_t st);
+// Column indices of a mask given as bits and row pointers (rows of any length).
+sea_status launch_fill_col_idx_bits(const sea_shape& s, const uint32_t* mask_bits, const int32_t* row_ptr,
+                                    int32_t* col_idx, int64_t nnz_cap, int32_t* status, cudaStream_t st);
+// Causal-aware per-query selection (sea_topk.cu): a causal row only chooses among the columns
+// that hold a key it may see.  mask_bits is written in full.
+sea_status launch_topk_mask_aware(const sea_shape& s, const float* A_hat, uint32_t* mask_bits,
+                                  int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                                  int32_t* row_counts, int32_t* tile_sums, int32_t* status,
+                                  cudaStream_t st);
 // Where each row parks its unnormalised probabilities when rows keep differing numbers of columns:
 // the (b, t) slabs of H*k_hat*r floats follow one another, the heads inside a slab.  Rows of a slab
 // that keeps more than H*k_hat columns get -1 and SEA_DEV_ROW_OVERFLOW is raised.

@@ -24,17 +24,21 @@ constexpr int kThreadMaxK = 32;    // Kc * k_hat min/max pairs per row, the bit 
 constexpr int kHistBins = 256;
 constexpr int kHistShift = 17;
 
-// One warp per row; lane l holds columns l, l+32, ... (VPL of them).
+// One warp per row; lane l holds columns l, l+32, ... (VPL of them).  `aware`: a causal row i only
+// chooses among the columns that hold a key j <= i (columns 0 .. i / r) and keeps at most as many
+// as there are; sel may be null then (rows keep differing numbers of columns).
 template <int VPL>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
-                 int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc, int k_hat,
-                 int seq_len, int r, int causal) {
+                 int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc_all, int k_all,
+                 int seq_len, int r, int causal, int aware) {
   __shared__ int hist_all[kWarpsPerCta][kHistBins];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kWarpsPerCta + warp;
   if (row >= rows) return;
-  const float* a = A_hat + (size_t)row * Kc;
+  const float* a = A_hat + (size_t)row * Kc_all;
+  const int Kc = aware ? min(Kc_all, (row % seq_len) / r + 1) : Kc_all;  // columns that compete
+  const int k_hat = min(k_all, Kc);
   uint32_t key[VPL];
 #pragma unroll
   for (int t = 0; t < VPL; ++t) {
@@ -149,7 +153,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
   const uint32_t lt_mask = (1u << lane) - 1u;
   const int i = row % seq_len;
   int out_base = 0, tie_seen = 0, cnt = 0;
-  int32_t* my_sel = sel + (size_t)row * k_hat;
+  int32_t* my_sel = sel != nullptr ? sel + (size_t)row * k_all : nullptr;
 #pragma unroll
   for (int t = 0; t < VPL; ++t) {
     const bool tie = key[t] == tau;
@@ -158,10 +162,10 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
     const uint32_t sb = __ballot_sync(0xffffffffu, take);
     if (take) {
       const int col = lane + 32 * t;
-      my_sel[out_base + __popc(sb & lt_mask)] = col;
+      if (my_sel != nullptr) my_sel[out_base + __popc(sb & lt_mask)] = col;
       cnt += causal ? max(0, min(r, i + 1 - col * r)) : r;
     }
-    if (mask_bits != nullptr && lane == 0 && 32 * t < Kc) mask_bits[(size_t)row * ((Kc + 31) / 32) + t] = sb;
+    if (mask_bits != nullptr && lane == 0 && 32 * t < Kc_all) mask_bits[(size_t)row * ((Kc_all + 31) / 32) + t] = sb;
     tie_seen += __popc(tb);
     out_base += __popc(sb);
   }
@@ -376,10 +380,25 @@ fill_col_idx_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__
 
 template <int VPL>
 void launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, uint32_t* mask_bits, int rows,
-                 const sea_shape& s, cudaStream_t st) {
+                 const sea_shape& s, bool aware, cudaStream_t st) {
   const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
   topk_rows_kernel<VPL><<<grid, kWarpsPerCta * 32, 0, st>>>(A_hat, sel, counts, mask_bits, rows, s.Kc, s.k_hat,
-                                                             s.T, s.T / s.Kc, s.causal);
+                                                             s.T, s.T / s.Kc, s.causal, aware ? 1 : 0);
+}
+
+// The warp-per-row kernel for a row of `vpl` values per lane.
+bool launch_topk_rows(const float* A_hat, int32_t* sel, int32_t* counts, uint32_t* mask_bits, int rows,
+                      const sea_shape& s, bool aware, cudaStream_t st) {
+  const int vpl = (s.Kc + 31) / 32;
+  if (vpl <= 1) launch_topk<1>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  else if (vpl <= 2) launch_topk<2>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  else if (vpl <= 4) launch_topk<4>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  else if (vpl <= 8) launch_topk<8>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  else if (vpl <= 16) launch_topk<16>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  else if (vpl <= 32) launch_topk<32>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  else if (vpl <= 64) launch_topk<64>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  else return false;
+  return true;
 }
 
 }  // namespace
@@ -404,7 +423,6 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
   const int rows = s.B * s.H * s.T;
   const int r = s.T / s.Kc;
   int32_t* counts = s.causal ? row_counts : nullptr;
-  const int vpl = (s.Kc + 31) / 32;
   sea_status rc = SEA_OK;
   if (selected) {
     // sel, the counts and the bits are in place already
@@ -425,14 +443,7 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
     else SEA_TOPK_THREAD(32);
 #undef SEA_TOPK_THREAD
   }
-  else if (vpl <= 1) launch_topk<1>(A_hat, sel, counts, mask_bits, rows, s, st);
-  else if (vpl <= 2) launch_topk<2>(A_hat, sel, counts, mask_bits, rows, s, st);
-  else if (vpl <= 4) launch_topk<4>(A_hat, sel, counts, mask_bits, rows, s, st);
-  else if (vpl <= 8) launch_topk<8>(A_hat, sel, counts, mask_bits, rows, s, st);
-  else if (vpl <= 16) launch_topk<16>(A_hat, sel, counts, mask_bits, rows, s, st);
-  else if (vpl <= 32) launch_topk<32>(A_hat, sel, counts, mask_bits, rows, s, st);
-  else if (vpl <= 64) launch_topk<64>(A_hat, sel, counts, mask_bits, rows, s, st);
-  else return SEA_ERR_UNSUPPORTED;
+  else if (!launch_topk_rows(A_hat, sel, counts, mask_bits, rows, s, false, st)) return SEA_ERR_UNSUPPORTED;
   if (!selected && (rc = check_launch()) != SEA_OK) return rc;
 
   if (s.causal) {
@@ -450,6 +461,19 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
                                                             rows, s.k_hat, r, log2r, status);
     if ((rc = check_launch()) != SEA_OK) return rc;
   }
+  return SEA_OK;
+}
+
+// Causal-aware per-query selection: bits, row lengths, row pointers and (optionally) column indices.
+sea_status launch_topk_mask_aware(const sea_shape& s, const float* A_hat, uint32_t* mask_bits, int32_t* row_ptr,
+                                  int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts, int32_t* tile_sums,
+                                  int32_t* status, cudaStream_t st) {
+  const int rows = s.B * s.H * s.T;
+  if (!launch_topk_rows(A_hat, nullptr, row_counts, mask_bits, rows, s, true, st)) return SEA_ERR_UNSUPPORTED;
+  sea_status rc = check_launch();
+  if (rc != SEA_OK) return rc;
+  if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
+  if (col_idx != nullptr) return launch_fill_col_idx_bits(s, mask_bits, row_ptr, col_idx, nnz_cap, status, st);
   return SEA_OK;
 }
 

@@ -438,16 +438,21 @@ sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint
   sea_status rc = check_launch();
   if (rc != SEA_OK) return rc;
   if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
-  if (col_idx != nullptr) {
-    int log2r = -1;
-    for (int l = 0; l < 31; ++l)
-      if ((1 << l) == r) log2r = l;
-    const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
-    fill_col_idx_bits_kernel<<<grid, kWarpsPerCta * 32, 0, st>>>(mask_bits, row_ptr, col_idx, (long long)nnz_cap, rows,
-                                                                 (s.Kc + 31) / 32, r, log2r, status);
-    if ((rc = check_launch()) != SEA_OK) return rc;
-  }
+  if (col_idx != nullptr) return launch_fill_col_idx_bits(s, mask_bits, row_ptr, col_idx, nnz_cap, status, st);
   return SEA_OK;
+}
+
+sea_status launch_fill_col_idx_bits(const sea_shape& s, const uint32_t* mask_bits, const int32_t* row_ptr,
+                                    int32_t* col_idx, int64_t nnz_cap, int32_t* status, cudaStream_t st) {
+  const int rows = s.B * s.H * s.T;
+  const int r = s.T / s.Kc;
+  int log2r = -1;
+  for (int l = 0; l < 31; ++l)
+    if ((1 << l) == r) log2r = l;
+  const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+  fill_col_idx_bits_kernel<<<grid, kWarpsPerCta * 32, 0, st>>>(mask_bits, row_ptr, col_idx, (long long)nnz_cap, rows,
+                                                               (s.Kc + 31) / 32, r, log2r, status);
+  return check_launch();
 }
 
 sea_status launch_park_offsets(const sea_shape& s, const uint32_t* mask_bits, int32_t* park_off, int32_t* status,

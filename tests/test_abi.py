@@ -111,6 +111,14 @@ def test_grouped_entry_points_reject_bad_arguments_before_launch(lib):
     rc = lib.sea_attention_grouped(ctypes.byref(shp), fake, fake, fake, fake, fake, None, fake, None, None, None,
                                    None, 0, fake, fake, 1 << 40, None)
     assert rc == binding.SEA_ERR_INVALID_ARG  # P without col_idx
+    nc = sea.make_shape(WORKLOADS["bert_base"])  # not causal
+    rc = lib.sea_topk_mask_causal_aware(ctypes.byref(nc), fake, None, fake, None, 0, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_UNSUPPORTED
+    rc = lib.sea_topk_mask_causal_aware(ctypes.byref(shp), fake, None, None, None, 0, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # row_ptr is required
+    rc = lib.sea_attention_causal_aware(ctypes.byref(shp), fake, fake, fake, fake, fake, None, fake, None, None, None,
+                                        None, 0, fake, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # P without col_idx
     f32 = sea.make_shape(WORKLOADS["tiny_f32"])
     rc = lib.sea_attention_grouped(ctypes.byref(f32), fake, fake, fake, None, None, fake, fake, None, None, None,
                                    None, 0, None, fake, 1 << 40, None)

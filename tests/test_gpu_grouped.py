@@ -302,3 +302,122 @@ def test_grouped_full_size_sampled_heads_and_global_properties(name):
         o_ref, p_ref = orc.sparse_attention(Q[t:t + 1], K, V, np.array([0, hi - lo]), cols, scale_of(w))
         check_float(np64(run.O[b, h, t]), o_ref[0], w.dtype, "O")
         check_float(np64(run.P[lo:hi]), p_ref, w.dtype, "P")
+
+
+# ---------------------------------------------------------------------------------------
+# Causal-aware per-query selection: a causal row chooses among the columns it can see.
+# ---------------------------------------------------------------------------------------
+class AwareRun(GroupedRun):
+    def topk(self):
+        sea.sea_topk_mask_causal_aware(self.shape, self.A_hat, self.bits, self.row_ptr, self.col_idx, self.ws)
+
+    def fused(self):
+        given = "A_hat" in self.d
+        sea.sea_attention_causal_aware(self.shape, self.d["Q"], self.d["K"], self.d["V"], self.d.get("omega"),
+                                       self.d.get("W_dec"), self.O, self.ws,
+                                       A_hat_in=self.A_hat if given else None, A_hat=None if given else self.A_hat,
+                                       mask_bits=self.bits, row_ptr=self.row_ptr, col_idx=self.col_idx, P=self.P)
+
+
+def check_aware_head(run: AwareRun, b: int, h: int):
+    w = run.w
+    Q, K, V = (np64(run.host[n][b, h]) for n in ("Q", "K", "V"))
+    A = run.A_hat[b, h].cpu().numpy()
+    cols = orc.topk_select_causal_aware(A, w.k_hat, w.T)
+    got = run.cols_of(b, h)
+    for t in range(w.T):
+        assert list(got[t]) == list(cols[t]), f"selection differs at b={b} h={h} t={t}"
+    row_ptr, col_idx = orc.expand_mask(cols, w.T, w.Kc, True)
+    O, P = orc.sparse_attention(Q, K, V, row_ptr, col_idx, scale_of(w))
+    bh = b * w.H + h
+    rp = run.row_ptr[bh * w.T:(bh + 1) * w.T + 1].cpu().numpy().astype(np.int64)
+    lo, hi = int(rp[0]), int(rp[-1])
+    np.testing.assert_array_equal(rp - lo, row_ptr)
+    np.testing.assert_array_equal(run.col_idx[lo:hi].cpu().numpy().astype(np.int64), col_idx)
+    check_float(np64(run.O[b, h]), O, w.dtype, "O")
+    got_p = np64(run.P[lo:hi])
+    check_float(got_p, P, w.dtype, "P")
+    sums = np.add.reduceat(np.append(got_p, 0.0), row_ptr[:-1])
+    assert np.all(np.abs(sums - 1.0) <= TOL[w.dtype]["row_sum"])  # no row is empty
+
+
+AWARE_CASES = [
+    small("a_f32", H=2, causal=True, T=96, Kc=32, k_hat=5, m=16),                       # r = 3, per-row kernels
+    small("a_bf16_r4", dtype="bf16", B=2, H=3, T=384, Kc=96, k_hat=9, causal=True, m=64),
+    small("a_bf16_r16", dtype="bf16", H=4, T=512, Kc=32, k_hat=4, causal=True, m=128),
+    small("a_k1", dtype="bf16", H=2, T=256, Kc=16, k_hat=1, causal=True),                # one column per row, never empty
+    small("a_wide", dtype="bf16", H=2, T=2048, Kc=512, k_hat=24, causal=True, m=64),     # 16 values per lane, histogram path
+    small("a_full", dtype="bf16", H=2, T=256, Kc=16, k_hat=16, causal=True),             # dense causal attention
+]
+
+
+@pytest.mark.parametrize("w", AWARE_CASES, ids=lambda w: w.name)
+def test_causal_aware_stages_and_fused_call_match_oracle(w):
+    a = AwareRun(w)
+    a.estimate(); a.topk(); a.sparse(); a.sync()
+    assert a.status() == 0
+    for b in range(w.B):
+        for h in range(w.H):
+            check_aware_head(a, b, h)
+    counts = (a.row_ptr[1:] - a.row_ptr[:-1])
+    assert int(counts.min()) >= 1
+    f = AwareRun(w)
+    f.fused(); f.sync()
+    assert f.status() == 0
+    nnz = int(a.row_ptr[-1])
+    for name in ("A_hat", "bits", "row_ptr", "O"):
+        assert torch.equal(getattr(a, name), getattr(f, name)), name
+    assert torch.equal(a.col_idx[:nnz], f.col_idx[:nnz])
+    assert torch.equal(a.P[:nnz].view(torch.int16 if w.dtype == "bf16" else torch.int32),
+                       f.P[:nnz].view(torch.int16 if w.dtype == "bf16" else torch.int32))
+
+
+def test_causal_aware_needs_a_causal_shape_and_handles_ties():
+    w = small("a_nc", H=1, T=128, Kc=32, k_hat=4, m=0)
+    run = AwareRun(w, inputs=make_inputs(w, with_a_hat=True))
+    with pytest.raises(sea.SeaError) as e:
+        run.topk()
+    assert e.value.code == binding.SEA_ERR_UNSUPPORTED
+    w = small("a_ties", H=1, T=128, Kc=32, k_hat=4, m=0, causal=True)
+    host = make_inputs(w, with_a_hat=True)
+    host["A_hat"] = (torch.round(host["A_hat"] * 2) / 2).contiguous()
+    host["A_hat"][0, 0, 50, :] = 0.0
+    host["A_hat"][0, 0, 51, ::2] = -0.0
+    run = AwareRun(w, inputs=host)
+    run.fused(); run.sync()
+    assert run.status() == 0
+    check_aware_head(run, 0, 0)
+
+
+def test_causal_aware_full_size_properties_and_sampled_rows():
+    w = WORKLOADS["opt_1p3b"]
+    run = AwareRun(w)
+    run.fused(); run.sync()
+    assert run.status() == 0
+    r = w.r
+    bits = run.bits.long() & 0xFFFFFFFF
+    shifts = torch.arange(32, device=run.dev)
+    sel = ((bits[:, :, None] >> shifts) & 1).reshape(w.rows, -1)[:, :w.Kc]
+    i = (torch.arange(w.rows, device=run.dev) % w.T)
+    visible = i // r + 1
+    assert bool((sel.sum(1) == torch.clamp(visible, max=w.k_hat)).all()), "a row keeps min(k_hat, visible) columns"
+    c = torch.arange(w.Kc, device=run.dev)[None, :]
+    assert bool(((sel == 0) | (c < visible[:, None])).all()), "a selected column holds no visible key"
+    counts = (sel * torch.clamp(i[:, None] + 1 - c * r, 0, r)).sum(1)
+    rp = run.row_ptr.long()
+    assert bool((rp[1:] - rp[:-1] == counts).all()) and int(counts.min()) >= 1
+    b, h = w.B - 1, 5
+    A = run.A_hat[b, h].cpu().numpy()
+    cols = orc.topk_select_causal_aware(A, w.k_hat, w.T)
+    got = run.cols_of(b, h)
+    for t in (0, 15, 16, 255, 256, 1000, w.T - 1):
+        assert list(got[t]) == list(cols[t])
+    Q, K, V = (np64(run.host[n][b, h]) for n in ("Q", "K", "V"))
+    bh = b * w.H + h
+    rph = run.row_ptr[bh * w.T:(bh + 1) * w.T + 1].cpu().numpy().astype(np.int64)
+    for t in (0, 3, 100, w.T - 1):
+        lo, hi = int(rph[t]), int(rph[t + 1])
+        cidx = run.col_idx[lo:hi].cpu().numpy().astype(np.int64)
+        o_ref, p_ref = orc.sparse_attention(Q[t:t + 1], K, V, np.array([0, hi - lo]), cidx, scale_of(w))
+        check_float(np64(run.O[b, h, t]), o_ref[0], w.dtype, "O")
+        check_float(np64(run.P[lo:hi]), p_ref, w.dtype, "P")
