@@ -5,6 +5,8 @@
 
 #include <stdint.h>
 
+#include <utility>
+
 namespace sea {
 namespace select {
 
@@ -15,20 +17,35 @@ __device__ __forceinline__ void cmp_exchange(float& x, float& y) {
   x = kDescending ? hi : lo;
   y = kDescending ? lo : hi;
 }
+// Batcher's odd-even merge sort as a list of compare-exchange pairs built at compile time: 19 pairs
+// for 8 values, 63 for 16, 191 for 32 (a bitonic sorter needs 24, 80 and 240).
 template <int N>
-__device__ __forceinline__ void bitonic_sort_ascending(float (&a)[N]) {
-#pragma unroll
-  for (int k = 2; k <= N; k <<= 1)
-#pragma unroll
-    for (int j = k >> 1; j > 0; j >>= 1)
-#pragma unroll
-      for (int i = 0; i < N; ++i) {
-        const int l = i ^ j;
-        if (l > i) {
-          if ((i & k) == 0) cmp_exchange<false>(a[i], a[l]);
-          else cmp_exchange<true>(a[i], a[l]);
-        }
-      }
+struct BatcherNet {
+  static constexpr int kMax = N * 8;
+  int lo[kMax] = {}, hi[kMax] = {};
+  int count = 0;
+  constexpr BatcherNet() {
+    for (int p = 1; p < N; p <<= 1)
+      for (int k = p; k >= 1; k >>= 1)
+        for (int j = k % p; j <= N - 1 - k; j += 2 * k)
+          for (int i = 0; i < k && i <= N - j - k - 1; ++i)
+            if ((i + j) / (2 * p) == (i + j + k) / (2 * p)) {
+              lo[count] = i + j;
+              hi[count] = i + j + k;
+              ++count;
+            }
+  }
+};
+template <int N, int... I>
+__device__ __forceinline__ void apply_net(float (&a)[N], std::integer_sequence<int, I...>) {
+  constexpr BatcherNet<N> net{};
+  (cmp_exchange<false>(a[net.lo[I]], a[net.hi[I]]), ...);  // every index is a compile-time constant
+}
+// Ascending sort of N registers (N a power of two).
+template <int N>
+__device__ __forceinline__ void sort_ascending(float (&a)[N]) {
+  constexpr BatcherNet<N> net{};
+  apply_net<N>(a, std::make_integer_sequence<int, net.count>{});
 }
 template <int N>
 __device__ __forceinline__ void bitonic_merge_descending(float (&a)[N]) {
@@ -43,7 +60,7 @@ __device__ __forceinline__ void bitonic_merge_descending(float (&a)[N]) {
 // top (descending) <- the KMAX largest of top and grp (any order; destroyed)
 template <int KMAX>
 __device__ __forceinline__ void merge_group(float (&top)[KMAX], float (&grp)[KMAX]) {
-  bitonic_sort_ascending<KMAX>(grp);
+  sort_ascending<KMAX>(grp);
 #pragma unroll
   for (int s = 0; s < KMAX; ++s) top[s] = fmaxf(top[s], grp[s]);
   bitonic_merge_descending<KMAX>(top);
