@@ -18,6 +18,8 @@ metric is quoted.  One JSON line is printed by rank 0.
              against the measured dense bf16 peak.
   stages     per-stage milliseconds from a second pass that calls the three stage entry points
              with events between them (same kernels as the fused call).
+  lean       the fused call asked for O and the CSR mask only (the estimate and the probabilities are
+             never written out); per-rank, not part of `value`.
   grouped, causal_aware
              the same step with the causal-per-batch grouping (sea_attention_grouped) and with the
              causal-aware per-query selection (sea_attention_causal_aware) on this rank, and their
@@ -294,6 +296,32 @@ def main():
     if not torch.equal(hO, O.cpu()):
         raise SystemExit("host entry point and device entry point disagree")
 
+    # ---- timed region 3b: the fused call with the required outputs only (O and the CSR mask) ------
+    O_lean = torch.empty_like(O)
+    rp_lean = torch.empty_like(row_ptr)
+
+    def lean_step():
+        sea.sea_attention(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O_lean, ws, row_ptr=rp_lean,
+                          col_idx=col_idx)
+
+    for _ in range(3):
+        flush.zero_()
+        lean_step()
+    lean_launches = sea.sea_last_launch_count()
+    lev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    torch.cuda.synchronize(dev)
+    for a, b in lev:
+        flush.zero_()
+        a.record()
+        lean_step()
+        b.record()
+    torch.cuda.synchronize(dev)
+    lean_ms = sum(a.elapsed_time(b) for a, b in lev) / args.steps
+    if not (torch.equal(O_lean, O) and torch.equal(rp_lean, row_ptr)):
+        raise SystemExit("the call without the optional outputs gives a different O or row_ptr")
+    lean = {"outputs": "O, row_ptr and col_idx only (no A_hat, sel, P)", "ms_per_step": lean_ms,
+            "value": w.B * w.T / (lean_ms / 1e3), "unit": "tokens/s", "gpu_launches_per_step": lean_launches}
+
     # ---- timed region 4: the selections that leave as bit masks (fused call, then the stages) ----
     def time_bits_mode(label, fused_fn, topk_fn):
         bits = torch.empty((w.rows, (w.Kc + 31) // 32), dtype=torch.int32, device=dev)
@@ -374,6 +402,7 @@ def main():
             "clocks": clocks,
             "stages_ms": {"estimate": stage_ms[0], "topk_mask": stage_ms[1], "sparse_attn": stage_ms[2]},
             "nnz": nnz,
+            "lean": lean,
             "grouped": grouped,
             "causal_aware": causal_aware,
             "roofline": {"kernel": "sparse_attn_tiles_tc_kernel" if tiled else "sparse_attn_blocks_tma_kernel",

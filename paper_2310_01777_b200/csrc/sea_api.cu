@@ -163,8 +163,10 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
   const float* a_use = A_hat_in;
   bool selected = false;
   if (estimate) {
-    // where the estimator can, it selects each row's columns while the row is still on chip
-    float* a_out = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
+    // where the estimator can, it selects each row's columns while the row is still on chip; the
+    // estimate then only leaves the chip if the caller asked for it
+    const bool on_chip = shape->io == SEA_BF16 && estimate_tc_selects(*shape);
+    float* a_out = A_hat ? A_hat : (on_chip ? nullptr : reinterpret_cast<float*>(w + L.a_hat));
     const SelectOut so{sel_buf, shape->causal ? counts : nullptr, bits};
     rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state),
                          w + L.est_split, &so, &selected, status, st);

@@ -434,12 +434,13 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   const int n_ct = (p.Kc + kWTile - 1) / kWTile;
   const bool single = n_ct == 1;
   const bool selecting = KSEL > 0 && p.sel != nullptr;  // the launcher only asks for it with a single pass
+  const bool keep_a = p.A_hat != nullptr;               // without it the tile is only read by the selecting warps
   const int n_items = p.BH * p.nchunk;
   if (tid == 0) {
     for (int i = 0; i < kO_NumBars; ++i) {
       const bool from_rows = i == kO_Phi || i == kO_P || i == kO_C;
       const bool tile_read = i >= kO_AFree && i < kO_AFree + 2;  // the rows, and the selecting warps
-      mbar_init(bar(i), tile_read ? kRowWarps + (selecting ? 4 : 0) : (from_rows ? kRowWarps : 1));
+      mbar_init(bar(i), tile_read ? (keep_a ? kRowWarps : 0) + (selecting ? 4 : 0) : (from_rows ? kRowWarps : 1));
     }
     *abort_flag = 0;
     mbar_init_fence();
@@ -800,9 +801,9 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         }
         warp_arrive(bar(kO_C), lane);
       }
-      // ---- decoder passes: tile out of tensor memory, then to A_hat
+      // ---- decoder passes: tile out of tensor memory, then to A_hat (when the caller keeps it)
       float* out = p.A_hat + grow * p.Kc;
-      for (int ct = 0; ct < n_ct; ++ct, ++g) {
+      for (int ct = 0; ct < n_ct && keep_a; ++ct, ++g) {
         const uint32_t b = g & 1;
         constexpr int kMine = 4 / kParts;  // chunks of the 128-column tile per thread
         uint32_t e[kMine][32];
@@ -906,9 +907,11 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   prm.causal = s.causal;
   // A_hat [BH][T][Kc] fp32 in boxes of 128 rows x 32 columns; without a map (rows that are no
   // multiple of 16 bytes) the rows store their values themselves
-  prm.tma_store = (s.Kc % 4 == 0 && make_map_3d(&ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, A_hat, s.Kc, s.T, BH, 32, kRows)) ? 1 : 0;
+  prm.tma_store = (A_hat != nullptr && s.Kc % 4 == 0 &&
+                   make_map_3d(&ma, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, A_hat, s.Kc, s.T, BH, 32, kRows)) ? 1 : 0;
   if (!prm.tma_store) ma = mq;  // a valid map that is never used
   const bool selecting = so != nullptr && so->sel != nullptr && estimate_tc_selects(s);
+  if (A_hat == nullptr && !selecting) return SEA_ERR_INVALID_ARG;  // the estimate would go nowhere
   if (selecting) {
     prm.sel = so->sel;
     prm.row_counts = so->row_counts;
