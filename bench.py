@@ -262,6 +262,11 @@ def main():
     total_ms = sum(a.elapsed_time(b) for a, b in ev)
 
     # ---- timed region 2: stage by stage (for the roofline of the dominant kernel) -------
+    for _ in range(2):  # the stage entry points launch kernels the fused call does not: load them first
+        sea.sea_estimate(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], A_hat, ws)
+        sea.sea_topk_mask(shape, A_hat, sel, row_ptr, col_idx, ws)
+        sea.sea_sparse_attn(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, sel, O, P, ws)
+    torch.cuda.synchronize(dev)
     sev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     for e in sev:
         flush.zero_()
@@ -343,6 +348,10 @@ def main():
             b.record()
         torch.cuda.synchronize(dev)
         g_ms = sum(a.elapsed_time(b) for a, b in gev) / args.steps
+        for _ in range(2):
+            topk_fn(shape, A_hat, bits, row_ptr, col_idx, ws)
+            sea.sea_sparse_attn_masked(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, bits, O, P, ws)
+        torch.cuda.synchronize(dev)
         gsev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
         for e in gsev:
             flush.zero_()
