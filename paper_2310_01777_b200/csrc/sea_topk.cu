@@ -24,26 +24,57 @@ constexpr int kThreadMaxK = 32;    // Kc * k_hat min/max pairs per row, the bit 
 constexpr int kHistBins = 256;
 constexpr int kHistShift = 17;
 
-// One warp per row; lane l holds columns l, l+32, ... (VPL of them).  `aware`: a causal row i only
+// One warp per row; lane l holds the VPL consecutive columns l * VPL ..., so that column order is lane
+// order and the selected columns of a lane can be emitted without looking at the others, after one
+// prefix sum over the lanes.  `aware`: a causal row i only
 // chooses among the columns that hold a key j <= i (columns 0 .. i / r) and keeps at most as many
 // as there are; sel may be null then (rows keep differing numbers of columns).
+// The row's keys: in registers, or (wide rows, which would need more registers than leave room for
+// enough warps) in the warp's part of shared memory, lane l's t-th key at word 32 t + l.
+template <int VPL, bool kShared>
+struct RowKeys;
 template <int VPL>
-__global__ void __launch_bounds__(kWarpsPerCta * 32)
+struct RowKeys<VPL, false> {
+  uint32_t k[VPL];
+  __device__ __forceinline__ RowKeys(uint32_t*) {}
+  __device__ __forceinline__ uint32_t get(int t) const { return k[t]; }
+  __device__ __forceinline__ void set(int t, uint32_t v) { k[t] = v; }
+};
+template <int VPL>
+struct RowKeys<VPL, true> {
+  uint32_t* p;
+  __device__ __forceinline__ RowKeys(uint32_t* warp_keys) : p(warp_keys + (threadIdx.x & 31)) {}
+  __device__ __forceinline__ uint32_t get(int t) const { return p[32 * t]; }
+  __device__ __forceinline__ void set(int t, uint32_t v) { p[32 * t] = v; }
+};
+
+template <int VPL, bool kShared>
+__global__ void __launch_bounds__(kWarpsPerCta * 32, kShared ? 3 : 4)
 topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
                  int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc_all, int k_all,
                  int seq_len, int r, int causal, int aware) {
   __shared__ int hist_all[kWarpsPerCta][kHistBins];
+  extern __shared__ uint32_t keys_all[];  // [kWarpsPerCta][VPL * 32] when kShared
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kWarpsPerCta + warp;
   if (row >= rows) return;
   const float* a = A_hat + (size_t)row * Kc_all;
   const int Kc = aware ? min(Kc_all, (row % seq_len) / r + 1) : Kc_all;  // columns that compete
   const int k_hat = min(k_all, Kc);
-  uint32_t key[VPL];
+  RowKeys<VPL, kShared> key(keys_all + (kShared ? warp * VPL * 32 : 0));
+  const int col0 = lane * VPL;  // this lane's first column
+  if (VPL % 4 == 0 && Kc_all % 4 == 0) {  // rows start on 16-byte boundaries
 #pragma unroll
-  for (int t = 0; t < VPL; ++t) {
-    const int col = lane + 32 * t;
-    key[t] = col < Kc ? order_key(__ldg(a + col)) : 0u;  // padding sorts below every real value
+    for (int t = 0; t < VPL; t += 4) {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (col0 + t < Kc_all) v = __ldg(reinterpret_cast<const float4*>(a + col0 + t));
+      const float x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) key.set(t + e, col0 + t + e < Kc ? order_key(x[e]) : 0u);  // padding sorts below every real value
+    }
+  } else {
+#pragma unroll
+    for (int t = 0; t < VPL; ++t) key.set(t, col0 + t < Kc ? order_key(__ldg(a + col0 + t)) : 0u);
   }
   // k_hat-th largest key: the largest tau with |{key >= tau}| >= k_hat.  First try: the row's
   // largest key `top`, a histogram of (top - key) >> kHistShift over the kHistBins steps below it
@@ -55,7 +86,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
     int* hist = hist_all[warp];
     uint32_t top = 0u;
 #pragma unroll
-    for (int t = 0; t < VPL; ++t) top = max(top, key[t]);
+    for (int t = 0; t < VPL; ++t) top = max(top, key.get(t));
     top = __reduce_max_sync(0xffffffffu, top);
     // step x is kept at word (x & 7) * 32 + (x >> 3): lane x >> 3 owns it and reads it without conflicts
 #pragma unroll
@@ -63,8 +94,8 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
     __syncwarp();
 #pragma unroll
     for (int t = 0; t < VPL; ++t) {
-      const uint32_t x = (top - key[t]) >> kHistShift;
-      if (x < (uint32_t)kHistBins && lane + 32 * t < Kc) atomicAdd(&hist[(x & 7u) * 32u + (x >> 3)], 1);
+      const uint32_t x = (top - key.get(t)) >> kHistShift;
+      if (x < (uint32_t)kHistBins && col0 + t < Kc) atomicAdd(&hist[(x & 7u) * 32u + (x >> 3)], 1);
     }
     __syncwarp();
     int bins[kHistBins / 32], mine = 0;
@@ -99,7 +130,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
       // the keys inside the step, one per lane when there are at most 32
       int inside = 0;
 #pragma unroll
-      for (int t = 0; t < VPL; ++t) inside += ((top - key[t]) >> kHistShift) == (uint32_t)step;
+      for (int t = 0; t < VPL; ++t) inside += ((top - key.get(t)) >> kHistShift) == (uint32_t)step;
       int pos = inside;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -114,7 +145,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
         constexpr uint32_t kFine = (1u << kHistShift) - 1u;
 #pragma unroll
         for (int t = 0; t < VPL; ++t) {
-          const uint32_t rel = top - key[t];
+          const uint32_t rel = top - key.get(t);
           if ((rel >> kHistShift) == (uint32_t)step) list[pos++] = kFine - (rel & kFine);  // grows with the key
         }
         __syncwarp();
@@ -139,35 +170,61 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
       const uint32_t cand = tau | (1u << bit);
       int c = 0;
 #pragma unroll
-      for (int t = 0; t < VPL; ++t) c += key[t] >= cand;
+      for (int t = 0; t < VPL; ++t) c += key.get(t) >= cand;
       c = __reduce_add_sync(0xffffffffu, c);
       if (c >= k_hat) tau = cand;
     }
   }
-  int n_gt = 0;
-#pragma unroll
-  for (int t = 0; t < VPL; ++t) n_gt += key[t] > tau;
-  n_gt = __reduce_add_sync(0xffffffffu, n_gt);
-  const int need = k_hat - n_gt;  // how many columns equal to tau are taken (lowest first)
-
-  const uint32_t lt_mask = (1u << lane) - 1u;
-  const int i = row % seq_len;
-  int out_base = 0, tie_seen = 0, cnt = 0;
-  int32_t* my_sel = sel != nullptr ? sel + (size_t)row * k_all : nullptr;
+  // per lane: the bits of its columns above tau and equal to it
+  uint64_t gt = 0ull, eq = 0ull;
 #pragma unroll
   for (int t = 0; t < VPL; ++t) {
-    const bool tie = key[t] == tau;
-    const uint32_t tb = __ballot_sync(0xffffffffu, tie);
-    const bool take = key[t] > tau || (tie && tie_seen + __popc(tb & lt_mask) < need);
-    const uint32_t sb = __ballot_sync(0xffffffffu, take);
-    if (take) {
-      const int col = lane + 32 * t;
-      if (my_sel != nullptr) my_sel[out_base + __popc(sb & lt_mask)] = col;
-      cnt += causal ? max(0, min(r, i + 1 - col * r)) : r;
+    gt |= (uint64_t)(key.get(t) > tau) << t;
+    eq |= (uint64_t)(key.get(t) == tau) << t;
+  }
+  const int my_gt = __popcll(gt), my_eq = __popcll(eq);
+  // inclusive prefix sums over the lanes of (columns above tau, columns equal to it), packed
+  int inc = (my_gt << 16) | my_eq;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += v;
+  }
+  const int tot = __shfl_sync(0xffffffffu, inc, 31);
+  const int need = k_hat - (tot >> 16);  // how many columns equal to tau are taken (lowest first)
+  // of this lane's equal columns, the first `mine` are taken
+  const int eq_before = (inc & 0xffff) - my_eq;
+  int mine = min(max(need - eq_before, 0), my_eq);
+  uint64_t take = gt;
+  for (uint64_t e = eq; mine > 0; --mine) {
+    const uint64_t low = e & (0ull - e);
+    take |= low;
+    e ^= low;
+  }
+  const int taken_before = (inc >> 16) - my_gt + min(eq_before, max(need, 0));
+
+  const int i = row % seq_len;
+  int cnt = 0;
+  int32_t* my_sel = sel != nullptr ? sel + (size_t)row * k_all + taken_before : nullptr;
+  for (uint64_t tk = take; tk != 0ull; tk &= tk - 1ull) {
+    const int col = col0 + __ffsll((long long)tk) - 1;
+    if (my_sel != nullptr) *my_sel++ = col;
+    cnt += causal ? max(0, min(r, i + 1 - col * r)) : r;
+  }
+  if (mask_bits != nullptr) {
+    uint32_t* words = mask_bits + (size_t)row * ((Kc_all + 31) / 32);
+    if constexpr (VPL >= 32) {
+#pragma unroll
+      for (int j = 0; j < VPL / 32; ++j)
+        if (col0 + 32 * j < Kc_all) words[lane * (VPL / 32) + j] = (uint32_t)(take >> (32 * j));
+    } else {
+      // 32 / VPL neighbouring lanes share a word
+      constexpr int kLanes = 32 / VPL;
+      uint32_t word = (uint32_t)take << ((lane % kLanes) * VPL);
+#pragma unroll
+      for (int o = 1; o < kLanes; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
+      if (lane % kLanes == 0 && col0 < Kc_all) words[lane / kLanes] = word;
     }
-    if (mask_bits != nullptr && lane == 0 && 32 * t < Kc_all) mask_bits[(size_t)row * ((Kc_all + 31) / 32) + t] = sb;
-    tie_seen += __popc(tb);
-    out_base += __popc(sb);
   }
   if (row_counts != nullptr) {
     cnt = __reduce_add_sync(0xffffffffu, cnt);
@@ -379,26 +436,31 @@ fill_col_idx_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__
 }
 
 template <int VPL>
-void launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, uint32_t* mask_bits, int rows,
+bool launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, uint32_t* mask_bits, int rows,
                  const sea_shape& s, bool aware, cudaStream_t st) {
   const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
-  topk_rows_kernel<VPL><<<grid, kWarpsPerCta * 32, 0, st>>>(A_hat, sel, counts, mask_bits, rows, s.Kc, s.k_hat,
-                                                             s.T, s.T / s.Kc, s.causal, aware ? 1 : 0);
+  constexpr bool kShared = VPL >= 32;  // beyond 512 columns the keys no longer fit the registers
+  const size_t smem = kShared ? (size_t)kWarpsPerCta * VPL * 32 * sizeof(uint32_t) : 0;
+  auto kern = topk_rows_kernel<VPL, kShared>;
+  if (smem > 40 * 1024 && cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return false;
+  kern<<<grid, kWarpsPerCta * 32, smem, st>>>(A_hat, sel, counts, mask_bits, rows, s.Kc, s.k_hat, s.T, s.T / s.Kc,
+                                              s.causal, aware ? 1 : 0);
+  return true;
 }
 
 // The warp-per-row kernel for a row of `vpl` values per lane.
 bool launch_topk_rows(const float* A_hat, int32_t* sel, int32_t* counts, uint32_t* mask_bits, int rows,
                       const sea_shape& s, bool aware, cudaStream_t st) {
   const int vpl = (s.Kc + 31) / 32;
-  if (vpl <= 1) launch_topk<1>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
-  else if (vpl <= 2) launch_topk<2>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
-  else if (vpl <= 4) launch_topk<4>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
-  else if (vpl <= 8) launch_topk<8>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
-  else if (vpl <= 16) launch_topk<16>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
-  else if (vpl <= 32) launch_topk<32>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
-  else if (vpl <= 64) launch_topk<64>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
-  else return false;
-  return true;
+  if (vpl <= 1) return launch_topk<1>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  if (vpl <= 2) return launch_topk<2>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  if (vpl <= 4) return launch_topk<4>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  if (vpl <= 8) return launch_topk<8>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  if (vpl <= 16) return launch_topk<16>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  if (vpl <= 32) return launch_topk<32>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  if (vpl <= 64) return launch_topk<64>(A_hat, sel, counts, mask_bits, rows, s, aware, st);
+  return false;
 }
 
 }  // namespace
