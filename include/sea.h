@@ -233,8 +233,9 @@ sea_status sea_attention_causal_aware(const sea_shape* shape, const void* Q, con
  * is copied back to hO.  The heads are independent, so the call is a pipeline
  * over up to eight slices of them: a slice is computed on `cuda_stream` while
  * the next slice's inputs arrive and the previous slice's O leaves on two
- * streams that the call creates and destroys (with a few events); this overlap
- * needs pinned host memory, pageable memory gives the same result serially.
+ * streams of the library's own (created, with a few events, by a host thread's
+ * first call on a device and kept by that thread); this overlap needs pinned
+ * host memory, pageable memory gives the same result serially.
  * Bytes needed: sea_workspace_host_bytes().  The call returns after all its work
  * has finished, so hO is valid on return.  Not for use during stream capture.
  * The paper has no counterpart; this is the end-to-end form of the call above.

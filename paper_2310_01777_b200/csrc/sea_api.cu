@@ -59,6 +59,54 @@ WsLayout ws_layout(const sea_shape& s) {
 
 using namespace sea;
 
+namespace {
+// The two copy streams and the events of sea_attention_host's pipeline.  Creating them costs more
+// than a slice of the pipeline takes, so a host thread creates them once per device it calls from
+// and keeps them until it exits.
+constexpr int kMaxSlices = 8;
+struct HostPipe {
+  int device = -1;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t ev_begin = nullptr, ev_in[kMaxSlices] = {}, ev_done[kMaxSlices] = {};
+  void release() {
+    for (int c = 0; c < kMaxSlices; ++c) {
+      if (ev_in[c]) cudaEventDestroy(ev_in[c]);
+      if (ev_done[c]) cudaEventDestroy(ev_done[c]);
+      ev_in[c] = ev_done[c] = nullptr;
+    }
+    if (ev_begin) cudaEventDestroy(ev_begin);
+    if (s_in) cudaStreamDestroy(s_in);
+    if (s_out) cudaStreamDestroy(s_out);
+    ev_begin = nullptr;
+    s_in = s_out = nullptr;
+    device = -1;
+  }
+  bool prepare() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (dev == device) return true;
+    release();
+    bool good = cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess &&
+                cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess &&
+                cudaEventCreateWithFlags(&ev_begin, cudaEventDisableTiming) == cudaSuccess;
+    for (int c = 0; c < kMaxSlices && good; ++c)
+      good = cudaEventCreateWithFlags(&ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&ev_done[c], cudaEventDisableTiming) == cudaSuccess;
+    if (!good) {
+      release();
+      return false;
+    }
+    device = dev;
+    return true;
+  }
+  ~HostPipe() {}  // at thread exit the CUDA runtime may already be gone: the handles are left to it
+};
+HostPipe& host_pipe() {
+  static thread_local HostPipe pipe;
+  return pipe;
+}
+}  // namespace
+
 extern "C" {
 
 sea_status sea_workspace_bytes(const sea_shape* shape, size_t* bytes) {
@@ -380,16 +428,12 @@ sea_status sea_attention_host(const sea_shape* shape, const void* hQ, const void
   sub.H = BH / nslice;
   const size_t slice_b = qkv_b / nslice;
 
-  constexpr int kMaxSlices = 8;
-  cudaStream_t s_in = nullptr, s_out = nullptr;
-  cudaEvent_t ev_begin = nullptr, ev_in[kMaxSlices] = {}, ev_done[kMaxSlices] = {};
-  bool good = cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaEventCreateWithFlags(&ev_begin, cudaEventDisableTiming) == cudaSuccess;
-  for (int c = 0; c < nslice && good; ++c)
-    good = cudaEventCreateWithFlags(&ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
-           cudaEventCreateWithFlags(&ev_done[c], cudaEventDisableTiming) == cudaSuccess;
-  rc = good ? SEA_OK : SEA_ERR_CUDA;
+  HostPipe& pipe = host_pipe();
+  rc = pipe.prepare() ? SEA_OK : SEA_ERR_CUDA;
+  cudaStream_t s_in = pipe.s_in, s_out = pipe.s_out;
+  cudaEvent_t ev_begin = pipe.ev_begin;
+  cudaEvent_t* ev_in = pipe.ev_in;
+  cudaEvent_t* ev_done = pipe.ev_done;
   int launches = 0;
   // the staging areas may still be read by work the caller enqueued earlier on `st`
   if (rc == SEA_OK && (cudaEventRecord(ev_begin, st) != cudaSuccess || cudaStreamWaitEvent(s_in, ev_begin, 0) != cudaSuccess ||
@@ -416,17 +460,10 @@ sea_status sea_attention_host(const sea_shape* shape, const void* hQ, const void
         cudaMemcpyAsync(static_cast<char*>(hO) + off, dO + off, slice_b, cudaMemcpyDeviceToHost, s_out) != cudaSuccess)
       rc = SEA_ERR_CUDA;
   }
-  // everything enqueued has to finish before the streams and events go away, success or not
+  // the call returns with all of its work finished, success or not
   if (s_in && cudaStreamSynchronize(s_in) != cudaSuccess && rc == SEA_OK) rc = SEA_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess && rc == SEA_OK) rc = SEA_ERR_CUDA;
   if (s_out && cudaStreamSynchronize(s_out) != cudaSuccess && rc == SEA_OK) rc = SEA_ERR_CUDA;
-  for (int c = 0; c < kMaxSlices; ++c) {
-    if (ev_in[c]) cudaEventDestroy(ev_in[c]);
-    if (ev_done[c]) cudaEventDestroy(ev_done[c]);
-  }
-  if (ev_begin) cudaEventDestroy(ev_begin);
-  if (s_in) cudaStreamDestroy(s_in);
-  if (s_out) cudaStreamDestroy(s_out);
   Launch::count() = launches;
   return rc;
 }
