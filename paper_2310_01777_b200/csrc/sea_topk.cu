@@ -235,7 +235,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
 // Selection with one thread per row, for short rows and small k_hat: no cross-lane traffic at
 // all.  Every thread walks its row (16-byte loads; a row is a few cache lines that the thread
 // reads front to back) in groups of KMAX values and keeps the KMAX largest values seen so far as
-// a descending list in registers: a group is sorted ascending by a bitonic network, the
+// a descending list in registers: a group is sorted ascending by an odd-even merge network, the
 // element-wise maximum with the list is then a bitonic sequence holding the KMAX largest of
 // both, and a bitonic merge sorts it again - all compare-exchanges on fixed registers, no
 // branches.  That leaves the k_hat-th largest value tau in the last slot; a second walk over
