@@ -40,6 +40,8 @@ the paper's steps in the paper's order:
                         up-sampling of the compressed mask done on indices; a
                         selected column c covers keys c*r .. c*r+r-1, r = T/Kc;
                         causal rows drop keys j > i.  Output is a flat CSR.
+                        With k_star: the appendix's cap for long sequences, at
+                        most k_star uniformly spaced keys per selected column.
     sparse_attention    Sec. 3.1.1 "Sparse Attention Mechanism": rho (scores at
                         mask positions), sigma (softmax over a row's non-zeros),
                         then C = A* V.
@@ -185,15 +187,25 @@ def topk_select_causal_aware(A_hat, k_hat: int, T: int):
     return cols
 
 
-def expand_mask(sel, T: int, Kc: int, causal: bool, query_index=None):
+def expand_mask(sel, T: int, Kc: int, causal: bool, query_index=None, k_star=None):
     """Flat CSR (row_ptr [n+1], col_idx [nnz]) of the up-sampled mask of one head.
 
     Row t of ``sel`` (an array [n, k_hat], or a list of n column arrays of any
     lengths) belongs to query ``query_index[t]`` (default: t, all T queries).
+
+    ``k_star`` (App. "Sparse Interpolation", the case k K / T < 1): a selected column is
+    replicated to at most k_star of its r = T / Kc keys, spaced uniformly over the run:
+    keys c*r + floor(u * r / k_star), u = 0 .. k_star-1.  None or k_star >= r: the whole run.
     """
     if T % Kc != 0:
         raise ValueError("T must be a multiple of Kc")
     r = T // Kc
+    if k_star is None or k_star >= r:
+        offsets = list(range(r))
+    else:
+        if k_star < 1:
+            raise ValueError("k_star must be positive")
+        offsets = [(u * r) // k_star for u in range(k_star)]
     n = len(sel)
     if query_index is None:
         query_index = np.arange(n)
@@ -203,7 +215,8 @@ def expand_mask(sel, T: int, Kc: int, causal: bool, query_index=None):
         i = int(query_index[t])
         row = []
         for c in sel[t]:
-            for j in range(int(c) * r, int(c) * r + r):
+            for o in offsets:
+                j = int(c) * r + o
                 if causal and j > i:
                     continue
                 row.append(j)

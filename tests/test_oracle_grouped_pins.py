@@ -216,3 +216,64 @@ def test_causal_aware_first_rows_are_dense_causal_attention():
     n_dense = k_hat * r
     np.testing.assert_allclose(O[:n_dense], ref[:n_dense], atol=1e-12)
     assert np.array_equal(np.diff(row_ptr)[:n_dense], np.arange(1, n_dense + 1))
+
+
+# ---------------------------------------------------------------------------
+# Capped replication for long sequences (App. "Sparse Interpolation", k K / T < 1):
+# at most k_star uniformly spaced keys per selected column.
+# ---------------------------------------------------------------------------
+def test_capped_expansion_invariants_and_special_cases():
+    g = rng(41)
+    T, Kc, k_hat = 96, 8, 2
+    r = T // Kc  # 12
+    A = g.standard_normal((T, Kc))
+    sel = orc.topk_select(A, k_hat)
+    full_rp, full_ci = orc.expand_mask(sel, T, Kc, False)
+    for k_star in (r, r + 5, None):  # no cap: the whole run
+        rp, ci = orc.expand_mask(sel, T, Kc, False, k_star=k_star)
+        assert np.array_equal(rp, full_rp) and np.array_equal(ci, full_ci)
+    for k_star in (1, 3, 4, 5, 7):
+        rp, ci = orc.expand_mask(sel, T, Kc, False, k_star=k_star)
+        assert np.all(np.diff(rp) == k_hat * k_star)  # the paper's constant number of non-zeros per row
+        for i in range(T):
+            js = ci[rp[i]:rp[i + 1]]
+            assert np.all(np.diff(js) > 0)
+            for n, c in enumerate(sel[i]):
+                run = js[n * k_star:(n + 1) * k_star] - c * r
+                assert run[0] == 0 and np.all((0 <= run) & (run < r))
+                gaps = np.diff(np.append(run, r))  # uniformly spaced: gaps differ by at most one
+                assert gaps.max() - gaps.min() <= 1
+            assert set(js) <= set(full_ci[full_rp[i]:full_rp[i + 1]])  # a subset of the uncapped mask
+        crp, cci = orc.expand_mask(sel, T, Kc, True, k_star=k_star)
+        for i in range(T):
+            js = ci[rp[i]:rp[i + 1]]
+            assert list(cci[crp[i]:crp[i + 1]]) == [j for j in js if j <= i]
+    # k_star dividing r: every (r / k_star)-th key of the run
+    rp, ci = orc.expand_mask(sel[:1], T, Kc, False, k_star=4)
+    c0 = sel[0][0]
+    assert list(ci[:4]) == [c0 * r + o for o in (0, 3, 6, 9)]
+
+
+def test_capped_mask_attention_is_masked_dense_attention():
+    g = rng(42)
+    T, Kc, d, k_hat, k_star = 64, 4, 8, 1, 5
+    r = T // Kc
+    Q, K, V = (g.standard_normal((T, d)) for _ in range(3))
+    A = g.standard_normal((T, Kc))
+    sel = orc.topk_select(A, k_hat)
+    for causal in (False, True):
+        rp, ci = orc.expand_mask(sel, T, Kc, causal, k_star=k_star)
+        O, P = orc.sparse_attention(Q, K, V, rp, ci, 0.3)
+        mask = torch.zeros(T, T, dtype=torch.bool)
+        for i in range(T):
+            for c in sel[i]:
+                for u in range(k_star):
+                    j = int(c) * r + (u * r) // k_star
+                    if not causal or j <= i:
+                        mask[i, j] = True
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(Q)[None], torch.from_numpy(K)[None], torch.from_numpy(V)[None],
+            attn_mask=mask[None], scale=0.3)[0].numpy()
+        nonempty = mask.any(dim=1).numpy()
+        np.testing.assert_allclose(O[nonempty], ref[nonempty], atol=1e-12)
+        assert np.all(O[~nonempty] == 0.0)
