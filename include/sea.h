@@ -228,6 +228,25 @@ sea_status sea_attention_causal_aware(const sea_shape* shape, const void* Q, con
                                       void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Capped replication for long sequences, App. "Sparse Interpolation": when
+ * k*K/T < 1 the paper selects a single column per row (k_hat = 1) and limits its
+ * replication to k* = min(k, ceil(T/K)) keys instead of the whole run of T/K,
+ * sampled uniformly; the spacing is not given and is taken as the keys
+ * c*r + floor(u*r/k_star), u = 0 .. k_star-1 (k_star >= r keeps the whole run).
+ * Causal rows drop keys j > i.  Works for any k_hat; T % Kc == 0 is still
+ * required.  col_idx is required (the sparse stage walks the CSR with the per-row
+ * kernels); nnz_cap rows*k_hat*min(k_star, r) always suffices.
+ */
+sea_status sea_topk_mask_capped(const sea_shape* shape, int32_t k_star, const float* A_hat, int32_t* sel,
+                                int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                                void* ws, size_t ws_bytes, void* cuda_stream);
+sea_status sea_attention_capped(const sea_shape* shape, int32_t k_star, const void* Q, const void* K,
+                                const void* V, const float* omega, const float* W_dec,
+                                const float* A_hat_in, void* O, float* A_hat, int32_t* sel,
+                                int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* P,
+                                void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * sea_attention for callers whose tensors live in HOST memory.  hQ, hK, hV,
  * homega, hW_dec are copied to staging areas inside `ws`, the layer runs, and O
  * is copied back to hO.  The heads are independent, so the call is a pipeline

@@ -30,7 +30,7 @@ SEA_DEV_NONFINITE = 2
 EXPORTS = (
     "sea_workspace_bytes", "sea_estimate", "sea_topk_mask", "sea_topk_mask_static", "sea_sparse_attn",
     "sea_attention", "sea_topk_mask_grouped", "sea_sparse_attn_masked", "sea_attention_grouped",
-    "sea_topk_mask_causal_aware", "sea_attention_causal_aware",
+    "sea_topk_mask_causal_aware", "sea_attention_causal_aware", "sea_topk_mask_capped", "sea_attention_capped",
     "sea_workspace_host_bytes", "sea_attention_host", "sea_device_status", "sea_last_launch_count",
     "sea_status_string",
 )
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     lib.sea_attention_grouped.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
     lib.sea_topk_mask_causal_aware.argtypes = lib.sea_topk_mask_grouped.argtypes
     lib.sea_attention_causal_aware.argtypes = lib.sea_attention_grouped.argtypes
+    lib.sea_topk_mask_capped.argtypes = [shp, i32, vp, vp, vp, vp, i64, vp, sz, vp]
+    lib.sea_attention_capped.argtypes = [shp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
     lib.sea_attention_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sea_device_status.argtypes = [vp, ctypes.POINTER(i32), i32, vp]
     lib.sea_last_launch_count.argtypes = []
@@ -223,6 +225,26 @@ def sea_attention_causal_aware(shape, Q, K, V, omega, W_dec, O, ws, A_hat_in=Non
                                                      _ptr(mask_bits), _ptr(row_ptr), _ptr(col_idx), nnz_cap, _ptr(P),
                                                      _ptr(ws), ws.numel(), _stream(ws.device)),
            "sea_attention_causal_aware")
+
+
+def sea_topk_mask_capped(shape, k_star: int, A_hat, sel, row_ptr, col_idx, ws, nnz_cap: Optional[int] = None):
+    """Per-query selection, each selected column replicated to at most k_star uniformly spaced keys."""
+    if nnz_cap is None:
+        nnz_cap = col_idx.numel()
+    _check(load_library().sea_topk_mask_capped(ctypes.byref(shape), k_star, _ptr(A_hat), _ptr(sel), _ptr(row_ptr),
+                                               _ptr(col_idx), nnz_cap, _ptr(ws), ws.numel(), _stream(ws.device)),
+           "sea_topk_mask_capped")
+
+
+def sea_attention_capped(shape, k_star: int, Q, K, V, omega, W_dec, O, ws, col_idx, A_hat_in=None, A_hat=None, sel=None,
+                         row_ptr=None, P=None, nnz_cap: Optional[int] = None):
+    if nnz_cap is None:
+        nnz_cap = col_idx.numel()
+    _check(load_library().sea_attention_capped(ctypes.byref(shape), k_star, _ptr(Q), _ptr(K), _ptr(V), _ptr(omega),
+                                               _ptr(W_dec), _ptr(A_hat_in), _ptr(O), _ptr(A_hat), _ptr(sel),
+                                               _ptr(row_ptr), _ptr(col_idx), nnz_cap, _ptr(P), _ptr(ws), ws.numel(),
+                                               _stream(ws.device)),
+           "sea_attention_capped")
 
 
 def sea_attention_host(shape, hQ, hK, hV, homega, hW_dec, hO, ws):

@@ -378,6 +378,66 @@ sea_status sea_attention_causal_aware(const sea_shape* shape, const void* Q, con
                         col_idx, nnz_cap, P, ws, ws_bytes, cuda_stream);
 }
 
+sea_status sea_topk_mask_capped(const sea_shape* shape, int32_t k_star, const float* A_hat, int32_t* sel,
+                                int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* ws, size_t ws_bytes,
+                                void* cuda_stream) {
+  Launch::count() = 0;
+  const sea_status rc = validate_shape(shape, false);
+  if (rc != SEA_OK) return rc;
+  if (k_star < 1 || !A_hat || !row_ptr || !col_idx || !ws) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(A_hat) || !aligned16(row_ptr) || !aligned16(col_idx) || !aligned16(ws) || (sel && !aligned16(sel)))
+    return SEA_ERR_INVALID_ARG;
+  if (nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
+  if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  const WsLayout L = ws_layout(*shape);
+  if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
+  return launch_topk_mask_capped(*shape, k_star, A_hat, sel_buf, row_ptr, col_idx, nnz_cap,
+                                 reinterpret_cast<int32_t*>(w + L.row_counts),
+                                 reinterpret_cast<int32_t*>(w + L.tile_sums), reinterpret_cast<int32_t*>(w + L.status),
+                                 static_cast<cudaStream_t>(cuda_stream));
+}
+
+sea_status sea_attention_capped(const sea_shape* shape, int32_t k_star, const void* Q, const void* K, const void* V,
+                                const float* omega, const float* W_dec, const float* A_hat_in, void* O, float* A_hat,
+                                int32_t* sel, int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* P, void* ws,
+                                size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  const bool estimate = A_hat_in == nullptr;
+  sea_status rc = validate_shape(shape, estimate);
+  if (rc != SEA_OK) return rc;
+  if (k_star < 1 || !Q || !K || !V || !O || !ws || !col_idx) return SEA_ERR_INVALID_ARG;
+  if (estimate && (!omega || !W_dec)) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(ws) || !aligned16(col_idx) ||
+      (omega && !aligned16(omega)) || (W_dec && !aligned16(W_dec)) || (A_hat_in && !aligned16(A_hat_in)) ||
+      (A_hat && !aligned16(A_hat)) || (sel && !aligned16(sel)) || (row_ptr && !aligned16(row_ptr)) || (P && !aligned16(P)))
+    return SEA_ERR_INVALID_ARG;
+  if (nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
+  if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  const WsLayout L = ws_layout(*shape);
+  if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
+  const float* a_use = A_hat_in;
+  if (estimate) {
+    float* a_out = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
+    rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state),
+                         w + L.est_split, nullptr, nullptr, status, st);
+    if (rc != SEA_OK) return rc;
+    a_use = a_out;
+  }
+  int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
+  int32_t* rp_buf = row_ptr ? row_ptr : reinterpret_cast<int32_t*>(w + L.row_ptr);
+  rc = launch_topk_mask_capped(*shape, k_star, a_use, sel_buf, rp_buf, col_idx, nnz_cap,
+                               reinterpret_cast<int32_t*>(w + L.row_counts),
+                               reinterpret_cast<int32_t*>(w + L.tile_sums), status, st);
+  if (rc != SEA_OK) return rc;
+  // rows keep scattered keys, not runs: the per-row kernels walk the CSR
+  return launch_sparse_attn_rows(*shape, Q, K, V, rp_buf, col_idx, nullptr, O, P, st);
+}
+
 sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes) {
   if (bytes == nullptr) return SEA_ERR_INVALID_ARG;
   const sea_status rc = validate_shape(shape, true);

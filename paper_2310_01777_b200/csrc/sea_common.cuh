@@ -90,6 +90,11 @@ sea_status launch_topk_mask_aware(const sea_shape& s, const float* A_hat, uint32
                                   int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
                                   int32_t* row_counts, int32_t* tile_sums, int32_t* status,
                                   cudaStream_t st);
+// Per-query selection whose selected columns are replicated to at most k_star uniformly spaced keys
+// (sea_topk.cu); col_idx is required, the sparse stage then walks the CSR.
+sea_status launch_topk_mask_capped(const sea_shape& s, int k_star, const float* A_hat, int32_t* sel,
+                                   int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts,
+                                   int32_t* tile_sums, int32_t* status, cudaStream_t st);
 // Where each row parks its unnormalised probabilities when rows keep differing numbers of columns:
 // the (b, t) slabs of H*k_hat*r floats follow one another, the heads inside a slab.  Rows of a slab
 // that keeps more than H*k_hat columns get -1 and SEA_DEV_ROW_OVERFLOW is raised.

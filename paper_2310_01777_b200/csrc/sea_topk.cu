@@ -526,6 +526,67 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
   return SEA_OK;
 }
 
+// ---- capped replication (App. "Sparse Interpolation", the case k K / T < 1) --------------------
+// A selected column c keeps at most k_star of its r keys, spaced uniformly over the run:
+// c r + floor(u r / k_star), u = 0 .. k_star - 1.  A causal row i keeps those <= i: with
+// m = i - c r >= 0 that is min(k_star, ceil((m + 1) k_star / r)) of them, a prefix.
+__global__ void capped_counts_kernel(const int32_t* __restrict__ sel, int32_t* __restrict__ row_counts, int rows,
+                                     int k_hat, int seq_len, int r, int k_star, int causal) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= rows) return;
+  const int i = row % seq_len;
+  int cnt = 0;
+  for (int e = 0; e < k_hat; ++e) {
+    if (!causal) {
+      cnt += k_star;
+    } else {
+      const long long m = (long long)i - (long long)__ldg(sel + (size_t)row * k_hat + e) * r;
+      if (m >= 0) cnt += (int)min((long long)k_star, ((m + 1) * k_star + r - 1) / r);
+    }
+  }
+  row_counts[row] = cnt;
+}
+
+// One warp per row: position n of the row is key number n % k_star of its (n / k_star)-th column.
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+fill_col_idx_capped_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__ row_ptr,
+                           int32_t* __restrict__ col_idx, long long nnz_cap, int rows, int k_hat, int r, int k_star,
+                           int32_t* __restrict__ status) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kWarpsPerCta + warp;
+  if (row >= rows) return;
+  const int base = row_ptr[row];
+  int n = row_ptr[row + 1] - base;
+  if ((long long)base + n > nnz_cap) {
+    if (lane == 0) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
+    n = (int)max(0ll, min((long long)n, nnz_cap - base));
+  }
+  const int32_t* my_sel = sel + (size_t)row * k_hat;
+  for (int pos = lane; pos < n; pos += 32) {
+    const int b = pos / k_star, u = pos - b * k_star;
+    col_idx[(size_t)base + pos] = __ldg(my_sel + b) * r + (int)(((long long)u * r) / k_star);
+  }
+}
+
+sea_status launch_topk_mask_capped(const sea_shape& s, int k_star, const float* A_hat, int32_t* sel, int32_t* row_ptr,
+                                   int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts, int32_t* tile_sums,
+                                   int32_t* status, cudaStream_t st) {
+  const int rows = s.B * s.H * s.T;
+  const int r = s.T / s.Kc;
+  if (k_star >= r)  // no cap: the whole run
+    return launch_topk_mask(s, A_hat, sel, row_ptr, col_idx, nnz_cap, row_counts, tile_sums, nullptr, false, status, st);
+  // the selection as usual (its row pointers are those of whole runs and are replaced below)
+  sea_status rc = launch_topk_mask(s, A_hat, sel, row_ptr, nullptr, 0, row_counts, tile_sums, nullptr, false, status, st);
+  if (rc != SEA_OK) return rc;
+  capped_counts_kernel<<<(rows + 255) / 256, 256, 0, st>>>(sel, row_counts, rows, s.k_hat, s.T, r, k_star, s.causal);
+  if ((rc = check_launch()) != SEA_OK) return rc;
+  if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
+  const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+  fill_col_idx_capped_kernel<<<grid, kWarpsPerCta * 32, 0, st>>>(sel, row_ptr, col_idx, (long long)nnz_cap, rows, s.k_hat, r,
+                                                                 k_star, status);
+  return check_launch();
+}
+
 // Causal-aware per-query selection: bits, row lengths, row pointers and (optionally) column indices.
 sea_status launch_topk_mask_aware(const sea_shape& s, const float* A_hat, uint32_t* mask_bits, int32_t* row_ptr,
                                   int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts, int32_t* tile_sums,

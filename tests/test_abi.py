@@ -119,6 +119,13 @@ def test_grouped_entry_points_reject_bad_arguments_before_launch(lib):
     rc = lib.sea_attention_causal_aware(ctypes.byref(shp), fake, fake, fake, fake, fake, None, fake, None, None, None,
                                         None, 0, fake, fake, 1 << 40, None)
     assert rc == binding.SEA_ERR_INVALID_ARG  # P without col_idx
+    rc = lib.sea_topk_mask_capped(ctypes.byref(shp), 0, fake, None, fake, fake, 1024, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # k_star must be positive
+    rc = lib.sea_topk_mask_capped(ctypes.byref(shp), 4, fake, None, fake, None, 0, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # col_idx is required
+    rc = lib.sea_attention_capped(ctypes.byref(shp), 4, fake, fake, fake, fake, fake, None, fake, None, None, None,
+                                  None, 0, None, fake, 1 << 40, None)
+    assert rc == binding.SEA_ERR_INVALID_ARG  # col_idx is required
     f32 = sea.make_shape(WORKLOADS["tiny_f32"])
     rc = lib.sea_attention_grouped(ctypes.byref(f32), fake, fake, fake, None, None, fake, fake, None, None, None,
                                    None, 0, None, fake, 1 << 40, None)
