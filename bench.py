@@ -130,7 +130,8 @@ def oracle_tokens_per_s(w, n_heads: int, repeats: int = 1):
     small = w.scaled(B=1, H=n_heads)
     host = make_inputs(small)
     f64 = lambda t: t.to(dtype=__import__("torch").float64).numpy()
-    om, wd = f64(host["omega"]), f64(host["W_dec"])
+    given = "A_hat" in host  # workloads without an estimator stage bring the estimate along
+    om, wd = (None, None) if given else (f64(host["omega"]), f64(host["W_dec"]))
     scale = 1.0 / np.sqrt(w.d)
     best = None
     with threadpool_limits(limits=1):
@@ -138,7 +139,8 @@ def oracle_tokens_per_s(w, n_heads: int, repeats: int = 1):
             t0 = time.perf_counter()
             for h in range(n_heads):
                 orc.sea_attention_head(f64(host["Q"][0, h]), f64(host["K"][0, h]), f64(host["V"][0, h]), w.k_hat,
-                                       w.Kc, w.causal, scale, omega=om, W_dec=wd)
+                                       w.Kc, w.causal, scale, A_hat=f64(host["A_hat"][0, h]) if given else None,
+                                       omega=om, W_dec=wd)
             dt = time.perf_counter() - t0
             best = dt if best is None else min(best, dt)
     tokens = n_heads * w.T / w.H  # a token passes through all H heads of the layer
@@ -170,6 +172,19 @@ def run_reference(args, w):
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of timings over all ranks: the job is as slow as its slowest
+    replica.  Without a process group (one GPU) the values come back unchanged."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
 
 
 def workload_config(w):
@@ -377,11 +392,7 @@ def main():
         causal_aware = time_bits_mode("causal-aware per-query", sea.sea_attention_causal_aware,
                                       sea.sea_topk_mask_causal_aware)
 
-    ms_per_step = total_ms / args.steps
-    if world > 1:
-        t = torch.tensor([ms_per_step, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step, e2e_ms = max_over_ranks([total_ms / args.steps, e2e_ms], dev)
     tokens = w.B * w.T * world
     elem = 2 if w.dtype == "bf16" else 4
     h2d = sum(host[k].numel() * host[k].element_size() for k in ("Q", "K", "V", "omega", "W_dec"))
