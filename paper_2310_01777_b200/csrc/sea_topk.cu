@@ -313,7 +313,7 @@ topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ s
   if (row_counts != nullptr) row_counts[row] = cnt;
 }
 
-// ---- exclusive scan of row_counts -> row_ptr (three small kernels) -------------------
+// ---- exclusive scan of row_counts -> row_ptr (two small kernels) ---------------------
 __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int& block_total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int inc = v;
@@ -355,24 +355,15 @@ scan_tile_sums_kernel(const int32_t* __restrict__ counts, int32_t* __restrict__ 
   if (threadIdx.x == 0) tile_sums[blockIdx.x] = total;
 }
 
-__global__ void __launch_bounds__(1024)
-scan_tile_offsets_kernel(int32_t* __restrict__ tile_sums, int ntiles) {
-  __shared__ int warp_tot[33];
-  int carry = 0;
-  for (int c0 = 0; c0 < ntiles; c0 += 1024) {
-    const int idx = c0 + threadIdx.x;
-    const int v = idx < ntiles ? tile_sums[idx] : 0;
-    int total;
-    const int ex = block_exclusive_scan(v, warp_tot, total);
-    if (idx < ntiles) tile_sums[idx] = carry + ex;
-    carry += total;
-  }
-}
-
 __global__ void __launch_bounds__(kScanThreads)
-scan_write_row_ptr_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ tile_offs,
+scan_write_row_ptr_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ tile_sums,
                           int32_t* __restrict__ row_ptr, int rows) {
   __shared__ int warp_tot[33];
+  // the tile's offset: the sum of the tiles before it (a few hundred values at most)
+  int before = 0;
+  for (int t = threadIdx.x; t < (int)blockIdx.x; t += kScanThreads) before += tile_sums[t];
+  int tile_off;
+  block_exclusive_scan(before, warp_tot, tile_off);
   const int base = blockIdx.x * kScanTile + threadIdx.x * kScanPerThread;
   int v[kScanPerThread];
   int s = 0;
@@ -382,7 +373,7 @@ scan_write_row_ptr_kernel(const int32_t* __restrict__ counts, const int32_t* __r
     s += v[e];
   }
   int total;
-  int run = block_exclusive_scan(s, warp_tot, total) + tile_offs[blockIdx.x];
+  int run = block_exclusive_scan(s, warp_tot, total) + tile_off;
 #pragma unroll
   for (int e = 0; e < kScanPerThread; ++e) {
     if (base + e < rows) row_ptr[base + e] = run;
@@ -471,8 +462,6 @@ sea_status launch_row_ptr_scan(const int32_t* row_counts, int32_t* tile_sums, in
   sea_status rc;
   const int ntiles = (rows + kScanTile - 1) / kScanTile;
   scan_tile_sums_kernel<<<ntiles, kScanThreads, 0, st>>>(row_counts, tile_sums, rows);
-  if ((rc = check_launch()) != SEA_OK) return rc;
-  scan_tile_offsets_kernel<<<1, 1024, 0, st>>>(tile_sums, ntiles);
   if ((rc = check_launch()) != SEA_OK) return rc;
   scan_write_row_ptr_kernel<<<ntiles, kScanThreads, 0, st>>>(row_counts, tile_sums, row_ptr, rows);
   return check_launch();
