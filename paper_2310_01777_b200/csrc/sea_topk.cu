@@ -24,78 +24,90 @@ constexpr int kThreadMaxK = 32;    // Kc * k_hat min/max pairs per row, the bit 
 constexpr int kHistBins = 256;
 constexpr int kHistShift = 17;
 
-// One warp per row; lane l holds the VPL consecutive columns l * VPL ..., so that column order is lane
-// order and the selected columns of a lane can be emitted without looking at the others, after one
-// prefix sum over the lanes.  `aware`: a causal row i only
-// chooses among the columns that hold a key j <= i (columns 0 .. i / r) and keeps at most as many
-// as there are; sel may be null then (rows keep differing numbers of columns).
+// ---- one warp per row ---------------------------------------------------------------------------
+// Lane l holds the VPL consecutive columns l * VPL ..., so that column order is lane order and the
+// selected columns of a lane can be emitted without looking at the others, after one prefix sum over
+// the lanes.  `aware`: a causal row i only chooses among the columns that hold a key j <= i (columns
+// 0 .. i / r) and keeps at most as many as there are; sel may be null then (rows keep differing
+// numbers of columns).
+//
 // The row's keys: in registers, or (wide rows, which would need more registers than leave room for
-// enough warps) in the warp's part of shared memory, lane l's t-th key at word 32 t + l.
+// enough warps) in the warp's part of shared memory, lane l's t-th key at word l (VPL + 1) + t: the
+// lanes read their t-th keys from different banks, and the row can be fetched with neighbouring lanes
+// on neighbouring 16-byte pieces (a lane that fetched its own VPL columns instead would touch every
+// cache line of the row with every load, and the rows of a CTA's warps do not fit the L1 cache).
 template <int VPL, bool kShared>
 struct RowKeys;
 template <int VPL>
 struct RowKeys<VPL, false> {
+  static constexpr int kSlots = VPL;
+  static constexpr bool kDense = true;  // slot t is column col0 + t
   uint32_t k[VPL];
-  __device__ __forceinline__ RowKeys(uint32_t*) {}
+  int col0;
+  __device__ __forceinline__ RowKeys(uint32_t*, int first) : col0(first) {}
   __device__ __forceinline__ uint32_t get(int t) const { return k[t]; }
   __device__ __forceinline__ void set(int t, uint32_t v) { k[t] = v; }
 };
 template <int VPL>
 struct RowKeys<VPL, true> {
+  static constexpr int kSlots = VPL;
+  static constexpr bool kDense = true;
+  static constexpr int kStride = VPL + 1;
+  uint32_t* base;
   uint32_t* p;
-  __device__ __forceinline__ RowKeys(uint32_t* warp_keys) : p(warp_keys + (threadIdx.x & 31)) {}
-  __device__ __forceinline__ uint32_t get(int t) const { return p[32 * t]; }
-  __device__ __forceinline__ void set(int t, uint32_t v) { p[32 * t] = v; }
+  int col0;
+  __device__ __forceinline__ RowKeys(uint32_t* warp_keys, int first)
+      : base(warp_keys), p(warp_keys + (threadIdx.x & 31) * kStride), col0(first) {}
+  __device__ __forceinline__ uint32_t get(int t) const { return p[t]; }
+  __device__ __forceinline__ void set(int t, uint32_t v) { p[t] = v; }
+  // the key of column `col`, whichever lane owns it
+  __device__ __forceinline__ void put(int col, uint32_t v) { base[(col / VPL) * kStride + (col % VPL)] = v; }
+};
+// A few keys of the lane's columns with their columns (ascending), the rest of the slots empty.
+template <int N>
+struct CandKeys {
+  static constexpr int kSlots = N;
+  static constexpr bool kDense = false;
+  uint32_t k[N];
+  int c[N];
+  __device__ __forceinline__ uint32_t get(int t) const { return k[t]; }
 };
 
-template <int VPL, bool kShared>
-__global__ void __launch_bounds__(kWarpsPerCta * 32, kShared ? 3 : 4)
-topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
-                 int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc_all, int k_all,
-                 int seq_len, int r, int causal, int aware) {
-  __shared__ int hist_all[kWarpsPerCta][kHistBins];
-  extern __shared__ uint32_t keys_all[];  // [kWarpsPerCta][VPL * 32] when kShared
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row = blockIdx.x * kWarpsPerCta + warp;
-  if (row >= rows) return;
-  const float* a = A_hat + (size_t)row * Kc_all;
-  const int Kc = aware ? min(Kc_all, (row % seq_len) / r + 1) : Kc_all;  // columns that compete
-  const int k_hat = min(k_all, Kc);
-  RowKeys<VPL, kShared> key(keys_all + (kShared ? warp * VPL * 32 : 0));
-  const int col0 = lane * VPL;  // this lane's first column
-  if (VPL % 4 == 0 && Kc_all % 4 == 0) {  // rows start on 16-byte boundaries
-#pragma unroll
-    for (int t = 0; t < VPL; t += 4) {
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (col0 + t < Kc_all) v = __ldg(reinterpret_cast<const float4*>(a + col0 + t));
-      const float x[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) key.set(t + e, col0 + t + e < Kc ? order_key(x[e]) : 0u);  // padding sorts below every real value
-    }
-  } else {
-#pragma unroll
-    for (int t = 0; t < VPL; ++t) key.set(t, col0 + t < Kc ? order_key(__ldg(a + col0 + t)) : 0u);
-  }
-  // k_hat-th largest key: the largest tau with |{key >= tau}| >= k_hat.  First try: the row's
-  // largest key `top`, a histogram of (top - key) >> kHistShift over the kHistBins steps below it
-  // (1/64 of an octave each: four octaves of magnitudes), a scan for the step that holds tau, and a
-  // search by ballots among the keys inside that step (one per lane).
+struct RowOut {
+  int32_t* sel;      // the row's part of sel, or null
+  uint32_t* words;   // the row's part of mask_bits, or null
+  int n_words;
+  int32_t* count;    // the row's entry of row_counts, or null
+  int i, r, causal;  // query index inside the sequence, keys per column
+};
+
+// Selection of the k_hat largest keys among the slots of all lanes (an empty slot holds key 0, which
+// sorts below every real value), ties to the lower column, and the row's outputs.  `hist`: the warp's
+// kHistBins words of shared memory.
+//
+// The k_hat-th largest key tau (the largest tau with |{key >= tau}| >= k_hat) is found from the
+// row's largest key `top`, a histogram of (top - key) >> kHistShift over the kHistBins steps below it
+// (1/64 of an octave each: four octaves of magnitudes), a scan for the step that holds tau, and a
+// search by ballots among the keys inside that step (one per lane); when the step holds more than
+// 32 keys, or tau lies below the histogram, bit by bit with warp-wide counts over all keys.
+template <typename Keys>
+__device__ __forceinline__ void select_row(const Keys& key, int* hist, int lane, int k_hat, const RowOut& out) {
+  constexpr int N = Keys::kSlots;
   uint32_t tau = 0u;
   bool found = false;
   {
-    int* hist = hist_all[warp];
     uint32_t top = 0u;
 #pragma unroll
-    for (int t = 0; t < VPL; ++t) top = max(top, key.get(t));
+    for (int t = 0; t < N; ++t) top = max(top, key.get(t));
     top = __reduce_max_sync(0xffffffffu, top);
     // step x is kept at word (x & 7) * 32 + (x >> 3): lane x >> 3 owns it and reads it without conflicts
 #pragma unroll
     for (int j = 0; j < kHistBins / 32; ++j) hist[j * 32 + lane] = 0;
     __syncwarp();
 #pragma unroll
-    for (int t = 0; t < VPL; ++t) {
+    for (int t = 0; t < N; ++t) {
       const uint32_t x = (top - key.get(t)) >> kHistShift;
-      if (x < (uint32_t)kHistBins && col0 + t < Kc) atomicAdd(&hist[(x & 7u) * 32u + (x >> 3)], 1);
+      if (x < (uint32_t)kHistBins && key.get(t) != 0u) atomicAdd(&hist[(x & 7u) * 32u + (x >> 3)], 1);
     }
     __syncwarp();
     int bins[kHistBins / 32], mine = 0;
@@ -130,7 +142,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
       // the keys inside the step, one per lane when there are at most 32
       int inside = 0;
 #pragma unroll
-      for (int t = 0; t < VPL; ++t) inside += ((top - key.get(t)) >> kHistShift) == (uint32_t)step;
+      for (int t = 0; t < N; ++t) inside += ((top - key.get(t)) >> kHistShift) == (uint32_t)step;
       int pos = inside;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -144,7 +156,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
         pos -= inside;
         constexpr uint32_t kFine = (1u << kHistShift) - 1u;
 #pragma unroll
-        for (int t = 0; t < VPL; ++t) {
+        for (int t = 0; t < N; ++t) {
           const uint32_t rel = top - key.get(t);
           if ((rel >> kHistShift) == (uint32_t)step) list[pos++] = kFine - (rel & kFine);  // grows with the key
         }
@@ -165,25 +177,25 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
   }
   if (!found) {
     // bit by bit with warp-wide counts over all keys
-#pragma unroll
+#pragma unroll 1
     for (int bit = 31; bit >= 0; --bit) {
       const uint32_t cand = tau | (1u << bit);
       int c = 0;
 #pragma unroll
-      for (int t = 0; t < VPL; ++t) c += key.get(t) >= cand;
+      for (int t = 0; t < N; ++t) c += key.get(t) >= cand;
       c = __reduce_add_sync(0xffffffffu, c);
       if (c >= k_hat) tau = cand;
     }
   }
-  // per lane: the bits of its columns above tau and equal to it
+  // per lane: the bits of its slots above tau and equal to it
   uint64_t gt = 0ull, eq = 0ull;
 #pragma unroll
-  for (int t = 0; t < VPL; ++t) {
+  for (int t = 0; t < N; ++t) {
     gt |= (uint64_t)(key.get(t) > tau) << t;
     eq |= (uint64_t)(key.get(t) == tau) << t;
   }
   const int my_gt = __popcll(gt), my_eq = __popcll(eq);
-  // inclusive prefix sums over the lanes of (columns above tau, columns equal to it), packed
+  // inclusive prefix sums over the lanes of (slots above tau, slots equal to it), packed
   int inc = (my_gt << 16) | my_eq;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -203,33 +215,138 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
   }
   const int taken_before = (inc >> 16) - my_gt + min(eq_before, max(need, 0));
 
-  const int i = row % seq_len;
   int cnt = 0;
-  int32_t* my_sel = sel != nullptr ? sel + (size_t)row * k_all + taken_before : nullptr;
-  for (uint64_t tk = take; tk != 0ull; tk &= tk - 1ull) {
-    const int col = col0 + __ffsll((long long)tk) - 1;
-    if (my_sel != nullptr) *my_sel++ = col;
-    cnt += causal ? max(0, min(r, i + 1 - col * r)) : r;
+  int32_t* my_sel = out.sel != nullptr ? out.sel + taken_before : nullptr;
+  if constexpr (Keys::kDense) {
+    for (uint64_t tk = take; tk != 0ull; tk &= tk - 1ull) {
+      const int col = key.col0 + __ffsll((long long)tk) - 1;
+      if (my_sel != nullptr) *my_sel++ = col;
+      cnt += out.causal ? max(0, min(out.r, out.i + 1 - col * out.r)) : out.r;
+    }
+    if (out.words != nullptr) {
+      if constexpr (N >= 32) {
+#pragma unroll
+        for (int j = 0; j < N / 32; ++j)
+          if (lane * (N / 32) + j < out.n_words) out.words[lane * (N / 32) + j] = (uint32_t)(take >> (32 * j));
+      } else {
+        // 32 / N neighbouring lanes share a word
+        constexpr int kLanes = 32 / N;
+        uint32_t word = (uint32_t)take << ((lane % kLanes) * N);
+#pragma unroll
+        for (int o = 1; o < kLanes; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
+        if (lane % kLanes == 0 && lane / kLanes < out.n_words) out.words[lane / kLanes] = word;
+      }
+    }
+  } else {
+    // scattered columns: the bits are gathered in the warp's shared memory first
+    uint32_t* words = reinterpret_cast<uint32_t*>(hist);
+    __syncwarp();
+    for (int wv = lane; wv < out.n_words; wv += 32) words[wv] = 0u;
+    __syncwarp();
+#pragma unroll
+    for (int t = 0; t < N; ++t)
+      if ((take >> t) & 1ull) {
+        const int col = key.c[t];
+        if (my_sel != nullptr) *my_sel++ = col;
+        cnt += out.causal ? max(0, min(out.r, out.i + 1 - col * out.r)) : out.r;
+        if (out.words != nullptr) atomicOr(&words[col >> 5], 1u << (col & 31));
+      }
+    __syncwarp();
+    if (out.words != nullptr)
+      for (int wv = lane; wv < out.n_words; wv += 32) out.words[wv] = words[wv];
   }
-  if (mask_bits != nullptr) {
-    uint32_t* words = mask_bits + (size_t)row * ((Kc_all + 31) / 32);
-    if constexpr (VPL >= 32) {
+  if (out.count != nullptr) {
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if (lane == 0) *out.count = cnt;
+  }
+}
+
+constexpr int kCandSlots = 8;  // candidate keys a lane may bring to the second round
+
+template <int VPL, bool kShared>
+__global__ void __launch_bounds__(kWarpsPerCta * 32, kShared ? 3 : 4)
+topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
+                 int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc_all, int k_all,
+                 int seq_len, int r, int causal, int aware) {
+  static_assert(kHistBins >= 64, "the histogram words double as the row's bit words (Kc <= 2048)");
+  __shared__ int hist_all[kWarpsPerCta][kHistBins];
+  extern __shared__ uint32_t keys_all[];  // [kWarpsPerCta][32 * (VPL + 1)] when kShared
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kWarpsPerCta + warp;
+  if (row >= rows) return;
+  const float* a = A_hat + (size_t)row * Kc_all;
+  const int Kc = aware ? min(Kc_all, (row % seq_len) / r + 1) : Kc_all;  // columns that compete
+  const int k_hat = min(k_all, Kc);
+  const int col0 = lane * VPL;  // this lane's first column
+  RowKeys<VPL, kShared> key(keys_all + (kShared ? warp * (VPL + 1) * 32 : 0), col0);
+  if constexpr (kShared) {
+    if (Kc_all % 4 == 0) {
+#pragma unroll 4
+      for (int c = 4 * lane; c < 32 * VPL; c += 128) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < Kc_all) v = __ldg(reinterpret_cast<const float4*>(a + c));
+        const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int j = 0; j < VPL / 32; ++j)
-        if (col0 + 32 * j < Kc_all) words[lane * (VPL / 32) + j] = (uint32_t)(take >> (32 * j));
+        for (int e = 0; e < 4; ++e) key.put(c + e, c + e < Kc ? order_key(x[e]) : 0u);  // empty slots sort below every real value
+      }
     } else {
-      // 32 / VPL neighbouring lanes share a word
-      constexpr int kLanes = 32 / VPL;
-      uint32_t word = (uint32_t)take << ((lane % kLanes) * VPL);
+      for (int c = lane; c < 32 * VPL; c += 32) key.put(c, c < Kc ? order_key(__ldg(a + c)) : 0u);
+    }
+    __syncwarp();
+  } else if (VPL % 4 == 0 && Kc_all % 4 == 0) {  // rows start on 16-byte boundaries
 #pragma unroll
-      for (int o = 1; o < kLanes; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
-      if (lane % kLanes == 0 && col0 < Kc_all) words[lane / kLanes] = word;
+    for (int t = 0; t < VPL; t += 4) {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (col0 + t < Kc_all) v = __ldg(reinterpret_cast<const float4*>(a + col0 + t));
+      const float x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) key.set(t + e, col0 + t + e < Kc ? order_key(x[e]) : 0u);  // empty slots sort below every real value
+    }
+  } else {
+#pragma unroll
+    for (int t = 0; t < VPL; ++t) key.set(t, col0 + t < Kc ? order_key(__ldg(a + col0 + t)) : 0u);
+  }
+  RowOut out;
+  out.sel = sel != nullptr ? sel + (size_t)row * k_all : nullptr;
+  out.n_words = (Kc_all + 31) / 32;
+  out.words = mask_bits != nullptr ? mask_bits + (size_t)row * out.n_words : nullptr;
+  out.count = row_counts != nullptr ? row_counts + row : nullptr;
+  out.i = row % seq_len;
+  out.r = r;
+  out.causal = causal;
+
+  if constexpr (kShared) {
+    // A wide row first sheds most of its keys.  When every lane holds a column of the row, the
+    // smallest of the lanes' largest keys, L, has at least 32 keys at or above it, so with
+    // k_hat <= 32 every selected key is >= L; usually only a few keys per lane are.  They go, with
+    // their columns and in column order, through the same selection on kCandSlots slots per lane.
+    if (k_hat <= 32 && 31 * VPL < Kc) {
+      uint32_t lane_top = 0u;
+#pragma unroll 8
+      for (int t = 0; t < VPL; ++t) lane_top = max(lane_top, key.get(t));
+      const uint32_t low = __reduce_min_sync(0xffffffffu, lane_top);
+      uint64_t cand = 0ull;
+#pragma unroll 8
+      for (int t = 0; t < VPL; ++t) cand |= (uint64_t)(key.get(t) >= low) << t;
+      if (__reduce_max_sync(0xffffffffu, __popcll(cand)) <= kCandSlots && low != 0u) {
+        CandKeys<kCandSlots> ck;
+#pragma unroll
+        for (int j = 0; j < kCandSlots; ++j) {
+          ck.k[j] = 0u;
+          ck.c[j] = 0;
+          if (cand != 0ull) {
+            const int t = __ffsll((long long)cand) - 1;
+            cand &= cand - 1ull;
+            ck.k[j] = key.get(t);
+            ck.c[j] = col0 + t;
+          }
+        }
+        select_row(ck, hist_all[warp], lane, k_hat, out);
+        return;
+      }
     }
   }
-  if (row_counts != nullptr) {
-    cnt = __reduce_add_sync(0xffffffffu, cnt);
-    if (lane == 0) row_counts[row] = cnt;
-  }
+  select_row(key, hist_all[warp], lane, k_hat, out);
 }
 
 // Selection with one thread per row, for short rows and small k_hat: no cross-lane traffic at
@@ -431,7 +548,7 @@ bool launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, uint32_t* ma
                  const sea_shape& s, bool aware, cudaStream_t st) {
   const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
   constexpr bool kShared = VPL >= 32;  // beyond 512 columns the keys no longer fit the registers
-  const size_t smem = kShared ? (size_t)kWarpsPerCta * VPL * 32 * sizeof(uint32_t) : 0;
+  const size_t smem = kShared ? (size_t)kWarpsPerCta * (VPL + 1) * 32 * sizeof(uint32_t) : 0;
   auto kern = topk_rows_kernel<VPL, kShared>;
   if (smem > 40 * 1024 && cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return false;
