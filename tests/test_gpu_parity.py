@@ -259,8 +259,9 @@ def test_causality_by_perturbation_on_device():
     assert torch.equal(a.P[:n].view(torch.int16), b.P[:n].view(torch.int16))
 
 
-def test_host_entry_point_matches_device_entry_point():
-    w = small("host", causal=True, dtype="bf16", T=256, Kc=32, k_hat=6, m=64)
+@pytest.mark.parametrize("B,H", [(1, 2), (2, 16), (4, 16)])  # one slice, four and eight slices of heads
+def test_host_entry_point_matches_device_entry_point(B, H):
+    w = small("host", causal=True, dtype="bf16", T=256, Kc=32, k_hat=6, m=64, B=B, H=H)
     dev_run = GpuRun(w)
     dev_run.attention(); dev_run.sync()
     shp = sea.make_shape(w)
