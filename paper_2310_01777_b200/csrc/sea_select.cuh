@@ -68,7 +68,7 @@ __device__ __forceinline__ void merge_group(float (&top)[KMAX], float (&grp)[KMA
 
 // One block of 32 columns starting at j0: `gt` marks the columns above the k_hat-th largest value,
 // `eq` those equal to it, of which the lowest `ties_left` (over the whole row, in column order) are
-// still to be taken.  Appends the selected columns to my_sel (ascending), adds their keys after
+// still to be taken.  Appends the selected columns to my_sel (ascending; may be null), adds their keys after
 // up-sampling to cnt (column c covers keys c r .. c r + r - 1; a causal row i keeps those <= i) and
 // stores the block's word of the bit mask.
 __device__ __forceinline__ void emit_columns(uint32_t gt, uint32_t eq, int j0, int& ties_left, int32_t* my_sel, int& out,
@@ -88,7 +88,8 @@ __device__ __forceinline__ void emit_columns(uint32_t gt, uint32_t eq, int j0, i
   while (word) {
     const int j = j0 + __ffs(word) - 1;
     word &= word - 1u;
-    my_sel[out++] = j;
+    if (my_sel != nullptr) my_sel[out] = j;
+    ++out;
     cnt += causal ? max(0, min(r, i + 1 - j * r)) : r;
   }
 }

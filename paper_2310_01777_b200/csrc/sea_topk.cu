@@ -363,14 +363,18 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
 // as equal exactly as the bit search's keys do.
 constexpr int kThreadRows = 128;  // threads (= rows) per CTA
 
-template <int KMAX, bool kVec>
+template <int KMAX, bool kVec, bool kAware>
 __global__ void __launch_bounds__(kThreadRows)
 topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
-                        int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc,
-                        int k_hat, int seq_len, int r, int causal) {
+                        int32_t* __restrict__ row_counts, uint32_t* __restrict__ mask_bits, int rows, int Kc_all,
+                        int k_all, int seq_len, int r, int causal) {
   const int row = blockIdx.x * kThreadRows + threadIdx.x;
   if (row >= rows) return;
-  const float* a = A_hat + (size_t)row * Kc;
+  const float* a = A_hat + (size_t)row * Kc_all;
+  const int i = row % seq_len;
+  // kAware: only the columns that hold a key j <= i compete, and at most as many are kept
+  const int Kc = kAware ? min(Kc_all, i / r + 1) : Kc_all;
+  const int k_hat = min(k_all, Kc);
   // Descending list.  Its first KMAX - k_hat slots hold +inf, above every (finite) value, so the
   // k_hat-th largest value of the row always ends up in the last slot; -inf stands for columns
   // beyond the row.
@@ -379,12 +383,15 @@ topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ s
   for (int s = 0; s < KMAX; ++s) top[s] = s < KMAX - k_hat ? INFINITY : -INFINITY;
   for (int j0 = 0; j0 < Kc; j0 += KMAX) {
     float grp[KMAX];
-    if (kVec) {  // Kc % 4 == 0: rows start on 16-byte boundaries
+    if (kVec) {  // Kc_all % 4 == 0: rows start on 16-byte boundaries
 #pragma unroll
       for (int j = 0; j < KMAX; j += 4) {
         float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
         if (j0 + j < Kc) v = __ldg(reinterpret_cast<const float4*>(a + j0 + j));
-        grp[j] = v.x; grp[j + 1] = v.y; grp[j + 2] = v.z; grp[j + 3] = v.w;
+        grp[j] = v.x;
+        grp[j + 1] = !kAware || j0 + j + 1 < Kc ? v.y : -INFINITY;  // Kc_all is a multiple of 4, the visible part need not be
+        grp[j + 2] = !kAware || j0 + j + 2 < Kc ? v.z : -INFINITY;
+        grp[j + 3] = !kAware || j0 + j + 3 < Kc ? v.w : -INFINITY;
       }
     } else {
 #pragma unroll
@@ -398,11 +405,10 @@ topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ s
   for (int s = 0; s < KMAX; ++s) n_gt += (top[s] != INFINITY && top[s] > tau);
   int ties_left = k_hat - n_gt;  // how many columns equal to tau are still to be taken (lowest first)
 
-  const int i = row % seq_len;
-  const int words = (Kc + 31) / 32;
-  int32_t* my_sel = sel + (size_t)row * k_hat;
+  const int words = (Kc_all + 31) / 32;
+  int32_t* my_sel = sel != nullptr ? sel + (size_t)row * k_all : nullptr;
   int out = 0, cnt = 0;
-  for (int j0 = 0; j0 < Kc; j0 += 32) {
+  for (int j0 = 0; j0 < Kc_all; j0 += 32) {
     uint32_t gt = 0u, eq = 0u;
     if (kVec) {
 #pragma unroll
@@ -412,8 +418,9 @@ topk_rows_thread_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ s
         const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          gt |= (x[e] > tau ? 1u : 0u) << (j + e);
-          eq |= (x[e] == tau ? 1u : 0u) << (j + e);
+          const bool in = !kAware || j0 + j + e < Kc;
+          gt |= (in && x[e] > tau ? 1u : 0u) << (j + e);
+          eq |= (in && x[e] == tau ? 1u : 0u) << (j + e);
         }
       }
     } else {
@@ -600,11 +607,13 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
 #define SEA_TOPK_THREAD(KM)                                                                                     \
   do {                                                                                                          \
     if (s.Kc % 4 == 0)                                                                                          \
-      topk_rows_thread_kernel<KM, true><<<grid, kThreadRows, 0, st>>>(A_hat, sel, counts, mask_bits, rows,     \
-                                                                      s.Kc, s.k_hat, s.T, r, s.causal);        \
+      topk_rows_thread_kernel<KM, true, false><<<grid, kThreadRows, 0, st>>>(A_hat, sel, counts, mask_bits,    \
+                                                                             rows, s.Kc, s.k_hat, s.T, r,      \
+                                                                             s.causal);                        \
     else                                                                                                        \
-      topk_rows_thread_kernel<KM, false><<<grid, kThreadRows, 0, st>>>(A_hat, sel, counts, mask_bits, rows,    \
-                                                                       s.Kc, s.k_hat, s.T, r, s.causal);       \
+      topk_rows_thread_kernel<KM, false, false><<<grid, kThreadRows, 0, st>>>(A_hat, sel, counts, mask_bits,   \
+                                                                              rows, s.Kc, s.k_hat, s.T, r,     \
+                                                                              s.causal);                       \
   } while (0)
     if (s.k_hat <= 8) SEA_TOPK_THREAD(8);
     else if (s.k_hat <= 16) SEA_TOPK_THREAD(16);
@@ -698,7 +707,26 @@ sea_status launch_topk_mask_aware(const sea_shape& s, const float* A_hat, uint32
                                   int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts, int32_t* tile_sums,
                                   int32_t* status, cudaStream_t st) {
   const int rows = s.B * s.H * s.T;
-  if (!launch_topk_rows(A_hat, nullptr, row_counts, mask_bits, rows, s, true, st)) return SEA_ERR_UNSUPPORTED;
+  if (s.Kc <= kThreadMaxKc && s.k_hat <= kThreadMaxK) {
+    // a short row and few columns to keep: one thread per row
+    const int grid = (rows + kThreadRows - 1) / kThreadRows;
+    const int r = s.T / s.Kc;
+#define SEA_AWARE_THREAD(KM)                                                                                          \
+  do {                                                                                                                \
+    if (s.Kc % 4 == 0)                                                                                                \
+      topk_rows_thread_kernel<KM, true, true><<<grid, kThreadRows, 0, st>>>(A_hat, nullptr, row_counts, mask_bits,   \
+                                                                            rows, s.Kc, s.k_hat, s.T, r, s.causal);  \
+    else                                                                                                              \
+      topk_rows_thread_kernel<KM, false, true><<<grid, kThreadRows, 0, st>>>(A_hat, nullptr, row_counts, mask_bits,  \
+                                                                             rows, s.Kc, s.k_hat, s.T, r, s.causal); \
+  } while (0)
+    if (s.k_hat <= 8) SEA_AWARE_THREAD(8);
+    else if (s.k_hat <= 16) SEA_AWARE_THREAD(16);
+    else SEA_AWARE_THREAD(32);
+#undef SEA_AWARE_THREAD
+  } else if (!launch_topk_rows(A_hat, nullptr, row_counts, mask_bits, rows, s, true, st)) {
+    return SEA_ERR_UNSUPPORTED;
+  }
   sea_status rc = check_launch();
   if (rc != SEA_OK) return rc;
   if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
