@@ -296,7 +296,7 @@ sea_status sea_sparse_attn_masked(const sea_shape* shape, const void* Q, const v
   const WsLayout L = ws_layout(*shape);
   const bool full = ws && ws_bytes >= L.total && shape->io == SEA_BF16;
   return launch_sparse_attn_masked(*shape, Q, K, V, row_ptr, col_idx, mask_bits, O, P,
-                                   full ? reinterpret_cast<int32_t*>(w + L.park_off) : nullptr, false,
+                                   full ? reinterpret_cast<int32_t*>(w + L.park_off) : nullptr, false, false,
                                    full ? reinterpret_cast<float*>(w + L.p_scratch) : nullptr,
                                    static_cast<int32_t*>(ws), static_cast<cudaStream_t>(cuda_stream));
 }
@@ -352,11 +352,11 @@ sea_status attention_bits(BitsMode mode, const sea_shape* shape, const void* Q, 
     rc = launch_topk_mask_grouped(*shape, a_use, bits, rp_buf, col_idx, nnz_cap, counts, sums, tiles && P ? park : nullptr,
                                   status, st);
     if (rc != SEA_OK) return rc;
-    return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, true, scratch, status, st);
+    return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, true, false, scratch, status, st);
   }
   rc = launch_topk_mask_aware(*shape, a_use, bits, rp_buf, col_idx, nnz_cap, counts, sums, status, st);
   if (rc != SEA_OK) return rc;
-  return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, false, scratch, status, st);
+  return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, false, true, scratch, status, st);
 }
 }  // namespace
 

@@ -101,11 +101,13 @@ sea_status launch_topk_mask_capped(const sea_shape& s, int k_star, const float* 
 sea_status launch_park_offsets(const sea_shape& s, const uint32_t* mask_bits, int32_t* park_off,
                                int32_t* status, cudaStream_t st);
 // Sparse stage for a mask given as bits with its row_ptr (rows of any length).  park_valid:
-// park_off already holds the offsets that belong to mask_bits.
+// park_off already holds the offsets that belong to mask_bits.  rows_within_k_hat: no row keeps
+// more than k_hat columns, so the per-query parking layout serves and no offsets are needed.
 sea_status launch_sparse_attn_masked(const sea_shape& s, const void* Q, const void* K, const void* V,
                                      const int32_t* row_ptr, const int32_t* col_idx,
                                      const uint32_t* mask_bits, void* O, void* P, int32_t* park_off,
-                                     bool park_valid, float* p_scratch, int32_t* status, cudaStream_t st);
+                                     bool park_valid, bool rows_within_k_hat, float* p_scratch,
+                                     int32_t* status, cudaStream_t st);
 // mask_bits and p_scratch (workspace areas of the tensor-core kernel) may be null: the per-row
 // kernels are used then.  bits_valid: mask_bits already holds the bit strings of `sel`
 // (launch_topk_mask wrote them); otherwise they are derived from `sel` first.

@@ -380,9 +380,12 @@ sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, 
 
 sea_status launch_sparse_attn_masked(const sea_shape& s, const void* Q, const void* K, const void* V,
                                      const int32_t* row_ptr, const int32_t* col_idx, const uint32_t* mask_bits,
-                                     void* O, void* P, int32_t* park_off, bool park_valid, float* p_scratch,
-                                     int32_t* status, cudaStream_t st) {
+                                     void* O, void* P, int32_t* park_off, bool park_valid, bool rows_within_k_hat,
+                                     float* p_scratch, int32_t* status, cudaStream_t st) {
   if (park_off != nullptr && sparse_attn_tc_applicable(s, nullptr, true, status, mask_bits, p_scratch)) {
+    if (P != nullptr && rows_within_k_hat)  // every row fits the per-query parking layout
+      return launch_sparse_attn_tc(s, Q, K, V, row_ptr, nullptr, O, P, const_cast<uint32_t*>(mask_bits), true, p_scratch,
+                                   nullptr, status, st);
     if (P != nullptr && !park_valid) {
       const sea_status rc = launch_park_offsets(s, mask_bits, park_off, status, st);
       if (rc != SEA_OK) return rc;
