@@ -47,9 +47,9 @@ METRIC = "SEA attention-layer tokens/s on 1 B200 (all stages)"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparse-attention launch, from the ncu capture
-# summarised in profiles/sparse_attn_tiles_tc_opt_1p3b.md (one launch covers the whole workload; 298.2 MB
-# read + 200.9 MB written).
-NCU_TRAFFIC_BYTES = {"opt_1p3b": 499.2e6}
+# summarised in profiles/sparse_attn_tiles_tc_opt_1p3b.md (one launch covers the whole workload; 290.6 MB
+# read + 200.7 MB written).
+NCU_TRAFFIC_BYTES = {"opt_1p3b": 491.3e6}
 
 
 def measured_peaks():
