@@ -214,6 +214,9 @@ def main():
         run_reference(args, w)
         return
 
+    if w.m == 0:
+        raise SystemExit(f"bench.py times workloads that start at the estimator; {w.name} is a parity-test case")
+
     import torch
     import torch.distributed as dist
 
