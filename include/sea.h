@@ -12,7 +12,10 @@
  *   - Pointers named Q, K, V, O, P, A_hat, sel, row_ptr, col_idx, omega, W_dec
  *     and ws are DEVICE pointers owned by the caller, 16-byte aligned, dense and
  *     row-major with the last index fastest.  The library never allocates or
- *     frees device memory and keeps no state between calls except inside `ws`.
+ *     frees device memory.  State kept between calls: the contents of `ws`; the
+ *     two copy streams and the events of sea_attention_host, which a host thread
+ *     creates on its first call on a device and keeps until it exits; and the
+ *     static scratch array of sea_topk_mask_static (see there).
  *   - Q, K, V, O are [B, H, T, d] in the dtype `shape->io`; d must be 64.
  *   - A "row" is one query: row = (b*H + h)*T + i, rows = B*H*T.
  *   - r = T / Kc keys are covered by one compressed column (T % Kc == 0).
@@ -23,6 +26,12 @@
  *     Anomalies only visible on the device (a row longer than nnz_cap allows, a
  *     non-finite normaliser) set bits in a status word inside `ws`, the kernel
  *     finishes safely, and sea_device_status() reads the word back.
+ *   - The sparse stage finds a row's entries of col_idx and P through row_ptr alone
+ *     and never sees a capacity.  In sea_sparse_attn / sea_sparse_attn_masked the
+ *     caller guarantees that col_idx and P hold row_ptr[rows] elements.  The fused
+ *     calls return SEA_ERR_TOO_LARGE, launching nothing, when P is requested (or
+ *     the sparse stage has to walk col_idx) and nnz_cap is below the largest mask
+ *     the shape allows (rows*k_hat*r; capped calls: rows*k_hat*min(k_star, r)).
  *   - Inputs must be finite.
  *   - Calls that share a workspace must be ordered on one stream.
  */
@@ -51,7 +60,7 @@ typedef enum { SEA_F32 = 0, SEA_BF16 = 1 } sea_dtype;
 enum {
   SEA_DEV_ROW_OVERFLOW = 1, /* a CSR row did not fit below nnz_cap and was truncated */
   SEA_DEV_NONFINITE = 2,    /* the estimator met a zero or non-finite normaliser */
-  SEA_DEV_TIMEOUT = 4       /* a bounded wait on an asynchronous copy ran out; the affected rows of O are zero */
+  SEA_DEV_TIMEOUT = 4       /* a bounded wait on an asynchronous copy or tensor-core product ran out: the output of that call is not valid */
 };
 
 typedef struct sea_shape {
@@ -235,8 +244,12 @@ sea_status sea_attention_causal_aware(const sea_shape* shape, const void* Q, con
  * c*r + floor(u*r/k_star), u = 0 .. k_star-1 (k_star >= r keeps the whole run).
  * Causal rows drop keys j > i.  Works for any k_hat; T % Kc == 0 is still
  * required.  col_idx is required (the sparse stage walks the CSR with the per-row
- * kernels); nnz_cap rows*k_hat*min(k_star, r) always suffices.
+ * kernels); nnz_cap rows*k_hat*min(k_star, r) always suffices, and it is this
+ * product, not the uncapped mask, that has to fit int32 (T = 131072, Kc = 128,
+ * k_hat = 1, k_star = 64 with 32 heads is within range).  sea_workspace_bytes_capped
+ * is sea_workspace_bytes under that limit.
  */
+sea_status sea_workspace_bytes_capped(const sea_shape* shape, int32_t k_star, size_t* bytes);
 sea_status sea_topk_mask_capped(const sea_shape* shape, int32_t k_star, const float* A_hat, int32_t* sel,
                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
                                 void* ws, size_t ws_bytes, void* cuda_stream);
@@ -271,6 +284,11 @@ sea_status sea_device_status(void* ws, int32_t* out, int32_t clear, void* cuda_s
 /* Number of kernel launches the last call of each entry point enqueued from
  * this thread (for benchmark bookkeeping). */
 int32_t sea_last_launch_count(void);
+
+/* Name of the kernel that the sparse stage of this thread's last call launched
+ * ("none" before the first one): the stage chooses among several kernels by shape,
+ * dtype and workspace, and a benchmark has to know which one it timed. */
+const char* sea_last_sparse_kernel(void);
 
 const char* sea_status_string(sea_status s);
 

@@ -273,25 +273,3 @@ def sea_attention_grouped_batch(Q, K, V, k_hat: int, Kc: int, causal: bool, scal
         O, P = sparse_attention(Q[h], K[h], V[h], row_ptr, col_idx, scale)
         out.append(dict(A_hat=_f64(A_hat[h]), cols=cols[h], row_ptr=row_ptr, col_idx=col_idx, O=O, P=P))
     return out
-
-
-def flatten_heads(per_head, T: int):
-    """Join per-head results in flat row order ((b*H + h)*T + i).
-
-    ``per_head`` is the list of ``sea_attention_head`` dicts in (b, h) order.
-    Row pointers become global offsets into the concatenated col_idx / P.
-    """
-    row_ptr = [np.zeros(1, dtype=np.int64)]
-    base = 0
-    for r in per_head:
-        row_ptr.append(r["row_ptr"][1:] + base)
-        base += int(r["row_ptr"][-1])
-    out = dict(
-        row_ptr=np.concatenate(row_ptr),
-        col_idx=np.concatenate([r["col_idx"] for r in per_head]),
-        P=np.concatenate([r["P"] for r in per_head]),
-        sel=np.concatenate([r["sel"] for r in per_head], axis=0) if "sel" in per_head[0] else None,
-        O=np.concatenate([r["O"] for r in per_head], axis=0),
-        A_hat=np.concatenate([r["A_hat"] for r in per_head], axis=0),
-    )
-    return out

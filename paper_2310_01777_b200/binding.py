@@ -26,12 +26,15 @@ SEA_F32 = 0
 SEA_BF16 = 1
 SEA_DEV_ROW_OVERFLOW = 1
 SEA_DEV_NONFINITE = 2
+SEA_DEV_TIMEOUT = 4
 
 EXPORTS = (
     "sea_workspace_bytes", "sea_estimate", "sea_topk_mask", "sea_topk_mask_static", "sea_sparse_attn",
     "sea_attention", "sea_topk_mask_grouped", "sea_sparse_attn_masked", "sea_attention_grouped",
-    "sea_topk_mask_causal_aware", "sea_attention_causal_aware", "sea_topk_mask_capped", "sea_attention_capped",
+    "sea_topk_mask_causal_aware", "sea_attention_causal_aware", "sea_workspace_bytes_capped", "sea_topk_mask_capped",
+    "sea_attention_capped",
     "sea_workspace_host_bytes", "sea_attention_host", "sea_device_status", "sea_last_launch_count",
+    "sea_last_sparse_kernel",
     "sea_status_string",
 )
 
@@ -77,17 +80,20 @@ def load_library() -> ctypes.CDLL:
     lib.sea_attention_grouped.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
     lib.sea_topk_mask_causal_aware.argtypes = lib.sea_topk_mask_grouped.argtypes
     lib.sea_attention_causal_aware.argtypes = lib.sea_attention_grouped.argtypes
+    lib.sea_workspace_bytes_capped.argtypes = [shp, i32, ctypes.POINTER(sz)]
     lib.sea_topk_mask_capped.argtypes = [shp, i32, vp, vp, vp, vp, i64, vp, sz, vp]
     lib.sea_attention_capped.argtypes = [shp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
     lib.sea_attention_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sea_device_status.argtypes = [vp, ctypes.POINTER(i32), i32, vp]
     lib.sea_last_launch_count.argtypes = []
     lib.sea_last_launch_count.restype = i32
+    lib.sea_last_sparse_kernel.argtypes = []
+    lib.sea_last_sparse_kernel.restype = ctypes.c_char_p
     lib.sea_status_string.argtypes = [ctypes.c_int]
     lib.sea_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
         fn = getattr(lib, name)
-        if name not in ("sea_last_launch_count", "sea_status_string"):
+        if name not in ("sea_last_launch_count", "sea_last_sparse_kernel", "sea_status_string"):
             fn.restype = ctypes.c_int
     _lib = lib
     return lib
@@ -122,6 +128,13 @@ def _check(code: int, where: str):
 def sea_workspace_bytes(shape: SeaShape) -> int:
     out = ctypes.c_size_t(0)
     _check(load_library().sea_workspace_bytes(ctypes.byref(shape), ctypes.byref(out)), "sea_workspace_bytes")
+    return out.value
+
+
+def sea_workspace_bytes_capped(shape: SeaShape, k_star: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(load_library().sea_workspace_bytes_capped(ctypes.byref(shape), k_star, ctypes.byref(out)),
+           "sea_workspace_bytes_capped")
     return out.value
 
 
@@ -266,3 +279,7 @@ def sea_device_status(ws, clear: bool = True) -> int:
 
 def sea_last_launch_count() -> int:
     return load_library().sea_last_launch_count()
+
+
+def sea_last_sparse_kernel() -> str:
+    return load_library().sea_last_sparse_kernel().decode()

@@ -9,7 +9,15 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 size_t io_bytes(const sea_shape& s) { return s.io == SEA_BF16 ? 2 : 4; }
 }  // namespace
 
-sea_status validate_shape(const sea_shape* s, bool need_estimator) {
+// Largest number of CSR entries the mask of this shape can hold: every row keeps k_hat columns of
+// min(r, k_star) keys (k_star <= 0: whole runs).
+long long mask_entries_bound(const sea_shape& s, int k_star) {
+  const long long r = s.T / s.Kc;
+  const long long per_col = k_star > 0 && k_star < r ? k_star : r;
+  return (long long)s.B * s.H * s.T * s.k_hat * per_col;
+}
+
+sea_status validate_shape(const sea_shape* s, bool need_estimator, int k_star) {
   if (s == nullptr) return SEA_ERR_INVALID_ARG;
   if (s->B <= 0 || s->H <= 0 || s->T <= 0 || s->Kc <= 0 || s->k_hat <= 0) return SEA_ERR_INVALID_ARG;
   if (s->causal != 0 && s->causal != 1) return SEA_ERR_INVALID_ARG;
@@ -22,9 +30,8 @@ sea_status validate_shape(const sea_shape* s, bool need_estimator) {
   if (s->Kc > 2048) return SEA_ERR_UNSUPPORTED;
   if (need_estimator && (s->m < 16 || s->m > 128 || s->m % 16 != 0)) return SEA_ERR_UNSUPPORTED;
   const long long rows = (long long)s->B * s->H * s->T;
-  const long long r = s->T / s->Kc;
   const long long lim = 2147483647ll;
-  if (rows + 1 > lim || rows * s->k_hat * r > lim) return SEA_ERR_TOO_LARGE;
+  if (rows + 1 > lim || mask_entries_bound(*s, k_star) > lim) return SEA_ERR_TOO_LARGE;
   return SEA_OK;
 }
 
@@ -49,7 +56,7 @@ WsLayout ws_layout(const sea_shape& s) {
   L.sel = take(rows * (size_t)s.k_hat * sizeof(int32_t));
   L.row_ptr = take((rows + 1) * sizeof(int32_t));
   L.mask_bits = take(sparse_attn_tc_bits_bytes(s));
-  L.p_scratch = take(s.io == SEA_BF16 ? sparse_attn_tc_scratch_bytes(s) : 0);
+  L.p_scratch = take(sparse_attn_tc_shape_ok(s) ? sparse_attn_tc_scratch_bytes(s) : 0);  // only the tile kernel parks
   L.park_off = take(s.io == SEA_BF16 ? rows * sizeof(int32_t) : 0);
   L.total = off;
   return L;
@@ -198,6 +205,10 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
     return SEA_ERR_INVALID_ARG;
   if (col_idx && nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
   if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  // The sparse stage writes P at the positions row_ptr gives and never learns nnz_cap: a capacity
+  // that a long mask could exceed is refused here.  (col_idx alone may be shorter: the fill
+  // truncates and reports, and the sparse stage walks `sel`, not col_idx.)
+  if (P && nnz_cap < mask_entries_bound(*shape, 0)) return SEA_ERR_TOO_LARGE;
   const WsLayout L = ws_layout(*shape);
   if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
   char* w = static_cast<char*>(ws);
@@ -332,8 +343,11 @@ sea_status attention_bits(BitsMode mode, const sea_shape* shape, const void* Q, 
   uint32_t* bits = mask_bits ? mask_bits : reinterpret_cast<uint32_t*>(w + L.mask_bits);
   float* scratch = shape->io == SEA_BF16 ? reinterpret_cast<float*>(w + L.p_scratch) : nullptr;
   int32_t* park = shape->io == SEA_BF16 ? reinterpret_cast<int32_t*>(w + L.park_off) : nullptr;
-  if (!col_idx && !(park && sparse_attn_tc_applicable(*shape, nullptr, true, status, bits, scratch)))
-    return SEA_ERR_INVALID_ARG;
+  const bool tiles_ok = park && sparse_attn_tc_applicable(*shape, nullptr, true, status, bits, scratch);
+  if (!col_idx && !tiles_ok) return SEA_ERR_INVALID_ARG;
+  // P is written at the positions row_ptr gives, and without the tile kernel the sparse stage walks
+  // col_idx; neither learns nnz_cap, so a capacity that the mask could exceed is refused here
+  if (col_idx && (P || !tiles_ok) && nnz_cap < mask_entries_bound(*shape, 0)) return SEA_ERR_TOO_LARGE;
 
   const float* a_use = A_hat_in;
   if (estimate) {
@@ -348,8 +362,7 @@ sea_status attention_bits(BitsMode mode, const sea_shape* shape, const void* Q, 
   int32_t* sums = reinterpret_cast<int32_t*>(w + L.tile_sums);
   if (mode == BitsMode::kPerBatch) {
     // the selection also lays out the parking area of the tile kernel when P is wanted
-    const bool tiles = park && sparse_attn_tc_applicable(*shape, nullptr, true, status, bits, scratch);
-    rc = launch_topk_mask_grouped(*shape, a_use, bits, rp_buf, col_idx, nnz_cap, counts, sums, tiles && P ? park : nullptr,
+    rc = launch_topk_mask_grouped(*shape, a_use, bits, rp_buf, col_idx, nnz_cap, counts, sums, tiles_ok && P ? park : nullptr,
                                   status, st);
     if (rc != SEA_OK) return rc;
     return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, true, false, scratch, status, st);
@@ -378,13 +391,22 @@ sea_status sea_attention_causal_aware(const sea_shape* shape, const void* Q, con
                         col_idx, nnz_cap, P, ws, ws_bytes, cuda_stream);
 }
 
+sea_status sea_workspace_bytes_capped(const sea_shape* shape, int32_t k_star, size_t* bytes) {
+  if (bytes == nullptr || k_star < 1) return SEA_ERR_INVALID_ARG;
+  const sea_status rc = validate_shape(shape, false, k_star);
+  if (rc != SEA_OK) return rc;
+  *bytes = ws_layout(*shape).total;
+  return SEA_OK;
+}
+
 sea_status sea_topk_mask_capped(const sea_shape* shape, int32_t k_star, const float* A_hat, int32_t* sel,
                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* ws, size_t ws_bytes,
                                 void* cuda_stream) {
   Launch::count() = 0;
-  const sea_status rc = validate_shape(shape, false);
+  if (k_star < 1) return SEA_ERR_INVALID_ARG;
+  const sea_status rc = validate_shape(shape, false, k_star);
   if (rc != SEA_OK) return rc;
-  if (k_star < 1 || !A_hat || !row_ptr || !col_idx || !ws) return SEA_ERR_INVALID_ARG;
+  if (!A_hat || !row_ptr || !col_idx || !ws) return SEA_ERR_INVALID_ARG;
   if (!aligned16(A_hat) || !aligned16(row_ptr) || !aligned16(col_idx) || !aligned16(ws) || (sel && !aligned16(sel)))
     return SEA_ERR_INVALID_ARG;
   if (nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
@@ -405,9 +427,10 @@ sea_status sea_attention_capped(const sea_shape* shape, int32_t k_star, const vo
                                 size_t ws_bytes, void* cuda_stream) {
   Launch::count() = 0;
   const bool estimate = A_hat_in == nullptr;
-  sea_status rc = validate_shape(shape, estimate);
+  if (k_star < 1) return SEA_ERR_INVALID_ARG;
+  sea_status rc = validate_shape(shape, estimate, k_star);
   if (rc != SEA_OK) return rc;
-  if (k_star < 1 || !Q || !K || !V || !O || !ws || !col_idx) return SEA_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !O || !ws || !col_idx) return SEA_ERR_INVALID_ARG;
   if (estimate && (!omega || !W_dec)) return SEA_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(ws) || !aligned16(col_idx) ||
       (omega && !aligned16(omega)) || (W_dec && !aligned16(W_dec)) || (A_hat_in && !aligned16(A_hat_in)) ||
@@ -415,6 +438,8 @@ sea_status sea_attention_capped(const sea_shape* shape, int32_t k_star, const vo
     return SEA_ERR_INVALID_ARG;
   if (nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
   if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  // the sparse stage walks col_idx (and writes P) by row_ptr alone: the capacity must hold any mask
+  if (nnz_cap < mask_entries_bound(*shape, k_star)) return SEA_ERR_TOO_LARGE;
   const WsLayout L = ws_layout(*shape);
   if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
   char* w = static_cast<char*>(ws);
@@ -474,8 +499,8 @@ sea_status sea_attention_host(const sea_shape* shape, const void* hQ, const void
 
   // The heads are independent, so the call runs as a pipeline over slices of them: while one slice
   // is computed on the caller's stream, the next one's Q, K, V come in on a second stream and the
-  // previous one's O goes out on a third (the link carries both directions at once).  The streams
-  // and events live for this call only.
+  // previous one's O goes out on a third (the link carries both directions at once).  The two
+  // copy streams and the events belong to the calling host thread, which creates them once.
   const int BH = shape->B * shape->H;
   int nslice = 1;
   for (int c = 8; c >= 2; c >>= 1)
@@ -538,6 +563,8 @@ sea_status sea_device_status(void* ws, int32_t* out, int32_t clear, void* cuda_s
 }
 
 int32_t sea_last_launch_count(void) { return Launch::count(); }
+
+const char* sea_last_sparse_kernel(void) { return Launch::sparse_kernel(); }
 
 const char* sea_status_string(sea_status s) {
   switch (s) {

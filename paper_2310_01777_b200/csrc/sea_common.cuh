@@ -13,10 +13,14 @@ constexpr int kHeadDim = 64;        // d, fixed by the interface
 constexpr int kStatusBytes = 256;   // head of every workspace: the device status word
 constexpr int kEstChunk = 64;       // rows per estimator chunk (prefix-state granularity)
 
-struct Launch {  // per-thread launch bookkeeping behind sea_last_launch_count()
+struct Launch {  // per-thread launch bookkeeping behind sea_last_launch_count() / sea_last_sparse_kernel()
   static int& count() {
     static thread_local int c = 0;
     return c;
+  }
+  static const char*& sparse_kernel() {
+    static thread_local const char* k = "none";
+    return k;
   }
 };
 
@@ -39,7 +43,9 @@ struct WsLayout {
 };
 
 WsLayout ws_layout(const sea_shape& s);
-sea_status validate_shape(const sea_shape* s, bool need_estimator);
+// k_star > 0: a selected column keeps at most k_star keys (capped replication), which bounds the mask.
+sea_status validate_shape(const sea_shape* s, bool need_estimator, int k_star = 0);
+long long mask_entries_bound(const sea_shape& s, int k_star);
 
 // Where the per-query selection goes when the estimator's output kernel performs it (see
 // estimate_tc_selects): the same three arrays launch_topk_mask's selection kernel writes.
@@ -118,6 +124,8 @@ sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, 
 sea_status launch_sparse_attn_rows(const sea_shape& s, const void* Q, const void* K, const void* V,
                                    const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
                                    void* O, void* P, cudaStream_t st);
+// the shape alone allows the tensor-core tile kernel (dtype, T, r, density)
+bool sparse_attn_tc_shape_ok(const sea_shape& s);
 size_t sparse_attn_tc_bits_bytes(const sea_shape& s);
 size_t sparse_attn_tc_scratch_bytes(const sea_shape& s);
 // have_bits: mask_bits already holds the mask (sel may then be null)

@@ -402,6 +402,7 @@ sea_status launch_sparse_attn_masked(const sea_shape& s, const void* Q, const vo
 sea_status launch_sparse_attn_rows(const sea_shape& s, const void* Q, const void* K, const void* V,
                                    const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel, void* O,
                                    void* P, cudaStream_t st) {
+  Launch::sparse_kernel() = s.io == SEA_BF16 ? "sparse_attn_rows_mma_kernel" : "sparse_attn_rows_kernel";
   if (s.io == SEA_BF16) {
     using T = __nv_bfloat16;
     const int rows = s.B * s.H * s.T;

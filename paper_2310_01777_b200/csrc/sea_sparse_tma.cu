@@ -13,56 +13,32 @@
 // its K blocks, then all its V blocks - so the ring stays full while a row's softmax runs and
 // while the next row starts.  The warp is its own producer: after a block has been read, lane 0
 // issues the copy that is kSlots ahead in the stream; the row metadata that the producer needs
-// (row_ptr pair, selected columns) is fetched one row early into registers.  Waits are bounded:
-// a wait that runs out sets SEA_DEV_TIMEOUT in the status word and the warp stops.
+// (row_ptr pair, selected columns) is fetched one row early into registers.  Waits are bounded by
+// a clock: when one runs out the warp sets SEA_DEV_TIMEOUT in the status word, waits (bounded again)
+// for the copies it still has in flight, writes zeros to the output rows it leaves undone and stops.
 #include <cuda.h>
 
 #include "sea_common.cuh"
+#include "sea_tc.cuh"
 
 namespace sea {
 namespace {
+
+using namespace tc;
 
 constexpr int kWarps = 8;
 constexpr int kSlots = 4;              // ring depth per warp (power of two)
 constexpr int kSlotBytes = 16 * 128;   // 16 keys x 64 bf16
 constexpr int kMaxBlocks = 64;         // 16-key blocks per row (k_hat * r <= 1024, so k_hat <= 64)
-constexpr uint32_t kWaitPolls = 1u << 16;
 
 struct alignas(1024) WarpRing {
   unsigned char slot[kSlots][kSlotBytes];
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait for the given phase parity; false when the poll budget ran out.
-__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  if (mbar_try(bar, parity)) return true;  // the usual case: the copy landed long ago
-  for (uint32_t i = 0; i < kWaitPolls; ++i)
-    if (mbar_try(bar, parity)) return true;
-  return false;
-}
 __device__ __forceinline__ float ex2(float x) {  // 2^x for x <= 0 (flushes denormal results to zero)
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void ldsm4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -193,7 +169,8 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
   for (int i = 0; i < kSlots; ++i) pump();
 
   bool ok = true;
-  for (int row = wg; row < rows && ok; row += stride) {
+  int row = wg;
+  for (; row < rows; row += stride) {
     const int base = n_rp0, n = n_rp1 - n_rp0;
     uint32_t qw[8];  // q as the B operand of every k-step: b0 = dims 16s+2t.., b1 = dims 16s+8+2t..
 #pragma unroll
@@ -214,7 +191,8 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     float mx = -INFINITY;
     for (int b = 0; b < nb; ++b) {
       const uint32_t slot = c_s & (kSlots - 1);
-      ok &= mbar_wait(bars + 8 * slot, (c_s / kSlots) & 1);
+      ok = __all_sync(0xffffffffu, mbar_wait_alone(bars + 8 * slot, (c_s / kSlots) & 1));
+      if (!ok) break;  // nothing more is consumed or issued once a wait has run out
       const uint32_t sbase = ring + slot * kSlotBytes;
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -235,7 +213,6 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
       ++c_s;
       pump();
     }
-    ok = __all_sync(0xffffffffu, ok);  // a wait that ran out ends the warp's work after this row's K pass
     if (!ok) break;
     mx = warp_max(mx);
 
@@ -270,7 +247,8 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
       for (int e = 0; e < 4; ++e) acc_o[i][e] = 0.f;
     for (int b = 0; b < nb; ++b) {
       const uint32_t slot = c_s & (kSlots - 1);
-      ok &= mbar_wait(bars + 8 * slot, (c_s / kSlots) & 1);
+      ok = __all_sync(0xffffffffu, mbar_wait_alone(bars + 8 * slot, (c_s / kSlots) & 1));
+      if (!ok) break;  // nothing more is consumed or issued once a wait has run out
       const uint32_t sbase = ring + slot * kSlotBytes;
       const uint2 pa = pairs[8 * b + t];      // positions 16b+2t, 16b+2t+1
       const uint2 pb = pairs[8 * b + 4 + t];  // positions 16b+8+2t, 16b+9+2t
@@ -285,7 +263,6 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
       ++c_s;
       pump();
     }
-    ok = __all_sync(0xffffffffu, ok);
     if (!ok) break;
     // every lane of a quad holds the same sums; lane t writes tile t: dims 16t + g and 16t + 8 + g
     {
@@ -297,36 +274,16 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
       out[16 * t + 8 + g] = __float2bfloat16_rn(hi);
     }
   }
-  if (!ok && lane == 0) atomicOr(status, SEA_DEV_TIMEOUT);
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      return nullptr;
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
-// [total_rows][64] bf16, boxes of 16 rows x 64 columns, 128-byte swizzle.
-bool make_rows_map(CUtensorMap* map, const void* ptr, unsigned long long total_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {kHeadDim, total_rows};
-  const cuuint64_t strides[1] = {kHeadDim * sizeof(__nv_bfloat16)};
-  const cuuint32_t box[2] = {kHeadDim, 16};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  if (!ok) {
+    if (lane == 0) atomicOr(status, SEA_DEV_TIMEOUT);
+    // copies already issued still land in this CTA's shared memory: wait for them before leaving
+    for (; c_s != p_s; ++c_s) mbar_wait_drain(bars + 8 * (c_s & (kSlots - 1)), (c_s / kSlots) & 1);
+    for (; row < rows; row += stride) {  // the rows this warp leaves undone read as zero
+      __nv_bfloat16* out = O + (size_t)row * kHeadDim;
+      out[2 * lane] = __float2bfloat16_rn(0.f);
+      out[2 * lane + 1] = __float2bfloat16_rn(0.f);
+    }
+  }
 }
 
 template <bool kWriteP>
@@ -366,7 +323,8 @@ sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void*
   using T = __nv_bfloat16;
   const unsigned long long rows = (unsigned long long)s.B * s.H * s.T;
   CUtensorMap map_k, map_v;
-  if (!make_rows_map(&map_k, K, rows) || !make_rows_map(&map_v, V, rows)) return SEA_ERR_CUDA;
+  if (!make_rows_map_bf16(&map_k, K, rows, 16) || !make_rows_map_bf16(&map_v, V, rows, 16)) return SEA_ERR_CUDA;
+  Launch::sparse_kernel() = "sparse_attn_blocks_tma_kernel";
   if (P) return launch_tma<true>(s, map_k, map_v, (const T*)Q, row_ptr, sel, (T*)O, (T*)P, status, st);
   return launch_tma<false>(s, map_k, map_v, (const T*)Q, row_ptr, sel, (T*)O, nullptr, status, st);
 }

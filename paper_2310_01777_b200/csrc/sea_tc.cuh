@@ -36,14 +36,19 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 // Waits for the phase with the given parity; gives up (and raises the CTA's abort flag) after
-// kWaitNs, or as soon as another thread of the CTA has raised the flag.
+// kWaitNs, or as soon as another thread of the CTA has raised the flag.  kSleepNs > 0 backs off
+// between polls: for roles whose hand-offs happen once per work item and that are off the critical
+// path, so that their polling takes no issue slots from the warps that compute.
+template <int kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 32; ++i)
+    for (int i = 0; i < 32; ++i) {
       if (mbar_try(bar, parity)) return true;
+      if (kSleepNs > 0) __nanosleep(kSleepNs);
+    }
     if (*abort_flag) return false;
     if (global_ns() - t0 > kWaitNs) {
       *abort_flag = 1;
@@ -51,22 +56,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
-// The same for a role whose hand-offs happen once per work item and that is off the critical path:
-// it sleeps between polls, so that its polling takes no issue slots from the warps that compute.
 __device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait<200>(bar, parity, abort_flag);
+}
+// Waits for two barriers; the first polls of both are issued together so that their latencies
+// overlap (for single issuing threads whose every instruction is on the critical path).
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
+                                           volatile int* abort_flag) {
+  const uint32_t ra = mbar_try(bar_a, par_a), rb = mbar_try(bar_b, par_b);
+  if (ra & rb) return true;
+  if (!ra && !mbar_wait(bar_a, par_a, abort_flag)) return false;
+  if (!rb && !mbar_wait(bar_b, par_b, abort_flag)) return false;
+  return true;
+}
+// The same wait for a warp that shares no abort flag with others: bounded by time alone.
+__device__ __forceinline__ bool mbar_wait_alone(uint32_t bar, uint32_t parity) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 32; ++i) {
+    for (int i = 0; i < 32; ++i)
       if (mbar_try(bar, parity)) return true;
-      __nanosleep(200);
-    }
-    if (*abort_flag) return false;
-    if (global_ns() - t0 > kWaitNs) {
-      *abort_flag = 1;
-      return false;
-    }
+    if (global_ns() - t0 > kWaitNs) return false;
   }
 }
 // For the way out: waits for an armed copy barrier whatever the abort flag says (a CTA must not
@@ -191,6 +202,18 @@ inline bool make_map_3d(CUtensorMap* map, CUtensorMapDataType type, unsigned ele
   const cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, type, 3, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// [total_rows][64] bf16 tensor, boxes of box_rows rows x 64 columns, 128-byte swizzle.
+inline bool make_rows_map_bf16(CUtensorMap* map, const void* ptr, unsigned long long total_rows, unsigned box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {64, total_rows};
+  const cuuint64_t strides[1] = {64 * sizeof(__nv_bfloat16)};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 inline bool make_map_bf16_3d(CUtensorMap* map, const void* ptr, unsigned long long d0, unsigned long long d1,

@@ -142,7 +142,7 @@ __device__ __forceinline__ void select_row(const Keys& key, int* hist, int lane,
       // the keys inside the step, one per lane when there are at most 32
       int inside = 0;
 #pragma unroll
-      for (int t = 0; t < N; ++t) inside += ((top - key.get(t)) >> kHistShift) == (uint32_t)step;
+      for (int t = 0; t < N; ++t) inside += key.get(t) != 0u && ((top - key.get(t)) >> kHistShift) == (uint32_t)step;  // 0: an empty slot
       int pos = inside;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -158,7 +158,7 @@ __device__ __forceinline__ void select_row(const Keys& key, int* hist, int lane,
 #pragma unroll
         for (int t = 0; t < N; ++t) {
           const uint32_t rel = top - key.get(t);
-          if ((rel >> kHistShift) == (uint32_t)step) list[pos++] = kFine - (rel & kFine);  // grows with the key
+          if (key.get(t) != 0u && (rel >> kHistShift) == (uint32_t)step) list[pos++] = kFine - (rel & kFine);  // grows with the key
         }
         __syncwarp();
         const bool have = lane < n_in;

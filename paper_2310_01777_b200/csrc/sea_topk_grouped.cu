@@ -173,7 +173,7 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
 #pragma unroll
       for (int i = 0; i < VI; ++i)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) inside += ((top - key[i][e]) >> kFineBits) == step;
+        for (int e = 0; e < 4; ++e) inside += key[i][e] != 0u && ((top - key[i][e]) >> kFineBits) == step;  // 0: a padding slot
       if (inside > 0) {
         int at = atomicAdd(&list_n, inside);
         if (at + inside <= kListCap) {
@@ -182,7 +182,7 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const uint32_t rel = top - key[i][e];
-              if ((rel >> kFineBits) == step) list[at++] = kFineMask - (rel & kFineMask);  // grows with the key
+              if (key[i][e] != 0u && (rel >> kFineBits) == step) list[at++] = kFineMask - (rel & kFineMask);  // grows with the key
             }
         }
       }

@@ -98,3 +98,44 @@ def test_capped_rejects_bad_arguments():
     with pytest.raises(sea.SeaError) as e:
         sea.sea_topk_mask_capped(run.shape, 0, run.A_hat, run.sel, run.row_ptr, run.col_idx, run.ws)
     assert e.value.code == binding.SEA_ERR_INVALID_ARG
+
+
+def test_capped_fused_call_refuses_a_capacity_below_the_largest_mask():
+    """The per-row sparse kernels walk col_idx by row_ptr alone: a buffer that the mask could
+    overrun is refused on the host and nothing is launched."""
+    w = small("cap_short", T=256, Kc=16, k_hat=2)
+    k_star = 5
+    run = GpuRun(w)
+    run.col_idx.fill_(0)
+    need = w.rows * w.k_hat * k_star
+    with pytest.raises(sea.SeaError) as e:
+        sea.sea_attention_capped(run.shape, k_star, run.d["Q"], run.d["K"], run.d["V"], run.d["omega"], run.d["W_dec"],
+                                 run.O, run.ws, run.col_idx, row_ptr=run.row_ptr, P=run.P, nnz_cap=need - 1)
+    assert e.value.code == binding.SEA_ERR_TOO_LARGE
+    run.sync()
+    assert bool((run.col_idx == 0).all()) and bool((run.row_ptr == -1).all())
+    sea.sea_attention_capped(run.shape, k_star, run.d["Q"], run.d["K"], run.d["V"], run.d["omega"], run.d["W_dec"],
+                             run.O, run.ws, run.col_idx, row_ptr=run.row_ptr, P=run.P, nnz_cap=need)
+    run.sync()
+    assert run.status() == 0 and int(run.row_ptr[-1]) <= need
+
+
+def test_capped_shape_limit_counts_the_capped_mask():
+    """T = 131072 with Kc = 128 and 32 heads: the uncapped mask (rows * r = 2^32 entries) is beyond
+    int32, the capped one (rows * 64) is not, and only the capped calls accept the shape."""
+    w = Workload(name="cap_131k", B=1, H=32, T=131072, d=64, m=128, Kc=128, k_hat=1, causal=True, dtype="bf16", seed=0)
+    shape = sea.make_shape(w)
+    lib = binding.load_library()
+    import ctypes
+    n = ctypes.c_size_t(0)
+    assert lib.sea_workspace_bytes(ctypes.byref(shape), ctypes.byref(n)) == binding.SEA_ERR_TOO_LARGE
+    assert 0 < sea.sea_workspace_bytes_capped(shape, 64) < 8 << 30
+    x = torch.zeros(64, dtype=torch.float32, device="cuda:0")
+    i = torch.zeros(64, dtype=torch.int32, device="cuda:0")
+    # argument checks run in order: the shape passes (no TOO_LARGE), the tiny workspace is what is refused
+    with pytest.raises(sea.SeaError) as e:
+        sea.sea_topk_mask_capped(shape, 64, x, i, i, i, x.view(torch.uint8), nnz_cap=64)
+    assert e.value.code == binding.SEA_ERR_WORKSPACE
+    with pytest.raises(sea.SeaError) as e:
+        sea.sea_topk_mask_capped(shape, 2048, x, i, i, i, x.view(torch.uint8), nnz_cap=64)
+    assert e.value.code == binding.SEA_ERR_TOO_LARGE

@@ -221,6 +221,7 @@ def test_wide_row_selection_paths_are_bit_exact(Kc, k_hat):
     a[0, 0, 5, :] = a[0, 0, 5, :] * 1e-30                   # tiny magnitudes
     a[0, 0, 6, :] = a[0, 0, 6, :].abs() * 1e30              # huge magnitudes
     a[0, 0, 7, :] = -a[0, 0, 7, :].abs() - 0.5              # all negative
+    a[0, 0, 8, :] = -3.0e38 - a[0, 0, 8, :].abs() * 1e36    # every key close to the smallest finite one
     run = GpuRun(w, inputs=host)
     run.topk_mask(); run.sparse_attn(); run.sync()
     assert run.status() == 0
@@ -237,6 +238,36 @@ def test_small_nnz_cap_sets_status_and_stays_in_bounds():
     assert run.status() & binding.SEA_DEV_ROW_OVERFLOW
     assert run.status() == 0  # cleared by the read above
     assert bool((guard[cap:] == -7).all()) and bool((guard[:cap] >= 0).all())
+
+
+@pytest.mark.parametrize("dtype,causal", [("bf16", True), ("f32", False)])
+def test_fused_call_refuses_a_capacity_the_mask_could_exceed(dtype, causal):
+    """The sparse stage writes P by row_ptr alone, so the fused call must not start with a P
+    buffer that a long mask could overrun: it returns an error and touches nothing.  With col_idx
+    alone a short capacity is allowed: the fill stops at nnz_cap, reports it, and O is unaffected."""
+    w = small("fused_cap", causal=causal, dtype=dtype, T=256, Kc=32, k_hat=6, H=2, m=32)
+    full = GpuRun(w)
+    full.attention(); full.sync()
+    assert full.status() == 0
+    nnz = int(full.row_ptr[-1])
+    cap = nnz // 2 + 3
+    run = GpuRun(w)
+    run.col_idx.fill_(0)   # guard values that are valid key indices
+    run.P.fill_(7.0)
+    with pytest.raises(binding.SeaError) as err:
+        sea.sea_attention(run.shape, run.d["Q"], run.d["K"], run.d["V"], run.d["omega"], run.d["W_dec"], run.O, run.ws,
+                          sel=run.sel, row_ptr=run.row_ptr, col_idx=run.col_idx, P=run.P, nnz_cap=cap)
+    assert err.value.code == binding.SEA_ERR_TOO_LARGE
+    run.sync()
+    assert bool((run.col_idx == 0).all()) and bool((run.P == 7.0).all()) and bool((run.row_ptr == -1).all())
+    # the mask alone, into a buffer that is too short
+    sea.sea_attention(run.shape, run.d["Q"], run.d["K"], run.d["V"], run.d["omega"], run.d["W_dec"], run.O, run.ws,
+                      sel=run.sel, row_ptr=run.row_ptr, col_idx=run.col_idx, nnz_cap=cap)
+    run.sync()
+    assert run.status() & binding.SEA_DEV_ROW_OVERFLOW
+    assert bool((run.col_idx[cap:] == 0).all())
+    assert torch.equal(run.col_idx[:cap], full.col_idx[:cap])
+    assert torch.equal(run.row_ptr, full.row_ptr) and torch.equal(run.O, full.O)
 
 
 def test_causality_by_perturbation_on_device():
