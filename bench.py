@@ -7,24 +7,29 @@ A step is one sea_attention call (all stages) over one synthetic batch of the wo
 The default workload is the OPT-1.3B-shaped causal bf16 configuration, on which the headline
 metric is quoted.  One JSON line is printed by rank 0.
 
-  value      tokens/s (B*T per step, all ranks) with inputs resident in HBM, CUDA events per step,
-             L2 flushed between steps, max over ranks.
+  value      tokens/s (B*T per step, all ranks) with inputs resident in HBM: mean of K per-step CUDA
+             event pairs, L2 flushed between steps, max over ranks; `ms_stats` adds median and min.
   e2e        the same through sea_attention_host: pinned host Q, K, V, omega, W_dec in, O out.
-  roofline   the sparse-attention kernel: algorithmic bytes (Q + O + every row's gathered K/V)
-             over its CUDA-event time, against the measured HBM copy bandwidth.  The kernel forms
-             the masked products as dense tiles on the tensor cores and gathers nothing, so this
-             figure exceeds 1; `tensor` inside it gives the FLOPs the kernel really executes
-             (every key tile a query tile may see, Q K^T twice and P V as head + remainder)
-             against the measured dense bf16 peak.
-  stages     per-stage milliseconds from a second pass that calls the three stage entry points
+  clocks     nvidia-smi samples taken while the K timed steps and an untimed continuation of the
+             same steps run (the K steps alone last a few milliseconds, less than one sample).
+  stages_ms  per-stage milliseconds from a second pass that calls the three stage entry points
              with events between them (same kernels as the fused call).
+  roofline   the sparse-attention kernel, against the resource that binds the kernel that ran.  The
+             tile kernel forms the masked products as dense tiles on the tensor cores: achieved =
+             the FLOPs it executes / its time, peak = the measured dense bf16 rate.  The per-row
+             kernels gather: achieved = Q + O + every row's gathered K/V bytes / time against the
+             measured HBM copy bandwidth.  `gather_model` always gives that byte figure (the
+             benchmark definition's) without calling it a fraction of anything when the kernel
+             gathers nothing; `bounds_ms` lists the time each resource alone would need.
+  roofline_estimate, roofline_mask
+             the other two stages against HBM: their compulsory bytes / stage time.
   lean       the fused call asked for O and the CSR mask only (the estimate and the probabilities are
              never written out); per-rank, not part of `value`.
   grouped, causal_aware
              the same step with the causal-per-batch grouping (sea_attention_grouped) and with the
              causal-aware per-query selection (sea_attention_causal_aware) on this rank, and their
              selection and sparse stages; per-rank, not part of `value`.
-  cpu_baseline  the fp64 oracle on a bounded sample of heads, on this machine's host cores.
+  cpu_baseline  the fp64 oracle on a bounded sample of heads, one head per host core at a time.
 
 With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no
 exchange step between GPUs); value sums the ranks' tokens over the slowest rank's time.
@@ -32,8 +37,10 @@ exchange step between GPUs); value sums the ranks' tokens over the slowest rank'
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import statistics
 import subprocess
 import sys
 import threading
@@ -46,10 +53,15 @@ if ROOT not in sys.path:
 METRIC = "SEA attention-layer tokens/s on 1 B200 (all stages)"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one sparse-attention launch, from the ncu capture
-# summarised in profiles/sparse_attn_tiles_tc_opt_1p3b.md (one launch covers the whole workload; 290.6 MB
-# read + 200.7 MB written).
-NCU_TRAFFIC_BYTES = {"opt_1p3b": 491.3e6}
+SM_COUNT = 148
+XU_PER_CLK_PER_SM = 16  # ex2 results per clock and SM
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+KERNEL_SOURCES = {
+    "sparse_attn_tiles_tc_kernel": "sea_sparse_tc.cu",
+    "sparse_attn_blocks_tma_kernel": "sea_sparse_tma.cu",
+    "sparse_attn_rows_mma_kernel": "sea_sparse.cu",
+    "sparse_attn_rows_kernel": "sea_sparse.cu",
+}
 
 
 def measured_peaks():
@@ -61,6 +73,23 @@ def measured_peaks():
         return float(j["hbm_gbs"]), float(j["bf16_tflops"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
+
+
+def ncu_traffic(workload: str, kernel: str):
+    """DRAM bytes of one launch of `kernel` on `workload` from the tracked ncu record, or None when
+    there is none or the kernel's source file has changed since the capture."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            rec = json.load(f).get(workload, {}).get(kernel)
+        if rec is None:
+            return None
+        src = os.path.join(ROOT, "paper_2310_01777_b200", "csrc", KERNEL_SOURCES[kernel])
+        with open(src, "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != rec["source_sha256"]:
+                return None
+        return float(rec["dram_bytes_read"]) + float(rec["dram_bytes_write"])
+    except Exception:
+        return None
 
 
 class ClockSampler:
@@ -92,7 +121,6 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
-        time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -115,36 +143,70 @@ class ClockSampler:
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
         sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+        return {"sm_mhz": sm[len(sm) // 2], "sm_min_mhz": sm[0], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
                 "samples": len(sm)}
 
 
-def oracle_tokens_per_s(w, n_heads: int, repeats: int = 1):
-    """The fp64 oracle, as it stands, on the first n_heads (b, h) units of the workload."""
+# ---- the CPU oracle, timed ---------------------------------------------------------------------
+def _oracle_heads(job):
+    """Worker: the fp64 oracle, as it stands, on heads [lo, hi) of the workload; returns seconds."""
+    name, lo, hi = job
     import numpy as np
+    import torch
     from threadpoolctl import threadpool_limits
 
     from oracle import sea_oracle as orc
-    from paper_2310_01777_b200.inputs import make_inputs
+    from paper_2310_01777_b200.inputs import WORKLOADS, make_inputs
 
-    small = w.scaled(B=1, H=n_heads)
+    w = WORKLOADS[name]
+    torch.set_num_threads(1)
+    small = w.scaled(B=1, H=hi)
     host = make_inputs(small)
-    f64 = lambda t: t.to(dtype=__import__("torch").float64).numpy()
+    f64 = lambda t: t.to(dtype=torch.float64).numpy()
     given = "A_hat" in host  # workloads without an estimator stage bring the estimate along
     om, wd = (None, None) if given else (f64(host["omega"]), f64(host["W_dec"]))
     scale = 1.0 / np.sqrt(w.d)
-    best = None
     with threadpool_limits(limits=1):
-        for _ in range(repeats):
-            t0 = time.perf_counter()
-            for h in range(n_heads):
-                orc.sea_attention_head(f64(host["Q"][0, h]), f64(host["K"][0, h]), f64(host["V"][0, h]), w.k_hat,
-                                       w.Kc, w.causal, scale, A_hat=f64(host["A_hat"][0, h]) if given else None,
-                                       omega=om, W_dec=wd)
-            dt = time.perf_counter() - t0
-            best = dt if best is None else min(best, dt)
+        t0 = time.perf_counter()
+        for h in range(lo, hi):
+            orc.sea_attention_head(f64(host["Q"][0, h]), f64(host["K"][0, h]), f64(host["V"][0, h]), w.k_hat,
+                                   w.Kc, w.causal, scale, A_hat=f64(host["A_hat"][0, h]) if given else None,
+                                   omega=om, W_dec=wd)
+        return time.perf_counter() - t0
+
+
+def oracle_tokens_per_s(w, n_heads: int, cores: int):
+    """Oracle throughput on the first n_heads (b, h) units, the heads dealt out to `cores` worker
+    processes (each one runs the unchanged single-threaded oracle).  Returns (tokens/s, seconds,
+    workers used).  Must run before this process initialises CUDA (the workers are forked)."""
+    import multiprocessing as mp
+
+    cores = max(1, min(cores, n_heads))
+    per = (n_heads + cores - 1) // cores
+    jobs = [(w.name, lo, min(lo + per, n_heads)) for lo in range(0, n_heads, per)]
+    if len(jobs) == 1:
+        secs = [_oracle_heads(jobs[0])]
+    else:
+        with mp.get_context("fork").Pool(len(jobs)) as pool:
+            secs = pool.map(_oracle_heads, jobs)
+    wall = max(secs)  # the workers run side by side; input generation is not part of the oracle
     tokens = n_heads * w.T / w.H  # a token passes through all H heads of the layer
-    return tokens / best, best
+    return tokens / wall, wall, len(jobs)
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(w, n_heads: int, max_cores: int):
+    cores = min(host_cores(), max_cores)
+    v, dt, used = oracle_tokens_per_s(w, n_heads, cores)
+    return {"value": v, "unit": "tokens/s", "cores": used, "kind": "oracle",
+            "sample": f"first {n_heads} of {w.B * w.H} heads of {w.name}, fp64 numpy oracle, {dt:.1f} s wall, "
+                      f"{used} worker processes of one thread each"}
 
 
 def run_reference(args, w):
@@ -153,21 +215,23 @@ def run_reference(args, w):
     if rank != 0:
         return
     n_heads = args.ref_heads
+    cores = min(host_cores(), args.cpu_cores, n_heads)
     for _ in range(args.warmup):
-        oracle_tokens_per_s(w, 1)
-    times = []
+        oracle_tokens_per_s(w, 1, 1)
+    times, used = [], 1
     for _ in range(args.steps):
-        _, dt = oracle_tokens_per_s(w, n_heads)
+        _, dt, used = oracle_tokens_per_s(w, n_heads, cores)
         times.append(dt)
     ms = 1e3 * sum(times) / len(times)
     value = (n_heads * w.T / w.H) / (ms / 1e3)
-    sample = f"{n_heads} of {w.B * w.H} heads of {w.name} per step, fp64 numpy oracle, BLAS threads limited to 1"
+    sample = (f"{n_heads} of {w.B * w.H} heads of {w.name} per step, fp64 numpy oracle, {used} worker processes of "
+              "one thread each")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(w),
-        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": used, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -194,6 +258,57 @@ def workload_config(w):
             "outputs": "O, A_hat, sel, row_ptr, col_idx and P all materialised"}
 
 
+def ms_stats(ms):
+    return {"mean": sum(ms) / len(ms), "median": statistics.median(ms), "min": min(ms), "n": len(ms)}
+
+
+def sparse_roofline(w, kernel, exec_flops, nnz, sparse_ms, peaks, clocks):
+    """Roofline block of the sparse-attention stage (see the module docstring)."""
+    hbm_peak, tc_peak, kind = peaks
+    elem = 2 if w.dtype == "bf16" else 4
+    t = sparse_ms / 1e3
+    gather_bytes = 2 * w.rows * w.d * elem + 2 * nnz * w.d * elem  # Q + O + every row's gathered K and V
+    useful_flops = 4 * nnz * w.d
+    # bytes that must cross HBM whatever the kernel: Q, K, V in, O and P out, sel and row_ptr in
+    compulsory = 4 * w.rows * w.d * elem + nnz * elem + w.rows * w.k_hat * 4 + (w.rows + 1) * 4
+    block = {"kernel": kernel, "ms": sparse_ms, "useful_flops": useful_flops,
+             "sparse_stage_tokens_per_s": w.B * w.T / t,
+             "gather_model": {"algorithmic_gather_bytes": gather_bytes, "gbs": gather_bytes / t / 1e9,
+                              "frac_of_gather_model": gather_bytes / t / 1e9 / hbm_peak,
+                              "note": "Q + O + gathered K/V of every row over the HBM copy bandwidth; the tile kernel "
+                                      "gathers nothing, so this is not a fraction of a resource it uses"},
+             "compulsory_hbm_bytes": compulsory, "compulsory_hbm_gbs": compulsory / t / 1e9,
+             "traffic": ncu_traffic(w.name, kernel),
+             "traffic_source": "profiles/ncu_traffic.json (one ncu capture; null when the kernel's source changed since)"}
+    bounds = {"hbm_compulsory": compulsory / (hbm_peak * 1e9) * 1e3}
+    if kernel == "sparse_attn_tiles_tc_kernel" and exec_flops:
+        mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        n_ex2 = exec_flops / (2 * w.d) / 2  # one exponential per entry of every executed score tile
+        bounds["tensor"] = exec_flops / (tc_peak * 1e12) * 1e3
+        bounds["xu_ex2"] = n_ex2 / (XU_PER_CLK_PER_SM * SM_COUNT * mhz * 1e6) * 1e3
+        achieved = exec_flops / t / 1e12
+        block.update({"bound": "tensor", "achieved": achieved, "peak": tc_peak, "unit": "TFLOP/s",
+                      "frac": achieved / tc_peak, "peak_source": f"{kind} dense bf16 (burst)",
+                      "executed_flops": exec_flops, "useful_over_executed": useful_flops / exec_flops})
+    else:
+        achieved = gather_bytes / t / 1e9
+        block.update({"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                      "frac": achieved / hbm_peak, "peak_source": f"{kind} HBM copy bandwidth",
+                      "note": "K and V of a head stay in L2 between the rows that gather them, so the gathered bytes "
+                              "mostly never cross HBM and this figure can exceed 1"})
+    block["bounds_ms"] = bounds
+    block["frac_of_tightest_bound"] = max(bounds.values()) / sparse_ms
+    return block
+
+
+def hbm_roofline(kernels, nbytes, ms, peaks, what):
+    hbm_peak, _, kind = peaks
+    achieved = nbytes / (ms / 1e3) / 1e9
+    return {"kernels": kernels, "bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+            "frac": achieved / hbm_peak, "peak_source": f"{kind} HBM copy bandwidth", "algorithmic_bytes": nbytes,
+            "ms": ms, "bytes": what}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -201,9 +316,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="opt_1p3b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--ref-heads", type=int, default=8, help="heads per step of the reference arm")
+    ap.add_argument("--ref-heads", type=int, default=16, help="heads per step of the reference arm")
     ap.add_argument("--cpu-heads", type=int, default=64, help="heads in the cpu_baseline sample")
+    ap.add_argument("--cpu-cores", type=int, default=32, help="most worker processes the oracle is dealt out to")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-modes", action="store_true", help="skip the grouped / causal-aware / lean regions")
+    ap.add_argument("--soak-s", type=float, default=1.2, help="seconds of steps the clock sampler watches")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -217,14 +335,20 @@ def main():
     if w.m == 0:
         raise SystemExit(f"bench.py times workloads that start at the estimator; {w.name} is a parity-test case")
 
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    # the oracle's worker processes are forked, which has to happen before CUDA is initialised
+    cpu_line = None
+    if rank == 0 and not args.no_cpu_baseline:
+        cpu_line = cpu_baseline(w, min(args.cpu_heads, w.B * w.H), args.cpu_cores)
+
     import torch
     import torch.distributed as dist
 
     import paper_2310_01777_b200 as sea
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: libsea has no CPU fallback")
     torch.cuda.set_device(local_rank)
@@ -250,6 +374,18 @@ def main():
     P = torch.empty((w.nnz_cap,), dtype=io, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
+    def timed(fn, steps):
+        """Per-step milliseconds of `steps` calls of fn, each bracketed by its own event pair on the
+        launching stream, the L2 flushed before each."""
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in ev:
+            flush.zero_()
+            a.record()
+            fn()
+            b.record()
+        torch.cuda.synchronize(dev)
+        return [a.elapsed_time(b) for a, b in ev]
+
     def step():
         sea.sea_attention(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O, ws, A_hat=A_hat, sel=sel,
                           row_ptr=row_ptr, col_idx=col_idx, P=P)
@@ -264,27 +400,38 @@ def main():
 
     sampler = ClockSampler(_gpu_index(local_rank))
     # ---- timed region 1: the fused call ------------------------------------------------
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     barrier()
     torch.cuda.synchronize(dev)
     if rank == 0:
         sampler.start()
-    for a, b in ev:
-        flush.zero_()
-        a.record()
-        step()
-        b.record()
-    torch.cuda.synchronize(dev)
+    step_ms = timed(step, args.steps)
     barrier()
+    # The K steps above are the measurement.  They last milliseconds, less than one nvidia-smi sample,
+    # so the same steps go on untimed until the sampler has seen the GPU under this load for a while.
+    soak_steps = 0
+    if rank == 0:
+        t_end = time.perf_counter() + 8.0
+        t_soak = time.perf_counter() + args.soak_s
+        while (time.perf_counter() < t_soak or len(sampler.rows) < 12) and time.perf_counter() < t_end:
+            for _ in range(50):
+                flush.zero_()
+                step()
+            torch.cuda.synchronize(dev)
+            soak_steps += 50
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    if clocks is not None:
+        clocks["watched"] = f"the {args.steps} timed steps and {soak_steps} more untimed ones of the same call"
+    barrier()
 
-    # ---- timed region 2: stage by stage (for the roofline of the dominant kernel) -------
+    # ---- timed region 2: stage by stage (for the rooflines) ----------------------------
     for _ in range(2):  # the stage entry points launch kernels the fused call does not: load them first
         sea.sea_estimate(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], A_hat, ws)
         sea.sea_topk_mask(shape, A_hat, sel, row_ptr, col_idx, ws)
         sea.sea_sparse_attn(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, sel, O, P, ws)
     torch.cuda.synchronize(dev)
+    sparse_kernel = sea.sea_last_sparse_kernel()
+    sparse_flops = sea.sea_last_sparse_flops()
+    sparse_launches = sea.sea_last_launch_count()
     sev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     for e in sev:
         flush.zero_()
@@ -296,158 +443,133 @@ def main():
         sea.sea_sparse_attn(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, sel, O, P, ws)
         e[3].record()
     torch.cuda.synchronize(dev)
-    stage_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in sev) / args.steps for i in range(3)]
+    stage_all = [[e[i].elapsed_time(e[i + 1]) for e in sev] for i in range(3)]
+    stage_ms = [sum(x) / len(x) for x in stage_all]
     nnz = int(row_ptr[-1])
 
     # ---- timed region 3: end to end from pinned host memory ---------------------------
     hp = {k: v.pin_memory() for k, v in host.items()}
     hO = torch.empty((w.B, w.H, w.T, w.d), dtype=io).pin_memory()
     e2e_steps = max(3, min(args.steps, 20))
+
+    def host_step():
+        sea.sea_attention_host(shape, hp["Q"], hp["K"], hp["V"], hp["omega"], hp["W_dec"], hO, ws)
+
     for _ in range(2):
-        sea.sea_attention_host(shape, hp["Q"], hp["K"], hp["V"], hp["omega"], hp["W_dec"], hO, ws)
-    eev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(e2e_steps)]
+        host_step()
     barrier()
     torch.cuda.synchronize(dev)
-    for a, b in eev:
-        flush.zero_()
-        a.record()
-        sea.sea_attention_host(shape, hp["Q"], hp["K"], hp["V"], hp["omega"], hp["W_dec"], hO, ws)
-        b.record()
-    torch.cuda.synchronize(dev)
+    e2e_all = timed(host_step, e2e_steps)
     barrier()
-    e2e_ms = sum(a.elapsed_time(b) for a, b in eev) / e2e_steps
+    e2e_ms = sum(e2e_all) / e2e_steps
     if not torch.equal(hO, O.cpu()):
         raise SystemExit("host entry point and device entry point disagree")
 
-    # ---- timed region 3b: the fused call with the required outputs only (O and the CSR mask) ------
-    O_lean = torch.empty_like(O)
-    rp_lean = torch.empty_like(row_ptr)
+    lean = grouped = causal_aware = None
+    if not args.no_modes:
+        # ---- timed region 3b: the fused call with the required outputs only (O and the CSR mask) ------
+        O_lean = torch.empty_like(O)
+        rp_lean = torch.empty_like(row_ptr)
 
-    def lean_step():
-        sea.sea_attention(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O_lean, ws, row_ptr=rp_lean,
-                          col_idx=col_idx)
-
-    for _ in range(3):
-        flush.zero_()
-        lean_step()
-    lean_launches = sea.sea_last_launch_count()
-    lev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    torch.cuda.synchronize(dev)
-    for a, b in lev:
-        flush.zero_()
-        a.record()
-        lean_step()
-        b.record()
-    torch.cuda.synchronize(dev)
-    lean_ms = sum(a.elapsed_time(b) for a, b in lev) / args.steps
-    if not (torch.equal(O_lean, O) and torch.equal(rp_lean, row_ptr)):
-        raise SystemExit("the call without the optional outputs gives a different O or row_ptr")
-    lean = {"outputs": "O, row_ptr and col_idx only (no A_hat, sel, P)", "ms_per_step": lean_ms,
-            "value": w.B * w.T / (lean_ms / 1e3), "unit": "tokens/s", "gpu_launches_per_step": lean_launches}
-
-    # ---- timed region 4: the selections that leave as bit masks (fused call, then the stages) ----
-    def time_bits_mode(label, fused_fn, topk_fn):
-        bits = torch.empty((w.rows, (w.Kc + 31) // 32), dtype=torch.int32, device=dev)
-
-        def gstep():
-            fused_fn(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O, ws, A_hat=A_hat, mask_bits=bits,
-                     row_ptr=row_ptr, col_idx=col_idx, P=P)
+        def lean_step():
+            sea.sea_attention(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O_lean, ws, row_ptr=rp_lean,
+                              col_idx=col_idx)
 
         for _ in range(3):
             flush.zero_()
-            gstep()
-        g_launches = sea.sea_last_launch_count()
-        gev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+            lean_step()
+        lean_launches = sea.sea_last_launch_count()
         torch.cuda.synchronize(dev)
-        for a, b in gev:
-            flush.zero_()
-            a.record()
-            gstep()
-            b.record()
-        torch.cuda.synchronize(dev)
-        g_ms = sum(a.elapsed_time(b) for a, b in gev) / args.steps
-        for _ in range(2):
-            topk_fn(shape, A_hat, bits, row_ptr, col_idx, ws)
-            sea.sea_sparse_attn_masked(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, bits, O, P, ws)
-        torch.cuda.synchronize(dev)
-        gsev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-        for e in gsev:
-            flush.zero_()
-            e[0].record()
-            topk_fn(shape, A_hat, bits, row_ptr, col_idx, ws)
-            e[1].record()
-            sea.sea_sparse_attn_masked(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, bits, O, P, ws)
-            e[2].record()
-        torch.cuda.synchronize(dev)
-        if sea.sea_device_status(ws) != 0:
-            raise SystemExit(f"device status word set by the {label} path")
-        return {"selection": label, "ms_per_step": g_ms, "value": w.B * w.T / (g_ms / 1e3), "unit": "tokens/s",
-                "gpu_launches_per_step": g_launches,
-                "stages_ms": {"topk_mask": sum(e[0].elapsed_time(e[1]) for e in gsev) / args.steps,
-                              "sparse_attn_masked": sum(e[1].elapsed_time(e[2]) for e in gsev) / args.steps},
-                "nnz": int(row_ptr[-1])}
+        lean_all = timed(lean_step, args.steps)
+        lean_ms = sum(lean_all) / args.steps
+        if not (torch.equal(O_lean, O) and torch.equal(rp_lean, row_ptr)):
+            raise SystemExit("the call without the optional outputs gives a different O or row_ptr")
+        lean = {"outputs": "O, row_ptr and col_idx only (no A_hat, sel, P)", "ms_per_step": lean_ms,
+                "ms_stats": ms_stats(lean_all), "value": w.B * w.T / (lean_ms / 1e3), "unit": "tokens/s",
+                "gpu_launches_per_step": lean_launches}
 
-    grouped = None
-    if w.Kc % 4 == 0 and w.H * w.Kc <= 32768:
-        grouped = time_bits_mode("causal-per-batch", sea.sea_attention_grouped, sea.sea_topk_mask_grouped)
-    causal_aware = None
-    if w.causal:
-        causal_aware = time_bits_mode("causal-aware per-query", sea.sea_attention_causal_aware,
-                                      sea.sea_topk_mask_causal_aware)
+        # ---- timed region 4: the selections that leave as bit masks (fused call, then the stages) ----
+        def time_bits_mode(label, fused_fn, topk_fn):
+            bits = torch.empty((w.rows, (w.Kc + 31) // 32), dtype=torch.int32, device=dev)
 
-    ms_per_step, e2e_ms = max_over_ranks([total_ms / args.steps, e2e_ms], dev)
+            def gstep():
+                fused_fn(shape, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O, ws, A_hat=A_hat, mask_bits=bits,
+                         row_ptr=row_ptr, col_idx=col_idx, P=P)
+
+            for _ in range(3):
+                flush.zero_()
+                gstep()
+            g_launches = sea.sea_last_launch_count()
+            torch.cuda.synchronize(dev)
+            g_all = timed(gstep, args.steps)
+            g_ms = sum(g_all) / args.steps
+            for _ in range(2):
+                topk_fn(shape, A_hat, bits, row_ptr, col_idx, ws)
+                sea.sea_sparse_attn_masked(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, bits, O, P, ws)
+            torch.cuda.synchronize(dev)
+            gsev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+            for e in gsev:
+                flush.zero_()
+                e[0].record()
+                topk_fn(shape, A_hat, bits, row_ptr, col_idx, ws)
+                e[1].record()
+                sea.sea_sparse_attn_masked(shape, d["Q"], d["K"], d["V"], row_ptr, col_idx, bits, O, P, ws)
+                e[2].record()
+            torch.cuda.synchronize(dev)
+            if sea.sea_device_status(ws) != 0:
+                raise SystemExit(f"device status word set by the {label} path")
+            return {"selection": label, "ms_per_step": g_ms, "ms_stats": ms_stats(g_all),
+                    "value": w.B * w.T / (g_ms / 1e3), "unit": "tokens/s", "gpu_launches_per_step": g_launches,
+                    "stages_ms": {"topk_mask": sum(e[0].elapsed_time(e[1]) for e in gsev) / args.steps,
+                                  "sparse_attn_masked": sum(e[1].elapsed_time(e[2]) for e in gsev) / args.steps},
+                    "nnz": int(row_ptr[-1])}
+
+        if w.Kc % 4 == 0 and w.H * w.Kc <= 32768:
+            grouped = time_bits_mode("causal-per-batch", sea.sea_attention_grouped, sea.sea_topk_mask_grouped)
+        if w.causal:
+            causal_aware = time_bits_mode("causal-aware per-query", sea.sea_attention_causal_aware,
+                                          sea.sea_topk_mask_causal_aware)
+
+    ms_per_step, e2e_ms = max_over_ranks([sum(step_ms) / args.steps, e2e_ms], dev)
     tokens = w.B * w.T * world
     elem = 2 if w.dtype == "bf16" else 4
     h2d = sum(host[k].numel() * host[k].element_size() for k in ("Q", "K", "V", "omega", "W_dec"))
     d2h = O.numel() * O.element_size()
 
     if rank == 0:
-        peak, tc_peak, peak_kind = measured_peaks()
-        alg_bytes = 2 * w.rows * w.d * elem + 2 * nnz * w.d * elem  # Q + O + gathered K and V
-        # what the tile kernel executes: per (query tile, key tile) pair S = Q K^T in both passes and
-        # P V with P as bf16 head + remainder, 2 * 128 * 128 * 64 FLOPs each
-        r = w.T // w.Kc
-        tiled = w.dtype == "bf16" and w.T % 128 == 0 and r >= 4 and r & (r - 1) == 0 and w.k_hat * 40 >= w.Kc
-        nq = w.T // 128
-        pairs = w.B * w.H * (nq * (nq + 1) // 2 if w.causal else nq * nq)
-        exec_flops = pairs * 4 * (2 * 128 * 128 * w.d) if tiled else None
-        sparse_s = stage_ms[2] / 1e3
-        unique_bytes = 4 * w.rows * w.d * elem + nnz * elem + w.rows * w.k_hat * 4 + (w.rows + 1) * 4
-        achieved = alg_bytes / sparse_s / 1e9
+        peaks = measured_peaks()
+        qkv_bytes = 3 * w.rows * w.d * elem
+        a_hat_bytes = w.rows * w.Kc * 4
+        mask_out = w.rows * w.k_hat * 4 + (w.rows + 1) * 4 + nnz * 4
         line = {
             "metric": METRIC, "value": tokens / (ms_per_step / 1e3), "unit": "tokens/s", "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "ms_stats": ms_stats(step_ms),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": workload_config(w),
             "e2e": {"value": tokens / (e2e_ms / 1e3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "ms_stats": ms_stats(e2e_all)},
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
+            "clock_x_time": None if not clocks or not clocks.get("sm_mhz") else
+            {"mhz_ms_per_step": clocks["sm_mhz"] * ms_per_step, "note": "median SM MHz x ms per step"},
             "stages_ms": {"estimate": stage_ms[0], "topk_mask": stage_ms[1], "sparse_attn": stage_ms[2]},
+            "stages_ms_stats": {"estimate": ms_stats(stage_all[0]), "topk_mask": ms_stats(stage_all[1]),
+                                "sparse_attn": ms_stats(stage_all[2])},
             "nnz": nnz,
             "lean": lean,
             "grouped": grouped,
             "causal_aware": causal_aware,
-            "roofline": {"kernel": "sparse_attn_tiles_tc_kernel" if tiled else "sparse_attn_blocks_tma_kernel",
-                         "bound": "hbm", "achieved": achieved, "peak": peak,
-                         "unit": "GB/s", "frac": achieved / peak, "peak_source": f"{peak_kind} HBM copy bandwidth",
-                         "algorithmic_bytes": alg_bytes, "traffic": NCU_TRAFFIC_BYTES.get(w.name) if tiled else None,
-                         "ms": stage_ms[2], "sparse_stage_tokens_per_s": w.B * w.T / sparse_s,
-                         "tensor": None if not tiled else {
-                             "executed_flops": exec_flops, "achieved": exec_flops / sparse_s / 1e12, "peak": tc_peak,
-                             "unit": "TFLOP/s", "frac": exec_flops / sparse_s / 1e12 / tc_peak,
-                             "peak_source": f"{peak_kind} dense bf16 (burst)"},
-                         # K and V of every head fit the L2 together, so the bytes that must cross HBM are
-                         # far fewer than the algorithmic ones: Q, K, V once, O and P once, sel and row_ptr
-                         "compulsory_hbm_bytes": unique_bytes,
-                         "compulsory_hbm_gbs": unique_bytes / sparse_s / 1e9},
+            "roofline": sparse_roofline(w, sparse_kernel, sparse_flops, nnz, stage_ms[2], peaks, clocks),
+            "roofline_estimate": hbm_roofline("favor_prep_tc / favor_state_tc / favor_scan_tc / favor_output_tc",
+                                              qkv_bytes + a_hat_bytes, stage_ms[0], peaks,
+                                              "Q, K, V in, A_hat (fp32) out"),
+            "roofline_mask": hbm_roofline("top-k selection, row_ptr scan, fill_col_idx", a_hat_bytes + mask_out,
+                                          stage_ms[1], peaks, "A_hat in; sel, row_ptr, col_idx out"),
         }
-        if not args.no_cpu_baseline and world == 1:
-            n = min(args.cpu_heads, w.B * w.H)
-            v, dt = oracle_tokens_per_s(w, n)
-            line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": 1, "kind": "oracle",
-                                    "sample": f"first {n} of {w.B * w.H} heads, fp64 numpy oracle, {dt:.1f} s, "
-                                              "BLAS threads limited to 1"}
+        line["roofline"]["launches_in_timed_call"] = sparse_launches
+        if cpu_line is not None:
+            line["cpu_baseline"] = cpu_line
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

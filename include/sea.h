@@ -289,6 +289,10 @@ int32_t sea_last_launch_count(void);
  * ("none" before the first one): the stage chooses among several kernels by shape,
  * dtype and workspace, and a benchmark has to know which one it timed. */
 const char* sea_last_sparse_kernel(void);
+/* Floating-point operations that launch executes when they follow from the shape alone (the
+ * tile kernel visits every key tile a query tile may see, whatever the mask); 0 for the per-row
+ * kernels, whose work is 4 * nnz * d. */
+double sea_last_sparse_flops(void);
 
 const char* sea_status_string(sea_status s);
 

@@ -8,7 +8,7 @@ from .binding import (  # noqa: F401
     SeaError, SeaShape, make_shape, new_workspace, sea_attention, sea_attention_host, sea_attention_grouped, sea_attention_causal_aware, sea_topk_mask_causal_aware,
     sea_attention_capped, sea_topk_mask_capped,
     sea_sparse_attn_masked, sea_topk_mask_grouped,
-    sea_device_status, sea_estimate, sea_last_launch_count, sea_last_sparse_kernel, sea_sparse_attn, sea_topk_mask, sea_topk_mask_static,
+    sea_device_status, sea_estimate, sea_last_launch_count, sea_last_sparse_kernel, sea_last_sparse_flops, sea_sparse_attn, sea_topk_mask, sea_topk_mask_static,
     sea_workspace_bytes, sea_workspace_bytes_capped, sea_workspace_host_bytes,
 )
 from .inputs import WORKLOADS, Workload, make_inputs  # noqa: F401

@@ -34,7 +34,7 @@ EXPORTS = (
     "sea_topk_mask_causal_aware", "sea_attention_causal_aware", "sea_workspace_bytes_capped", "sea_topk_mask_capped",
     "sea_attention_capped",
     "sea_workspace_host_bytes", "sea_attention_host", "sea_device_status", "sea_last_launch_count",
-    "sea_last_sparse_kernel",
+    "sea_last_sparse_kernel", "sea_last_sparse_flops",
     "sea_status_string",
 )
 
@@ -89,11 +89,13 @@ def load_library() -> ctypes.CDLL:
     lib.sea_last_launch_count.restype = i32
     lib.sea_last_sparse_kernel.argtypes = []
     lib.sea_last_sparse_kernel.restype = ctypes.c_char_p
+    lib.sea_last_sparse_flops.argtypes = []
+    lib.sea_last_sparse_flops.restype = ctypes.c_double
     lib.sea_status_string.argtypes = [ctypes.c_int]
     lib.sea_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
         fn = getattr(lib, name)
-        if name not in ("sea_last_launch_count", "sea_last_sparse_kernel", "sea_status_string"):
+        if name not in ("sea_last_launch_count", "sea_last_sparse_kernel", "sea_last_sparse_flops", "sea_status_string"):
             fn.restype = ctypes.c_int
     _lib = lib
     return lib
@@ -279,6 +281,10 @@ def sea_device_status(ws, clear: bool = True) -> int:
 
 def sea_last_launch_count() -> int:
     return load_library().sea_last_launch_count()
+
+
+def sea_last_sparse_flops() -> float:
+    return load_library().sea_last_sparse_flops()
 
 
 def sea_last_sparse_kernel() -> str:

@@ -566,6 +566,8 @@ int32_t sea_last_launch_count(void) { return Launch::count(); }
 
 const char* sea_last_sparse_kernel(void) { return Launch::sparse_kernel(); }
 
+double sea_last_sparse_flops(void) { return Launch::sparse_flops(); }
+
 const char* sea_status_string(sea_status s) {
   switch (s) {
     case SEA_OK: return "ok";

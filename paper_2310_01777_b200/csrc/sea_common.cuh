@@ -22,6 +22,10 @@ struct Launch {  // per-thread launch bookkeeping behind sea_last_launch_count()
     static thread_local const char* k = "none";
     return k;
   }
+  static double& sparse_flops() {
+    static thread_local double f = 0.0;
+    return f;
+  }
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

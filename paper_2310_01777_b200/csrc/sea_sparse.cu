@@ -403,6 +403,7 @@ sea_status launch_sparse_attn_rows(const sea_shape& s, const void* Q, const void
                                    const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel, void* O,
                                    void* P, cudaStream_t st) {
   Launch::sparse_kernel() = s.io == SEA_BF16 ? "sparse_attn_rows_mma_kernel" : "sparse_attn_rows_kernel";
+  Launch::sparse_flops() = 0.0;  // depends on the mask: 4 * nnz * d
   if (s.io == SEA_BF16) {
     using T = __nv_bfloat16;
     const int rows = s.B * s.H * s.T;

@@ -779,6 +779,13 @@ sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* 
     if (rc != SEA_OK) return rc;
   }
   Launch::sparse_kernel() = "sparse_attn_tiles_tc_kernel";
+  {
+    // every (query tile, key tile) pair a query tile may see: S = Q K^T in both passes and P V with P
+    // as a bf16 head plus a bf16 remainder, 2 * 128 * 128 * 64 FLOPs each
+    const double nq = s.T / kTile;
+    const double pairs = (double)s.B * s.H * (s.causal ? nq * (nq + 1) / 2 : nq * nq);
+    Launch::sparse_flops() = pairs * 4.0 * (2.0 * kTile * kTile * kHeadDim);
+  }
   const int L = prm.log2r < 7 ? prm.log2r : 7;
 #define SEA_TC(LL)                                                                   \
   case LL:                                                                           \

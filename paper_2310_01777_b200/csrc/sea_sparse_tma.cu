@@ -325,6 +325,7 @@ sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void*
   CUtensorMap map_k, map_v;
   if (!make_rows_map_bf16(&map_k, K, rows, 16) || !make_rows_map_bf16(&map_v, V, rows, 16)) return SEA_ERR_CUDA;
   Launch::sparse_kernel() = "sparse_attn_blocks_tma_kernel";
+  Launch::sparse_flops() = 0.0;  // depends on the mask: 4 * nnz * d
   if (P) return launch_tma<true>(s, map_k, map_v, (const T*)Q, row_ptr, sel, (T*)O, (T*)P, status, st);
   return launch_tma<false>(s, map_k, map_v, (const T*)Q, row_ptr, sel, (T*)O, nullptr, status, st);
 }
