@@ -12,15 +12,23 @@
 // is every column, so all tiles are visited; at the densities this layer runs at (k_hat / Kc
 // of 1/8 to 1/64) the dense products cost less than gathering every row's K and V rows.
 //
-// Two passes over the key tiles of a work item: the first finds every row's maximum over its
-// kept scores, the second forms exp2((s - max) * scale * log2 e), the row sums and P V.  The
-// unnormalised fp32 probabilities of kept keys are parked in a scratch array and written to P
-// (rounded once, after the division by the row sum) when the item ends.
+// One pass over the key tiles of a work item with an online softmax.  The two threads of a row
+// (one per half of a tile's columns) each keep a reference value m of their own: probabilities are
+// formed as exp2((s - m) * scale * log2 e), summed in fp32, and accumulated by the P V product into
+// an output buffer of the thread's half (two accumulators of 64 columns per item).  m starts as the
+// maximum of the first tile that holds a kept score and is only raised when a later tile's maximum
+// exceeds it by more than 2^8 in the exponent's units; the thread then waits for the P V products
+// issued so far, multiplies its accumulator row and its sum by exp2((m_old - m_new) * ...) and goes
+// on - a rare event, since a reference within 2^8 of the maximum keeps every probability and sum
+// far inside the fp32 range.  When the item ends the halves exchange (m, sum), and the output row is
+// (O_0 w_0 + O_1 w_1) / (l_0 w_0 + l_1 w_1) with w_h = exp2((m_h - max(m_0, m_1)) * ...).
+// The raw scores of kept keys are parked in a scratch array as they are read; the last warpgroup
+// turns them into P = exp2((s - M) * ...) / l, rounded once, when the item ends.
 //
 // Warp roles (warpgroups that re-balance their registers): warp 0 issues the TMA copies (the
 // item's mask bits and Q tile, K and V tiles through rings of 16 KB stages), warp 1 issues the
 // Q K^T MMAs, warp 2 the P V MMAs; the row warpgroups own the query rows (per thread a row and 128 / kSplit of every
-// tile's columns); the last warpgroup turns the parked probabilities into P.  All hand-offs are
+// tile's columns); the last warpgroup turns the parked scores into P.  All hand-offs are
 // mbarriers; every wait is bounded by a clock and a wait that runs out sets SEA_DEV_TIMEOUT,
 // after which all roles drain and leave.
 #include <cuda.h>
@@ -54,7 +62,8 @@ static_assert(kRegsLaunch * kThreads <= 65536, "launch allocation exceeds the re
 constexpr uint32_t kTmemCols = 512;
 constexpr int kNS = 3;                    // S / P buffers of 128 columns: the MMAs run up to two tiles ahead of the rows
 constexpr uint32_t kColS = 0;
-constexpr uint32_t kColO = 128 * kNS;     // two O buffers of 64 columns
+constexpr uint32_t kColO = 128 * kNS;     // the output accumulators of the two column halves, 64 columns each
+constexpr float kLazyBits = 8.f;          // the reference may lag the running maximum by 2^8
 static_assert(kColO + 128 <= kTmemCols, "tensor memory budget");
 
 // Barrier indices inside the shared-memory barrier block.
@@ -66,10 +75,9 @@ enum {
   kBarVFull = kBarKEmpty + kNK,  // [kNV]
   kBarVEmpty = kBarVFull + kNV,  // [kNV]
   kBarSFull = kBarVEmpty + kNV,  // [kNS]  S tile written by the MMA
-  kBarSDone = kBarSFull + kNS,   // [kNS]  S tile read (first pass) / P written (second pass)
-  kBarOFull = kBarSDone + kNS,   // [2]
-  kBarOEmpty = kBarOFull + 2,    // [2]
-  kBarBitsFull = kBarOEmpty + 2,      // [2]  the item's mask bits have landed
+  kBarSDone = kBarSFull + kNS,   // [kNS][kSplit]  a column half of P written over the S tile (and, for an item's first tile, the previous item's output read)
+  kBarOFull = kBarSDone + kNS * kSplit,  // [2]  the item's last P V product has finished (items alternate between the two)
+  kBarBitsFull = kBarOFull + 2,       // [2]  the item's mask bits have landed
   kBarBitsEmpty = kBarBitsFull + 2,   // [2]
   kBarFixFull = kBarBitsEmpty + 2,    // [2]  row normalisers handed to the P writers
   kBarFixEmpty = kBarFixFull + 2,     // [2]
@@ -185,75 +193,72 @@ __device__ __forceinline__ int next_rank(int rank_base, uint32_t tb, int t, int 
   return (((t + 1) >> sh) != (t >> sh)) ? rank_base + (int)tb : rank_base;
 }
 
-// Maximum over the kept scores of one 32-column chunk (chunk cg of the tile; lim = last kept
-// column inside the chunk on the diagonal tile).
-template <int L, bool kDiag>
-__device__ __forceinline__ float chunk_max(const uint32_t (&v)[32], uint32_t tb, int cg, int lim, float mx) {
-  float m[4] = {mx, -INFINITY, -INFINITY, -INFINITY};
-  if constexpr (L >= 5) {
-    const int g = L >= 7 ? 0 : (32 * cg) >> L;
-    if ((tb >> g) & 1u) {
-#pragma unroll
-      for (int e = 0; e < 32; ++e)
-        if (!kDiag || e <= lim) m[e & 3] = fmaxf(m[e & 3], __uint_as_float(v[e]));
-    }
-  } else {
-    constexpr int R = 1 << L;
-    const uint32_t gb = tb >> ((32 * cg) >> L);
-#pragma unroll
-    for (int gi = 0; gi < 32 / R; ++gi) {
-      if ((gb >> gi) & 1u) {
-#pragma unroll
-        for (int e = gi * R; e < gi * R + R; ++e)
-          if (!kDiag || e <= lim) m[e & 3] = fmaxf(m[e & 3], __uint_as_float(v[e]));
-      }
-    }
-  }
-  return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
-// Probabilities of one 32-column chunk: p = 2^(s * cs + bias) with bias = -max * cs for kept
-// columns and -inf otherwise; the row sum grows by them; hi / lo receive the bf16 head
-// (truncated) and the bf16 remainder, two columns per word.  With kWriteP the kept
-// probabilities are parked as fp32: run `rank` of the row starts at rank * r.
-template <int L, bool kDiag, bool kWriteP>
-__device__ __forceinline__ void chunk_probs(const uint32_t (&v)[32], uint32_t tb, int cg, int lim, float cs,
-                                            float neg_mc, float2& la, float2& lb, uint32_t (&hi)[16],
-                                            uint32_t (&lo)[16], float* my_scratch, bool park, int rank_base, int off0) {
+// Exponents of one 32-column chunk, in place: x = s * cs + bias with bias = -(reference, in the
+// exponent's units) for kept columns and -inf otherwise (chunk cg of the tile; lim = last kept
+// column inside the chunk on the diagonal tile).  Returns the maximum of mx and the exponents.
+template <int L, bool kDiag>
+__device__ __forceinline__ float chunk_exponents(uint32_t (&v)[32], uint32_t tb, int cg, int lim, float cs, float neg_ref,
+                                                 float mx) {
   constexpr int R = 1 << (L < 5 ? L : 5);  // columns of this chunk per group
   const float2 cs2 = make_float2(cs, cs);
-  const float2 m1 = make_float2(-1.f, -1.f);
+  float m0 = mx, m1 = -INFINITY;
 #pragma unroll
   for (int gi = 0; gi < 32 / R; ++gi) {
     const int g = L >= 7 ? 0 : ((32 * cg) >> L) + (L < 5 ? gi : 0);
-    const bool live = (tb >> g) & 1u;
-    const float bias = live ? neg_mc : -INFINITY;
-    float4* dst = nullptr;
-    if (kWriteP) {
-      const int off = L >= 7 ? off0 + 32 * cg
-                             : ((rank_base + __popc(tb & ((1u << g) - 1u))) << L) + (32 * cg + gi * R - (g << L));
-      dst = reinterpret_cast<float4*>(my_scratch + off);
-    }
-    float2 prev = make_float2(0.f, 0.f);
+    const float bias = (tb >> g) & 1u ? neg_ref : -INFINITY;
 #pragma unroll
     for (int e2 = gi * R / 2; e2 < (gi + 1) * R / 2; ++e2) {
       const float b0 = (!kDiag || 2 * e2 <= lim) ? bias : -INFINITY;
       const float b1 = (!kDiag || 2 * e2 + 1 <= lim) ? bias : -INFINITY;
       const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * e2]), __uint_as_float(v[2 * e2 + 1])), cs2, make_float2(b0, b1));
-      const float2 pp = make_float2(ex2(x.x), ex2(x.y));
-      if (e2 & 1) lb = __fadd2_rn(lb, pp); else la = __fadd2_rn(la, pp);
-      const uint32_t h0 = __float_as_uint(pp.x) & 0xffff0000u, h1 = __float_as_uint(pp.y) & 0xffff0000u;
-      hi[e2] = __byte_perm(h0, h1, 0x7632);
-      const float2 rem = __ffma2_rn(make_float2(__uint_as_float(h0), __uint_as_float(h1)), m1, pp);  // p - head, exact
-      const __nv_bfloat162 l2 = __floats2bfloat162_rn(rem.x, rem.y);
-      lo[e2] = *reinterpret_cast<const uint32_t*>(&l2);
-      if (kWriteP) {
-        if (e2 & 1) {
-          if (live && park) dst[(e2 - gi * R / 2) >> 1] = make_float4(prev.x, prev.y, pp.x, pp.y);
-        } else {
-          prev = pp;
-        }
-      }
+      v[2 * e2] = __float_as_uint(x.x);
+      v[2 * e2 + 1] = __float_as_uint(x.y);
+      if (e2 & 1) m1 = fmax3(m1, x.x, x.y); else m0 = fmax3(m0, x.x, x.y);
+    }
+  }
+  return fmaxf(m0, m1);
+}
+
+// Probabilities of one 32-column chunk from its exponents: p = 2^(x - adj); the row sum grows by
+// them; hi / lo receive the bf16 head (truncated) and the bf16 remainder, two columns per word.
+__device__ __forceinline__ void chunk_probs(const uint32_t (&v)[32], float adj, float2& la, float2& lb, uint32_t (&hi)[16],
+                                            uint32_t (&lo)[16]) {
+  const float2 m1 = make_float2(-1.f, -1.f);
+#pragma unroll
+  for (int e2 = 0; e2 < 16; ++e2) {
+    const float2 pp = make_float2(ex2(__uint_as_float(v[2 * e2]) - adj), ex2(__uint_as_float(v[2 * e2 + 1]) - adj));
+    if (e2 & 1) lb = __fadd2_rn(lb, pp); else la = __fadd2_rn(la, pp);
+    const uint32_t h0 = __float_as_uint(pp.x) & 0xffff0000u, h1 = __float_as_uint(pp.y) & 0xffff0000u;
+    hi[e2] = __byte_perm(h0, h1, 0x7632);
+    const float2 rem = __ffma2_rn(make_float2(__uint_as_float(h0), __uint_as_float(h1)), m1, pp);  // p - head, exact
+    const __nv_bfloat162 l2 = __floats2bfloat162_rn(rem.x, rem.y);
+    lo[e2] = *reinterpret_cast<const uint32_t*>(&l2);
+  }
+}
+
+// Parks the raw scores of the kept groups of one 32-column chunk: run `rank` of the row starts at
+// rank * r floats inside the row's part of the scratch array (the writers cut a causal row's last
+// run by the row's length, so whole groups are stored).
+template <int L>
+__device__ __forceinline__ void chunk_park(const uint32_t (&v)[32], uint32_t tb, int cg, float* my_scratch, int rank_base,
+                                           int off0) {
+  constexpr int R = 1 << (L < 5 ? L : 5);
+#pragma unroll
+  for (int gi = 0; gi < 32 / R; ++gi) {
+    const int g = L >= 7 ? 0 : ((32 * cg) >> L) + (L < 5 ? gi : 0);
+    if ((tb >> g) & 1u) {
+      const int off = L >= 7 ? off0 + 32 * cg
+                             : ((rank_base + __popc(tb & ((1u << g) - 1u))) << L) + (32 * cg + gi * R - (g << L));
+      uint4* dst = reinterpret_cast<uint4*>(my_scratch + off);
+#pragma unroll
+      for (int e4 = 0; e4 < R / 4; ++e4)
+        dst[e4] = make_uint4(v[gi * R + 4 * e4], v[gi * R + 4 * e4 + 1], v[gi * R + 4 * e4 + 2], v[gi * R + 4 * e4 + 3]);
     }
   }
 }
@@ -266,6 +271,8 @@ __device__ __forceinline__ bool rows_all(bool ok) {
       : "=r"(r) : "r"((uint32_t)ok), "n"(kRowThreads) : "memory");
   return r != 0;
 }
+
+constexpr int kBarBlockBytes = (8 * kNumBars + 8 + 15) / 16 * 16;  // barriers, tensor-memory slot, abort flag
 
 template <int kRegs>
 __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegs)); }
@@ -285,10 +292,12 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
   const uint32_t bars = smem_u32(tail);                      // kNumBars x 8 B
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8 * kNumBars + 4);
-  float* xch = reinterpret_cast<float*>(tail + 8 * kNumBars + 8);       // [kSplit][128] partial maxima
-  float* xch_l = xch + kSplit * kTile;                                   // [kSplit][128] partial sums
-  float* fix_inv = xch_l + kSplit * kTile;                                      // [2 slots][128]
-  int* fix_base = reinterpret_cast<int*>(fix_inv + 2 * kTile);           // [2][128]
+  // the arrays begin on a 16-byte boundary: the mask bits at their end are the target of a bulk copy
+  float* xch_m = reinterpret_cast<float*>(tail + kBarBlockBytes);       // [2 items][kSplit][128] the halves' references
+  float* xch_l = xch_m + 2 * kSplit * kTile;                             // [2 items][kSplit][128] the halves' sums
+  float* fix_inv = xch_l + 2 * kSplit * kTile;                           // [2 slots][128] 1 / row sum
+  float* fix_nmc = fix_inv + 2 * kTile;                                  // [2][128] -(row reference, in the exponent's units)
+  int* fix_base = reinterpret_cast<int*>(fix_nmc + 2 * kTile);           // [2][128]
   int* fix_cnt = fix_base + 2 * kTile;                                   // [2][128]
   int* fix_off = fix_cnt + 2 * kTile;                                    // [2][128]
   uint32_t* bits = reinterpret_cast<uint32_t*>(fix_off + 2 * kTile);     // [2 slots][128 rows][words]
@@ -298,19 +307,15 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
   if (tid == 0) {
     for (int i = 0; i < kNumBars; ++i) {
       uint32_t count = 1;
-      if ((i >= kBarSDone && i < kBarSDone + kNS) || (i >= kBarOEmpty && i < kBarOEmpty + 2) ||
-          (i >= kBarBitsEmpty && i < kBarBitsEmpty + 2))
-        count = kRowWarps;  // one arrival per row warp
+      if (i >= kBarBitsEmpty && i < kBarBitsEmpty + 2) count = kRowWarps;  // one arrival per row warp
+      if (i >= kBarSDone && i < kBarSDone + kNS * kSplit) count = 4;       // one arrival per row warp of the half
       if ((i >= kBarFixFull && i < kBarFixFull + 2) || (i >= kBarFixEmpty && i < kBarFixEmpty + 2)) count = 4;
       mbar_init(bar(i), count);
     }
     *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    mbar_init_fence();
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
-  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
   fence_before();
   __syncthreads();
   fence_after();
@@ -336,81 +341,57 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         mbar_expect_tx(bar(kBarQFull + qb), kTileBytes);
         tma_load_2d(sQ + qb * kTileBytes, &map_q, 0, it.row0, bar(kBarQFull + qb));
         ++q_it;
-        for (int pass = 0; pass < 2 && ok; ++pass) {
-          for (int t = 0; t < it.nt; ++t) {
-            const uint32_t ks = k_it % kNK;
-            ok = mbar_wait<100>(bar(kBarKEmpty + ks), ((k_it / kNK) & 1) ^ 1, abort_flag);
-            if (!ok) break;
-            mbar_expect_tx(bar(kBarKFull + ks), kTileBytes);
-            tma_load_2d(sK + ks * kTileBytes, &map_k, 0, it.bh * p.T + t * kTile, bar(kBarKFull + ks));
-            ++k_it;
-            if (pass == 1) {
-              const uint32_t vs = v_it % kNV;
-              ok = mbar_wait<100>(bar(kBarVEmpty + vs), ((v_it / kNV) & 1) ^ 1, abort_flag);
-              if (!ok) break;
-              mbar_expect_tx(bar(kBarVFull + vs), kTileBytes);
-              tma_load_2d(sV + vs * kTileBytes, &map_v, 0, it.bh * p.T + t * kTile, bar(kBarVFull + vs));
-              ++v_it;
-            }
-          }
+        for (int t = 0; t < it.nt; ++t) {
+          const uint32_t ks = k_it % kNK;
+          ok = mbar_wait<100>(bar(kBarKEmpty + ks), ((k_it / kNK) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(bar(kBarKFull + ks), kTileBytes);
+          tma_load_2d(sK + ks * kTileBytes, &map_k, 0, it.bh * p.T + t * kTile, bar(kBarKFull + ks));
+          ++k_it;
+          const uint32_t vs = v_it % kNV;
+          ok = mbar_wait<100>(bar(kBarVEmpty + vs), ((v_it / kNV) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(bar(kBarVFull + vs), kTileBytes);
+          tma_load_2d(sV + vs * kTileBytes, &map_v, 0, it.bh * p.T + t * kTile, bar(kBarVFull + vs));
+          ++v_it;
         }
       }
       // copies still in flight must land before the CTA may leave: wait for the last use of every stage
-      for (uint32_t i = (k_it > kNK ? k_it - kNK : 0); i < k_it; ++i) mbar_wait(bar(kBarKFull + i % kNK), (i / kNK) & 1, abort_flag);
-      for (uint32_t i = (v_it > kNV ? v_it - kNV : 0); i < v_it; ++i) mbar_wait(bar(kBarVFull + i % kNV), (i / kNV) & 1, abort_flag);
+      for (uint32_t i = (k_it > kNK ? k_it - kNK : 0); i < k_it; ++i) mbar_wait_drain(bar(kBarKFull + i % kNK), (i / kNK) & 1);
+      for (uint32_t i = (v_it > kNV ? v_it - kNV : 0); i < v_it; ++i) mbar_wait_drain(bar(kBarVFull + i % kNV), (i / kNV) & 1);
       for (uint32_t i = (q_it > 2 ? q_it - 2 : 0); i < q_it; ++i) {
-        mbar_wait(bar(kBarQFull + (i & 1)), (i >> 1) & 1, abort_flag);
-        mbar_wait(bar(kBarBitsFull + (i & 1)), (i >> 1) & 1, abort_flag);
+        mbar_wait_drain(bar(kBarQFull + (i & 1)), (i >> 1) & 1);
+        mbar_wait_drain(bar(kBarBitsFull + (i & 1)), (i >> 1) & 1);
       }
     } else if (warp == 1 && lane == 0) {
       // ---------------------------------------------------------------- issuer of S = Q K^T
-      // S/P buffer u % kNS serves use u (the tiles of the first pass, then of the second pass, item
-      // after item).  Before a buffer is written again its previous use must be over: the rows have
-      // read S (first-pass use, barrier SDone) or the P V product has consumed P (second-pass use,
-      // barrier PFree, committed by the other issuer).
-      uint32_t q_it = 0, k_it = 0, s_it = 0;
-      uint32_t b = 0, round = 0;  // use s_it = round * kNS + b occupies buffer b
+      // S/P buffer u % kNS serves use u (tile after tile, item after item).  Before a buffer is
+      // written again the P V product of its previous use must have consumed it (barrier PFree,
+      // committed by the other issuer, one phase per use).
+      uint32_t q_it = 0, k_it = 0;
+      uint32_t b = 0, round = 0;  // use round * kNS + b occupies buffer b
       const uint64_t k_desc0 = smem_desc(sK, 16, 1024);  // a stage further on: + 16 KB / 16
-      uint32_t prev_second = 0;  // bit b: the last use of buffer b belonged to a second pass
-      uint32_t pfree_par = 0;    // bit b: parity of the PFree phase that ends that use
-      uint32_t pfree_cnt = 0;    // bit b: parity of the number of second-pass uses of buffer b so far
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const Item it = decode_item(item, p);
         const uint32_t qb = q_it & 1;
         ok = mbar_wait(bar(kBarQFull + qb), (q_it >> 1) & 1, abort_flag);
         const uint64_t q_desc = smem_desc(sQ + qb * kTileBytes, 16, 1024);
-        for (int pass = 0; pass < 2 && ok; ++pass) {
-          for (int t = 0; t < it.nt && ok; ++t) {
-            const uint32_t u = s_it;
-            const uint32_t ks = k_it % kNK;
-            const uint32_t kbar = bar(kBarKFull + ks), kpar = (k_it / kNK) & 1;
-            if (u >= (uint32_t)kNS) {
-              // the buffer's previous use is over (its round number is one less than this use's)
-              if ((prev_second >> b) & 1u) ok = mbar_wait2(bar(kBarPFree + b), (pfree_par >> b) & 1u, kbar, kpar, abort_flag);
-              else ok = mbar_wait2(bar(kBarSDone + b), (round & 1u) ^ 1u, kbar, kpar, abort_flag);
-            } else {
-              ok = mbar_wait(kbar, kpar, abort_flag);
-            }
-            if (!ok) break;
-            fence_after();
-            issue_qk_mmas(tmem + kColS + 128 * b, q_desc, k_desc0 + 1024ull * ks);
-            mma_commit(bar(kBarKEmpty + ks));
-            mma_commit(bar(kBarSFull + b));
-            if (pass == 1 && t == it.nt - 1) mma_commit(bar(kBarQEmpty + qb));
-            if (pass == 1) {
-              prev_second |= 1u << b;
-              pfree_par = (pfree_par & ~(1u << b)) | (pfree_cnt & (1u << b));
-              pfree_cnt ^= 1u << b;
-            } else {
-              prev_second &= ~(1u << b);
-            }
-            ++s_it;
-            ++k_it;
-            if (++b == (uint32_t)kNS) {
-              b = 0;
-              ++round;
-            }
+        for (int t = 0; t < it.nt && ok; ++t) {
+          const uint32_t ks = k_it % kNK;
+          const uint32_t kbar = bar(kBarKFull + ks), kpar = (k_it / kNK) & 1;
+          if (round > 0) ok = mbar_wait2(bar(kBarPFree + b), (round & 1u) ^ 1u, kbar, kpar, abort_flag);
+          else ok = mbar_wait(kbar, kpar, abort_flag);
+          if (!ok) break;
+          fence_after();
+          issue_qk_mmas(tmem + kColS + 128 * b, q_desc, k_desc0 + 1024ull * ks);
+          mma_commit(bar(kBarKEmpty + ks));
+          mma_commit(bar(kBarSFull + b));
+          if (t == it.nt - 1) mma_commit(bar(kBarQEmpty + qb));
+          ++k_it;
+          if (++b == (uint32_t)kNS) {
+            b = 0;
+            ++round;
           }
         }
         ++q_it;
@@ -419,37 +400,40 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       mma_commit(bar(kBarDrain));
       mbar_wait(bar(kBarDrain), 0, abort_flag);
     } else if (warp == 2 && lane == 0) {
-      // ---------------------------------------------------------------- issuer of O += P V
-      uint32_t v_it = 0, o_it = 0, use0 = 0, s_waited = 0;
+      // ---------------------------------------------------------------- issuer of O_h += P_h V
+      uint32_t v_it = 0, o_it = 0;
+      uint32_t b = 0, round = 0;
       const uint64_t v_desc0 = smem_desc(sV, 8192, 1024);  // a stage further on: + 16 KB / 16
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const Item it = decode_item(item, p);
-        const uint32_t ob = o_it & 1;
-        const uint32_t d = tmem + kColO + 64 * ob;
         for (int t = 0; t < it.nt && ok; ++t) {
-          const uint32_t u = use0 + it.nt + t, b = u % kNS;  // the second pass follows the item's first
-          // the rows have written P.  A parity wait only tells the current phase from the one before
-          // it, so this thread follows SDone through every use, the first-pass ones included.
-          while (ok && s_waited < u) {
-            ok = mbar_wait(bar(kBarSDone + s_waited % kNS), (s_waited / kNS) & 1, abort_flag);
-            ++s_waited;
-          }
-          if (ok && t == 0) ok = mbar_wait(bar(kBarOEmpty + ob), ((o_it >> 1) & 1) ^ 1, abort_flag);
+          // the rows have written P (and, before an item's first tile, read the previous item's output)
+          // Each column half has its own accumulator and its own barrier, so a half's product starts as
+          // soon as its rows are done.  Every row thread reads both accumulators when an item ends: the
+          // first product of an item waits for both halves.
           const uint32_t vs = v_it % kNV;
-          if (ok) ok = mbar_wait2(bar(kBarSDone + b), (u / kNS) & 1, bar(kBarVFull + vs), (v_it / kNV) & 1, abort_flag);
-          ++s_waited;
+          ok = mbar_wait2(bar(kBarSDone + kSplit * b), round & 1u, bar(kBarVFull + vs), (v_it / kNV) & 1, abort_flag);
+          if (ok && t == 0) ok = mbar_wait(bar(kBarSDone + kSplit * b + 1), round & 1u, abort_flag);
           if (!ok) break;
           fence_after();
           const uint64_t vd = v_desc0 + 1024ull * vs;
-          issue_pv_half(d, tmem + kColS + 128 * b, vd, 0, t == 0 ? 0u : 1u);
-          issue_pv_half(d, tmem + kColS + 128 * b, vd, 1, 1u);
+          issue_pv_half(tmem + kColO, tmem + kColS + 128 * b, vd, 0, t == 0 ? 0u : 1u);
+          if (t != 0) {
+            ok = mbar_wait(bar(kBarSDone + kSplit * b + 1), round & 1u, abort_flag);
+            if (!ok) break;
+            fence_after();
+          }
+          issue_pv_half(tmem + kColO + 64, tmem + kColS + 128 * b, vd, 1, t == 0 ? 0u : 1u);
           mma_commit(bar(kBarVEmpty + vs));
           mma_commit(bar(kBarPFree + b));
-          if (t == it.nt - 1) mma_commit(bar(kBarOFull + ob));
+          if (t == it.nt - 1) mma_commit(bar(kBarOFull + (o_it & 1)));
           ++v_it;
+          if (++b == (uint32_t)kNS) {
+            b = 0;
+            ++round;
+          }
         }
-        use0 += 2 * it.nt;
         ++o_it;
       }
       mma_commit(bar(kBarDrain2));
@@ -463,42 +447,43 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     const int part = (warp - 4) >> 2;      // columns (128 / kSplit) * part .. of every tile
     const int rt = quarter * 32 + lane;    // row inside the work item
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t my_o = lane_addr + kColO + 64 * part;  // this half's accumulator row
     const int log2r = p.log2r;
     const int KR = p.k_hat << log2r;
     const float cs = p.scale_log2;
-    uint32_t s_it = 0, it_cnt = 0;
+    uint32_t b = 0, round = 0, it_cnt = 0;  // use round * kNS + b of the S / P buffers
     bool ok = true;
     struct {
       bool active;
-      float inv;
+      float w0, w1, inv, nmc;  // weights of the two halves' accumulators (normaliser included), 1 / sum, -(row reference)
       int row, p_base, p_cnt, p_off;
       uint32_t it_cnt;
-    } pend = {false, 0.f, 0, 0, 0, 0, 0u};
-    // Output row of the pending item (this thread: 64 / kSplit of its columns), and the hand-over
-    // of the rows' normalisers to the warps that write P.
+    } pend = {false, 0.f, 0.f, 0.f, 0.f, 0, 0, 0, 0, 0u};
+    // Output row of the pending item (this thread: 32 of its columns, from both halves'
+    // accumulators), and the hand-over of the rows' normalisers to the warps that write P.
     auto epilogue = [&]() -> bool {
       if (!pend.active) return true;
       pend.active = false;
-      const uint32_t ob = pend.it_cnt & 1, pslot = pend.it_cnt & 1;
-      bool good = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull + ob), (pend.it_cnt >> 1) & 1, abort_flag));
+      const uint32_t pslot = pend.it_cnt & 1;
+      bool good = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull + pslot), (pend.it_cnt >> 1) & 1, abort_flag));
       if (!good) return false;
       fence_after();
       constexpr int kOC = 64 / kSplit;
       static_assert(kOC == 32, "the output row is read 32 columns at a time");
-      uint32_t o[kOC];
-      tmem_ld32(lane_addr + kColO + 64 * ob + kOC * part, o);
+      uint32_t o0[kOC], o1[kOC];
+      tmem_ld32(lane_addr + kColO + kOC * part, o0);
+      tmem_ld32(lane_addr + kColO + 64 + kOC * part, o1);
       tmem_ld_wait();
       fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(kBarOEmpty + ob));
       uint4* out = reinterpret_cast<uint4*>(p.O + (size_t)pend.row * kHeadDim + kOC * part);
 #pragma unroll
       for (int e = 0; e < kOC / 8; ++e) {
         uint32_t w[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(o[8 * e + 2 * k]) * pend.inv,
-                                                         __uint_as_float(o[8 * e + 2 * k + 1]) * pend.inv);
+          const float x = __uint_as_float(o0[8 * e + 2 * k]) * pend.w0 + __uint_as_float(o1[8 * e + 2 * k]) * pend.w1;
+          const float y = __uint_as_float(o0[8 * e + 2 * k + 1]) * pend.w0 + __uint_as_float(o1[8 * e + 2 * k + 1]) * pend.w1;
+          const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
           w[k] = *reinterpret_cast<const uint32_t*>(&h);
         }
         out[e] = make_uint4(w[0], w[1], w[2], w[3]);
@@ -507,6 +492,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         good = __all_sync(0xffffffffu, mbar_wait(bar(kBarFixEmpty + pslot), ((pend.it_cnt >> 1) & 1) ^ 1, abort_flag));
         if (!good) return false;
         fix_inv[pslot * kTile + rt] = pend.inv;
+        fix_nmc[pslot * kTile + rt] = pend.nmc;
         fix_base[pslot * kTile + rt] = pend.p_base;
         fix_cnt[pslot * kTile + rt] = pend.p_cnt;
         fix_off[pslot * kTile + rt] = pend.p_off;
@@ -534,47 +520,12 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       }
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarBitsFull + slot), (it_cnt >> 1) & 1, abort_flag));
       const uint32_t* my_bits = bits + slot * (kTile * p.words) + rt * p.words;
-      // ---- first pass: the row's maximum over its kept scores
-      float mx = -INFINITY;
-      for (int t = 0; t < it.nt && ok; ++t) {
-        const uint32_t b = s_it % kNS;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + b), (s_it / kNS) & 1, abort_flag));
-        if (!ok) break;
-        fence_after();
-        int off0;
-        const uint32_t tb = tile_bits<L>(my_bits, t, log2r, 0, off0);
-        const uint32_t src = lane_addr + kColS + 128 * b + 32 * kChunks * part;
-        uint32_t v[kChunks][32];
-#pragma unroll
-        for (int c = 0; c < kChunks; ++c) tmem_ld32(src + 32 * c, v[c]);
-        tmem_ld_wait();
-        const bool diag = p.causal && t == it.qt;
-#pragma unroll
-        for (int c = 0; c < kChunks; ++c) {
-          const int cg = kChunks * part + c;
-          if (diag) mx = chunk_max<L, true>(v[c], tb, cg, rt - 32 * cg, mx);
-          else mx = chunk_max<L, false>(v[c], tb, cg, 0, mx);
-        }
-        fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(kBarSDone + b));
-        ++s_it;
-      }
-      if (ok) ok = epilogue();  // the previous item's output row
-      xch[part * kTile + rt] = mx;
-      ok = rows_all(ok);
-      if (!ok) break;
-#pragma unroll
-      for (int q = 0; q < kSplit; ++q) mx = fmaxf(mx, xch[q * kTile + rt]);
-      if (mx == -INFINITY) mx = 0.f;  // a row that keeps no key: every probability is zero below
-      const float neg_mc = -mx * cs;
       float* my_scratch = kWriteP ? p.p_scratch + p_off : nullptr;
-      // ---- second pass: probabilities, row sum, P into tensor memory
+      float mb = -INFINITY;  // this half's reference in the exponent's units (score * cs); -inf while it has met no kept score
       float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
       int rank_base = 0;
       for (int t = 0; t < it.nt && ok; ++t) {
-        const uint32_t b = s_it % kNS;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + b), (s_it / kNS) & 1, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + b), round & 1u, abort_flag));
         if (!ok) break;
         fence_after();
         int off0;
@@ -585,40 +536,101 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         for (int c = 0; c < kChunks; ++c) tmem_ld32(src + 32 * c, v[c]);
         tmem_ld_wait();
         const bool diag = p.causal && t == it.qt;
+        // exponents under the current reference (0 while there is none), and their maximum
+        const float neg_ref = mb == -INFINITY ? 0.f : -mb;
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          const int cg = kChunks * part + c;
+          if (kWriteP && park) chunk_park<L>(v[c], tb, cg, my_scratch, rank_base, off0);
+          if (diag) mx = chunk_exponents<L, true>(v[c], tb, cg, rt - 32 * cg, cs, neg_ref, mx);
+          else mx = chunk_exponents<L, false>(v[c], tb, cg, 0, cs, neg_ref, mx);
+        }
+        // The reference moves to the tile's maximum when that lies more than kLazyBits above it, or
+        // when this is the row half's first kept score; the exponents then shift by adj.
+        const bool raise = mb == -INFINITY ? mx > -INFINITY : mx > kLazyBits;
+        float adj = 0.f;
+        if (__any_sync(0xffffffffu, raise)) {
+          // What the row has accumulated under the old reference is multiplied by 2^-adj; with no
+          // kept score so far the sum and the accumulator row are exactly zero and stay so.
+          const bool rescale = raise && mb != -INFINITY;
+          if (raise) {
+            adj = mx;
+            mb = rescale ? mb + mx : mx;
+          }
+          const float f = rescale ? ex2(-adj) : 1.f;
+          la.x *= f; la.y *= f; lb.x *= f; lb.y *= f;
+          if (__any_sync(0xffffffffu, rescale)) {
+            // rare: the P V products issued so far (the last one belongs to the previous use) must have finished
+            const uint32_t pb = b == 0 ? kNS - 1 : b - 1, pround = b == 0 ? round - 1 : round;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarPFree + pb), pround & 1u, abort_flag));
+            if (!ok) break;
+            fence_after();
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              uint32_t o[16];
+              tmem_ld16(my_o + 16 * c, o);
+              tmem_ld_wait();
+#pragma unroll
+              for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
+              tmem_st16(my_o + 16 * c, o);
+            }
+          }
+        }
 #pragma unroll
         for (int c = 0; c < kChunks; ++c) {
           uint32_t hi[16], lo[16];
-          const int cg = kChunks * part + c;
-          if (diag) chunk_probs<L, true, kWriteP>(v[c], tb, cg, rt - 32 * cg, cs, neg_mc, la, lb, hi, lo, my_scratch, park, rank_base, off0);
-          else chunk_probs<L, false, kWriteP>(v[c], tb, cg, 0, cs, neg_mc, la, lb, hi, lo, my_scratch, park, rank_base, off0);
+          chunk_probs(v[c], adj, la, lb, hi, lo);
           tmem_st16(src + 32 * c, hi);
           tmem_st16(src + 32 * c + 16, lo);
         }
         rank_base = next_rank<L>(rank_base, tb, t, log2r);
+        // the previous item's output row leaves the accumulators before this item's first product
+        // may overwrite them: by now that item's last product has long finished
+        if (t == 0 && !epilogue()) {
+          ok = false;
+          break;
+        }
         tmem_st_wait();
         fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar(kBarSDone + b));
-        ++s_it;
+        if (lane == 0) mbar_arrive(bar(kBarSDone + kSplit * b + part));
+        if (++b == (uint32_t)kNS) {
+          b = 0;
+          ++round;
+        }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kBarBitsEmpty + slot));
-      xch_l[part * kTile + rt] = (la.x + la.y) + (lb.x + lb.y);
+      // The halves exchange their references and sums.  Items alternate between two exchange areas:
+      // a thread can only write an area again after the barrier of the item in between, which every
+      // thread reaches after it has read what it needs here.
+      float* xm = xch_m + slot * (kSplit * kTile);
+      float* xl = xch_l + slot * (kSplit * kTile);
+      xm[part * kTile + rt] = mb;
+      xl[part * kTile + rt] = (la.x + la.y) + (lb.x + lb.y);
       ok = rows_all(ok);
       if (!ok) break;
-      float l = 0.f;
-#pragma unroll
-      for (int q = 0; q < kSplit; ++q) l += xch_l[q * kTile + rt];
-      const float inv = l > 0.f ? 1.f / l : 0.f;
-      // the item's output row is written while the next item's first pass runs (by then the last
-      // P V product has long finished); remember what that needs
-      pend.active = true;
-      pend.inv = inv;
-      pend.row = row;
-      pend.it_cnt = it_cnt;
-      pend.p_base = p_base;
-      pend.p_cnt = p_cnt;
-      pend.p_off = p_off;
+      {
+        const float m0 = xm[rt], m1 = xm[kTile + rt];
+        const float M = fmaxf(m0, m1);
+        const float w0 = m0 == -INFINITY ? 0.f : ex2(m0 - M);  // a half without kept scores has weight 0
+        const float w1 = m1 == -INFINITY ? 0.f : ex2(m1 - M);
+        const float l = xl[rt] * w0 + xl[kTile + rt] * w1;
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        // the item's output row is written while the next item's first tile is worked on; remember
+        // what that needs
+        pend.active = true;
+        pend.w0 = w0 * inv;
+        pend.w1 = w1 * inv;
+        pend.inv = inv;
+        pend.nmc = M == -INFINITY ? 0.f : -M;
+        pend.row = row;
+        pend.it_cnt = it_cnt;
+        pend.p_base = p_base;
+        pend.p_cnt = p_cnt;
+        pend.p_off = p_off;
+      }
     }
     if (ok) ok = epilogue();
   } else {
@@ -626,17 +638,19 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
     reg_dec<kRegsFix>();
     if (kWriteP) {
       const int w4 = warp - (4 + kRowWarps);
+      const float cs = p.scale_log2;
       uint32_t it_cnt = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it_cnt) {
         const uint32_t slot = it_cnt & 1;
         ok = __all_sync(0xffffffffu, mbar_wait<500>(bar(kBarFixFull + slot), (it_cnt >> 1) & 1, abort_flag));
         if (!ok) break;
-        // P = parked probability / row sum, rounded once.  Rows are taken eight at a time, in
+        // P = 2^((parked score - M) cs) / row sum, rounded once.  Rows are taken eight at a time, in
         // slices of 128 keys (one 16-byte load per lane and row), so that eight loads are in flight.
         const int* cnt_s = fix_cnt + slot * kTile + 32 * w4;
         const int* base_s = fix_base + slot * kTile + 32 * w4;
         const float* inv_s = fix_inv + slot * kTile + 32 * w4;
+        const float* nmc_s = fix_nmc + slot * kTile + 32 * w4;
         const int* off_s = fix_off + slot * kTile + 32 * w4;
         const int longest_all = __reduce_max_sync(0xffffffffu, cnt_s[lane]);
         for (int u0 = 0; u0 < longest_all; u0 += 128) {
@@ -654,9 +668,10 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               const int n = cnt_s[r0 + j];
-              const float inv = inv_s[r0 + j];
+              const float inv = inv_s[r0 + j], nmc = nmc_s[r0 + j];
               __nv_bfloat16* dst = p.P + (size_t)base_s[r0 + j] + u;
-              const float f[4] = {val[j].x * inv, val[j].y * inv, val[j].z * inv, val[j].w * inv};
+              const float f[4] = {ex2(fmaf(val[j].x, cs, nmc)) * inv, ex2(fmaf(val[j].y, cs, nmc)) * inv,
+                                  ex2(fmaf(val[j].z, cs, nmc)) * inv, ex2(fmaf(val[j].w, cs, nmc)) * inv};
 #pragma unroll
               for (int e = 0; e < 4; ++e)
                 if (u + e < n) dst[e] = __float2bfloat16_rn(f[e]);
@@ -674,7 +689,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
   if (warp == 1) {
     __syncwarp();
     fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    tmem_dealloc(tmem, kTmemCols);
   }
   if (tid == 0 && *abort_flag) atomicOr(p.status, SEA_DEV_TIMEOUT);
 }
@@ -712,7 +727,7 @@ int log2_exact(int x) {
 template <int L, bool kWriteP>
 sea_status launch_tc(const sea_shape& s, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                      const TcParams& prm, cudaStream_t st) {
-  const size_t smem = 1024 + (size_t)(2 + kNK + kNV) * kTileBytes + 8 * kNumBars + 8 + (size_t)(2 * kSplit + 8) * kTile * 4 +
+  const size_t smem = 1024 + (size_t)(2 + kNK + kNV) * kTileBytes + kBarBlockBytes + (size_t)(4 * kSplit + 10) * kTile * 4 +
                       2 * (size_t)prm.words * kTile * 4;
   auto kern = sparse_attn_tiles_tc_kernel<L, kWriteP>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SEA_ERR_CUDA;
@@ -780,11 +795,11 @@ sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* 
   }
   Launch::sparse_kernel() = "sparse_attn_tiles_tc_kernel";
   {
-    // every (query tile, key tile) pair a query tile may see: S = Q K^T in both passes and P V with P
-    // as a bf16 head plus a bf16 remainder, 2 * 128 * 128 * 64 FLOPs each
+    // every (query tile, key tile) pair a query tile may see: S = Q K^T and P V with P as a bf16
+    // head plus a bf16 remainder, 2 * 128 * 128 * 64 FLOPs each
     const double nq = s.T / kTile;
     const double pairs = (double)s.B * s.H * (s.causal ? nq * (nq + 1) / 2 : nq * nq);
-    Launch::sparse_flops() = pairs * 4.0 * (2.0 * kTile * kTile * kHeadDim);
+    Launch::sparse_flops() = pairs * 3.0 * (2.0 * kTile * kTile * kHeadDim);
   }
   const int L = prm.log2r < 7 ? prm.log2r : 7;
 #define SEA_TC(LL)                                                                   \

@@ -77,6 +77,37 @@ def test_tile_kernel_and_row_kernels_both_match_oracle(w):
         global_mask_properties(run)
 
 
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("profile", ["rising", "sawtooth", "late_spike"])
+def test_tile_kernel_moves_its_softmax_reference(causal, profile):
+    """The tile kernel keeps a softmax reference per row that it only raises when a later key tile
+    exceeds it by a wide margin, rescaling what it has accumulated.  Inputs whose scores grow along
+    the keys (by far more than that margin per tile), go up and down, or jump at the end make it
+    do so; O and P still have to match the oracle, which knows no such thing."""
+    w = small(f"rescale_{profile}", dtype="bf16", T=1024, Kc=64, k_hat=40, causal=causal, H=2, m=0)
+    host = make_inputs(w)
+    g = torch.Generator().manual_seed(5)
+    j = torch.arange(w.T, dtype=torch.float32)
+    if profile == "rising":
+        gain = 60.0 * j / w.T                     # q.k / 8 grows by 7.5 nats = 11 bits per 128 keys
+    elif profile == "sawtooth":
+        gain = 10.0 * ((j // 128) % 3) + 0.01 * j  # up and down between tiles, 14 bits a step
+    else:
+        gain = torch.where(j >= w.T - 40, torch.tensor(40.0), 0.002 * j)  # one jump of 58 bits near the end
+    u = torch.ones(w.d)
+    host["Q"][:] = (u + 0.25 * torch.randn(host["Q"].shape, generator=g)).to(torch.bfloat16)
+    host["K"][:] = (gain[None, None, :, None] / 8.0 * u + 0.1 * torch.randn(host["K"].shape, generator=g)).to(torch.bfloat16)
+    run = GpuRun(w, inputs=host)
+    run.topk_mask(); run.sync()
+    for lean in (False, True):
+        run.O.fill_(float("nan")); run.P.fill_(float("nan"))
+        run.sparse_attn(lean_ws=lean)
+        run.sync()
+        assert run.status() == 0
+        for h in range(w.H):
+            check_head_against_oracle(run, 0, h, check_estimate=False)
+
+
 EST_CASES = [
     small("est_m16", dtype="bf16", causal=True, T=256, Kc=32, m=16),
     small("est_m48", dtype="bf16", T=384, Kc=32, m=48),                              # features padded to 64
