@@ -27,7 +27,8 @@
 //
 // Warp roles (warpgroups that re-balance their registers): warp 0 issues the TMA copies (the
 // item's mask bits and Q tile, K and V tiles through rings of 16 KB stages), warp 1 issues the
-// Q K^T MMAs, warp 2 the P V MMAs; the row warpgroups own the query rows (per thread a row and 128 / kSplit of every
+// Q K^T MMAs, warp 2 the P V MMAs (whole warps, so that what feeds the MMAs stays in uniform
+// registers; one elected lane issues); the row warpgroups own the query rows (per thread a row and 128 / kSplit of every
 // tile's columns); the last warpgroup turns the parked scores into P.  All hand-offs are
 // mbarriers; every wait is bounded by a clock and a wait that runs out sets SEA_DEV_TIMEOUT,
 // after which all roles drain and leave.
@@ -154,6 +155,16 @@ struct TcParams {
   float scale_log2;
 };
 
+// The k-th work item of this CTA, or -1 when it has no more.  Items are numbered in order of
+// descending cost and dealt out to the CTAs stripe by stripe, back and forth (the CTA that got a
+// stripe's most expensive item gets the next stripe's cheapest), which evens out the CTAs' totals
+// without any exchange between them.
+__device__ __forceinline__ int cta_item(int k, int n_items) {
+  const int g = (int)gridDim.x, c = (int)blockIdx.x;
+  const int item = k * g + ((k & 1) ? g - 1 - c : c);
+  return item < n_items ? item : -1;
+}
+
 struct Item {
   int bh, qt, nt, row0;
 };
@@ -199,12 +210,13 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return d;
 }
 
-// Exponents of one 32-column chunk, in place: x = s * cs + bias with bias = -(reference, in the
+// Exponents of one 32-column chunk (kept apart from the scores, which the parking stores still
+// read): x = s * cs + bias with bias = -(reference, in the
 // exponent's units) for kept columns and -inf otherwise (chunk cg of the tile; lim = last kept
 // column inside the chunk on the diagonal tile).  Returns the maximum of mx and the exponents.
 template <int L, bool kDiag>
-__device__ __forceinline__ float chunk_exponents(uint32_t (&v)[32], uint32_t tb, int cg, int lim, float cs, float neg_ref,
-                                                 float mx) {
+__device__ __forceinline__ float chunk_exponents(const uint32_t (&v)[32], uint32_t (&x)[32], uint32_t tb, int cg, int lim,
+                                                 float cs, float neg_ref, float mx) {
   constexpr int R = 1 << (L < 5 ? L : 5);  // columns of this chunk per group
   const float2 cs2 = make_float2(cs, cs);
   float m0 = mx, m1 = -INFINITY;
@@ -216,10 +228,10 @@ __device__ __forceinline__ float chunk_exponents(uint32_t (&v)[32], uint32_t tb,
     for (int e2 = gi * R / 2; e2 < (gi + 1) * R / 2; ++e2) {
       const float b0 = (!kDiag || 2 * e2 <= lim) ? bias : -INFINITY;
       const float b1 = (!kDiag || 2 * e2 + 1 <= lim) ? bias : -INFINITY;
-      const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * e2]), __uint_as_float(v[2 * e2 + 1])), cs2, make_float2(b0, b1));
-      v[2 * e2] = __float_as_uint(x.x);
-      v[2 * e2 + 1] = __float_as_uint(x.y);
-      if (e2 & 1) m1 = fmax3(m1, x.x, x.y); else m0 = fmax3(m0, x.x, x.y);
+      const float2 xx = __ffma2_rn(make_float2(__uint_as_float(v[2 * e2]), __uint_as_float(v[2 * e2 + 1])), cs2, make_float2(b0, b1));
+      x[2 * e2] = __float_as_uint(xx.x);
+      x[2 * e2 + 1] = __float_as_uint(xx.y);
+      if (e2 & 1) m1 = fmax3(m1, xx.x, xx.y); else m0 = fmax3(m0, xx.x, xx.y);
     }
   }
   return fmaxf(m0, m1);
@@ -329,7 +341,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       // ---------------------------------------------------------------- TMA producer
       uint32_t q_it = 0, k_it = 0, v_it = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      for (int k = 0, item; (item = cta_item(k, n_items)) >= 0 && ok; ++k) {
         const Item it = decode_item(item, p);
         const uint32_t qb = q_it & 1;
         ok = mbar_wait<100>(bar(kBarBitsEmpty + qb), ((q_it >> 1) & 1) ^ 1, abort_flag);
@@ -363,7 +375,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         mbar_wait_drain(bar(kBarQFull + (i & 1)), (i >> 1) & 1);
         mbar_wait_drain(bar(kBarBitsFull + (i & 1)), (i >> 1) & 1);
       }
-    } else if (warp == 1 && lane == 0) {
+    } else if (warp == 1) {
       // ---------------------------------------------------------------- issuer of S = Q K^T
       // S/P buffer u % kNS serves use u (tile after tile, item after item).  Before a buffer is
       // written again the P V product of its previous use must have consumed it (barrier PFree,
@@ -372,22 +384,25 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       uint32_t b = 0, round = 0;  // use round * kNS + b occupies buffer b
       const uint64_t k_desc0 = smem_desc(sK, 16, 1024);  // a stage further on: + 16 KB / 16
       bool ok = true;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      for (int k = 0, item; (item = cta_item(k, n_items)) >= 0 && ok; ++k) {
         const Item it = decode_item(item, p);
         const uint32_t qb = q_it & 1;
-        ok = mbar_wait(bar(kBarQFull + qb), (q_it >> 1) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarQFull + qb), (q_it >> 1) & 1, abort_flag));
         const uint64_t q_desc = smem_desc(sQ + qb * kTileBytes, 16, 1024);
         for (int t = 0; t < it.nt && ok; ++t) {
           const uint32_t ks = k_it % kNK;
           const uint32_t kbar = bar(kBarKFull + ks), kpar = (k_it / kNK) & 1;
-          if (round > 0) ok = mbar_wait2(bar(kBarPFree + b), (round & 1u) ^ 1u, kbar, kpar, abort_flag);
-          else ok = mbar_wait(kbar, kpar, abort_flag);
+          if (round > 0) ok = __all_sync(0xffffffffu, mbar_wait2(bar(kBarPFree + b), (round & 1u) ^ 1u, kbar, kpar, abort_flag));
+          else ok = __all_sync(0xffffffffu, mbar_wait(kbar, kpar, abort_flag));
           if (!ok) break;
           fence_after();
-          issue_qk_mmas(tmem + kColS + 128 * b, q_desc, k_desc0 + 1024ull * ks);
-          mma_commit(bar(kBarKEmpty + ks));
-          mma_commit(bar(kBarSFull + b));
-          if (t == it.nt - 1) mma_commit(bar(kBarQEmpty + qb));
+          if (elect_one()) {
+            issue_qk_mmas(tmem + kColS + 128 * b, q_desc, k_desc0 + 1024ull * ks);
+            mma_commit(bar(kBarKEmpty + ks));
+            mma_commit(bar(kBarSFull + b));
+            if (t == it.nt - 1) mma_commit(bar(kBarQEmpty + qb));
+          }
+          __syncwarp();
           ++k_it;
           if (++b == (uint32_t)kNS) {
             b = 0;
@@ -397,15 +412,17 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         ++q_it;
       }
       // every MMA issued by this thread must have finished before tensor memory is released
-      mma_commit(bar(kBarDrain));
+      if (elect_one()) mma_commit(bar(kBarDrain));
+      __syncwarp();
       mbar_wait(bar(kBarDrain), 0, abort_flag);
-    } else if (warp == 2 && lane == 0) {
+      __syncwarp();
+    } else if (warp == 2) {
       // ---------------------------------------------------------------- issuer of O_h += P_h V
       uint32_t v_it = 0, o_it = 0;
       uint32_t b = 0, round = 0;
       const uint64_t v_desc0 = smem_desc(sV, 8192, 1024);  // a stage further on: + 16 KB / 16
       bool ok = true;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      for (int k = 0, item; (item = cta_item(k, n_items)) >= 0 && ok; ++k) {
         const Item it = decode_item(item, p);
         for (int t = 0; t < it.nt && ok; ++t) {
           // the rows have written P (and, before an item's first tile, read the previous item's output)
@@ -413,21 +430,25 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
           // soon as its rows are done.  Every row thread reads both accumulators when an item ends: the
           // first product of an item waits for both halves.
           const uint32_t vs = v_it % kNV;
-          ok = mbar_wait2(bar(kBarSDone + kSplit * b), round & 1u, bar(kBarVFull + vs), (v_it / kNV) & 1, abort_flag);
-          if (ok && t == 0) ok = mbar_wait(bar(kBarSDone + kSplit * b + 1), round & 1u, abort_flag);
+          ok = __all_sync(0xffffffffu, mbar_wait2(bar(kBarSDone + kSplit * b), round & 1u, bar(kBarVFull + vs), (v_it / kNV) & 1, abort_flag));
+          if (ok && t == 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSDone + kSplit * b + 1), round & 1u, abort_flag));
           if (!ok) break;
           fence_after();
           const uint64_t vd = v_desc0 + 1024ull * vs;
-          issue_pv_half(tmem + kColO, tmem + kColS + 128 * b, vd, 0, t == 0 ? 0u : 1u);
+          if (elect_one()) issue_pv_half(tmem + kColO, tmem + kColS + 128 * b, vd, 0, t == 0 ? 0u : 1u);
+          __syncwarp();
           if (t != 0) {
-            ok = mbar_wait(bar(kBarSDone + kSplit * b + 1), round & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSDone + kSplit * b + 1), round & 1u, abort_flag));
             if (!ok) break;
             fence_after();
           }
-          issue_pv_half(tmem + kColO + 64, tmem + kColS + 128 * b, vd, 1, t == 0 ? 0u : 1u);
-          mma_commit(bar(kBarVEmpty + vs));
-          mma_commit(bar(kBarPFree + b));
-          if (t == it.nt - 1) mma_commit(bar(kBarOFull + (o_it & 1)));
+          if (elect_one()) {
+            issue_pv_half(tmem + kColO + 64, tmem + kColS + 128 * b, vd, 1, t == 0 ? 0u : 1u);
+            mma_commit(bar(kBarVEmpty + vs));
+            mma_commit(bar(kBarPFree + b));
+            if (t == it.nt - 1) mma_commit(bar(kBarOFull + (o_it & 1)));
+          }
+          __syncwarp();
           ++v_it;
           if (++b == (uint32_t)kNS) {
             b = 0;
@@ -436,8 +457,10 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         }
         ++o_it;
       }
-      mma_commit(bar(kBarDrain2));
+      if (elect_one()) mma_commit(bar(kBarDrain2));
+      __syncwarp();
       mbar_wait(bar(kBarDrain2), 0, abort_flag);
+      __syncwarp();
     }
   } else if (warp < 4 + kRowWarps) {
     // ---------------------------------------------------------------- row warps: a query row and
@@ -501,7 +524,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       }
       return true;
     };
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it_cnt) {
+    for (int k = 0, item; (item = cta_item(k, n_items)) >= 0; ++k, ++it_cnt) {
       const Item it = decode_item(item, p);
       const int row = it.row0 + rt;
       const uint32_t slot = it_cnt & 1;
@@ -539,12 +562,13 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         // exponents under the current reference (0 while there is none), and their maximum
         const float neg_ref = mb == -INFINITY ? 0.f : -mb;
         float mx = -INFINITY;
+        uint32_t x[kChunks][32];
 #pragma unroll
         for (int c = 0; c < kChunks; ++c) {
           const int cg = kChunks * part + c;
           if (kWriteP && park) chunk_park<L>(v[c], tb, cg, my_scratch, rank_base, off0);
-          if (diag) mx = chunk_exponents<L, true>(v[c], tb, cg, rt - 32 * cg, cs, neg_ref, mx);
-          else mx = chunk_exponents<L, false>(v[c], tb, cg, 0, cs, neg_ref, mx);
+          if (diag) mx = chunk_exponents<L, true>(v[c], x[c], tb, cg, rt - 32 * cg, cs, neg_ref, mx);
+          else mx = chunk_exponents<L, false>(v[c], x[c], tb, cg, 0, cs, neg_ref, mx);
         }
         // The reference moves to the tile's maximum when that lies more than kLazyBits above it, or
         // when this is the row half's first kept score; the exponents then shift by adj.
@@ -580,7 +604,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
 #pragma unroll
         for (int c = 0; c < kChunks; ++c) {
           uint32_t hi[16], lo[16];
-          chunk_probs(v[c], adj, la, lb, hi, lo);
+          chunk_probs(x[c], adj, la, lb, hi, lo);
           tmem_st16(src + 32 * c, hi);
           tmem_st16(src + 32 * c + 16, lo);
         }
@@ -641,7 +665,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       const float cs = p.scale_log2;
       uint32_t it_cnt = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it_cnt) {
+      for (int k = 0, item; (item = cta_item(k, n_items)) >= 0 && ok; ++k, ++it_cnt) {
         const uint32_t slot = it_cnt & 1;
         ok = __all_sync(0xffffffffu, mbar_wait<500>(bar(kBarFixFull + slot), (it_cnt >> 1) & 1, abort_flag));
         if (!ok) break;
