@@ -42,6 +42,12 @@ the paper's steps in the paper's order:
                         causal rows drop keys j > i.  Output is a flat CSR.
                         With k_star: the appendix's cap for long sequences, at
                         most k_star uniformly spaced keys per selected column.
+    expand_mask_resized App. "Sparse Interpolation" at any ratio of T to Kc, and App.
+                        "Visualization of intermediate buffers" for causal rows:
+                        nearest-neighbour resize of row i of the compressed mask
+                        from Kc pixels to a target width W (T; or, with
+                        ``row_widths``, the causal row's own width i + 1): key j
+                        looks at pixel floor(j * Kc / W).
     sparse_attention    Sec. 3.1.1 "Sparse Attention Mechanism": rho (scores at
                         mask positions), sigma (softmax over a row's non-zeros),
                         then C = A* V.
@@ -76,6 +82,7 @@ __all__ = [
     "topk_select_causal_aware",
     "sea_attention_grouped_batch",
     "expand_mask",
+    "expand_mask_resized",
     "sparse_attention",
     "sea_attention_head",
     "k_hat_from_k",
@@ -219,6 +226,35 @@ def expand_mask(sel, T: int, Kc: int, causal: bool, query_index=None, k_star=Non
                 j = int(c) * r + o
                 if causal and j > i:
                     continue
+                row.append(j)
+        cols.extend(row)
+        row_ptr[t + 1] = row_ptr[t] + len(row)
+    return row_ptr, np.asarray(cols, dtype=np.int64)
+
+
+def expand_mask_resized(sel, T: int, Kc: int, causal: bool, row_widths: bool, query_index=None):
+    """Flat CSR of the mask obtained by resizing every row of the compressed mask by nearest
+    neighbour, for any T and Kc (T need not be a multiple of Kc).
+
+    Row i of the compressed mask has Kc pixels, those listed in ``sel[i]`` set.  It is resized to
+    W pixels, W = T, or W = i + 1 when ``row_widths`` (the paper resizes every causal row to the
+    row's own width): key j < W is kept when pixel floor(j * Kc / W) is set.  ``causal`` drops
+    keys j > i (with row_widths there are none).
+    """
+    n = len(sel)
+    if query_index is None:
+        query_index = np.arange(n)
+    row_ptr = np.zeros(n + 1, dtype=np.int64)
+    cols = []
+    for t in range(n):
+        i = int(query_index[t])
+        W = i + 1 if row_widths else T
+        chosen = set(int(c) for c in sel[t])
+        row = []
+        for j in range(W):
+            if causal and j > i:
+                continue
+            if (j * Kc) // W in chosen:
                 row.append(j)
         cols.extend(row)
         row_ptr[t + 1] = row_ptr[t] + len(row)
