@@ -18,7 +18,9 @@
  *     static scratch array of sea_topk_mask_static (see there).
  *   - Q, K, V, O are [B, H, T, d] in the dtype `shape->io`; d must be 64.
  *   - A "row" is one query: row = (b*H + h)*T + i, rows = B*H*T.
- *   - r = T / Kc keys are covered by one compressed column (T % Kc == 0).
+ *   - r = T / Kc keys are covered by one compressed column (T % Kc == 0; only
+ *     sea_estimate, sea_sparse_attn without `sel` and the *_resized calls take
+ *     other ratios).
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL =
  *     the default stream) and the call returns without synchronising.
  *   - Host-detectable errors (null pointer, bad shape, too small a workspace or
@@ -258,6 +260,34 @@ sea_status sea_attention_capped(const sea_shape* shape, int32_t k_star, const vo
                                 const float* A_hat_in, void* O, float* A_hat, int32_t* sel,
                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* P,
                                 void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Nearest-neighbour resize of the compressed mask at any ratio, App. "Sparse
+ * Interpolation" and App. "Visualization of intermediate buffers".  The selection
+ * is that of sea_topk_mask (per query, k_hat of the Kc pixels of a row); the
+ * up-sampling treats row i of the compressed mask as an image of Kc pixels that is
+ * resized to W pixels: key j < W looks at pixel floor(j * Kc / W), so a selected
+ * pixel c covers the keys ceil(c*W/Kc) .. ceil((c+1)*W/Kc) - 1.
+ *   row_widths == 0: W = T for every row; T need not be a multiple of Kc (for
+ *     T % Kc == 0 the result is that of sea_topk_mask); causal rows drop keys j > i.
+ *   row_widths == 1 (causal shapes only): W = i + 1, the paper's handling of causal
+ *     rows ("each row ... is resized with different target widths according to the
+ *     token index"): a row's k_hat pixels spread over the keys it may see, so its
+ *     length grows with i, and only rows narrower than Kc keys can lose pixels.
+ * Outputs as for sea_topk_mask; nnz_cap rows*k_hat*ceil(T/Kc) always suffices and is
+ * what sea_attention_resized requires (its sparse stage walks col_idx with the
+ * per-row kernels, so col_idx is required there).  sea_workspace_bytes_resized is
+ * sea_workspace_bytes without the T % Kc == 0 condition.
+ */
+sea_status sea_workspace_bytes_resized(const sea_shape* shape, size_t* bytes);
+sea_status sea_topk_mask_resized(const sea_shape* shape, int32_t row_widths, const float* A_hat, int32_t* sel,
+                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap,
+                                 void* ws, size_t ws_bytes, void* cuda_stream);
+sea_status sea_attention_resized(const sea_shape* shape, int32_t row_widths, const void* Q, const void* K,
+                                 const void* V, const float* omega, const float* W_dec,
+                                 const float* A_hat_in, void* O, float* A_hat, int32_t* sel,
+                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* P,
+                                 void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
  * sea_attention for callers whose tensors live in HOST memory.  hQ, hK, hV,

@@ -32,7 +32,7 @@ EXPORTS = (
     "sea_workspace_bytes", "sea_estimate", "sea_topk_mask", "sea_topk_mask_static", "sea_sparse_attn",
     "sea_attention", "sea_topk_mask_grouped", "sea_sparse_attn_masked", "sea_attention_grouped",
     "sea_topk_mask_causal_aware", "sea_attention_causal_aware", "sea_workspace_bytes_capped", "sea_topk_mask_capped",
-    "sea_attention_capped",
+    "sea_attention_capped", "sea_workspace_bytes_resized", "sea_topk_mask_resized", "sea_attention_resized",
     "sea_workspace_host_bytes", "sea_attention_host", "sea_device_status", "sea_last_launch_count",
     "sea_last_sparse_kernel", "sea_last_sparse_flops",
     "sea_status_string",
@@ -83,6 +83,9 @@ def load_library() -> ctypes.CDLL:
     lib.sea_workspace_bytes_capped.argtypes = [shp, i32, ctypes.POINTER(sz)]
     lib.sea_topk_mask_capped.argtypes = [shp, i32, vp, vp, vp, vp, i64, vp, sz, vp]
     lib.sea_attention_capped.argtypes = [shp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
+    lib.sea_workspace_bytes_resized.argtypes = [shp, ctypes.POINTER(sz)]
+    lib.sea_topk_mask_resized.argtypes = [shp, i32, vp, vp, vp, vp, i64, vp, sz, vp]
+    lib.sea_attention_resized.argtypes = [shp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
     lib.sea_attention_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sea_device_status.argtypes = [vp, ctypes.POINTER(i32), i32, vp]
     lib.sea_last_launch_count.argtypes = []
@@ -260,6 +263,32 @@ def sea_attention_capped(shape, k_star: int, Q, K, V, omega, W_dec, O, ws, col_i
                                                _ptr(row_ptr), _ptr(col_idx), nnz_cap, _ptr(P), _ptr(ws), ws.numel(),
                                                _stream(ws.device)),
            "sea_attention_capped")
+
+
+def sea_workspace_bytes_resized(shape: SeaShape) -> int:
+    out = ctypes.c_size_t(0)
+    _check(load_library().sea_workspace_bytes_resized(ctypes.byref(shape), ctypes.byref(out)), "sea_workspace_bytes_resized")
+    return out.value
+
+
+def sea_topk_mask_resized(shape, row_widths: bool, A_hat, sel, row_ptr, col_idx, ws, nnz_cap: Optional[int] = None):
+    """Nearest-neighbour resize at any ratio of T to Kc; row_widths: causal rows resized to their own width."""
+    if nnz_cap is None:
+        nnz_cap = col_idx.numel() if col_idx is not None else 0
+    _check(load_library().sea_topk_mask_resized(ctypes.byref(shape), int(row_widths), _ptr(A_hat), _ptr(sel), _ptr(row_ptr),
+                                                _ptr(col_idx), nnz_cap, _ptr(ws), ws.numel(), _stream(ws.device)),
+           "sea_topk_mask_resized")
+
+
+def sea_attention_resized(shape, row_widths: bool, Q, K, V, omega, W_dec, O, ws, col_idx, A_hat_in=None, A_hat=None,
+                          sel=None, row_ptr=None, P=None, nnz_cap: Optional[int] = None):
+    if nnz_cap is None:
+        nnz_cap = col_idx.numel()
+    _check(load_library().sea_attention_resized(ctypes.byref(shape), int(row_widths), _ptr(Q), _ptr(K), _ptr(V),
+                                                _ptr(omega), _ptr(W_dec), _ptr(A_hat_in), _ptr(O), _ptr(A_hat), _ptr(sel),
+                                                _ptr(row_ptr), _ptr(col_idx), nnz_cap, _ptr(P), _ptr(ws), ws.numel(),
+                                                _stream(ws.device)),
+           "sea_attention_resized")
 
 
 def sea_attention_host(shape, hQ, hK, hV, homega, hW_dec, hO, ws):

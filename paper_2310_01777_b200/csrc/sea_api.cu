@@ -12,12 +12,12 @@ size_t io_bytes(const sea_shape& s) { return s.io == SEA_BF16 ? 2 : 4; }
 // Largest number of CSR entries the mask of this shape can hold: every row keeps k_hat columns of
 // min(r, k_star) keys (k_star <= 0: whole runs).
 long long mask_entries_bound(const sea_shape& s, int k_star) {
-  const long long r = s.T / s.Kc;
+  const long long r = (s.T + s.Kc - 1) / s.Kc;
   const long long per_col = k_star > 0 && k_star < r ? k_star : r;
   return (long long)s.B * s.H * s.T * s.k_hat * per_col;
 }
 
-sea_status validate_shape(const sea_shape* s, bool need_estimator, int k_star) {
+sea_status validate_shape(const sea_shape* s, bool need_estimator, int k_star, bool ragged) {
   if (s == nullptr) return SEA_ERR_INVALID_ARG;
   if (s->B <= 0 || s->H <= 0 || s->T <= 0 || s->Kc <= 0 || s->k_hat <= 0) return SEA_ERR_INVALID_ARG;
   if (s->causal != 0 && s->causal != 1) return SEA_ERR_INVALID_ARG;
@@ -26,7 +26,7 @@ sea_status validate_shape(const sea_shape* s, bool need_estimator, int k_star) {
   if (s->m < 0) return SEA_ERR_INVALID_ARG;
   if (s->k_hat > s->Kc) return SEA_ERR_INVALID_ARG;
   if (s->d != kHeadDim) return SEA_ERR_UNSUPPORTED;
-  if (s->T % s->Kc != 0) return SEA_ERR_UNSUPPORTED;
+  if (!ragged && s->T % s->Kc != 0) return SEA_ERR_UNSUPPORTED;
   if (s->Kc > 2048) return SEA_ERR_UNSUPPORTED;
   if (need_estimator && (s->m < 16 || s->m > 128 || s->m % 16 != 0)) return SEA_ERR_UNSUPPORTED;
   const long long rows = (long long)s->B * s->H * s->T;
@@ -128,7 +128,7 @@ sea_status sea_estimate(const sea_shape* shape, const void* Q, const void* K, co
                         const float* omega, const float* W_dec, float* A_hat, void* ws,
                         size_t ws_bytes, void* cuda_stream) {
   Launch::count() = 0;
-  const sea_status rc = validate_shape(shape, true);
+  const sea_status rc = validate_shape(shape, true, 0, true);  // the estimate does not depend on the ratio of T to Kc
   if (rc != SEA_OK) return rc;
   if (!Q || !K || !V || !omega || !W_dec || !A_hat || !ws) return SEA_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(omega) || !aligned16(W_dec) ||
@@ -168,7 +168,7 @@ sea_status sea_sparse_attn(const sea_shape* shape, const void* Q, const void* K,
                            const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel, void* O,
                            void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
   Launch::count() = 0;
-  const sea_status rc = validate_shape(shape, false);
+  const sea_status rc = validate_shape(shape, false, 0, sel == nullptr);  // a plain CSR may come from any up-sampling
   if (rc != SEA_OK) return rc;
   if (!Q || !K || !V || !row_ptr || !O || (!col_idx && !sel)) return SEA_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(row_ptr) ||
@@ -460,6 +460,79 @@ sea_status sea_attention_capped(const sea_shape* shape, int32_t k_star, const vo
                                reinterpret_cast<int32_t*>(w + L.tile_sums), status, st);
   if (rc != SEA_OK) return rc;
   // rows keep scattered keys, not runs: the per-row kernels walk the CSR
+  return launch_sparse_attn_rows(*shape, Q, K, V, rp_buf, col_idx, nullptr, O, P, st);
+}
+
+sea_status sea_workspace_bytes_resized(const sea_shape* shape, size_t* bytes) {
+  if (bytes == nullptr) return SEA_ERR_INVALID_ARG;
+  const sea_status rc = validate_shape(shape, false, 0, true);
+  if (rc != SEA_OK) return rc;
+  *bytes = ws_layout(*shape).total;
+  return SEA_OK;
+}
+
+sea_status sea_topk_mask_resized(const sea_shape* shape, int32_t row_widths, const float* A_hat, int32_t* sel,
+                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* ws, size_t ws_bytes,
+                                 void* cuda_stream) {
+  Launch::count() = 0;
+  const sea_status rc = validate_shape(shape, false, 0, true);
+  if (rc != SEA_OK) return rc;
+  if (row_widths != 0 && row_widths != 1) return SEA_ERR_INVALID_ARG;
+  if (row_widths && !shape->causal) return SEA_ERR_UNSUPPORTED;  // a row's own width is a causal notion
+  if (!A_hat || !row_ptr || !ws) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(A_hat) || !aligned16(row_ptr) || !aligned16(ws) || (sel && !aligned16(sel)) || (col_idx && !aligned16(col_idx)))
+    return SEA_ERR_INVALID_ARG;
+  if (col_idx && nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
+  if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  const WsLayout L = ws_layout(*shape);
+  if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
+  return launch_topk_mask_resized(*shape, row_widths, A_hat, sel_buf, row_ptr, col_idx, nnz_cap,
+                                  reinterpret_cast<int32_t*>(w + L.row_counts), reinterpret_cast<int32_t*>(w + L.tile_sums),
+                                  reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
+}
+
+sea_status sea_attention_resized(const sea_shape* shape, int32_t row_widths, const void* Q, const void* K, const void* V,
+                                 const float* omega, const float* W_dec, const float* A_hat_in, void* O, float* A_hat,
+                                 int32_t* sel, int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* P, void* ws,
+                                 size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  const bool estimate = A_hat_in == nullptr;
+  sea_status rc = validate_shape(shape, estimate, 0, true);
+  if (rc != SEA_OK) return rc;
+  if (row_widths != 0 && row_widths != 1) return SEA_ERR_INVALID_ARG;
+  if (row_widths && !shape->causal) return SEA_ERR_UNSUPPORTED;
+  if (!Q || !K || !V || !O || !ws || !col_idx) return SEA_ERR_INVALID_ARG;
+  if (estimate && (!omega || !W_dec)) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(ws) || !aligned16(col_idx) ||
+      (omega && !aligned16(omega)) || (W_dec && !aligned16(W_dec)) || (A_hat_in && !aligned16(A_hat_in)) ||
+      (A_hat && !aligned16(A_hat)) || (sel && !aligned16(sel)) || (row_ptr && !aligned16(row_ptr)) || (P && !aligned16(P)))
+    return SEA_ERR_INVALID_ARG;
+  if (nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
+  if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  // the sparse stage walks col_idx (and writes P) by row_ptr alone: the capacity must hold any mask
+  if (nnz_cap < mask_entries_bound(*shape, 0)) return SEA_ERR_TOO_LARGE;
+  const WsLayout L = ws_layout(*shape);
+  if (ws_bytes < L.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
+  const float* a_use = A_hat_in;
+  if (estimate) {
+    float* a_out = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
+    rc = launch_estimate(*shape, Q, K, V, omega, W_dec, a_out, reinterpret_cast<float*>(w + L.est_state),
+                         w + L.est_split, nullptr, nullptr, status, st);
+    if (rc != SEA_OK) return rc;
+    a_use = a_out;
+  }
+  int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
+  int32_t* rp_buf = row_ptr ? row_ptr : reinterpret_cast<int32_t*>(w + L.row_ptr);
+  rc = launch_topk_mask_resized(*shape, row_widths, a_use, sel_buf, rp_buf, col_idx, nnz_cap,
+                                reinterpret_cast<int32_t*>(w + L.row_counts), reinterpret_cast<int32_t*>(w + L.tile_sums),
+                                status, st);
+  if (rc != SEA_OK) return rc;
+  // a pixel's keys are runs of differing lengths: the per-row kernels walk the CSR
   return launch_sparse_attn_rows(*shape, Q, K, V, rp_buf, col_idx, nullptr, O, P, st);
 }
 

@@ -48,7 +48,8 @@ struct WsLayout {
 
 WsLayout ws_layout(const sea_shape& s);
 // k_star > 0: a selected column keeps at most k_star keys (capped replication), which bounds the mask.
-sea_status validate_shape(const sea_shape* s, bool need_estimator, int k_star = 0);
+// ragged: T need not be a multiple of Kc (the resized expansion); a column then covers up to ceil(T / Kc) keys.
+sea_status validate_shape(const sea_shape* s, bool need_estimator, int k_star = 0, bool ragged = false);
 long long mask_entries_bound(const sea_shape& s, int k_star);
 
 // Where the per-query selection goes when the estimator's output kernel performs it (see
@@ -105,6 +106,11 @@ sea_status launch_topk_mask_aware(const sea_shape& s, const float* A_hat, uint32
 sea_status launch_topk_mask_capped(const sea_shape& s, int k_star, const float* A_hat, int32_t* sel,
                                    int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts,
                                    int32_t* tile_sums, int32_t* status, cudaStream_t st);
+// Nearest-neighbour resize of the compressed mask at any ratio of T to Kc; row_widths: a causal row
+// is resized to its own width i + 1 (sea_topk.cu).  col_idx may be null.
+sea_status launch_topk_mask_resized(const sea_shape& s, int row_widths, const float* A_hat, int32_t* sel, int32_t* row_ptr,
+                                    int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts, int32_t* tile_sums,
+                                    int32_t* status, cudaStream_t st);
 // Where each row parks its unnormalised probabilities when rows keep differing numbers of columns:
 // the (b, t) slabs of H*k_hat*r floats follow one another, the heads inside a slab.  Rows of a slab
 // that keeps more than H*k_hat columns get -1 and SEA_DEV_ROW_OVERFLOW is raised.

@@ -344,7 +344,7 @@ sea_status launch_typed(const sea_shape& s, const T* Q, const T* K, const T* V,
                         const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel, T* O,
                         T* P, cudaStream_t st) {
   const int rows = s.B * s.H * s.T;
-  const int r = s.T / s.Kc;
+  const int r = (s.T + s.Kc - 1) / s.Kc;  // a column's keys (the most, when T is no multiple of Kc)
   const long long cap = (long long)s.k_hat * r;
   int chunk = (int)((cap + 31) / 32 * 32);
   if (chunk > 1024) chunk = 1024;
@@ -407,7 +407,7 @@ sea_status launch_sparse_attn_rows(const sea_shape& s, const void* Q, const void
   if (s.io == SEA_BF16) {
     using T = __nv_bfloat16;
     const int rows = s.B * s.H * s.T;
-    const int r = s.T / s.Kc;
+    const int r = (s.T + s.Kc - 1) / s.Kc;  // a column's keys (the most, when T is no multiple of Kc)
     const long long cap = (long long)s.k_hat * r;
     int chunk = (int)((cap + 63) / 64 * 64);
     if (chunk > 1024) chunk = 1024;

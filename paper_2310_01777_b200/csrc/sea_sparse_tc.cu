@@ -776,7 +776,7 @@ size_t sparse_attn_tc_scratch_bytes(const sea_shape& s) {
 bool sparse_attn_tc_shape_ok(const sea_shape& s) {
   if (s.io != SEA_BF16) return false;
   const int r = s.T / s.Kc;
-  if (s.T % kTile != 0 || log2_exact(r) < 2) return false;
+  if (s.T % s.Kc != 0 || s.T % kTile != 0 || log2_exact(r) < 2) return false;
   // dense tiles pay off while a row keeps at least about 1/40 of the keys it may see: measured at
   // k_hat / Kc = 1/32 the tiles take 0.77 of the per-row gather's time, at 1/64 they take 1.43 of it
   return (long long)s.k_hat * 40 >= s.Kc;

@@ -702,6 +702,95 @@ sea_status launch_topk_mask_capped(const sea_shape& s, int k_star, const float* 
   return check_launch();
 }
 
+// ---- nearest-neighbour resize at any ratio (App. "Sparse Interpolation"; App. "Visualization of
+// intermediate buffers": every causal row is resized to its own width) --------------------------
+// Row i of the compressed mask (Kc pixels) is resized to W pixels, W = T or, with row_widths, i + 1:
+// key j looks at pixel floor(j Kc / W), so a selected pixel c covers the keys
+// ceil(c W / Kc) .. ceil((c + 1) W / Kc) - 1 (none when W < Kc skips the pixel).  Causal rows keep j <= i.
+__device__ __forceinline__ int resized_first_key(int c, int W, int Kc) { return (int)(((long long)c * W + Kc - 1) / Kc); }
+__device__ __forceinline__ void resized_run(int c, int i, int T, int Kc, int causal, int row_widths, int& start, int& len) {
+  const int W = row_widths ? i + 1 : T;
+  start = resized_first_key(c, W, Kc);
+  int end = resized_first_key(c + 1, W, Kc);
+  if (causal) end = min(end, i + 1);
+  len = max(0, end - start);
+}
+
+__global__ void resized_counts_kernel(const int32_t* __restrict__ sel, int32_t* __restrict__ row_counts, int rows, int k_hat,
+                                      int T, int Kc, int causal, int row_widths) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= rows) return;
+  const int i = row % T;
+  int cnt = 0;
+  for (int e = 0; e < k_hat; ++e) {
+    int start, len;
+    resized_run(__ldg(sel + (size_t)row * k_hat + e), i, T, Kc, causal, row_widths, start, len);
+    cnt += len;
+  }
+  row_counts[row] = cnt;
+}
+
+// One warp per row, 32 selected pixels at a time: the lanes hold the pixels' runs and the running
+// sum of their lengths; every entry of the row finds its run by a search over those sums.
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+fill_col_idx_resized_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__ row_ptr,
+                            int32_t* __restrict__ col_idx, long long nnz_cap, int rows, int k_hat, int T, int Kc, int causal,
+                            int row_widths, int32_t* __restrict__ status) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kWarpsPerCta + warp;
+  if (row >= rows) return;
+  const int i = row % T;
+  const long long base = row_ptr[row];
+  long long room = nnz_cap - base;  // entries of this row that still fit
+  if (base + (row_ptr[row + 1] - base) > nnz_cap && lane == 0) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
+  int done = 0;
+  for (int e0 = 0; e0 < k_hat; e0 += 32) {
+    int start = 0, len = 0;
+    if (e0 + lane < k_hat) resized_run(__ldg(sel + (size_t)row * k_hat + e0 + lane), i, T, Kc, causal, row_widths, start, len);
+    int inc = len;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += v;
+    }
+    const int total = __shfl_sync(0xffffffffu, inc, 31);
+    const int n_up = (total + 31) & ~31;  // every lane takes part in the shuffles
+    for (int pos = lane; pos < n_up; pos += 32) {
+      // the first lane whose running sum exceeds pos
+      int lo = 0;
+#pragma unroll
+      for (int step = 16; step > 0; step >>= 1) {
+        const int v = __shfl_sync(0xffffffffu, inc, lo + step - 1);
+        if (v <= pos) lo += step;
+      }
+      const int run_start = __shfl_sync(0xffffffffu, start, lo);
+      const int before = __shfl_sync(0xffffffffu, inc - len, lo);
+      if (pos < total && (long long)(done + pos) < room) col_idx[base + done + pos] = run_start + (pos - before);
+    }
+    done += total;
+  }
+}
+
+sea_status launch_topk_mask_resized(const sea_shape& s, int row_widths, const float* A_hat, int32_t* sel, int32_t* row_ptr,
+                                    int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts, int32_t* tile_sums,
+                                    int32_t* status, cudaStream_t st) {
+  const int rows = s.B * s.H * s.T;
+  // the selection as usual, on a copy of the shape that asks for no row lengths (the row pointers it
+  // writes are replaced below)
+  sea_shape plain = s;
+  plain.causal = 0;
+  sea_status rc = launch_topk_mask(plain, A_hat, sel, row_ptr, nullptr, 0, row_counts, tile_sums, nullptr, false, status, st);
+  if (rc != SEA_OK) return rc;
+  resized_counts_kernel<<<(rows + 255) / 256, 256, 0, st>>>(sel, row_counts, rows, s.k_hat, s.T, s.Kc, s.causal, row_widths);
+  if ((rc = check_launch()) != SEA_OK) return rc;
+  if ((rc = launch_row_ptr_scan(row_counts, tile_sums, row_ptr, rows, st)) != SEA_OK) return rc;
+  if (col_idx == nullptr) return SEA_OK;
+  const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
+  fill_col_idx_resized_kernel<<<grid, kWarpsPerCta * 32, 0, st>>>(sel, row_ptr, col_idx, (long long)nnz_cap, rows, s.k_hat, s.T,
+                                                                  s.Kc, s.causal, row_widths, status);
+  return check_launch();
+}
+
 // Causal-aware per-query selection: bits, row lengths, row pointers and (optionally) column indices.
 sea_status launch_topk_mask_aware(const sea_shape& s, const float* A_hat, uint32_t* mask_bits, int32_t* row_ptr,
                                   int32_t* col_idx, int64_t nnz_cap, int32_t* row_counts, int32_t* tile_sums,
