@@ -283,7 +283,8 @@ def sparse_roofline(w, kernel, exec_flops, nnz, sparse_ms, peaks, clocks):
     bounds = {"hbm_compulsory": compulsory / (hbm_peak * 1e9) * 1e3}
     if kernel == "sparse_attn_tiles_tc_kernel" and exec_flops:
         mhz = (clocks or {}).get("sm_mhz") or 1965.0
-        n_ex2 = exec_flops / (2 * w.d) / 2  # one exponential per entry of every executed score tile
+        nq = w.T // 128
+        n_ex2 = w.B * w.H * (nq * (nq + 1) // 2 if w.causal else nq * nq) * 128 * 128  # one per entry of every score tile
         bounds["tensor"] = exec_flops / (tc_peak * 1e12) * 1e3
         bounds["xu_ex2"] = n_ex2 / (XU_PER_CLK_PER_SM * SM_COUNT * mhz * 1e6) * 1e3
         achieved = exec_flops / t / 1e12
@@ -309,6 +310,70 @@ def hbm_roofline(kernels, nbytes, ms, peaks, what):
             "ms": ms, "bytes": what}
 
 
+# Latencies the paper reports for its own implementation on one RTX 2080 Ti (App. Tables A.1 / A.2:
+# bidirectional, K = 128, random inputs; batch and head counts not stated): context, not a target.
+PAPER_SWEEP_MS = {32: {4096: 1.45, 8192: 3.07, 16384: 6.21, 32768: 12.00, 65536: 25.74, 131072: 50.89},
+                  64: {4096: 1.77, 8192: 3.69, 16384: 7.40, 32768: 13.46, 65536: 28.74, 131072: 56.46},
+                  128: {4096: 2.39, 8192: 4.89, 16384: 9.81, 32768: 16.49, 65536: 37.94, 131072: 72.59}}
+
+
+def run_capped_sweep(args):
+    """The paper's long-sequence setting with a fixed compressed width: K = 128, k in {32, 64, 128},
+    T = 4096 .. 131072, not causal; k_hat = max(1, round(k K / T)) and every selected column keeps
+    k* = min(k, ceil(T / K)) uniformly spaced keys (sea_attention_capped).  One JSON line."""
+    import torch
+
+    import paper_2310_01777_b200 as sea
+    from paper_2310_01777_b200.inputs import Workload, make_inputs
+
+    dev = torch.device("cuda", 0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    rows_out = []
+    for k in (32, 64, 128):
+        for T in (4096, 8192, 16384, 32768, 65536, 131072):
+            Kc = 128
+            k_hat = max(1, round(k * Kc / T))  # Sec. 3.1; Python rounds halves to even
+            k_star = min(k, -(-T // Kc))
+            w = Workload(f"sweep_T{T}_k{k}", args.sweep_B, args.sweep_H, T, 64, 128, Kc, k_hat, False, "bf16", 0)
+            host = make_inputs(w)
+            d = {n: v.to(dev) for n, v in host.items()}
+            shape = sea.make_shape(w)
+            ws = torch.empty(sea.sea_workspace_bytes_capped(shape, k_star), dtype=torch.uint8, device=dev)
+            ws[:256].zero_()
+            cap = w.rows * k_hat * min(k_star, T // Kc)
+            O = torch.empty_like(d["Q"])
+            col = torch.empty((cap,), dtype=torch.int32, device=dev)
+            P = torch.empty((cap,), dtype=torch.bfloat16, device=dev)
+            rp = torch.empty((w.rows + 1,), dtype=torch.int32, device=dev)
+
+            def step():
+                sea.sea_attention_capped(shape, k_star, d["Q"], d["K"], d["V"], d["omega"], d["W_dec"], O, ws, col,
+                                         row_ptr=rp, P=P)
+
+            for _ in range(3):
+                step()
+            torch.cuda.synchronize(dev)
+            ms = []
+            for _ in range(args.steps if args.steps <= 10 else 10):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); step(); b.record()
+                torch.cuda.synchronize(dev)
+                ms.append(a.elapsed_time(b))
+            if sea.sea_device_status(ws) != 0:
+                raise SystemExit("device status word set in the capped sweep")
+            rows_out.append({"T": T, "k": k, "k_hat": k_hat, "k_star": k_star, "nnz": int(rp[-1]), "ms": ms_stats(ms),
+                             "tokens_per_s": w.B * T / (statistics.median(ms) / 1e3), "paper_2080ti_ms": PAPER_SWEEP_MS[k][T]})
+            del d, ws, O, col, P, rp
+            torch.cuda.empty_cache()
+    print(json.dumps({"metric": "SEA attention latency on the paper's long-sequence sweep (all stages, with P)",
+                      "unit": "ms", "config": {"workload": f"B={args.sweep_B} H={args.sweep_H} d=64 m=128 K=128 not causal bf16, "
+                                                           "capped replication (App. Sparse Interpolation)",
+                                               "l2": "flushed between steps (256 MiB write)"},
+                      "note": "paper_2080ti_ms: the paper's own figures on its hardware, batch and heads unstated; context only",
+                      "sweep": rows_out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -322,6 +387,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-modes", action="store_true", help="skip the grouped / causal-aware / lean regions")
     ap.add_argument("--soak-s", type=float, default=1.2, help="seconds of steps the clock sampler watches")
+    ap.add_argument("--capped-sweep", action="store_true", help="time the paper's long-sequence sweep shape instead")
+    ap.add_argument("--sweep-B", type=int, default=1)
+    ap.add_argument("--sweep-H", type=int, default=12)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -330,6 +398,10 @@ def main():
     w = WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
+        return
+
+    if args.capped_sweep:
+        run_capped_sweep(args)
         return
 
     if w.m == 0:
