@@ -58,6 +58,7 @@ WsLayout ws_layout(const sea_shape& s) {
   L.mask_bits = take(sparse_attn_tc_bits_bytes(s));
   L.p_scratch = take(sparse_attn_tc_shape_ok(s) ? sparse_attn_tc_scratch_bytes(s) : 0);  // only the tile kernel parks
   L.park_off = take(s.io == SEA_BF16 ? rows * sizeof(int32_t) : 0);
+  L.tile_live = take(sparse_attn_tc_shape_ok(s) ? sparse_attn_tc_live_bytes(s) : 0);
   L.total = off;
   return L;
 }
@@ -184,6 +185,7 @@ sea_status sea_sparse_attn(const sea_shape* shape, const void* Q, const void* K,
   return launch_sparse_attn(*shape, Q, K, V, row_ptr, col_idx, sel, O, P,
                             full ? reinterpret_cast<uint32_t*>(w + L.mask_bits) : nullptr, false,
                             full ? reinterpret_cast<float*>(w + L.p_scratch) : nullptr,
+                            full ? reinterpret_cast<uint32_t*>(w + L.tile_live) : nullptr,
                             static_cast<int32_t*>(ws), static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -236,7 +238,7 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
                         reinterpret_cast<int32_t*>(w + L.tile_sums), bits, selected, status, st);
   if (rc != SEA_OK) return rc;
   return launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P, bits, true,
-                            reinterpret_cast<float*>(w + L.p_scratch), status, st);
+                            reinterpret_cast<float*>(w + L.p_scratch), reinterpret_cast<uint32_t*>(w + L.tile_live), status, st);
 }
 
 }  // extern "C"
@@ -309,6 +311,7 @@ sea_status sea_sparse_attn_masked(const sea_shape* shape, const void* Q, const v
   return launch_sparse_attn_masked(*shape, Q, K, V, row_ptr, col_idx, mask_bits, O, P,
                                    full ? reinterpret_cast<int32_t*>(w + L.park_off) : nullptr, false, false,
                                    full ? reinterpret_cast<float*>(w + L.p_scratch) : nullptr,
+                                   full ? reinterpret_cast<uint32_t*>(w + L.tile_live) : nullptr,
                                    static_cast<int32_t*>(ws), static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -365,11 +368,11 @@ sea_status attention_bits(BitsMode mode, const sea_shape* shape, const void* Q, 
     rc = launch_topk_mask_grouped(*shape, a_use, bits, rp_buf, col_idx, nnz_cap, counts, sums, tiles_ok && P ? park : nullptr,
                                   status, st);
     if (rc != SEA_OK) return rc;
-    return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, true, false, scratch, status, st);
+    return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, true, false, scratch, reinterpret_cast<uint32_t*>(w + L.tile_live), status, st);
   }
   rc = launch_topk_mask_aware(*shape, a_use, bits, rp_buf, col_idx, nnz_cap, counts, sums, status, st);
   if (rc != SEA_OK) return rc;
-  return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, false, true, scratch, status, st);
+  return launch_sparse_attn_masked(*shape, Q, K, V, rp_buf, col_idx, bits, O, P, park, false, true, scratch, reinterpret_cast<uint32_t*>(w + L.tile_live), status, st);
 }
 }  // namespace
 

@@ -43,6 +43,7 @@ struct WsLayout {
   size_t mask_bits;   // uint32 [rows][ceil(Kc/32)]   selected columns as bits (tensor-core sparse stage)
   size_t p_scratch;   // float [rows][k_hat*r]        unnormalised probabilities (tensor-core sparse stage)
   size_t park_off;    // int32 [rows]                 offsets into p_scratch (masks with rows of differing lengths)
+  size_t tile_live;   // uint32 [BH*T/128][..]        a bit per (work item, key tile) that holds a kept key (tensor-core sparse stage)
   size_t total;
 };
 
@@ -122,7 +123,7 @@ sea_status launch_park_offsets(const sea_shape& s, const uint32_t* mask_bits, in
 sea_status launch_sparse_attn_masked(const sea_shape& s, const void* Q, const void* K, const void* V,
                                      const int32_t* row_ptr, const int32_t* col_idx,
                                      const uint32_t* mask_bits, void* O, void* P, int32_t* park_off,
-                                     bool park_valid, bool rows_within_k_hat, float* p_scratch,
+                                     bool park_valid, bool rows_within_k_hat, float* p_scratch, uint32_t* tile_live,
                                      int32_t* status, cudaStream_t st);
 // mask_bits and p_scratch (workspace areas of the tensor-core kernel) may be null: the per-row
 // kernels are used then.  bits_valid: mask_bits already holds the bit strings of `sel`
@@ -130,7 +131,7 @@ sea_status launch_sparse_attn_masked(const sea_shape& s, const void* Q, const vo
 sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, const void* V,
                               const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
                               void* O, void* P, uint32_t* mask_bits, bool bits_valid, float* p_scratch,
-                              int32_t* status, cudaStream_t st);
+                              uint32_t* tile_live, int32_t* status, cudaStream_t st);
 sea_status launch_sparse_attn_rows(const sea_shape& s, const void* Q, const void* K, const void* V,
                                    const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
                                    void* O, void* P, cudaStream_t st);
@@ -138,6 +139,7 @@ sea_status launch_sparse_attn_rows(const sea_shape& s, const void* Q, const void
 bool sparse_attn_tc_shape_ok(const sea_shape& s);
 size_t sparse_attn_tc_bits_bytes(const sea_shape& s);
 size_t sparse_attn_tc_scratch_bytes(const sea_shape& s);
+size_t sparse_attn_tc_live_bytes(const sea_shape& s);
 // have_bits: mask_bits already holds the mask (sel may then be null)
 bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, bool have_bits, const int32_t* status,
                                const void* mask_bits, const void* p_scratch);
@@ -145,7 +147,7 @@ bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, bool have
 sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* K, const void* V,
                                  const int32_t* row_ptr, const int32_t* sel, void* O, void* P,
                                  uint32_t* mask_bits, bool bits_valid, float* p_scratch,
-                                 const int32_t* park_off, int32_t* status, cudaStream_t st);
+                                 const int32_t* park_off, uint32_t* tile_live, int32_t* status, cudaStream_t st);
 bool sparse_attn_tma_applicable(const sea_shape& s, const int32_t* sel, const int32_t* status);
 sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void* K, const void* V,
                                   const int32_t* row_ptr, const int32_t* sel, void* O, void* P,

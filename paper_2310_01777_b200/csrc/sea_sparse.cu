@@ -370,9 +370,9 @@ sea_status launch_typed(const sea_shape& s, const T* Q, const T* K, const T* V,
 sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, const void* V,
                               const int32_t* row_ptr, const int32_t* col_idx, const int32_t* sel,
                               void* O, void* P, uint32_t* mask_bits, bool bits_valid, float* p_scratch,
-                              int32_t* status, cudaStream_t st) {
-  if (sparse_attn_tc_applicable(s, sel, false, status, mask_bits, p_scratch))
-    return launch_sparse_attn_tc(s, Q, K, V, row_ptr, sel, O, P, mask_bits, bits_valid, p_scratch, nullptr, status, st);
+                              uint32_t* tile_live, int32_t* status, cudaStream_t st) {
+  if (tile_live != nullptr && sparse_attn_tc_applicable(s, sel, false, status, mask_bits, p_scratch))
+    return launch_sparse_attn_tc(s, Q, K, V, row_ptr, sel, O, P, mask_bits, bits_valid, p_scratch, nullptr, tile_live, status, st);
   if (sparse_attn_tma_applicable(s, sel, status))
     return launch_sparse_attn_tma(s, Q, K, V, row_ptr, sel, O, P, status, st);
   return launch_sparse_attn_rows(s, Q, K, V, row_ptr, col_idx, sel, O, P, st);
@@ -381,18 +381,18 @@ sea_status launch_sparse_attn(const sea_shape& s, const void* Q, const void* K, 
 sea_status launch_sparse_attn_masked(const sea_shape& s, const void* Q, const void* K, const void* V,
                                      const int32_t* row_ptr, const int32_t* col_idx, const uint32_t* mask_bits,
                                      void* O, void* P, int32_t* park_off, bool park_valid, bool rows_within_k_hat,
-                                     float* p_scratch, int32_t* status, cudaStream_t st) {
-  if (park_off != nullptr && sparse_attn_tc_applicable(s, nullptr, true, status, mask_bits, p_scratch)) {
+                                     float* p_scratch, uint32_t* tile_live, int32_t* status, cudaStream_t st) {
+  if (park_off != nullptr && tile_live != nullptr && sparse_attn_tc_applicable(s, nullptr, true, status, mask_bits, p_scratch)) {
     if (P != nullptr && rows_within_k_hat)  // every row fits the per-query parking layout
       return launch_sparse_attn_tc(s, Q, K, V, row_ptr, nullptr, O, P, const_cast<uint32_t*>(mask_bits), true, p_scratch,
-                                   nullptr, status, st);
+                                   nullptr, tile_live, status, st);
     if (P != nullptr && !park_valid) {
       const sea_status rc = launch_park_offsets(s, mask_bits, park_off, status, st);
       if (rc != SEA_OK) return rc;
     }
     // the bits are only read: bits_valid keeps the launcher from deriving them from a selection list
     return launch_sparse_attn_tc(s, Q, K, V, row_ptr, nullptr, O, P, const_cast<uint32_t*>(mask_bits), true, p_scratch,
-                                 P != nullptr ? park_off : nullptr, status, st);
+                                 P != nullptr ? park_off : nullptr, tile_live, status, st);
   }
   if (col_idx == nullptr) return SEA_ERR_INVALID_ARG;
   return launch_sparse_attn_rows(s, Q, K, V, row_ptr, col_idx, nullptr, O, P, st);

@@ -151,9 +151,51 @@ struct TcParams {
   float* p_scratch;             // unnormalised probabilities of kept keys: row `row` parks its runs at
   const int32_t* park_off;      // park_off[row] (negative: nowhere), or at row * k_hat * r when this is null
   int32_t* status;
-  int BH, T, words, log2r, k_hat, causal;
+  const uint32_t* tile_live;    // [work items][live_words] a bit per key tile: some row of the item keeps a key of it
+  const uint32_t* some_tile_unused;  // [n_unused_flags] non-zero: some item has a key tile in which none of its rows keeps a key
+  int n_unused_flags;
+  int BH, T, words, log2r, k_hat, causal, live_words;
   float scale_log2;
 };
+
+// The key tiles of a work item that its rows keep a key of, a bit per tile, read an item ahead.
+// Tiles that no row of the item selected anything in are not visited at all: no copy, no product,
+// no row work.  Walking a list that is only known on the device costs every role time on every tile
+// (the loops' bounds and counters no longer live in uniform registers), so the kernel exists twice:
+// kSkip = true walks the lists, kSkip = false visits every tile; both are launched, and the one
+// that the mask does not call for (tile_live[-1]: some tile of some item is unused) returns at once.
+constexpr int kLiveWords = 8;  // T <= 32768
+template <bool kSkip>
+struct LiveTiles {
+  uint32_t w[kSkip ? kLiveWords : 1];
+};
+template <bool kSkip>
+__device__ __forceinline__ LiveTiles<kSkip> load_live_tiles(const TcParams& p, int item) {  // item < 0: none
+  LiveTiles<kSkip> lt;
+  if constexpr (kSkip) {
+    const uint32_t* src = p.tile_live + (size_t)(item < 0 ? 0 : item) * p.live_words;
+#pragma unroll
+    for (int i = 0; i < kLiveWords; ++i) lt.w[i] = (item >= 0 && i < p.live_words) ? __ldg(src + i) : 0u;
+  } else {
+    lt.w[0] = 0u;
+  }
+  return lt;
+}
+// The first tile to visit that is >= from (from >= 0), or -1.
+template <bool kSkip>
+__device__ __forceinline__ int next_live_tile(const LiveTiles<kSkip>& lt, int from, int nt) {
+  if constexpr (!kSkip) return from < nt ? from : -1;
+  int t = -1;
+#pragma unroll
+  for (int i = 0; i < (kSkip ? kLiveWords : 1); ++i) {
+    const int skip = from - 32 * i;  // bits of this word below `from`
+    uint32_t m = lt.w[i];
+    if (skip >= 32) m = 0u;
+    else if (skip > 0) m &= 0xffffffffu << skip;
+    if (t < 0 && m != 0u) t = 32 * i + __ffs((int)m) - 1;
+  }
+  return t < nt ? t : -1;
+}
 
 // The k-th work item of this CTA, or -1 when it has no more.  Items are numbered in order of
 // descending cost and dealt out to the CTAs stripe by stripe, back and forth (the CTA that got a
@@ -291,10 +333,15 @@ __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.al
 template <int kRegs>
 __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegs)); }
 
-template <int L, bool kWriteP>
+template <int L, bool kWriteP, bool kSkip>
 __global__ void __launch_bounds__(kThreads, 1)
 sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                             const __grid_constant__ CUtensorMap map_v, const TcParams p) {
+  {
+    int unused = 0;
+    for (int i = threadIdx.x; i < p.n_unused_flags; i += kThreads) unused |= (int)__ldg(p.some_tile_unused + i);
+    if (kSkip != (__syncthreads_or(unused) != 0)) return;  // the other instance of the kernel does the work
+  }
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* sm = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   const uint32_t sQ = smem_u32(sm);                          // 2 x 16 KB
@@ -341,6 +388,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       // ---------------------------------------------------------------- TMA producer
       uint32_t q_it = 0, k_it = 0, v_it = 0;
       bool ok = true;
+      LiveTiles<kSkip> live_next = load_live_tiles<kSkip>(p, cta_item(0, n_items));  // read an item ahead: the latency hides behind the item before
       for (int k = 0, item; (item = cta_item(k, n_items)) >= 0 && ok; ++k) {
         const Item it = decode_item(item, p);
         const uint32_t qb = q_it & 1;
@@ -353,7 +401,9 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         mbar_expect_tx(bar(kBarQFull + qb), kTileBytes);
         tma_load_2d(sQ + qb * kTileBytes, &map_q, 0, it.row0, bar(kBarQFull + qb));
         ++q_it;
-        for (int t = 0; t < it.nt; ++t) {
+        const LiveTiles<kSkip> live = live_next;
+        live_next = load_live_tiles<kSkip>(p, cta_item(k + 1, n_items));
+        for (int t = next_live_tile<kSkip>(live, 0, it.nt); t >= 0; t = next_live_tile<kSkip>(live, t + 1, it.nt)) {
           const uint32_t ks = k_it % kNK;
           ok = mbar_wait<100>(bar(kBarKEmpty + ks), ((k_it / kNK) & 1) ^ 1, abort_flag);
           if (!ok) break;
@@ -384,12 +434,16 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       uint32_t b = 0, round = 0;  // use round * kNS + b occupies buffer b
       const uint64_t k_desc0 = smem_desc(sK, 16, 1024);  // a stage further on: + 16 KB / 16
       bool ok = true;
+      LiveTiles<kSkip> live_next = load_live_tiles<kSkip>(p, cta_item(0, n_items));  // read an item ahead: the latency hides behind the item before
       for (int k = 0, item; (item = cta_item(k, n_items)) >= 0 && ok; ++k) {
         const Item it = decode_item(item, p);
         const uint32_t qb = q_it & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarQFull + qb), (q_it >> 1) & 1, abort_flag));
         const uint64_t q_desc = smem_desc(sQ + qb * kTileBytes, 16, 1024);
-        for (int t = 0; t < it.nt && ok; ++t) {
+        const LiveTiles<kSkip> live = live_next;
+        live_next = load_live_tiles<kSkip>(p, cta_item(k + 1, n_items));
+        for (int t = next_live_tile<kSkip>(live, 0, it.nt), t_next; t >= 0 && ok; t = t_next) {
+          t_next = next_live_tile<kSkip>(live, t + 1, it.nt);
           const uint32_t ks = k_it % kNK;
           const uint32_t kbar = bar(kBarKFull + ks), kpar = (k_it / kNK) & 1;
           if (round > 0) ok = __all_sync(0xffffffffu, mbar_wait2(bar(kBarPFree + b), (round & 1u) ^ 1u, kbar, kpar, abort_flag));
@@ -400,7 +454,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
             issue_qk_mmas(tmem + kColS + 128 * b, q_desc, k_desc0 + 1024ull * ks);
             mma_commit(bar(kBarKEmpty + ks));
             mma_commit(bar(kBarSFull + b));
-            if (t == it.nt - 1) mma_commit(bar(kBarQEmpty + qb));
+            if (t_next < 0) mma_commit(bar(kBarQEmpty + qb));
           }
           __syncwarp();
           ++k_it;
@@ -422,31 +476,37 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       uint32_t b = 0, round = 0;
       const uint64_t v_desc0 = smem_desc(sV, 8192, 1024);  // a stage further on: + 16 KB / 16
       bool ok = true;
+      LiveTiles<kSkip> live_next = load_live_tiles<kSkip>(p, cta_item(0, n_items));  // read an item ahead: the latency hides behind the item before
       for (int k = 0, item; (item = cta_item(k, n_items)) >= 0 && ok; ++k) {
         const Item it = decode_item(item, p);
-        for (int t = 0; t < it.nt && ok; ++t) {
+        const LiveTiles<kSkip> live = live_next;
+        live_next = load_live_tiles<kSkip>(p, cta_item(k + 1, n_items));
+        const int t_first = next_live_tile<kSkip>(live, 0, it.nt);
+        for (int t = t_first, t_next; t >= 0 && ok; t = t_next) {
+          t_next = next_live_tile<kSkip>(live, t + 1, it.nt);
+          const bool first = t == t_first;
           // the rows have written P (and, before an item's first tile, read the previous item's output)
           // Each column half has its own accumulator and its own barrier, so a half's product starts as
           // soon as its rows are done.  Every row thread reads both accumulators when an item ends: the
           // first product of an item waits for both halves.
           const uint32_t vs = v_it % kNV;
           ok = __all_sync(0xffffffffu, mbar_wait2(bar(kBarSDone + kSplit * b), round & 1u, bar(kBarVFull + vs), (v_it / kNV) & 1, abort_flag));
-          if (ok && t == 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSDone + kSplit * b + 1), round & 1u, abort_flag));
+          if (ok && first) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSDone + kSplit * b + 1), round & 1u, abort_flag));
           if (!ok) break;
           fence_after();
           const uint64_t vd = v_desc0 + 1024ull * vs;
-          if (elect_one()) issue_pv_half(tmem + kColO, tmem + kColS + 128 * b, vd, 0, t == 0 ? 0u : 1u);
+          if (elect_one()) issue_pv_half(tmem + kColO, tmem + kColS + 128 * b, vd, 0, first ? 0u : 1u);
           __syncwarp();
-          if (t != 0) {
+          if (!first) {
             ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSDone + kSplit * b + 1), round & 1u, abort_flag));
             if (!ok) break;
             fence_after();
           }
           if (elect_one()) {
-            issue_pv_half(tmem + kColO + 64, tmem + kColS + 128 * b, vd, 1, t == 0 ? 0u : 1u);
+            issue_pv_half(tmem + kColO + 64, tmem + kColS + 128 * b, vd, 1, first ? 0u : 1u);
             mma_commit(bar(kBarVEmpty + vs));
             mma_commit(bar(kBarPFree + b));
-            if (t == it.nt - 1) mma_commit(bar(kBarOFull + (o_it & 1)));
+            if (t_next < 0) mma_commit(bar(kBarOFull + (o_it & 1)));
           }
           __syncwarp();
           ++v_it;
@@ -524,6 +584,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       }
       return true;
     };
+    LiveTiles<kSkip> live_next = load_live_tiles<kSkip>(p, cta_item(0, n_items));  // read an item ahead: the latency hides behind the item before
     for (int k = 0, item; (item = cta_item(k, n_items)) >= 0; ++k, ++it_cnt) {
       const Item it = decode_item(item, p);
       const int row = it.row0 + rt;
@@ -547,7 +608,10 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
       float mb = -INFINITY;  // this half's reference in the exponent's units (score * cs); -inf while it has met no kept score
       float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
       int rank_base = 0;
-      for (int t = 0; t < it.nt && ok; ++t) {
+      const LiveTiles<kSkip> live = live_next;
+      live_next = load_live_tiles<kSkip>(p, cta_item(k + 1, n_items));
+      const int t_first = next_live_tile<kSkip>(live, 0, it.nt);
+      for (int t = t_first; t >= 0 && ok; t = next_live_tile<kSkip>(live, t + 1, it.nt)) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + b), round & 1u, abort_flag));
         if (!ok) break;
         fence_after();
@@ -611,7 +675,7 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
         rank_base = next_rank<L>(rank_base, tb, t, log2r);
         // the previous item's output row leaves the accumulators before this item's first product
         // may overwrite them: by now that item's last product has long finished
-        if (t == 0 && !epilogue()) {
+        if (t == t_first && !epilogue()) {
           ok = false;
           break;
         }
@@ -718,6 +782,57 @@ sparse_attn_tiles_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __g
   if (tid == 0 && *abort_flag) atomicOr(p.status, SEA_DEV_TIMEOUT);
 }
 
+// One warp per work item (128 query rows): which key tiles does any of its rows keep a key of?
+// The union of the rows' bit strings, then a bit per key tile; an item whose rows keep nothing at
+// all still visits one tile, so that its output rows are written (as zeros) the usual way.
+// unused_flags [gridDim.x]: whether some item of this block has a key tile that it does not use.
+__global__ void __launch_bounds__(128)
+tile_live_kernel(const uint32_t* __restrict__ mask_bits, uint32_t* __restrict__ tile_live, uint32_t* __restrict__ unused_flags,
+                 int n_items, int BH, int T, int words, int log2r, int causal, int live_words) {
+  __shared__ uint32_t uni_all[4][32];  // Kc <= 1024: at most 32 words
+  const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int item = blockIdx.x * 4 + wid;
+  int unused = 0;
+  if (item < n_items) {
+    uint32_t* uni = uni_all[wid];
+    const int ntq = T / kTile;
+    const int qt = ntq - 1 - item / BH, bh = item % BH;
+    const int nt = causal ? qt + 1 : ntq;
+    const uint32_t* rows = mask_bits + ((size_t)bh * T + (size_t)qt * kTile) * words;
+    for (int w = 0; w < words; ++w) {
+      uint32_t acc = 0u;
+      for (int r = lane; r < kTile; r += 32) acc |= __ldg(rows + (size_t)r * words + w);
+      acc = __reduce_or_sync(0xffffffffu, acc);
+      if (lane == 0) uni[w] = acc;
+    }
+    __syncwarp();
+    uint32_t* out = tile_live + (size_t)item * live_words;
+    int n_live = 0;
+    for (int w0 = 0; w0 < live_words; ++w0) {
+      const int t = 32 * w0 + lane;
+      bool mine = false;
+      if (t < nt) {
+        if (log2r >= 7) {
+          const int c = t >> (log2r - 7);
+          mine = (uni[c >> 5] >> (c & 31)) & 1u;
+        } else {
+          const int G = 128 >> log2r;  // compressed columns per key tile: 1 .. 32, never across a word
+          const int c0 = t * G;
+          const uint32_t m = G >= 32 ? 0xffffffffu : ((1u << G) - 1u);
+          mine = ((uni[c0 >> 5] >> (c0 & 31)) & m) != 0u;
+        }
+      }
+      const uint32_t word = __ballot_sync(0xffffffffu, mine);
+      n_live += __popc(word);
+      if (lane == 0) out[w0] = word;
+    }
+    if (n_live == 0 && lane == 0) out[0] = 1u;
+    unused = n_live < nt;
+  }
+  unused = __syncthreads_or(unused);
+  if (threadIdx.x == 0) unused_flags[blockIdx.x] = unused ? 1u : 0u;
+}
+
 // One thread per row: the ascending selected columns become a bit string of `words` words.
 __global__ void sel_to_bits_kernel(const int32_t* __restrict__ sel, uint32_t* __restrict__ mask_bits, int rows, int k_hat,
                                    int words) {
@@ -748,12 +863,12 @@ int log2_exact(int x) {
   return (1 << l) == x ? l : -1;
 }
 
-template <int L, bool kWriteP>
-sea_status launch_tc(const sea_shape& s, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+template <int L, bool kWriteP, bool kSkip>
+sea_status launch_tc_one(const sea_shape& s, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                      const TcParams& prm, cudaStream_t st) {
   const size_t smem = 1024 + (size_t)(2 + kNK + kNV) * kTileBytes + kBarBlockBytes + (size_t)(4 * kSplit + 10) * kTile * 4 +
                       2 * (size_t)prm.words * kTile * 4;
-  auto kern = sparse_attn_tiles_tc_kernel<L, kWriteP>;
+  auto kern = sparse_attn_tiles_tc_kernel<L, kWriteP, kSkip>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SEA_ERR_CUDA;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -763,11 +878,24 @@ sea_status launch_tc(const sea_shape& s, const CUtensorMap& mq, const CUtensorMa
   kern<<<grid, kThreads, smem, st>>>(mq, mk, mv, prm);
   return check_launch();
 }
+// Both instances: the one that the mask does not call for returns at once.
+template <int L, bool kWriteP>
+sea_status launch_tc(const sea_shape& s, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                     const TcParams& prm, cudaStream_t st) {
+  const sea_status rc = launch_tc_one<L, kWriteP, false>(s, mq, mk, mv, prm, st);
+  if (rc != SEA_OK) return rc;
+  return launch_tc_one<L, kWriteP, true>(s, mq, mk, mv, prm, st);
+}
 
 }  // namespace
 
 size_t sparse_attn_tc_bits_bytes(const sea_shape& s) {
   return (size_t)s.B * s.H * s.T * (size_t)((s.Kc + 31) / 32) * sizeof(uint32_t);
+}
+size_t sparse_attn_tc_live_bytes(const sea_shape& s) {
+  const size_t ntq = (size_t)(s.T + kTile - 1) / kTile;
+  const size_t n_items = (size_t)s.B * s.H * ntq;
+  return n_items * ((ntq + 31) / 32) * sizeof(uint32_t) + ((n_items + 3) / 4) * sizeof(uint32_t);  // the lists, then the flags
 }
 size_t sparse_attn_tc_scratch_bytes(const sea_shape& s) {
   return (size_t)s.B * s.H * s.T * (size_t)s.k_hat * (size_t)(s.T / s.Kc) * sizeof(float);
@@ -777,6 +905,7 @@ bool sparse_attn_tc_shape_ok(const sea_shape& s) {
   if (s.io != SEA_BF16) return false;
   const int r = s.T / s.Kc;
   if (s.T % s.Kc != 0 || s.T % kTile != 0 || log2_exact(r) < 2) return false;
+  if (s.T / kTile > 32 * kLiveWords) return false;  // a bit per key tile of a work item, held in registers
   // dense tiles pay off while a row keeps at least about 1/40 of the keys it may see: measured at
   // k_hat / Kc = 1/32 the tiles take 0.77 of the per-row gather's time, at 1/64 they take 1.43 of it
   return (long long)s.k_hat * 40 >= s.Kc;
@@ -790,7 +919,8 @@ bool sparse_attn_tc_applicable(const sea_shape& s, const int32_t* sel, bool have
 
 sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* K, const void* V, const int32_t* row_ptr,
                                  const int32_t* sel, void* O, void* P, uint32_t* mask_bits, bool bits_valid,
-                                 float* p_scratch, const int32_t* park_off, int32_t* status, cudaStream_t st) {
+                                 float* p_scratch, const int32_t* park_off, uint32_t* tile_live, int32_t* status,
+                                 cudaStream_t st) {
   const unsigned long long rows = (unsigned long long)s.B * s.H * s.T;
   CUtensorMap mq, mk, mv;
   if (!make_rows_map_bf16(&mq, Q, rows, kTile) || !make_rows_map_bf16(&mk, K, rows, kTile) || !make_rows_map_bf16(&mv, V, rows, kTile)) return SEA_ERR_CUDA;
@@ -817,8 +947,21 @@ sea_status launch_sparse_attn_tc(const sea_shape& s, const void* Q, const void* 
     const sea_status rc = check_launch();
     if (rc != SEA_OK) return rc;
   }
+  {
+    const int n_items = prm.BH * (s.T / kTile);
+    prm.live_words = (s.T / kTile + 31) / 32;
+    prm.tile_live = tile_live;
+    uint32_t* flags = tile_live + (size_t)n_items * prm.live_words;  // a word per block of the kernel below, after the lists
+    prm.some_tile_unused = flags;
+    prm.n_unused_flags = (n_items + 3) / 4;
+    tile_live_kernel<<<prm.n_unused_flags, 128, 0, st>>>(mask_bits, tile_live, flags, n_items, prm.BH, s.T, prm.words, prm.log2r,
+                                                        s.causal, prm.live_words);
+    const sea_status rc = check_launch();
+    if (rc != SEA_OK) return rc;
+  }
   Launch::sparse_kernel() = "sparse_attn_tiles_tc_kernel";
   {
+    // (an upper bound when the mask leaves whole key tiles unused: those are skipped)
     // every (query tile, key tile) pair a query tile may see: S = Q K^T and P V with P as a bf16
     // head plus a bf16 remainder, 2 * 128 * 128 * 64 FLOPs each
     const double nq = s.T / kTile;

@@ -73,6 +73,22 @@ WORKLOADS: Dict[str, Workload] = {
 }
 
 
+def banded_estimate(w: Workload, width: float = 2.0, sink: bool = True, seed: int = 3) -> torch.Tensor:
+    """A compressed estimate [B, H, T, Kc] whose large entries lie in a band of about `width`
+    compressed columns around the diagonal (plus, with `sink`, column 0), with a little noise:
+    the structure the paper's figures show for trained SEA estimates (diagonal bands, a few
+    global columns), which the random-init decoder of the benchmark workloads does not have.
+    Only an input recipe: no arithmetic of the method."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    i = torch.arange(w.T, dtype=torch.float32)[:, None] / w.r
+    c = torch.arange(w.Kc, dtype=torch.float32)[None, :]
+    a = -(c - i).abs() / width + 0.05 * torch.randn((w.B, w.H, w.T, w.Kc), generator=g, dtype=torch.float32)
+    if sink:
+        a[..., 0] = 10.0
+    return a.contiguous()
+
+
 def torch_dtype(name: str) -> torch.dtype:
     if name == "f32":
         return torch.float32

@@ -6,7 +6,7 @@ import torch
 import paper_2310_01777_b200 as sea
 from oracle import sea_oracle as orc
 from paper_2310_01777_b200 import binding
-from paper_2310_01777_b200.inputs import WORKLOADS, Workload, make_inputs
+from paper_2310_01777_b200.inputs import WORKLOADS, Workload, banded_estimate, make_inputs
 from tests.helpers import (GpuRun, check_a_hat, check_float, check_head_against_oracle,
                            global_mask_properties, head_slices, np64, scale_of)
 
@@ -106,6 +106,28 @@ def test_tile_kernel_moves_its_softmax_reference(causal, profile):
         assert run.status() == 0
         for h in range(w.H):
             check_head_against_oracle(run, 0, h, check_estimate=False)
+
+
+@pytest.mark.parametrize("causal,sink", [(True, False), (True, True), (False, False)])
+def test_tile_kernel_skips_key_tiles_no_row_selected(causal, sink):
+    """With a banded mask most key tiles hold no kept key for any of the 128 rows of a work item:
+    the tile kernel leaves them out (no copy, no product); O, P and the mask still match the
+    oracle, the per-row kernels give the same, and rows of a tile that keep nothing come out zero."""
+    w = small("banded", dtype="bf16", T=1024, Kc=64, k_hat=5, causal=causal, H=2, m=0)
+    host = make_inputs(w)
+    host["A_hat"] = banded_estimate(w, 2.0, sink)
+    run = GpuRun(w, inputs=host)
+    run.topk_mask(); run.sync()
+    for lean in (False, True):
+        run.O.fill_(float("nan")); run.P.fill_(float("nan"))
+        run.sparse_attn(lean_ws=lean)
+        run.sync()
+        assert run.status() == 0
+        for h in range(w.H):
+            check_head_against_oracle(run, 0, h, check_estimate=False)
+    assert sea.sea_last_sparse_kernel() != "sparse_attn_tiles_tc_kernel"
+    run.sparse_attn(); run.sync()
+    assert sea.sea_last_sparse_kernel() == "sparse_attn_tiles_tc_kernel"
 
 
 EST_CASES = [
