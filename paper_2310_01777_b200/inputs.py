@@ -89,6 +89,31 @@ def banded_estimate(w: Workload, width: float = 2.0, sink: bool = True, seed: in
     return a.contiguous()
 
 
+def make_decoder_params(w: Workload, d_hidden: int = 64, c_s: int = 2, c_h: int = 4, seed: int = 1) -> Dict[str, torch.Tensor]:
+    """Random-init weights of the paper's estimator head (MLPs mu and nu, the three convolutions,
+    the two scalar heads, and for causal layers the positional embedding that replaces V_I), drawn
+    with fan-in scaling so that activations stay of order one.  fp32, except pos_emb which has the
+    I/O dtype of V (it is concatenated to V).  Only an input recipe: no arithmetic of the method."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    d, C, Wr = w.d, w.H * c_h, w.Kc // c_s
+
+    def n(shape, std):
+        return (torch.randn(shape, generator=g, dtype=torch.float32) * std).contiguous()
+
+    return {
+        "W_mu": n((3 * d, d_hidden), (1.0 / (3 * d)) ** 0.5), "b_mu": n((d_hidden,), 0.1),
+        "W_nu1": n((d_hidden, d_hidden), (2.0 / d_hidden) ** 0.5), "b_nu1": n((d_hidden,), 0.1),
+        "W_nu2": n((d_hidden, Wr * c_h), (2.0 / d_hidden) ** 0.5), "b_nu2": n((Wr * c_h,), 0.1),
+        "conv1_w": n((C, C, 3, 3), (2.0 / (9 * C)) ** 0.5), "conv1_b": n((C,), 0.1),
+        "conv2_w": n((C, C, 3, 3), (2.0 / (9 * C)) ** 0.5), "conv2_b": n((C,), 0.1),
+        "conv3_w": n((w.H, C, 3, 3), (8.0 / (9 * C)) ** 0.5), "conv3_b": n((w.H,), 0.1),
+        "pos_emb": torch.randn((w.T, d), generator=g, dtype=torch.float32).to(torch_dtype(w.dtype)).contiguous(),
+        "w_prob": n((d_hidden,), (1.0 / d_hidden) ** 0.5), "b_prob": n((1,), 0.5),
+        "w_mix": n((d_hidden,), (1.0 / d_hidden) ** 0.5), "b_mix": n((1,), 0.5),
+    }
+
+
 def torch_dtype(name: str) -> torch.dtype:
     if name == "f32":
         return torch.float32
