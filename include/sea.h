@@ -290,6 +290,62 @@ sea_status sea_attention_resized(const sea_shape* shape, int32_t row_widths, con
                                  void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The paper's estimator head and output mixing, with weights given by the caller (the
+ * benchmark workloads use random-init ones; trained weights would come from the paper's
+ * distillation, which is outside this library).
+ *
+ * Sec. 3.1 "Attention Matrix Estimation" / "CNN Decoder", App. "Attention Estimator CNN":
+ *   V_cat = [V_I ; V], V_I the identity I_d resized by nearest neighbour to T rows (causal
+ *   shapes: the positional embedding pos_emb [T, d] takes its place);
+ *   C_perf = FAVOR+(Q, K, V_cat) [T, 2d];  Z = relu([C_perf ; V] W_mu + b_mu) [T, d_hidden];
+ *   Z_hat = relu(Z W_nu1 + b_nu1) W_nu2 + b_nu2 [T, (Kc/c_s) c_h], reshaped over the heads to an
+ *   image [H c_h, T, Kc/c_s] (entry j Kc/c_s + x of head h: channel h c_h + j, column x);
+ *   conv 3x3 (C -> C, relu; not causal: stride c_s along T), conv 3x3 (C -> C, relu), nearest
+ *   resize to [C, T, Kc], conv 3x3 (C -> H), softmax over Kc.  Causal shapes keep the height and
+ *   pad every layer with two rows above and none below (row t sees rows t-2 .. t); the width is
+ *   padded by one on both sides.  Where the paper gives no detail (activations, layer counts of the
+ *   MLPs, paddings, the channel order) these are this library's readings.
+ * Sec. 3.1.1: s_prob = sigmoid(Z . w_prob + b_prob) re-scales the sparse attention's
+ *   probabilities and output; C_avg is, not causal, the V-average weighted by the column means
+ *   of A_hat resized to T keys, and, causal, the running mean of V; s_mix = sigmoid(Z . w_mix +
+ *   b_mix); C_sea = s_mix (s_prob C) + (1 - s_mix) C_avg.
+ *
+ * All weights are fp32 device arrays, row-major: W_mu [3d, d_hidden], W_nu1 [d_hidden, d_hidden],
+ * W_nu2 [d_hidden, (Kc/c_s) c_h], conv1_w / conv2_w [C, C, 3, 3], conv3_w [H, C, 3, 3] with
+ * C = H c_h, biases alongside, w_prob / w_mix [d_hidden]; pos_emb [T, d] has the io dtype.
+ * Requires Kc % c_s == 0 and, for shapes that are not causal, T % c_s == 0.
+ *
+ * sea_estimate_decoder writes A_hat [B, H, T, Kc] (rows sum to one) and Z [B, H, T, d_hidden].
+ * sea_mix_output turns O (the output C of sea_sparse_attn for a mask from that A_hat) into
+ * C_sea in place and multiplies P (may be NULL) by s_prob.  sea_attention_decoder chains
+ * sea_estimate_decoder -> sea_topk_mask -> sea_sparse_attn -> sea_mix_output; A_hat, sel,
+ * row_ptr, col_idx, P are optional outputs as for sea_attention.  Workspace:
+ * sea_workspace_bytes_decoder().  The arithmetic of the head is plain fp32.
+ */
+typedef struct sea_decoder {
+  int32_t d_hidden;           /* d' of the paper, 1 .. 1024 */
+  int32_t c_s, c_h;           /* width reduction and channel expansion (the paper uses 2 and 4) */
+  const float *W_mu, *b_mu;
+  const float *W_nu1, *b_nu1, *W_nu2, *b_nu2;
+  const float *conv1_w, *conv1_b, *conv2_w, *conv2_b, *conv3_w, *conv3_b;
+  const void* pos_emb;        /* causal shapes only */
+  const float *w_prob, *w_mix;
+  float b_prob, b_mix;
+} sea_decoder;
+
+sea_status sea_workspace_bytes_decoder(const sea_shape* shape, const sea_decoder* dec, size_t* bytes);
+sea_status sea_estimate_decoder(const sea_shape* shape, const sea_decoder* dec, const void* Q, const void* K,
+                                const void* V, const float* omega, float* A_hat, float* Z,
+                                void* ws, size_t ws_bytes, void* cuda_stream);
+sea_status sea_mix_output(const sea_shape* shape, const sea_decoder* dec, const float* Z, const float* A_hat,
+                          const void* V, const int32_t* row_ptr, void* O, void* P,
+                          void* ws, size_t ws_bytes, void* cuda_stream);
+sea_status sea_attention_decoder(const sea_shape* shape, const sea_decoder* dec, const void* Q, const void* K,
+                                 const void* V, const float* omega, void* O, float* A_hat, int32_t* sel,
+                                 int32_t* row_ptr, int32_t* col_idx, int64_t nnz_cap, void* P,
+                                 void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * sea_attention for callers whose tensors live in HOST memory.  hQ, hK, hV,
  * homega, hW_dec are copied to staging areas inside `ws`, the layer runs, and O
  * is copied back to hO.  The heads are independent, so the call is a pipeline

@@ -32,6 +32,7 @@ EXPORTS = (
     "sea_workspace_bytes", "sea_estimate", "sea_topk_mask", "sea_topk_mask_static", "sea_sparse_attn",
     "sea_attention", "sea_topk_mask_grouped", "sea_sparse_attn_masked", "sea_attention_grouped",
     "sea_topk_mask_causal_aware", "sea_attention_causal_aware", "sea_workspace_bytes_capped", "sea_topk_mask_capped",
+    "sea_workspace_bytes_decoder", "sea_estimate_decoder", "sea_mix_output", "sea_attention_decoder",
     "sea_attention_capped", "sea_workspace_bytes_resized", "sea_topk_mask_resized", "sea_attention_resized",
     "sea_workspace_host_bytes", "sea_attention_host", "sea_device_status", "sea_last_launch_count",
     "sea_last_sparse_kernel", "sea_last_sparse_flops",
@@ -45,6 +46,14 @@ class SeaShape(ctypes.Structure):
         ("m", ctypes.c_int32), ("Kc", ctypes.c_int32), ("k_hat", ctypes.c_int32),
         ("causal", ctypes.c_int32), ("io", ctypes.c_int32), ("scale", ctypes.c_float),
     ]
+
+
+class SeaDecoder(ctypes.Structure):
+    """Mirror of `sea_decoder`: sizes and device pointers of the estimator head's weights."""
+    _fields_ = [("d_hidden", ctypes.c_int32), ("c_s", ctypes.c_int32), ("c_h", ctypes.c_int32)] + \
+               [(n, ctypes.c_void_p) for n in ("W_mu", "b_mu", "W_nu1", "b_nu1", "W_nu2", "b_nu2", "conv1_w", "conv1_b",
+                                               "conv2_w", "conv2_b", "conv3_w", "conv3_b", "pos_emb", "w_prob", "w_mix")] + \
+               [("b_prob", ctypes.c_float), ("b_mix", ctypes.c_float)]
 
 
 class SeaError(RuntimeError):
@@ -86,6 +95,11 @@ def load_library() -> ctypes.CDLL:
     lib.sea_workspace_bytes_resized.argtypes = [shp, ctypes.POINTER(sz)]
     lib.sea_topk_mask_resized.argtypes = [shp, i32, vp, vp, vp, vp, i64, vp, sz, vp]
     lib.sea_attention_resized.argtypes = [shp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
+    dcp = ctypes.POINTER(SeaDecoder)
+    lib.sea_workspace_bytes_decoder.argtypes = [shp, dcp, ctypes.POINTER(sz)]
+    lib.sea_estimate_decoder.argtypes = [shp, dcp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sea_mix_output.argtypes = [shp, dcp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sea_attention_decoder.argtypes = [shp, dcp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
     lib.sea_attention_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sea_device_status.argtypes = [vp, ctypes.POINTER(i32), i32, vp]
     lib.sea_last_launch_count.argtypes = []
@@ -289,6 +303,51 @@ def sea_attention_resized(shape, row_widths: bool, Q, K, V, omega, W_dec, O, ws,
                                                 _ptr(row_ptr), _ptr(col_idx), nnz_cap, _ptr(P), _ptr(ws), ws.numel(),
                                                 _stream(ws.device)),
            "sea_attention_resized")
+
+
+def make_decoder(params, d_hidden: int, c_s: int, c_h: int, causal: bool) -> SeaDecoder:
+    """`sea_decoder` over the device tensors of `params` (keys as in inputs.make_decoder_params); the
+    caller keeps `params` alive while the struct is in use."""
+    d = SeaDecoder()
+    d.d_hidden, d.c_s, d.c_h = d_hidden, c_s, c_h
+    for name in ("W_mu", "b_mu", "W_nu1", "b_nu1", "W_nu2", "b_nu2", "conv1_w", "conv1_b", "conv2_w", "conv2_b", "conv3_w",
+                 "conv3_b", "w_prob", "w_mix"):
+        t = params[name]
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == torch.float32):
+            raise ValueError(f"{name}: a contiguous fp32 device tensor is needed")
+        setattr(d, name, t.data_ptr())
+    d.pos_emb = params["pos_emb"].data_ptr() if causal else None
+    d.b_prob, d.b_mix = float(params["b_prob"].reshape(-1)[0]), float(params["b_mix"].reshape(-1)[0])
+    return d
+
+
+def sea_workspace_bytes_decoder(shape: SeaShape, dec: SeaDecoder) -> int:
+    out = ctypes.c_size_t(0)
+    _check(load_library().sea_workspace_bytes_decoder(ctypes.byref(shape), ctypes.byref(dec), ctypes.byref(out)),
+           "sea_workspace_bytes_decoder")
+    return out.value
+
+
+def sea_estimate_decoder(shape, dec, Q, K, V, omega, A_hat, Z, ws):
+    _check(load_library().sea_estimate_decoder(ctypes.byref(shape), ctypes.byref(dec), _ptr(Q), _ptr(K), _ptr(V), _ptr(omega),
+                                               _ptr(A_hat), _ptr(Z), _ptr(ws), ws.numel(), _stream(ws.device)),
+           "sea_estimate_decoder")
+
+
+def sea_mix_output(shape, dec, Z, A_hat, V, row_ptr, O, P, ws):
+    _check(load_library().sea_mix_output(ctypes.byref(shape), ctypes.byref(dec), _ptr(Z), _ptr(A_hat), _ptr(V), _ptr(row_ptr),
+                                         _ptr(O), _ptr(P), _ptr(ws), ws.numel(), _stream(ws.device)),
+           "sea_mix_output")
+
+
+def sea_attention_decoder(shape, dec, Q, K, V, omega, O, ws, A_hat=None, sel=None, row_ptr=None, col_idx=None, P=None,
+                          nnz_cap: Optional[int] = None):
+    if nnz_cap is None:
+        nnz_cap = col_idx.numel() if col_idx is not None else 0
+    _check(load_library().sea_attention_decoder(ctypes.byref(shape), ctypes.byref(dec), _ptr(Q), _ptr(K), _ptr(V), _ptr(omega),
+                                                _ptr(O), _ptr(A_hat), _ptr(sel), _ptr(row_ptr), _ptr(col_idx), nnz_cap, _ptr(P),
+                                                _ptr(ws), ws.numel(), _stream(ws.device)),
+           "sea_attention_decoder")
 
 
 def sea_attention_host(shape, hQ, hK, hV, homega, hW_dec, hO, ws):

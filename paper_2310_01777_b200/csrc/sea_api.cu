@@ -539,6 +539,107 @@ sea_status sea_attention_resized(const sea_shape* shape, int32_t row_widths, con
   return launch_sparse_attn_rows(*shape, Q, K, V, rp_buf, col_idx, nullptr, O, P, st);
 }
 
+}  // extern "C"
+
+namespace {
+sea_status validate_decoder(const sea_shape* s, const sea_decoder* d) {
+  if (d == nullptr) return SEA_ERR_INVALID_ARG;
+  if (d->d_hidden < 1 || d->d_hidden > 1024 || d->c_s < 1 || d->c_h < 1) return SEA_ERR_INVALID_ARG;
+  if (s->Kc % d->c_s != 0 || (!s->causal && s->T % d->c_s != 0)) return SEA_ERR_UNSUPPORTED;
+  if (!d->W_mu || !d->b_mu || !d->W_nu1 || !d->b_nu1 || !d->W_nu2 || !d->b_nu2 || !d->conv1_w || !d->conv1_b || !d->conv2_w ||
+      !d->conv2_b || !d->conv3_w || !d->conv3_b || !d->w_prob || !d->w_mix || (s->causal && !d->pos_emb))
+    return SEA_ERR_INVALID_ARG;
+  if ((long long)s->B * s->H * d->c_h * s->T * (s->Kc / d->c_s) > 2147483647ll * 4) return SEA_ERR_TOO_LARGE;
+  return SEA_OK;
+}
+// the decoder's buffers follow the base layout
+size_t decoder_ws_offset(const sea_shape& s) { return align_up(ws_layout(s).total, 256); }
+}  // namespace
+
+extern "C" {
+
+sea_status sea_workspace_bytes_decoder(const sea_shape* shape, const sea_decoder* dec, size_t* bytes) {
+  if (bytes == nullptr) return SEA_ERR_INVALID_ARG;
+  sea_status rc = validate_shape(shape, true);
+  if (rc != SEA_OK) return rc;
+  if ((rc = validate_decoder(shape, dec)) != SEA_OK) return rc;
+  *bytes = decoder_ws_offset(*shape) + decoder_layout(*shape, *dec).total;
+  return SEA_OK;
+}
+
+sea_status sea_estimate_decoder(const sea_shape* shape, const sea_decoder* dec, const void* Q, const void* K, const void* V,
+                                const float* omega, float* A_hat, float* Z, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  sea_status rc = validate_shape(shape, true);
+  if (rc != SEA_OK) return rc;
+  if ((rc = validate_decoder(shape, dec)) != SEA_OK) return rc;
+  if (!Q || !K || !V || !omega || !A_hat || !ws) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(omega) || !aligned16(A_hat) || !aligned16(ws) ||
+      (Z && !aligned16(Z)))
+    return SEA_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*shape);
+  const size_t doff = decoder_ws_offset(*shape);
+  const DecoderLayout D = decoder_layout(*shape, *dec);
+  if (ws_bytes < doff + D.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  float* z = Z ? Z : reinterpret_cast<float*>(w + doff + D.z);
+  return launch_estimate_decoder(*shape, *dec, Q, K, V, omega, A_hat, z, w + doff, reinterpret_cast<float*>(w + L.est_state),
+                                 w + L.est_split, reinterpret_cast<int32_t*>(w + L.status), static_cast<cudaStream_t>(cuda_stream));
+}
+
+sea_status sea_mix_output(const sea_shape* shape, const sea_decoder* dec, const float* Z, const float* A_hat, const void* V,
+                          const int32_t* row_ptr, void* O, void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  sea_status rc = validate_shape(shape, true);
+  if (rc != SEA_OK) return rc;
+  if ((rc = validate_decoder(shape, dec)) != SEA_OK) return rc;
+  if (!Z || !A_hat || !V || !O || !ws || (P && !row_ptr)) return SEA_ERR_INVALID_ARG;
+  const size_t doff = decoder_ws_offset(*shape);
+  if (ws_bytes < doff + decoder_layout(*shape, *dec).total) return SEA_ERR_WORKSPACE;
+  return launch_mix_output(*shape, *dec, Z, A_hat, V, row_ptr, O, P, static_cast<char*>(ws) + doff,
+                           static_cast<cudaStream_t>(cuda_stream));
+}
+
+sea_status sea_attention_decoder(const sea_shape* shape, const sea_decoder* dec, const void* Q, const void* K, const void* V,
+                                 const float* omega, void* O, float* A_hat, int32_t* sel, int32_t* row_ptr, int32_t* col_idx,
+                                 int64_t nnz_cap, void* P, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Launch::count() = 0;
+  sea_status rc = validate_shape(shape, true);
+  if (rc != SEA_OK) return rc;
+  if ((rc = validate_decoder(shape, dec)) != SEA_OK) return rc;
+  if (!Q || !K || !V || !omega || !O || !ws) return SEA_ERR_INVALID_ARG;
+  if (P && !col_idx) return SEA_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(ws) || !aligned16(omega) ||
+      (A_hat && !aligned16(A_hat)) || (sel && !aligned16(sel)) || (row_ptr && !aligned16(row_ptr)) ||
+      (col_idx && !aligned16(col_idx)) || (P && !aligned16(P)))
+    return SEA_ERR_INVALID_ARG;
+  if (col_idx && nnz_cap <= 0) return SEA_ERR_INVALID_ARG;
+  if (nnz_cap > 2147483647ll) return SEA_ERR_TOO_LARGE;
+  if (P && nnz_cap < mask_entries_bound(*shape, 0)) return SEA_ERR_TOO_LARGE;
+  const WsLayout L = ws_layout(*shape);
+  const size_t doff = decoder_ws_offset(*shape);
+  const DecoderLayout D = decoder_layout(*shape, *dec);
+  if (ws_bytes < doff + D.total) return SEA_ERR_WORKSPACE;
+  char* w = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
+  float* a_buf = A_hat ? A_hat : reinterpret_cast<float*>(w + L.a_hat);
+  float* z = reinterpret_cast<float*>(w + doff + D.z);
+  rc = launch_estimate_decoder(*shape, *dec, Q, K, V, omega, a_buf, z, w + doff, reinterpret_cast<float*>(w + L.est_state),
+                               w + L.est_split, status, st);
+  if (rc != SEA_OK) return rc;
+  int32_t* sel_buf = sel ? sel : reinterpret_cast<int32_t*>(w + L.sel);
+  int32_t* rp_buf = row_ptr ? row_ptr : reinterpret_cast<int32_t*>(w + L.row_ptr);
+  uint32_t* bits = reinterpret_cast<uint32_t*>(w + L.mask_bits);
+  rc = launch_topk_mask(*shape, a_buf, sel_buf, rp_buf, col_idx, nnz_cap, reinterpret_cast<int32_t*>(w + L.row_counts),
+                        reinterpret_cast<int32_t*>(w + L.tile_sums), bits, false, status, st);
+  if (rc != SEA_OK) return rc;
+  rc = launch_sparse_attn(*shape, Q, K, V, rp_buf, col_idx, sel_buf, O, P, bits, true, reinterpret_cast<float*>(w + L.p_scratch),
+                          reinterpret_cast<uint32_t*>(w + L.tile_live), status, st);
+  if (rc != SEA_OK) return rc;
+  return launch_mix_output(*shape, *dec, z, a_buf, V, rp_buf, O, P, w + doff, st);
+}
+
 sea_status sea_workspace_host_bytes(const sea_shape* shape, size_t* bytes) {
   if (bytes == nullptr) return SEA_ERR_INVALID_ARG;
   const sea_status rc = validate_shape(shape, true);

@@ -153,6 +153,18 @@ sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void*
                                   const int32_t* row_ptr, const int32_t* sel, void* O, void* P,
                                   int32_t* status, cudaStream_t st);
 
+// The paper's estimator head and output mixing (sea_decoder.cu).  dws: the decoder's own part of
+// the workspace (decoder_layout), est_state / est_split: the estimator's scratch of the base layout.
+struct DecoderLayout {
+  size_t ident, first, c_first, c_value, z, hidden, image, conv_a, conv_b, s_prob, s_mix, c_avg, total;
+};
+DecoderLayout decoder_layout(const sea_shape& s, const sea_decoder& dec);
+sea_status launch_estimate_decoder(const sea_shape& s, const sea_decoder& dec, const void* Q, const void* K, const void* V,
+                                   const float* omega, float* A_hat, float* Z, char* dws, float* est_state, void* est_split,
+                                   int32_t* status, cudaStream_t st);
+sea_status launch_mix_output(const sea_shape& s, const sea_decoder& dec, const float* Z, const float* A_hat, const void* V,
+                             const int32_t* row_ptr, void* O, void* P, char* dws, cudaStream_t st);
+
 inline sea_status check_launch() {
   Launch::count()++;
   return cudaGetLastError() == cudaSuccess ? SEA_OK : SEA_ERR_CUDA;
