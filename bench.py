@@ -32,6 +32,8 @@ metric is quoted.  One JSON line is printed by rank 0.
   structured_mask
              the mask and sparse stages when the caller gives a banded estimate (the structure of
              trained SEA masks): the tile kernel skips the key tiles nothing was selected in.
+  decoder_head  (--decoder) the layer with the paper's estimator head (MLPs + three-layer CNN, random-init
+             weights) and output mixing through sea_attention_decoder: plain fp32 kernels.
   cpu_baseline  the fp64 oracle on a bounded sample of heads, one head per host core at a time.
 
 With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no
@@ -390,6 +392,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-modes", action="store_true", help="skip the grouped / causal-aware / lean regions")
     ap.add_argument("--soak-s", type=float, default=1.2, help="seconds of steps the clock sampler watches")
+    ap.add_argument("--decoder", action="store_true", help="also time the paper's MLP + CNN estimator head (tens of ms per step)")
     ap.add_argument("--capped-sweep", action="store_true", help="time the paper's long-sequence sweep shape instead")
     ap.add_argument("--sweep-B", type=int, default=1)
     ap.add_argument("--sweep-H", type=int, default=12)
@@ -636,6 +639,45 @@ def main():
         step()  # the outputs of the benchmark workload again, for what follows
         torch.cuda.synchronize(dev)
 
+    decoder = None
+    if args.decoder:
+        # ---- timed region 6: the paper's estimator head (MLPs + three-layer CNN) with random-init weights ----
+        from paper_2310_01777_b200.inputs import make_decoder_params
+
+        d_hidden, c_s, c_h = 64, 2, 4
+        dp = {k: v.to(dev) for k, v in make_decoder_params(w, d_hidden, c_s, c_h).items()}
+        dec = sea.make_decoder(dp, d_hidden, c_s, c_h, w.causal)
+        dws = torch.empty(sea.sea_workspace_bytes_decoder(shape, dec), dtype=torch.uint8, device=dev)
+        dws[:256].zero_()
+        Zb = torch.empty((w.B, w.H, w.T, d_hidden), dtype=torch.float32, device=dev)
+
+        def dstep():
+            sea.sea_attention_decoder(shape, dec, d["Q"], d["K"], d["V"], d["omega"], O, dws, A_hat=A_hat, sel=sel,
+                                      row_ptr=row_ptr, col_idx=col_idx, P=P)
+
+        for _ in range(2):
+            dstep()
+        d_launches = sea.sea_last_launch_count()
+        torch.cuda.synchronize(dev)
+        n_d = max(3, min(args.steps, 5))
+        d_all = timed(dstep, n_d)
+        e_all = timed(lambda: sea.sea_estimate_decoder(shape, dec, d["Q"], d["K"], d["V"], d["omega"], A_hat, Zb, dws), n_d)
+        C = w.H * c_h
+        conv_flops = 2 * 9 * w.B * (2 * C * C * w.T * (w.Kc // c_s) // (1 if w.causal else c_s) + C * w.H * w.T * w.Kc)
+        if not w.causal:  # the second layer also runs at the reduced height; the first writes it
+            conv_flops = 2 * 9 * w.B * (2 * C * C * (w.T // c_s) * (w.Kc // c_s) + C * w.H * w.T * w.Kc)
+        if sea.sea_device_status(dws) != 0:
+            raise SystemExit("device status word set by the decoder path")
+        d_ms = sum(d_all) / n_d
+        decoder = {"head": f"d_hidden={d_hidden} c_s={c_s} c_h={c_h}: V_cat, mu, nu, 3-layer CNN over {C} channels, softmax; "
+                           "s_prob, s_mix, C_avg mixing; random-init weights; fp32 FMA kernels",
+                   "ms_per_step": d_ms, "ms_stats": ms_stats(d_all), "value": w.B * w.T / (d_ms / 1e3), "unit": "tokens/s",
+                   "gpu_launches_per_step": d_launches, "estimate_decoder_ms": ms_stats(e_all),
+                   "conv_flops": conv_flops, "conv_tflops_if_all_time_were_conv": conv_flops / (sum(e_all) / n_d / 1e3) / 1e12}
+        step()
+        torch.cuda.synchronize(dev)
+        del dws, Zb
+
     ms_per_step, e2e_ms = max_over_ranks([sum(step_ms) / args.steps, e2e_ms], dev)
     tokens = w.B * w.T * world
     elem = 2 if w.dtype == "bf16" else 4
@@ -667,6 +709,7 @@ def main():
             "grouped": grouped,
             "causal_aware": causal_aware,
             "structured_mask": structured,
+            "decoder_head": decoder,
             "roofline": sparse_roofline(w, sparse_kernel, sparse_flops, nnz, stage_ms[2], peaks, clocks),
             "roofline_estimate": hbm_roofline("favor_prep_tc / favor_state_tc / favor_scan_tc / favor_output_tc",
                                               qkv_bytes + a_hat_bytes, stage_ms[0], peaks,

@@ -191,8 +191,7 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
     float mx = -INFINITY;
     for (int b = 0; b < nb; ++b) {
       const uint32_t slot = c_s & (kSlots - 1);
-      ok = __all_sync(0xffffffffu, mbar_wait_alone(bars + 8 * slot, (c_s / kSlots) & 1));
-      if (!ok) break;  // nothing more is consumed or issued once a wait has run out
+      ok = ok && mbar_wait_alone(bars + 8 * slot, (c_s / kSlots) & 1);
       const uint32_t sbase = ring + slot * kSlotBytes;
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -213,6 +212,7 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
       ++c_s;
       pump();
     }
+    ok = __all_sync(0xffffffffu, ok);  // a wait that ran out ends the warp's work after this row's K pass
     if (!ok) break;
     mx = warp_max(mx);
 
@@ -247,8 +247,7 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
       for (int e = 0; e < 4; ++e) acc_o[i][e] = 0.f;
     for (int b = 0; b < nb; ++b) {
       const uint32_t slot = c_s & (kSlots - 1);
-      ok = __all_sync(0xffffffffu, mbar_wait_alone(bars + 8 * slot, (c_s / kSlots) & 1));
-      if (!ok) break;  // nothing more is consumed or issued once a wait has run out
+      ok = ok && mbar_wait_alone(bars + 8 * slot, (c_s / kSlots) & 1);
       const uint32_t sbase = ring + slot * kSlotBytes;
       const uint2 pa = pairs[8 * b + t];      // positions 16b+2t, 16b+2t+1
       const uint2 pb = pairs[8 * b + 4 + t];  // positions 16b+8+2t, 16b+9+2t
@@ -263,6 +262,7 @@ sparse_attn_blocks_tma_kernel(const __grid_constant__ CUtensorMap map_k, const _
       ++c_s;
       pump();
     }
+    ok = __all_sync(0xffffffffu, ok);
     if (!ok) break;
     // every lane of a quad holds the same sums; lane t writes tile t: dims 16t + g and 16t + 8 + g
     {
