@@ -362,12 +362,21 @@ def test_host_entry_point_matches_device_entry_point(B, H):
 # (one sea_attention call).  The oracle checks a sample of heads element by element (all heads
 # for the tiny case); properties that hold at any size are checked over every row on the device.
 # ---------------------------------------------------------------------------------------
+def sampled_heads(w, n, seed):
+    """The first and the last head and n - 2 more drawn with a seed (distinct)."""
+    g = np.random.default_rng(seed)
+    picks = {(0, 0), (w.B - 1, w.H - 1)}
+    while len(picks) < min(n, w.B * w.H):
+        picks.add((int(g.integers(0, w.B)), int(g.integers(0, w.H))))
+    return sorted(picks)
+
+
 FULL = [
     ("tiny_f32", "all"),
-    ("bert_base", [(0, 0), (13, 5), (31, 11)]),
-    ("opt_125m", [(0, 0), (7, 11)]),
-    ("opt_1p3b", [(0, 0), (2, 17), (3, 31)]),
-    ("long_8k", [(0, 9)]),
+    ("bert_base", 12),
+    ("opt_125m", 8),
+    ("opt_1p3b", 12),
+    ("long_8k", 3),
 ]
 
 
@@ -383,6 +392,8 @@ def test_benchmark_workloads_full_size(name, heads):
         assert nnz == w.rows * w.k_hat * w.r  # the paper's constant T*k non-zeros per head
     if heads == "all":
         heads = [(b, h) for b in range(w.B) for h in range(w.H)]
+    else:
+        heads = sampled_heads(w, heads, seed=len(name))
     for b, h in heads:
         check_head_against_oracle(run, b, h, check_estimate=w.m > 0)
 
