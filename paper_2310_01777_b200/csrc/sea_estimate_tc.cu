@@ -221,31 +221,39 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   const uint32_t tmem = *tmem_slot;
 
   if (warp == kRowWarps) {
-    if (lane == 0) {
-      // ------------------------------------------------------------ copies and MMAs
+    {
+      // ------------------------------------------------------------ copies and MMAs: the whole warp
+      // walks the phases (so that descriptors stay in uniform registers), one elected lane issues
+      const bool leader = elect_one();
       bool ok = true;
-      mbar_expect_tx(bar(kS_Load), 2 * kTileBytes + 2 * MP * 128);
-      tma_load_3d(smem_u32(sK), &map_k, 0, chunk * kRows, bh, bar(kS_Load));
-      tma_load_3d(smem_u32(sV), &map_v, 0, chunk * kRows, bh, bar(kS_Load));
-      tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kS_Load));
-      tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kS_Load));
-      ok = mbar_wait(bar(kS_Load), 0, abort_flag);
+      if (leader) {
+        mbar_expect_tx(bar(kS_Load), 2 * kTileBytes + 2 * MP * 128);
+        tma_load_3d(smem_u32(sK), &map_k, 0, chunk * kRows, bh, bar(kS_Load));
+        tma_load_3d(smem_u32(sV), &map_v, 0, chunk * kRows, bh, bar(kS_Load));
+        tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kS_Load));
+        tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kS_Load));
+      }
+      __syncwarp();
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(kS_Load), 0, abort_flag));
       if (ok) {
         fence_after();
         // E = K omega'^T (head, then remainder of omega'), contraction over d in four steps
         const uint64_t dk = smem_desc(smem_u32(sK), 16, 1024);
         const uint64_t doh = smem_desc(smem_u32(sOm), 16, 1024), dol = smem_desc(smem_u32(sOm) + kTileBytes, 16, 1024);
         constexpr uint32_t idE = idesc_bf16(MP, false, false);
+        if (leader) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) mma_ss(tmem + kColE, dk + 2 * k, doh + 2 * k, idE, k > 0);
+          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColE, dk + 2 * k, doh + 2 * k, idE, k > 0);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) mma_ss(tmem + kColE, dk + 2 * k, dol + 2 * k, idE, 1);
-        mma_commit(bar(kS_E));
-        ok = mbar_wait(bar(kS_Phi), 0, abort_flag);
+          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColE, dk + 2 * k, dol + 2 * k, idE, 1);
+          mma_commit(bar(kS_E));
+        }
+        __syncwarp();
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kS_Phi), 0, abort_flag));
       }
       if (ok) {
         fence_after();
-        if (p.causal) {
+        if (p.causal && leader) {
           // the output kernel needs phi(K) of its own chunk again: keep the tiles (head atoms, remainder atoms)
           constexpr int kAtoms = MP > 64 ? 2 : 1;
           const int slice0 = (bh * p.nchunk + chunk) * 2 * kAtoms;
@@ -258,22 +266,26 @@ favor_state_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
         // tile of ones read MN-major; contraction over the 128 keys in eight steps
         constexpr uint32_t idS = idesc_bf16(64, true, true), idZ = idesc_bf16(16, true, true);
         const uint64_t dones = smem_desc(smem_u32(sOnes), 2048, 1024);
+        const uint64_t ah0 = smem_desc(smem_u32(sPhi), kTileBytes, 1024), al0 = smem_desc(smem_u32(sPhi) + 2 * kTileBytes, kTileBytes, 1024);
+        const uint64_t bv0 = smem_desc(smem_u32(sV), kTileBytes, 1024);
+        if (leader) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint64_t ah = smem_desc(smem_u32(sPhi) + 2048 * k, kTileBytes, 1024);
-          const uint64_t al = smem_desc(smem_u32(sPhi) + 2 * kTileBytes + 2048 * k, kTileBytes, 1024);
-          const uint64_t bv = smem_desc(smem_u32(sV) + 2048 * k, kTileBytes, 1024);
-          mma_ss(tmem + kColS, ah, bv, idS, k > 0);
-          mma_ss(tmem + kColS, al, bv, idS, 1);
-          mma_ss(tmem + kColZ, ah, dones, idZ, k > 0);
-          mma_ss(tmem + kColZ, al, dones, idZ, 1);
+          for (int k = 0; k < 8; ++k) {  // a step of 16 keys: 2048 bytes = 128 descriptor units
+            mma_ss(tmem + kColS, ah0 + 128 * k, bv0 + 128 * k, idS, k > 0);
+            mma_ss(tmem + kColS, al0 + 128 * k, bv0 + 128 * k, idS, 1);
+            mma_ss(tmem + kColZ, ah0 + 128 * k, dones, idZ, k > 0);
+            mma_ss(tmem + kColZ, al0 + 128 * k, dones, idZ, 1);
+          }
+          mma_commit(bar(kS_S));
         }
-        mma_commit(bar(kS_S));
+        __syncwarp();
       }
-      mma_commit(bar(kS_Drain));
+      if (leader) mma_commit(bar(kS_Drain));
+      __syncwarp();
       mbar_wait(bar(kS_Drain), 0, abort_flag);
       mbar_wait_drain(bar(kS_Load), 0);  // the copies have landed before the CTA may leave
-      bulk_wait_all();                   // and the stored tiles have left shared memory
+      if (leader) bulk_wait_all();       // and the stored tiles have left shared memory
+      __syncwarp();
     }
   } else {
     // -------------------------------------------------------------- row warps
@@ -525,14 +537,18 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     }
   } else if (warp >= kRowWarps) {
     reg_dec<kRegsOutCtl>();
-    if (warp == kRowWarps && lane == 0) {
-      // ------------------------------------------------------------ copies and MMAs
+    if (warp == kRowWarps) {
+      // ------------------------------------------------------------ copies and MMAs: the whole warp
+      // walks the phases (so that descriptors and counters stay in uniform registers), one elected
+      // lane issues the copies, the MMAs and their commits
+      const bool leader = elect_one();
       bool ok = true;
       uint32_t it = 0;          // items done: parity of the per-item barriers
       uint32_t g = 0;           // decoder passes issued so far: pass g uses buffers g & 1
       uint32_t w_next = 0;      // decoder passes whose columns have been requested
       uint32_t afree_next = 0;  // decoder passes whose tile the rows are known to have read
       auto load_qk = [&](int item) {
+        if (!leader) return;
         const int bh = item / p.nchunk, chunk = item - bh * p.nchunk;
         mbar_expect_tx(bar(kO_QK), kTileBytes);
         tma_load_3d(smem_u32(sQ), &map_q, 0, chunk * kRows, bh, bar(kO_QK));
@@ -540,6 +556,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       // phi(K) of the item's chunk, as the state kernel left it: head atoms, remainder atoms
       constexpr int kAtoms = MP > 64 ? 2 : 1;
       auto load_phik = [&](int item) {
+        if (!leader) return;
         mbar_expect_tx(bar(kO_PhiK), 2 * kAtoms * kTileBytes);
         for (int part = 0; part < 2; ++part)
           for (int a = 0; a < kAtoms; ++a)
@@ -547,6 +564,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         item * 2 * kAtoms + part * kAtoms + a, bar(kO_PhiK));
       };
       auto load_vs = [&](int item) {
+        if (!leader) return;
         const int bh = item / p.nchunk, chunk = item - bh * p.nchunk;
         const bool prefix = !causal || chunk > 0;
         const int state_idx = (bh * p.nchunk + (causal ? chunk : 0)) * 2;
@@ -562,26 +580,31 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       auto load_w = [&](int ct) {
         const int b = w_next & 1;
         const uint32_t dst = smem_u32(sPhi) + b * 2 * kTileBytes;
-        mbar_expect_tx(bar(kO_W + b), 4 * 8192);
-        for (int part = 0; part < 2; ++part)
-          for (int atom = 0; atom < 2; ++atom)
-            tma_load_3d(dst + part * kTileBytes + atom * 8192, &map_w, ct * kWTile + 64 * atom, 0, part, bar(kO_W + b));
+        if (leader) {
+          mbar_expect_tx(bar(kO_W + b), 4 * 8192);
+          for (int part = 0; part < 2; ++part)
+            for (int atom = 0; atom < 2; ++atom)
+              tma_load_3d(dst + part * kTileBytes + atom * 8192, &map_w, ct * kWTile + 64 * atom, 0, part, bar(kO_W + b));
+        }
         ++w_next;
       };
       auto wait_afree_upto = [&](uint32_t upto) {  // the rows have read the tiles of passes 0 .. upto-1
         while (ok && afree_next < upto) {
-          ok = mbar_wait(bar(kO_AFree + (afree_next & 1)), (afree_next >> 1) & 1, abort_flag);
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_AFree + (afree_next & 1)), (afree_next >> 1) & 1, abort_flag));
           ++afree_next;
         }
       };
       const int first = blockIdx.x;
       if (first < n_items) {
-        mbar_expect_tx(bar(kO_Om), 2 * MP * 128);
-        tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kO_Om));
-        tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kO_Om));
+        if (leader) {
+          mbar_expect_tx(bar(kO_Om), 2 * MP * 128);
+          tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kO_Om));
+          tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kO_Om));
+        }
         load_qk(first);
         load_vs(first);
-        ok = mbar_wait(bar(kO_Om), 0, abort_flag);
+        __syncwarp();
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Om), 0, abort_flag));
       }
       const uint64_t doh = smem_desc(smem_u32(sOm), 16, 1024), dol = smem_desc(smem_u32(sOm) + kTileBytes, 16, 1024);
       for (int item = first; item < n_items && ok; item += gridDim.x, ++it) {
@@ -589,62 +612,70 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         const bool has_prefix = !causal || chunk > 0;
         const int next = item + gridDim.x;
         const uint32_t par = it & 1;
-        ok = mbar_wait(bar(kO_QK), par, abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_QK), par, abort_flag));
         // the projections go where the previous item's A_hat tiles were, and phi(K) where its decoder
         // columns were: the rows have read the former (which also means the MMAs that read the
         // latter are complete); with a tile region of its own only the MMAs matter
         if (!single) wait_afree_upto(g);
-        else if (ok && g > 0) ok = mbar_wait(bar(kO_WDone + ((g - 1) & 1)), ((g - 1) >> 1) & 1, abort_flag);
+        else if (ok && g > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_WDone + ((g - 1) & 1)), ((g - 1) >> 1) & 1, abort_flag));
         if (!ok) break;
         fence_after();
         if (causal) load_phik(item);
         {
           constexpr uint32_t idE = idesc_bf16(MP, false, false);
           const uint64_t dq = smem_desc(smem_u32(sQ), 16, 1024);
+          if (leader) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, doh + 2 * k, idE, k > 0);
+            for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, doh + 2 * k, idE, k > 0);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, dol + 2 * k, idE, 1);
-          mma_commit(bar(kO_E));
+            for (int k = 0; k < 4; ++k) mma_ss(tmem + kColQ, dq + 2 * k, dol + 2 * k, idE, 1);
+            mma_commit(bar(kO_E));
+          }
+          __syncwarp();
         }
-        ok = mbar_wait(bar(kO_Phi), par, abort_flag);
-        if (ok) ok = mbar_wait(bar(kO_VS), par, abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Phi), par, abort_flag));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_VS), par, abort_flag));
         if (!ok) break;
         fence_after();
         // the rows have read the projections, so the Q tile is free for the next item
         if (next < n_items) load_qk(next);
         if (causal) {
-          ok = mbar_wait(bar(kO_PhiK), par, abort_flag);
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_PhiK), par, abort_flag));
           if (!ok) break;
           // in-chunk kernel matrix phi(Q) phi(K)^T: A = phi(Q) in tensor memory, B = phi(K) K-major
           constexpr uint32_t idA = idesc_bf16(128, false, false);
+          const uint64_t bh0 = smem_desc(smem_u32(sPhi), 16, 1024), bl0 = smem_desc(smem_u32(sPhi) + 2 * kTileBytes, 16, 1024);
+          if (leader) {
 #pragma unroll
-          for (int k = 0; k < MP / 16; ++k) {
-            const uint32_t off = (k >> 2) * kTileBytes + (k & 3) * 32;
-            const uint64_t bh_ = smem_desc(smem_u32(sPhi) + off, 16, 1024);
-            const uint64_t bl_ = smem_desc(smem_u32(sPhi) + 2 * kTileBytes + off, 16, 1024);
-            const uint32_t a = tmem + kColQ + a_col(k);
-            mma_ts(tmem + kColA, a, bh_, idA, k > 0);
-            mma_ts(tmem + kColA, a, bl_, idA, 1);
-            mma_ts(tmem + kColA, a + 16, bh_, idA, 1);
+            for (int k = 0; k < MP / 16; ++k) {
+              constexpr int kUnitsPerTile = kTileBytes / 16;
+              const uint32_t off = (k >> 2) * kUnitsPerTile + (k & 3) * 2;  // descriptor units of 16 bytes
+              const uint32_t a = tmem + kColQ + a_col(k);
+              mma_ts(tmem + kColA, a, bh0 + off, idA, k > 0);
+              mma_ts(tmem + kColA, a, bl0 + off, idA, 1);
+              mma_ts(tmem + kColA, a + 16, bh0 + off, idA, 1);
+            }
+            mma_commit(bar(kO_A));
           }
-          mma_commit(bar(kO_A));
+          __syncwarp();
         }
         if (has_prefix) {
           // phi(Q) S: B = the state read MN-major (16 features = 2048 bytes per step)
           constexpr uint32_t idN = idesc_bf16(64, false, true);
+          const uint64_t sh0 = smem_desc(smem_u32(sS), kTileBytes, 1024), sl0 = smem_desc(smem_u32(sS) + kTileBytes, kTileBytes, 1024);
+          if (leader) {
 #pragma unroll
-          for (int k = 0; k < MP / 16; ++k) {
-            const uint64_t bh_ = smem_desc(smem_u32(sS) + 2048 * k, kTileBytes, 1024);
-            const uint64_t bl_ = smem_desc(smem_u32(sS) + kTileBytes + 2048 * k, kTileBytes, 1024);
-            const uint32_t a = tmem + kColQ + a_col(k);
-            mma_ts(tmem + kColNum, a, bh_, idN, k > 0);
-            mma_ts(tmem + kColNum, a, bl_, idN, 1);
-            mma_ts(tmem + kColNum, a + 16, bh_, idN, 1);
+            for (int k = 0; k < MP / 16; ++k) {  // a step of 16 features: 2048 bytes = 128 descriptor units
+              const uint32_t a = tmem + kColQ + a_col(k);
+              mma_ts(tmem + kColNum, a, sh0 + 128 * k, idN, k > 0);
+              mma_ts(tmem + kColNum, a, sl0 + 128 * k, idN, 1);
+              mma_ts(tmem + kColNum, a + 16, sh0 + 128 * k, idN, 1);
+            }
           }
+          __syncwarp();
         }
         if (causal) {
-          ok = mbar_wait(bar(kO_P), par, abort_flag);
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_P), par, abort_flag));
           if (!ok) break;
           fence_after();
         }
@@ -654,16 +685,20 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         if (n_ct > 1) load_w(1);
         if (causal) {
           constexpr uint32_t idN = idesc_bf16(64, false, true);
+          const uint64_t bv0 = smem_desc(smem_u32(sV), kTileBytes, 1024);
+          if (leader) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint64_t bv = smem_desc(smem_u32(sV) + 2048 * k, kTileBytes, 1024);
-            const uint32_t a = tmem + kColA + a_col(k);
-            mma_ts(tmem + kColNum, a, bv, idN, (has_prefix || k > 0) ? 1u : 0u);
-            mma_ts(tmem + kColNum, a + 16, bv, idN, 1);
+            for (int k = 0; k < 8; ++k) {
+              const uint32_t a = tmem + kColA + a_col(k);
+              mma_ts(tmem + kColNum, a, bv0 + 128 * k, idN, (has_prefix || k > 0) ? 1u : 0u);
+              mma_ts(tmem + kColNum, a + 16, bv0 + 128 * k, idN, 1);
+            }
           }
+          __syncwarp();
         }
-        mma_commit(bar(kO_Num));
-        ok = mbar_wait(bar(kO_C), par, abort_flag);
+        if (leader) mma_commit(bar(kO_Num));
+        __syncwarp();
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_C), par, abort_flag));
         if (!ok) break;
         fence_after();
         // numerator complete and read: V, the state and its normaliser are free for the next item
@@ -672,7 +707,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         constexpr uint32_t idW = idesc_bf16(kWTile, false, true);
         for (int ct = 0; ct < n_ct && ok; ++ct, ++g) {
           const uint32_t b = g & 1;
-          ok = mbar_wait(bar(kO_W + b), (g >> 1) & 1, abort_flag);
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_W + b), (g >> 1) & 1, abort_flag));
           // the rows have read the tile that was in this buffer
           if (single) wait_afree_upto(g);
           else if (g >= 2) wait_afree_upto(g - 1);
@@ -680,25 +715,28 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           fence_after();
           const uint32_t wbase = smem_u32(sPhi) + b * 2 * kTileBytes;
           const uint32_t d = tmem + (single ? kColAh : (b ? kColA : kColQ));
+          const uint64_t wh0 = smem_desc(wbase, 8192, 1024), wl0 = smem_desc(wbase + kTileBytes, 8192, 1024);
+          if (leader) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const uint64_t wh = smem_desc(wbase + 2048 * k, 8192, 1024);
-            const uint64_t wl = smem_desc(wbase + kTileBytes + 2048 * k, 8192, 1024);
-            const uint32_t a = tmem + kColC + a_col(k);
-            mma_ts(d, a, wh, idW, k > 0);
-            mma_ts(d, a, wl, idW, 1);
-            mma_ts(d, a + 16, wh, idW, 1);
+            for (int k = 0; k < 4; ++k) {
+              const uint32_t a = tmem + kColC + a_col(k);
+              mma_ts(d, a, wh0 + 128 * k, idW, k > 0);
+              mma_ts(d, a, wl0 + 128 * k, idW, 1);
+              mma_ts(d, a + 16, wh0 + 128 * k, idW, 1);
+            }
+            mma_commit(bar(kO_Ahat + b));
+            mma_commit(bar(kO_WDone + b));
           }
-          mma_commit(bar(kO_Ahat + b));
-          mma_commit(bar(kO_WDone + b));
+          __syncwarp();
           if (ct >= 1 && ct + 1 < n_ct) {
             // columns of the next pass go where the previous pass read from
-            ok = mbar_wait(bar(kO_WDone + (b ^ 1)), ((g - 1) >> 1) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_WDone + (b ^ 1)), ((g - 1) >> 1) & 1, abort_flag));
             if (ok) load_w(ct + 1);
           }
         }
       }
-      mma_commit(bar(kO_Drain));
+      if (leader) mma_commit(bar(kO_Drain));
+      __syncwarp();
       mbar_wait(bar(kO_Drain), 0, abort_flag);
       // copies still in flight must land before the CTA may leave (only after a wait ran out can
       // any be outstanding here: every armed phase is waited for in the loop above)
