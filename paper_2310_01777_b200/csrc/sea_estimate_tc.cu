@@ -76,6 +76,23 @@ __global__ void favor_prep_tc_kernel(const float* __restrict__ omega, const floa
 }
 
 // ---- pieces shared by the two chunk kernels ----------------------------------------------------
+// |u|^2 / 16 = |x|^2 / 2 of row r of a [128][64] bf16 tile staged by a tiled copy with the
+// 128-byte swizzle (16-byte piece j of row r sits at piece j ^ (r & 7) of the row's 128 bytes).
+__device__ __forceinline__ float half_sq_norm_swizzled(const unsigned char* tile, int r) {
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint4 t = *reinterpret_cast<const uint4*>(tile + r * 128 + ((i ^ (r & 7)) << 4));
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xffff0000u);
+      s = fmaf(lo, lo, fmaf(hi, hi, s));
+    }
+  }
+  return s * (1.f / 16.f);
+}
+
 // |u|^2 / 16 = |x|^2 / 2 of one row of a bf16 [.][64] matrix.
 __device__ __forceinline__ float half_sq_norm(const __nv_bfloat16* row) {
   float s = 0.f;
@@ -154,7 +171,8 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
                ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory"); }
+template <int kPending = 0>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;\n" ::"n"(kPending) : "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory"); }
 struct EstParams {
   const __nv_bfloat16 *Q, *K;   // for the rows' norms
@@ -426,8 +444,8 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   unsigned char* sOm = sV + kTileBytes;                // head, remainder: 32 KB
   unsigned char* sS = sOm + 2 * kTileBytes;            // prefix state head, remainder [MP][64]: 32 KB
   unsigned char* sPhi = sS + 2 * kTileBytes;           // phi(K) head 32 KB, remainder 32 KB; later the decoder columns
-  unsigned char* sOut = sPhi + 4 * kTileBytes;         // kParts boxes of 128 rows x 32 fp32 on their way to A_hat
-  unsigned char* tail = sOut + kParts * kTileBytes;
+  unsigned char* sOut = sPhi + 4 * kTileBytes;         // four boxes of 128 rows x 32 fp32 (a pass's column groups) bound for A_hat
+  unsigned char* tail = sOut + 4 * kTileBytes;
   const uint32_t bars = smem_u32(tail);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * kO_NumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8 * kO_NumBars + 4);
@@ -754,7 +772,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     const int quarter = warp & 3, part = warp >> 2, rt = quarter * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     const bool elected = quarter == 0 && lane == 0;  // issues this column group's stores
-    unsigned char* my_box = sOut + part * kTileBytes;
+    unsigned char* my_boxes = sOut + part * (4 / kParts) * kTileBytes;  // one box per column group of a pass
     uint32_t it = 0, g = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
@@ -764,7 +782,10 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       const int row = chunk * kRows + rt;
       const bool row_ok = row < p.T;
       const size_t grow = (size_t)bh * p.T + row;
-      const float bias_q = feature_bias(row_ok ? half_sq_norm(p.Q + grow * kHeadDim) : 0.f, row_ok, p.m);
+      // the row's norm from the staged Q tile (the control warp refills it only after every row
+      // warp has arrived at kO_Phi below); rows past T are zero-filled by the copy
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_QK), par, abort_flag));
+      const float bias_q = feature_bias(ok ? half_sq_norm_swizzled(sQ, rt) : 0.f, row_ok, p.m);
       float den = 0.f;
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_E), par, abort_flag));
       if (ok && has_prefix) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_VS), par, abort_flag));  // z has landed
@@ -860,7 +881,8 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           if (p.tma_store) {
             // the column group's box: wait until its previous store has been read out, fill it
             // (128-byte rows, swizzled like the copy expects), hand it to the copy engine
-            if (elected) bulk_wait_read();
+            unsigned char* my_box = my_boxes + cc * kTileBytes;
+            if (elected) bulk_wait_read<kMine - 1>();  // every group but the last kMine - 1: this box's among them
             part_sync(2 + part);
             if (ok) {
 #pragma unroll
@@ -870,8 +892,8 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             }
             fence_async_smem();
             part_sync(2 + part);
-            if (elected && ok && col0 < p.Kc) {
-              tma_store_3d(&map_a, smem_u32(my_box), col0, chunk * kRows, bh);
+            if (elected) {  // one group per box and pass, stored or not, so that the count above holds
+              if (ok && col0 < p.Kc) tma_store_3d(&map_a, smem_u32(my_box), col0, chunk * kRows, bh);
               bulk_commit();
             }
           } else if (ok && row_ok) {
@@ -959,7 +981,7 @@ sea_status launch_mp(const sea_shape& s, const __nv_bfloat16* Q, const __nv_bflo
   }
 
   const size_t smem1 = 1024 + 5 * kTileBytes + 2048 + 8 * kS_NumBars + 16;
-  const size_t smem3 = 1024 + (10 + kParts) * kTileBytes + (8 * kO_NumBars + 8 + 127) / 128 * 128 + (1 + kParts) * 128 * 4;
+  const size_t smem3 = 1024 + (10 + 4) * kTileBytes + (8 * kO_NumBars + 8 + 127) / 128 * 128 + (1 + kParts) * 128 * 4;
   if (cudaFuncSetAttribute(favor_state_tc_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess)
     return SEA_ERR_CUDA;
   const dim3 grid(nchunk, BH);
