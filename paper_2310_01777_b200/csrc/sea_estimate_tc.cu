@@ -171,8 +171,7 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
                ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
-template <int kPending = 0>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;\n" ::"n"(kPending) : "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory"); }
 struct EstParams {
   const __nv_bfloat16 *Q, *K;   // for the rows' norms
@@ -419,7 +418,10 @@ enum {
   kO_QK,                   // the item's Q tile
   kO_PhiK,                 // the item's phi(K) tiles (causal)
   kO_VS,                   // the item's V tile, prefix state and its normaliser
-  kO_E, kO_Phi, kO_A, kO_P, kO_Num, kO_C,
+  kO_E,
+  kO_Phi,                  // phi(Q): every row warp has written its first chunk of features ...
+  kO_Phi2,                 // ... and all of them
+  kO_A, kO_P, kO_Num, kO_C,
   kO_W,                    // [2] decoder columns staged
   kO_WDone = kO_W + 2,     // [2] the MMAs that read them are complete
   kO_Ahat = kO_WDone + 2,  // [2] A_hat tile in tensor memory
@@ -468,7 +470,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   const int n_items = p.BH * p.nchunk;
   if (tid == 0) {
     for (int i = 0; i < kO_NumBars; ++i) {
-      const bool from_rows = i == kO_Phi || i == kO_P || i == kO_C;
+      const bool from_rows = i == kO_Phi || i == kO_Phi2 || i == kO_P || i == kO_C;
       const bool tile_read = i >= kO_AFree && i < kO_AFree + 2;  // the rows, and the selecting warps
       mbar_init(bar(i), tile_read ? (keep_a ? kRowWarps : 0) + (selecting ? 4 : 0) : (from_rows ? kRowWarps : 1));
     }
@@ -651,47 +653,61 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           }
           __syncwarp();
         }
+        // The contractions over the features start once every row warp has written its first chunk
+        // (features 0 .. 32 kParts - 1: steps 0 .. kStep1 - 1) and go on when all are there.
+        constexpr int kSteps = MP / 16, kStep1 = kSteps < 2 * kParts ? kSteps : 2 * kParts;
+        constexpr uint32_t idA = idesc_bf16(128, false, false);
+        constexpr uint32_t idS = idesc_bf16(64, false, true);
+        const uint64_t bh0 = smem_desc(smem_u32(sPhi), 16, 1024), bl0 = smem_desc(smem_u32(sPhi) + 2 * kTileBytes, 16, 1024);
+        const uint64_t sh0 = smem_desc(smem_u32(sS), kTileBytes, 1024), sl0 = smem_desc(smem_u32(sS) + kTileBytes, kTileBytes, 1024);
+        // in-chunk kernel matrix phi(Q) phi(K)^T: A = phi(Q) in tensor memory, B = phi(K) K-major
+        auto mma_kernel_matrix = [&](int k_lo, int k_hi) {
+          if (!leader) return;
+#pragma unroll
+          for (int k = k_lo; k < k_hi; ++k) {
+            constexpr int kUnitsPerTile = kTileBytes / 16;
+            const uint32_t off = (k >> 2) * kUnitsPerTile + (k & 3) * 2;  // descriptor units of 16 bytes
+            const uint32_t a = tmem + kColQ + a_col(k);
+            mma_ts(tmem + kColA, a, bh0 + off, idA, k > 0);
+            mma_ts(tmem + kColA, a, bl0 + off, idA, 1);
+            mma_ts(tmem + kColA, a + 16, bh0 + off, idA, 1);
+          }
+        };
+        // phi(Q) S: B = the state read MN-major (16 features = 2048 bytes = 128 descriptor units per step)
+        auto mma_prefix = [&](int k_lo, int k_hi) {
+          if (!leader) return;
+#pragma unroll
+          for (int k = k_lo; k < k_hi; ++k) {
+            const uint32_t a = tmem + kColQ + a_col(k);
+            mma_ts(tmem + kColNum, a, sh0 + 128 * k, idS, k > 0);
+            mma_ts(tmem + kColNum, a, sl0 + 128 * k, idS, 1);
+            mma_ts(tmem + kColNum, a + 16, sh0 + 128 * k, idS, 1);
+          }
+        };
         ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Phi), par, abort_flag));
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_VS), par, abort_flag));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(causal ? kO_PhiK : kO_VS), par, abort_flag));
         if (!ok) break;
         fence_after();
-        // the rows have read the projections, so the Q tile is free for the next item
+        if (causal) mma_kernel_matrix(0, kStep1);
+        else mma_prefix(0, kStep1);  // not causal: every item has a prefix (the total)
+        __syncwarp();
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Phi2), par, abort_flag));
+        if (!ok) break;
+        fence_after();
+        // the rows have read the projections (and the Q tile, for their norms): it is free for the next item
         if (next < n_items) load_qk(next);
         if (causal) {
-          ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_PhiK), par, abort_flag));
+          mma_kernel_matrix(kStep1, kSteps);
+          if (leader) mma_commit(bar(kO_A));
+          __syncwarp();
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_VS), par, abort_flag));
           if (!ok) break;
-          // in-chunk kernel matrix phi(Q) phi(K)^T: A = phi(Q) in tensor memory, B = phi(K) K-major
-          constexpr uint32_t idA = idesc_bf16(128, false, false);
-          const uint64_t bh0 = smem_desc(smem_u32(sPhi), 16, 1024), bl0 = smem_desc(smem_u32(sPhi) + 2 * kTileBytes, 16, 1024);
-          if (leader) {
-#pragma unroll
-            for (int k = 0; k < MP / 16; ++k) {
-              constexpr int kUnitsPerTile = kTileBytes / 16;
-              const uint32_t off = (k >> 2) * kUnitsPerTile + (k & 3) * 2;  // descriptor units of 16 bytes
-              const uint32_t a = tmem + kColQ + a_col(k);
-              mma_ts(tmem + kColA, a, bh0 + off, idA, k > 0);
-              mma_ts(tmem + kColA, a, bl0 + off, idA, 1);
-              mma_ts(tmem + kColA, a + 16, bh0 + off, idA, 1);
-            }
-            mma_commit(bar(kO_A));
-          }
-          __syncwarp();
+          fence_after();
+          if (has_prefix) mma_prefix(0, kSteps);
+        } else {
+          mma_prefix(kStep1, kSteps);
         }
-        if (has_prefix) {
-          // phi(Q) S: B = the state read MN-major (16 features = 2048 bytes per step)
-          constexpr uint32_t idN = idesc_bf16(64, false, true);
-          const uint64_t sh0 = smem_desc(smem_u32(sS), kTileBytes, 1024), sl0 = smem_desc(smem_u32(sS) + kTileBytes, kTileBytes, 1024);
-          if (leader) {
-#pragma unroll
-            for (int k = 0; k < MP / 16; ++k) {  // a step of 16 features: 2048 bytes = 128 descriptor units
-              const uint32_t a = tmem + kColQ + a_col(k);
-              mma_ts(tmem + kColNum, a, sh0 + 128 * k, idN, k > 0);
-              mma_ts(tmem + kColNum, a, sl0 + 128 * k, idN, 1);
-              mma_ts(tmem + kColNum, a + 16, sh0 + 128 * k, idN, 1);
-            }
-          }
-          __syncwarp();
-        }
+        __syncwarp();
         if (causal) {
           ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_P), par, abort_flag));
           if (!ok) break;
@@ -791,6 +807,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       if (ok && has_prefix) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_VS), par, abort_flag));  // z has landed
       if (ok) {
         fence_after();
+        bool first_chunk = true;
         for (int c = part; c < MP / 32; c += kParts) {
           uint32_t e[32];
           float phi[32];
@@ -807,9 +824,15 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           split32(phi, hi, lo);
           tmem_st16(lane_addr + kColQ + 32 * c, hi);
           tmem_st16(lane_addr + kColQ + 32 * c + 16, lo);
+          if (first_chunk) {  // the contractions may start on the first 32 kParts features
+            tmem_st_wait();
+            warp_arrive(bar(kO_Phi), lane);
+            first_chunk = false;
+          }
         }
+        if (first_chunk) warp_arrive(bar(kO_Phi), lane);  // no chunk of its own
         tmem_st_wait();
-        warp_arrive(bar(kO_Phi), lane);
+        warp_arrive(bar(kO_Phi2), lane);
         if (causal) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_A), par, abort_flag));
       }
       if (ok && causal) {
@@ -875,28 +898,33 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           tmem_ld_wait();
           warp_arrive(bar(kO_AFree + b), lane);
         }
+        if (p.tma_store) {
+          // the column groups' boxes: wait until their previous stores have been read out, fill them
+          // (128-byte rows, swizzled like the copy expects), hand them to the copy engine
+          if (elected) bulk_wait_read();
+          part_sync(2 + part);
+          if (ok) {
 #pragma unroll
-        for (int cc = 0; cc < kMine; ++cc) {
-          const int col0 = ct * kWTile + 32 * (part + kParts * cc);
-          if (p.tma_store) {
-            // the column group's box: wait until its previous store has been read out, fill it
-            // (128-byte rows, swizzled like the copy expects), hand it to the copy engine
-            unsigned char* my_box = my_boxes + cc * kTileBytes;
-            if (elected) bulk_wait_read<kMine - 1>();  // every group but the last kMine - 1: this box's among them
-            part_sync(2 + part);
-            if (ok) {
+            for (int cc = 0; cc < kMine; ++cc)
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<uint4*>(my_box + rt * 128 + ((j ^ (rt & 7)) << 4)) =
+                *reinterpret_cast<uint4*>(my_boxes + cc * kTileBytes + rt * 128 + ((j ^ (rt & 7)) << 4)) =
                     make_uint4(e[cc][4 * j], e[cc][4 * j + 1], e[cc][4 * j + 2], e[cc][4 * j + 3]);
+          }
+          fence_async_smem();
+          part_sync(2 + part);
+          if (elected && ok) {
+#pragma unroll
+            for (int cc = 0; cc < kMine; ++cc) {
+              const int col0 = ct * kWTile + 32 * (part + kParts * cc);
+              if (col0 < p.Kc) tma_store_3d(&map_a, smem_u32(my_boxes + cc * kTileBytes), col0, chunk * kRows, bh);
             }
-            fence_async_smem();
-            part_sync(2 + part);
-            if (elected) {  // one group per box and pass, stored or not, so that the count above holds
-              if (ok && col0 < p.Kc) tma_store_3d(&map_a, smem_u32(my_box), col0, chunk * kRows, bh);
-              bulk_commit();
-            }
-          } else if (ok && row_ok) {
+            bulk_commit();
+          }
+        } else if (ok && row_ok) {
+#pragma unroll
+          for (int cc = 0; cc < kMine; ++cc) {
+            const int col0 = ct * kWTile + 32 * (part + kParts * cc);
 #pragma unroll
             for (int i = 0; i < 32; ++i)
               if (col0 + i < p.Kc) out[col0 + i] = __uint_as_float(e[cc][i]);
