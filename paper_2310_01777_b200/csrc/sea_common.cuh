@@ -156,8 +156,17 @@ sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void*
 // The paper's estimator head and output mixing (sea_decoder.cu).  dws: the decoder's own part of
 // the workspace (decoder_layout), est_state / est_split: the estimator's scratch of the base layout.
 struct DecoderLayout {
-  size_t ident, first, c_first, c_value, z, hidden, image, conv_a, conv_b, s_prob, s_mix, c_avg, total;
+  size_t ident, first, c_first, c_value, z, hidden, image, conv_a, conv_b, s_prob, s_mix, c_avg;
+  size_t act0, w_tiles;  // tensor-core form of the convolutions only: the image as bf16 planes, the layers' weight tiles
+  size_t total;
 };
+// Tensor-core form of a 3 x 3 convolution layer (sea_conv_tc.cu).
+bool conv_tc_shape_ok(int c_in, int c_out, int h_in, int w_in, int up_h, int up_w, int stride_h);
+size_t conv_tc_weight_bytes(int c_in, int c_out, int up_h, int up_w);
+sea_status launch_nchw_to_nhwc_split(const float* in, void* out, int batch, int C, int h, int w, cudaStream_t st);
+sea_status launch_conv_tc(const void* act_in, int batch, int c_in, int h_in, int w_in, int up_h, int up_w, int stride_h,
+                          int pad_top, const float* w, const float* bias, int c_out, int relu, void* w_tiles, void* out_split,
+                          float* out_logits, int32_t* status, cudaStream_t st);
 DecoderLayout decoder_layout(const sea_shape& s, const sea_decoder& dec);
 sea_status launch_estimate_decoder(const sea_shape& s, const sea_decoder& dec, const void* Q, const void* K, const void* V,
                                    const float* omega, float* A_hat, float* Z, char* dws, float* est_state, void* est_split,

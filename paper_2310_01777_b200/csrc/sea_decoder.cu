@@ -285,6 +285,16 @@ sea_status linear(const float* x0, const float* x1, const T* x2, int k_in, const
 
 }  // namespace
 
+// True when all three convolutions of this shape run in the tensor-core form.
+static bool decoder_conv_tc(const sea_shape& s, const sea_decoder& dec) {
+  const int C = s.H * dec.c_h, wr = s.Kc / dec.c_s;
+  const int stride1 = s.causal ? 1 : dec.c_s;
+  const int t1 = conv_out_h(s.T, stride1);
+  if (t1 <= 0 || s.T % t1 != 0) return false;
+  return conv_tc_shape_ok(C, C, s.T, wr, 1, 1, stride1) && conv_tc_shape_ok(C, C, t1, wr, 1, 1, 1) &&
+         conv_tc_shape_ok(C, s.H, t1, wr, s.T / t1, dec.c_s, 1);
+}
+
 // Buffers of the decoder path inside its part of the workspace (all offsets 256-byte aligned).
 DecoderLayout decoder_layout(const sea_shape& s, const sea_decoder& dec) {
   DecoderLayout L{};
@@ -310,6 +320,10 @@ DecoderLayout decoder_layout(const sea_shape& s, const sea_decoder& dec) {
   L.s_prob = take(rows * sizeof(float));
   L.s_mix = take(rows * sizeof(float));
   L.c_avg = take((s.causal ? rows : (size_t)s.B * s.H) * kHeadDim * sizeof(float));
+  if (decoder_conv_tc(s, dec)) {
+    L.act0 = take((size_t)s.B * C * s.T * wr * 2 * sizeof(__nv_bfloat16));
+    L.w_tiles = take(3 * align_up(conv_tc_weight_bytes((int)C, 128, 1, 1), 256));  // 128: the most accumulator columns of a layer
+  }
   L.total = off;
   return L;
 }
@@ -356,6 +370,24 @@ static sea_status estimate_decoder_typed(const sea_shape& s, const sea_decoder& 
   const int pad_top = s.causal ? 2 : 1;
   const int stride1 = s.causal ? 1 : dec.c_s;
   const int t1 = conv_out_h(s.T, stride1);
+  if (decoder_conv_tc(s, dec)) {
+    // tensor-core form: activations as bf16 head / remainder planes, pixel-major
+    char* act0 = dws + L.act0;
+    char* wt = dws + L.w_tiles;
+    const size_t wt_step = align_up(conv_tc_weight_bytes(C, 128, 1, 1), 256);
+    if ((rc = launch_nchw_to_nhwc_split(image, act0, s.B, C, s.T, wr, st)) != SEA_OK) return rc;
+    if ((rc = launch_conv_tc(act0, s.B, C, s.T, wr, 1, 1, stride1, pad_top, dec.conv1_w, dec.conv1_b, C, 1, wt, conv_a, nullptr,
+                             status, st)) != SEA_OK)
+      return rc;
+    if ((rc = launch_conv_tc(conv_a, s.B, C, t1, wr, 1, 1, 1, pad_top, dec.conv2_w, dec.conv2_b, C, 1, wt + wt_step, conv_b, nullptr,
+                             status, st)) != SEA_OK)
+      return rc;
+    if ((rc = launch_conv_tc(conv_b, s.B, C, t1, wr, s.T / t1, dec.c_s, 1, pad_top, dec.conv3_w, dec.conv3_b, s.H, 0,
+                             wt + 2 * wt_step, nullptr, A_hat, status, st)) != SEA_OK)
+      return rc;
+    softmax_rows_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(A_hat, rows, s.Kc);
+    return check_launch();
+  }
   if ((rc = conv3x3(image, dec.conv1_w, dec.conv1_b, conv_a, s.B, C, s.T, wr, 1, 1, stride1, pad_top, C, 1, st)) != SEA_OK) return rc;
   if ((rc = conv3x3(conv_a, dec.conv2_w, dec.conv2_b, conv_b, s.B, C, t1, wr, 1, 1, 1, pad_top, C, 1, st)) != SEA_OK) return rc;
   // nearest resize to [T, Kc] folded into the last layer's reads (integer factors: T = t1 * up_h, Kc = wr * c_s)

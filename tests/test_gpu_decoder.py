@@ -109,6 +109,27 @@ def test_decoder_stages_and_fused_call_match_oracle(w):
     assert torch.equal(a.col_idx[:nnz], f.col_idx[:nnz]) and torch.equal(a.P[:nnz].view(view), f.P[:nnz].view(view))
 
 
+# Shapes whose convolutions run in the tensor-core form (H c_h a multiple of 64, image width a
+# divisor or multiple of 128): one and two blocks of input channels, both paddings, the strided
+# first layer, two and four phases of the folded resize, tiles that run past the last row.
+TC_CASES = [
+    small("dec_tc_causal", H=16, T=256, Kc=32, k_hat=4),
+    small("dec_tc_nc", causal=False, H=32, T=192, Kc=64, k_hat=6),
+    small("dec_tc_nc_ragged", causal=False, H=16, T=80, Kc=16, k_hat=3),
+    small("dec_tc_causal_ragged", H=16, T=80, Kc=16, k_hat=3, B=2),
+]
+
+
+@pytest.mark.parametrize("w", TC_CASES, ids=lambda w: w.name)
+def test_tensor_core_convolutions_match_oracle(w):
+    a = Run(w, c_h=4)
+    a.stages(); a.done()
+    assert bool(torch.isfinite(a.A_hat).all())
+    assert torch.allclose(a.A_hat.sum(-1), torch.ones_like(a.A_hat[..., 0]), atol=1e-5)
+    for b in range(w.B):
+        check_batch(a, b)
+
+
 def test_causal_decoder_on_device_does_not_look_ahead():
     w = small("dec_perturb", T=128, Kc=16)
     t = 70
