@@ -31,24 +31,27 @@ __global__ void identity64_kernel(float* __restrict__ w) {
   if (i < kHeadDim * kHeadDim) w[i] = (i / kHeadDim == i % kHeadDim) ? 1.f : 0.f;
 }
 
-// ---- y = act(x W + b) for 32 rows per block; x is the concatenation of up to three 64-wide
+// ---- y = act(x W + b) for 64 rows per block; x is the concatenation of up to three 64-wide
 // sources (two fp32, one in the io dtype) or one fp32 source of width k_in ----------------------
 // image != 0: the output row (b, h, t) of width c_h * wr goes to the image [B][H c_h][T][wr] instead
 // (entry j * wr + x -> channel h c_h + j, column x).
-constexpr int kLinRows = 32;
+// A thread: 16 rows of one output column at a time (a warp shares its rows: their inputs come
+// from shared memory as broadcasts, four values of k per load; the weights' reads run along n).
+constexpr int kLinRows = 64, kLinRowsPerThread = 16, kLinCols = 64;
 
 template <typename T>
 __global__ void __launch_bounds__(256)
 linear_kernel(const float* __restrict__ x0, const float* __restrict__ x1, const T* __restrict__ x2, int k_in,
               const float* __restrict__ W, const float* __restrict__ b, float* __restrict__ out, long long rows, int n_out,
               int relu, int image, int H, int seq_len, int c_h, int wr) {
-  extern __shared__ float xs[];  // [kLinRows][k_in]
+  extern __shared__ __align__(16) float xs[];  // [kLinRows][k_pad], k_pad = k_in rounded up to a multiple of 4
+  const int k_pad = (k_in + 3) & ~3;
   const long long row0 = (long long)blockIdx.x * kLinRows;
-  for (int i = threadIdx.x; i < kLinRows * k_in; i += blockDim.x) {
-    const int r = i / k_in, k = i - r * k_in;
+  for (int i = threadIdx.x; i < kLinRows * k_pad; i += blockDim.x) {
+    const int r = i / k_pad, k = i - r * k_pad;
     const long long row = row0 + r;
     float v = 0.f;
-    if (row < rows) {
+    if (row < rows && k < k_in) {
       if (x1 == nullptr && x2 == nullptr) v = x0[row * k_in + k];
       else if (k < kHeadDim) v = x0[row * kHeadDim + k];
       else if (k < 2 * kHeadDim) v = x1[row * kHeadDim + k - kHeadDim];
@@ -57,18 +60,29 @@ linear_kernel(const float* __restrict__ x0, const float* __restrict__ x1, const 
     xs[i] = v;
   }
   __syncthreads();
-  for (int n = threadIdx.x; n < n_out; n += blockDim.x) {
-    float acc[kLinRows];
+  const int tn = threadIdx.x % kLinCols, tr = threadIdx.x / kLinCols;
+  const float* my_x = xs + (size_t)tr * kLinRowsPerThread * k_pad;
+  for (int n = tn; n < n_out; n += kLinCols) {
+    float acc[kLinRowsPerThread];
+    const float bn = b[n];
 #pragma unroll
-    for (int r = 0; r < kLinRows; ++r) acc[r] = b[n];
-    for (int k = 0; k < k_in; ++k) {
-      const float w = __ldg(W + (size_t)k * n_out + n);
+    for (int r = 0; r < kLinRowsPerThread; ++r) acc[r] = bn;
+    for (int k = 0; k < k_pad; k += 4) {
+      float w[4];
 #pragma unroll
-      for (int r = 0; r < kLinRows; ++r) acc[r] = fmaf(xs[r * k_in + k], w, acc[r]);
+      for (int q = 0; q < 4; ++q) w[q] = (k + q < k_in) ? __ldg(W + (size_t)(k + q) * n_out + n) : 0.f;
+#pragma unroll
+      for (int r = 0; r < kLinRowsPerThread; ++r) {
+        const float4 x = *reinterpret_cast<const float4*>(my_x + r * k_pad + k);
+        acc[r] = fmaf(x.x, w[0], acc[r]);
+        acc[r] = fmaf(x.y, w[1], acc[r]);
+        acc[r] = fmaf(x.z, w[2], acc[r]);
+        acc[r] = fmaf(x.w, w[3], acc[r]);
+      }
     }
 #pragma unroll
-    for (int r = 0; r < kLinRows; ++r) {
-      const long long row = row0 + r;
+    for (int r = 0; r < kLinRowsPerThread; ++r) {
+      const long long row = row0 + tr * kLinRowsPerThread + r;
       if (row >= rows) break;
       const float y = relu ? fmaxf(acc[r], 0.f) : acc[r];
       if (!image) {
@@ -197,16 +211,26 @@ __global__ void scalers_kernel(const float* __restrict__ Z, const float* __restr
 }
 
 // ---- pooled context ---------------------------------------------------------------------------------
-// causal: running mean of V along the sequence, one thread per (head, column)
+// causal: running mean of V along the sequence.  One block per head: its 64 x 16 threads split the
+// sequence into 16 segments per column, sum their segments, take the sums of the segments before
+// theirs from shared memory and walk their segments again.
+constexpr int kMeanSegs = 16;
 template <typename T>
-__global__ void running_mean_kernel(const T* __restrict__ V, float* __restrict__ c_avg, int BH, int seq_len) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= BH * kHeadDim) return;
-  const int bh = i / kHeadDim, c = i - bh * kHeadDim;
+__global__ void __launch_bounds__(kHeadDim * kMeanSegs)
+running_mean_kernel(const T* __restrict__ V, float* __restrict__ c_avg, int seq_len) {
+  __shared__ float seg_sum[kMeanSegs][kHeadDim];
+  const int bh = blockIdx.x, c = threadIdx.x % kHeadDim, sg = threadIdx.x / kHeadDim;
+  const int seg_len = (seq_len + kMeanSegs - 1) / kMeanSegs;
+  const int t0 = min(seq_len, sg * seg_len), t1 = min(seq_len, t0 + seg_len);
   const T* v = V + (size_t)bh * seq_len * kHeadDim + c;
   float* o = c_avg + (size_t)bh * seq_len * kHeadDim + c;
   float sum = 0.f;
-  for (int t = 0; t < seq_len; ++t) {
+  for (int t = t0; t < t1; ++t) sum += Io<T>::from_io(v[(size_t)t * kHeadDim]);
+  seg_sum[sg][c] = sum;
+  __syncthreads();
+  sum = 0.f;
+  for (int q = 0; q < sg; ++q) sum += seg_sum[q][c];
+  for (int t = t0; t < t1; ++t) {
     sum += Io<T>::from_io(v[(size_t)t * kHeadDim]);
     o[(size_t)t * kHeadDim] = sum / (float)(t + 1);
   }
@@ -277,7 +301,10 @@ sea_status conv3x3(const float* in, const float* w, const float* b, float* out, 
 template <typename T>
 sea_status linear(const float* x0, const float* x1, const T* x2, int k_in, const float* W, const float* b, float* out,
                   long long rows, int n_out, int relu, int image, int H, int seq_len, int c_h, int wr, cudaStream_t st) {
-  const size_t smem = (size_t)kLinRows * k_in * sizeof(float);
+  const size_t smem = (size_t)kLinRows * ((k_in + 3) & ~3) * sizeof(float);
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(linear_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return SEA_ERR_CUDA;
   linear_kernel<T><<<(unsigned)((rows + kLinRows - 1) / kLinRows), 256, smem, st>>>(x0, x1, x2, k_in, W, b, out, rows, n_out,
                                                                                    relu, image, H, seq_len, c_h, wr);
   return check_launch();
@@ -420,7 +447,7 @@ static sea_status mix_typed(const sea_shape& s, const sea_decoder& dec, const fl
                                                                dec.d_hidden);
   if ((rc = check_launch()) != SEA_OK) return rc;
   const int BH = s.B * s.H;
-  if (s.causal) running_mean_kernel<T><<<(BH * kHeadDim + 127) / 128, 128, 0, st>>>(V, c_avg, BH, s.T);
+  if (s.causal) running_mean_kernel<T><<<BH, kHeadDim * kMeanSegs, 0, st>>>(V, c_avg, s.T);
   else pooled_kernel<T><<<BH, 256, (size_t)s.Kc * sizeof(float), st>>>(A_hat, V, c_avg, s.T, s.Kc);
   if ((rc = check_launch()) != SEA_OK) return rc;
   mix_kernel<T><<<(unsigned)((rows * kHeadDim + 255) / 256), 256, 0, st>>>(O, s_prob, s_mix, c_avg, rows, s.T, s.causal);
