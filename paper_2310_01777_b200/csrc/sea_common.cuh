@@ -158,8 +158,14 @@ sea_status launch_sparse_attn_tma(const sea_shape& s, const void* Q, const void*
 struct DecoderLayout {
   size_t ident, first, c_first, c_value, z, hidden, image, conv_a, conv_b, s_prob, s_mix, c_avg;
   size_t act0, w_tiles;  // tensor-core form of the convolutions only: the image as bf16 planes, the layers' weight tiles
+  size_t mlp_w;          // tensor-core form of the MLPs only: their weight tiles
   size_t total;
 };
+// Tensor-core form of the estimator head's MLPs (sea_mlp_tc.cu): Z and the CNN's input feature map.
+bool mlp_tc_shape_ok(int d_hidden, int n3);
+size_t mlp_tc_weight_bytes(int n3);
+sea_status launch_mlp_tc(const sea_shape& s, const sea_decoder& dec, const float* c_first, const float* c_value, const void* V, float* Z,
+                         void* act, void* w_tiles, int32_t* status, cudaStream_t st);
 // Tensor-core form of a 3 x 3 convolution layer (sea_conv_tc.cu).
 bool conv_tc_shape_ok(int c_in, int c_out, int h_in, int w_in, int up_h, int up_w, int stride_h);
 size_t conv_tc_weight_bytes(int c_in, int c_out, int up_h, int up_w);

@@ -350,6 +350,7 @@ DecoderLayout decoder_layout(const sea_shape& s, const sea_decoder& dec) {
   if (decoder_conv_tc(s, dec)) {
     L.act0 = take((size_t)s.B * C * s.T * wr * 2 * sizeof(__nv_bfloat16));
     L.w_tiles = take(3 * align_up(conv_tc_weight_bytes((int)C, 128, 1, 1), 256));  // 128: the most accumulator columns of a layer
+    if (mlp_tc_shape_ok(dec.d_hidden, (int)wr * dec.c_h)) L.mlp_w = take(mlp_tc_weight_bytes((int)wr * dec.c_h));
   }
   L.total = off;
   return L;
@@ -384,15 +385,21 @@ static sea_status estimate_decoder_typed(const sea_shape& s, const sea_decoder& 
   if ((rc = launch_estimate(e, Q, K, V, omega, ident, c_value, est_state, est_split, nullptr, nullptr, status, st)) != SEA_OK)
     return rc;
   const int wr = s.Kc / dec.c_s, C = s.H * dec.c_h;
+  // with the convolutions in their tensor-core form the MLPs can run in theirs, writing the CNN's input as bf16 planes
+  const bool mlp_tc = decoder_conv_tc(s, dec) && mlp_tc_shape_ok(dec.d_hidden, wr * dec.c_h);
   // Z = relu([C_perf ; V] W_mu + b_mu); Z_hat = relu(Z W_1 + b_1) W_2 + b_2, written as the image
-  if ((rc = linear<T>(c_first, c_value, V, 3 * kHeadDim, dec.W_mu, dec.b_mu, Z, rows, dec.d_hidden, 1, 0, 0, 0, 0, 0, st)) != SEA_OK)
-    return rc;
-  if ((rc = linear<T>(Z, nullptr, nullptr, dec.d_hidden, dec.W_nu1, dec.b_nu1, hidden, rows, dec.d_hidden, 1, 0, 0, 0, 0, 0, st)) !=
-      SEA_OK)
-    return rc;
-  if ((rc = linear<T>(hidden, nullptr, nullptr, dec.d_hidden, dec.W_nu2, dec.b_nu2, image, rows, wr * dec.c_h, 0, 1, s.H, s.T,
-                      dec.c_h, wr, st)) != SEA_OK)
-    return rc;
+  if (mlp_tc) {
+    if ((rc = launch_mlp_tc(s, dec, c_first, c_value, V, Z, dws + L.act0, dws + L.mlp_w, status, st)) != SEA_OK) return rc;
+  } else {
+    if ((rc = linear<T>(c_first, c_value, V, 3 * kHeadDim, dec.W_mu, dec.b_mu, Z, rows, dec.d_hidden, 1, 0, 0, 0, 0, 0, st)) != SEA_OK)
+      return rc;
+    if ((rc = linear<T>(Z, nullptr, nullptr, dec.d_hidden, dec.W_nu1, dec.b_nu1, hidden, rows, dec.d_hidden, 1, 0, 0, 0, 0, 0, st)) !=
+        SEA_OK)
+      return rc;
+    if ((rc = linear<T>(hidden, nullptr, nullptr, dec.d_hidden, dec.W_nu2, dec.b_nu2, image, rows, wr * dec.c_h, 0, 1, s.H, s.T,
+                        dec.c_h, wr, st)) != SEA_OK)
+      return rc;
+  }
   // the CNN: causal layers see rows t-2 .. t (two rows of padding above), the others pad one row on either side
   const int pad_top = s.causal ? 2 : 1;
   const int stride1 = s.causal ? 1 : dec.c_s;
@@ -402,7 +409,7 @@ static sea_status estimate_decoder_typed(const sea_shape& s, const sea_decoder& 
     char* act0 = dws + L.act0;
     char* wt = dws + L.w_tiles;
     const size_t wt_step = align_up(conv_tc_weight_bytes(C, 128, 1, 1), 256);
-    if ((rc = launch_nchw_to_nhwc_split(image, act0, s.B, C, s.T, wr, st)) != SEA_OK) return rc;
+    if (!mlp_tc && (rc = launch_nchw_to_nhwc_split(image, act0, s.B, C, s.T, wr, st)) != SEA_OK) return rc;
     if ((rc = launch_conv_tc(act0, s.B, C, s.T, wr, 1, 1, stride1, pad_top, dec.conv1_w, dec.conv1_b, C, 1, wt, conv_a, nullptr,
                              status, st)) != SEA_OK)
       return rc;

@@ -117,12 +117,16 @@ TC_CASES = [
     small("dec_tc_nc", causal=False, H=32, T=192, Kc=64, k_hat=6),
     small("dec_tc_nc_ragged", causal=False, H=16, T=80, Kc=16, k_hat=3),
     small("dec_tc_causal_ragged", H=16, T=80, Kc=16, k_hat=3, B=2),
+    small("dec_tc_wide", H=16, T=512, Kc=256, k_hat=8),   # Z_hat 512 wide: two chunks of W_2; image rows of 128 pixels
 ]
 
 
+# d' = 64 also takes the MLPs to their tensor-core form (feature map written as bf16 planes: four
+# channels at a time when the image is a multiple of 16 wide, else element by element)
+@pytest.mark.parametrize("d_hidden", [24, 64])
 @pytest.mark.parametrize("w", TC_CASES, ids=lambda w: w.name)
-def test_tensor_core_convolutions_match_oracle(w):
-    a = Run(w, c_h=4)
+def test_tensor_core_head_matches_oracle(w, d_hidden):
+    a = Run(w, d_hidden=d_hidden, c_h=4)
     a.stages(); a.done()
     assert bool(torch.isfinite(a.A_hat).all())
     assert torch.allclose(a.A_hat.sum(-1), torch.ones_like(a.A_hat[..., 0]), atol=1e-5)
