@@ -7,6 +7,9 @@
 // leaves the SM; Z_hat is written straight as the CNN's input feature map in the tensor-core
 // convolutions' layout, [hi, lo][B][T][K / c_s][H c_h] bf16 (row (b, h, t), entry j (K / c_s) + x
 // -> pixel (t, x), channel h c_h + j).
+// A tile is 128 rows: hg neighbouring heads (a power of two dividing H, at most 32) at 128 / hg
+// positions, heads fastest, so that a warp's stores of Z_hat fall on neighbouring channels of the
+// same pixels.
 // Roles: warps 0-3 own the tile's rows (thread = row = lane of tensor memory): they stage the
 // inputs, and take each product out (bias, ReLU, split) to feed the next; warp 4 copies the weights
 // in (once, or per 256-column chunk of W_2 when Z_hat is wider than that) and issues the MMAs.
@@ -37,6 +40,7 @@ struct MlpTcParams {
   long long rows;
   int n_tiles, n3, n_chunks, chunk;
   int H, seq_len, c_h, wr, batch;
+  int hg, tiles_t;                  // heads per tile (a power of two dividing H, at most 32); tiles along the sequence per group of heads
   int32_t* status;
 };
 
@@ -202,8 +206,12 @@ mlp_tc_kernel(const __grid_constant__ CUtensorMap map_wmu, const __grid_constant
     uint32_t it = 0, c_it = 0;
     for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
       const uint32_t par = it & 1;
-      const long long row = (long long)tile * 128 + r;
-      const bool live = row < p.rows;
+      // Row r of the tile is head h0 + r % hg at position t0 + r / hg: the threads of a warp hold
+      // neighbouring heads of the same positions, whose channels are neighbours in the feature map
+      const int tt = tile % p.tiles_t, grp = tile / p.tiles_t, groups = p.H / p.hg;
+      const int b = grp / groups, h = (grp - b * groups) * p.hg + r % p.hg, t = tt * (128 / p.hg) + r / p.hg;
+      const bool live = t < p.seq_len;
+      const long long row = ((long long)b * p.H + h) * p.seq_len + (live ? t : 0);
       // inputs: C_perf's two halves (fp32) and V, as head / remainder rows of the three blocks
 #pragma unroll 1
       for (int kb = 0; kb < 3; ++kb) {
@@ -290,9 +298,7 @@ mlp_tc_kernel(const __grid_constant__ CUtensorMap map_wmu, const __grid_constant
       fence_async_smem();
       ml_warp_arrive(bar(kMl_H), lane);
       // Z_hat + b_2 -> the feature map
-      const long long bh = live ? row / p.seq_len : 0;
-      const int t = live ? (int)(row - bh * p.seq_len) : 0, b = (int)(bh / p.H), h = (int)(bh - (long long)b * p.H);
-      __nv_bfloat16* pix = p.act + ((size_t)b * p.seq_len + t) * p.wr * C + (size_t)h * p.c_h;  // pixel (t, 0), channel h c_h
+      __nv_bfloat16* pix = p.act + ((size_t)b * p.seq_len + (live ? t : 0)) * p.wr * C + (size_t)h * p.c_h;  // pixel (t, 0), channel h c_h
       for (int c = 0; c < p.n_chunks && ok; ++c, ++c_it) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar(kMl_M3), c_it & 1, abort_flag));
         if (!ok) break;
@@ -400,7 +406,10 @@ static sea_status launch_mlp_tc_typed(const sea_shape& s, const sea_decoder& dec
   p.Z = Z;
   p.act = static_cast<__nv_bfloat16*>(act);
   p.rows = (long long)s.B * s.H * s.T;
-  p.n_tiles = (int)((p.rows + 127) / 128);
+  p.hg = 1;
+  while (p.hg < 32 && s.H % (2 * p.hg) == 0) p.hg *= 2;
+  p.tiles_t = (s.T + 128 / p.hg - 1) / (128 / p.hg);
+  p.n_tiles = s.B * (s.H / p.hg) * p.tiles_t;
   p.n3 = n3;
   p.chunk = n3 <= kMlChunk ? n3 : kMlChunk;
   p.n_chunks = n3 / p.chunk;
