@@ -33,7 +33,7 @@ metric is quoted.  One JSON line is printed by rank 0.
              the mask and sparse stages when the caller gives a banded estimate (the structure of
              trained SEA masks): the tile kernel skips the key tiles nothing was selected in.
   decoder_head  (--decoder) the layer with the paper's estimator head (MLPs + three-layer CNN, random-init
-             weights) and output mixing through sea_attention_decoder: plain fp32 kernels.
+             weights) and output mixing through sea_attention_decoder: MLPs and convolutions on tcgen05.
   cpu_baseline  the fp64 oracle on a bounded sample of heads, one head per host core at a time.
 
 With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no
@@ -392,7 +392,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-modes", action="store_true", help="skip the grouped / causal-aware / lean regions")
     ap.add_argument("--soak-s", type=float, default=1.2, help="seconds of steps the clock sampler watches")
-    ap.add_argument("--decoder", action="store_true", help="also time the paper's MLP + CNN estimator head (tens of ms per step)")
+    ap.add_argument("--decoder", action="store_true", help="also time the paper's MLP + CNN estimator head (a few ms per step)")
     ap.add_argument("--capped-sweep", action="store_true", help="time the paper's long-sequence sweep shape instead")
     ap.add_argument("--sweep-B", type=int, default=1)
     ap.add_argument("--sweep-H", type=int, default=12)
@@ -670,7 +670,8 @@ def main():
             raise SystemExit("device status word set by the decoder path")
         d_ms = sum(d_all) / n_d
         decoder = {"head": f"d_hidden={d_hidden} c_s={c_s} c_h={c_h}: V_cat, mu, nu, 3-layer CNN over {C} channels, softmax; "
-                           "s_prob, s_mix, C_avg mixing; random-init weights; fp32 FMA kernels",
+                           "s_prob, s_mix, C_avg mixing; random-init weights; MLPs and convolutions on tcgen05 "
+                           "(bf16 head/remainder operands, three products per step, fp32 accumulators)",
                    "ms_per_step": d_ms, "ms_stats": ms_stats(d_all), "value": w.B * w.T / (d_ms / 1e3), "unit": "tokens/s",
                    "gpu_launches_per_step": d_launches, "estimate_decoder_ms": ms_stats(e_all),
                    "conv_flops": conv_flops, "conv_tflops_if_all_time_were_conv": conv_flops / (sum(e_all) / n_d / 1e3) / 1e12}

@@ -519,33 +519,56 @@ fill_col_idx_kernel(const int32_t* __restrict__ sel, const int32_t* __restrict__
                     int32_t* __restrict__ col_idx, long long nnz_cap, int rows, int k_hat, int r, int log2r,
                     int32_t* __restrict__ status) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row = blockIdx.x * kWarpsPerCta + warp;
+  const int n_warps = gridDim.x * kWarpsPerCta;
+  int row = blockIdx.x * kWarpsPerCta + warp;
   if (row >= rows) return;
-  const int base = row_ptr[row];
-  int n = row_ptr[row + 1] - base;
-  if ((long long)base + n > nnz_cap) {
-    if (lane == 0) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
-    n = (int)max(0ll, min((long long)n, nnz_cap - base));
-  }
-  const int32_t* my_sel = sel + (size_t)row * k_hat;
   if (log2r >= 0 && k_hat <= 32) {
     // r a power of two: the run and the offset inside it are a shift and a mask; the row's
-    // selected columns sit one per lane and are fetched by shuffles
-    const int mine = lane < k_hat ? __ldg(my_sel + lane) << log2r : 0;
-    int32_t* out = col_idx + base;
-    const int n_up = (n + 31) & ~31;  // every lane takes part in the shuffles
+    // selected columns sit one per lane and are fetched by shuffles.  A warp walks rows row,
+    // row + n_warps, ...: the next row's pointers and columns are requested before this row's
+    // keys are written, so that their latency hides under the stores.
+    int base = __ldg(row_ptr + row), end = __ldg(row_ptr + row + 1);
+    int mine = lane < k_hat ? __ldg(sel + (size_t)row * k_hat + lane) << log2r : 0;
+    for (;;) {
+      const int next = row + n_warps;
+      int base_n = 0, end_n = 0, mine_n = 0;
+      if (next < rows) {
+        base_n = __ldg(row_ptr + next), end_n = __ldg(row_ptr + next + 1);
+        mine_n = lane < k_hat ? __ldg(sel + (size_t)next * k_hat + lane) << log2r : 0;
+      }
+      int n = end - base;
+      if ((long long)base + n > nnz_cap) {
+        if (lane == 0) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
+        n = (int)max(0ll, min((long long)n, nnz_cap - base));
+      }
+      int32_t* out = col_idx + base;
+      const int n_up = (n + 31) & ~31;  // every lane takes part in the shuffles
 #pragma unroll 4
-    for (int pos = lane; pos < n_up; pos += 32) {
-      const int start = __shfl_sync(0xffffffffu, mine, (pos >> log2r) & 31);
-      if (pos < n) out[pos] = start + (pos & (r - 1));
+      for (int pos = lane; pos < n_up; pos += 32) {
+        const int start = __shfl_sync(0xffffffffu, mine, (pos >> log2r) & 31);
+        if (pos < n) out[pos] = start + (pos & (r - 1));
+      }
+      if (next >= rows) break;
+      row = next, base = base_n, end = end_n, mine = mine_n;
     }
-  } else if (log2r >= 0) {
-    for (int pos = lane; pos < n; pos += 32)
-      col_idx[(size_t)base + pos] = (__ldg(my_sel + (pos >> log2r)) << log2r) + (pos & (r - 1));
-  } else {
-    for (int pos = lane; pos < n; pos += 32) {
-      const int b = pos / r;
-      col_idx[(size_t)base + pos] = __ldg(my_sel + b) * r + (pos - b * r);
+    return;
+  }
+  for (; row < rows; row += n_warps) {
+    const int base = row_ptr[row];
+    int n = row_ptr[row + 1] - base;
+    if ((long long)base + n > nnz_cap) {
+      if (lane == 0) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
+      n = (int)max(0ll, min((long long)n, nnz_cap - base));
+    }
+    const int32_t* my_sel = sel + (size_t)row * k_hat;
+    if (log2r >= 0) {
+      for (int pos = lane; pos < n; pos += 32)
+        col_idx[(size_t)base + pos] = (__ldg(my_sel + (pos >> log2r)) << log2r) + (pos & (r - 1));
+    } else {
+      for (int pos = lane; pos < n; pos += 32) {
+        const int b = pos / r;
+        col_idx[(size_t)base + pos] = __ldg(my_sel + b) * r + (pos - b * r);
+      }
     }
   }
 }
@@ -634,8 +657,13 @@ sea_status launch_topk_mask(const sea_shape& s, const float* A_hat, int32_t* sel
     int log2r = -1;
     for (int l = 0; l < 31; ++l)
       if ((1 << l) == r) log2r = l;
-    fill_col_idx_kernel<<<grid, kWarpsPerCta * 32, 0, st>>>(sel, row_ptr, col_idx, (long long)nnz_cap,
-                                                            rows, s.k_hat, r, log2r, status);
+    // a grid that fills the machine once: each warp then walks several rows
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return SEA_ERR_CUDA;
+    const int resident = sms * (2048 / (kWarpsPerCta * 32));
+    fill_col_idx_kernel<<<grid < resident ? grid : resident, kWarpsPerCta * 32, 0, st>>>(
+        sel, row_ptr, col_idx, (long long)nnz_cap, rows, s.k_hat, r, log2r, status);
     if ((rc = check_launch()) != SEA_OK) return rc;
   }
   return SEA_OK;
