@@ -279,7 +279,86 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
   const int k_hat = min(k_all, Kc);
   const int col0 = lane * VPL;  // this lane's first column
   RowKeys<VPL, kShared> key(keys_all + (kShared ? warp * (VPL + 1) * 32 : 0), col0);
+  RowOut out;
+  out.sel = sel != nullptr ? sel + (size_t)row * k_all : nullptr;
+  out.n_words = (Kc_all + 31) / 32;
+  out.words = mask_bits != nullptr ? mask_bits + (size_t)row * out.n_words : nullptr;
+  out.count = row_counts != nullptr ? row_counts + row : nullptr;
+  out.i = row % seq_len;
+  out.r = r;
+  out.causal = causal;
+
   if constexpr (kShared) {
+    // A wide row first sheds most of its values.  The row is fetched as 16-byte pieces (lane l takes
+    // pieces l, l + 32, ...) and parked in the warp's shared memory as it is; while fetching, every
+    // lane keeps the two largest values it met.  Those are 64 different entries of the row, so the
+    // k_hat-th largest of the 64, L (found bit by bit with ballots on their keys), has at least
+    // k_hat entries at or above it: every selected entry is >= L, and usually few more than k_hat
+    // are (L = 0 when fewer than k_hat of the 64 hold a column: no shortcut then).  Each lane then
+    // reads back its own VPL consecutive columns (piece q sits at q ^ (owner lane & 7): neither the
+    // writes nor these reads meet bank conflicts), and the entries >= L go, with their columns and in
+    // column order, through the same selection on kCandSlots slots per lane.
+    if (k_hat <= 32 && Kc_all % 4 == 0) {
+      constexpr int kPerLane = VPL / 4;  // pieces of a lane's own columns
+      static_assert(kPerLane >= 8, "the swizzle takes the owner's low three bits");
+      float4* stage = reinterpret_cast<float4*>(keys_all + warp * (VPL + 1) * 32);
+      float f1 = -INFINITY, f2 = -INFINITY;  // columns that do not compete count as -inf (inputs are finite)
+#pragma unroll 4
+      for (int q = lane; q < 8 * VPL; q += 32) {
+        float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (4 * q < Kc) v = __ldg(reinterpret_cast<const float4*>(a + 4 * q));
+        if (4 * q + 3 >= Kc) {  // the visible part of an aware row need not end on a piece
+          if (4 * q + 1 >= Kc) v.y = -INFINITY;
+          if (4 * q + 2 >= Kc) v.z = -INFINITY;
+          v.w = -INFINITY;
+        }
+        stage[q ^ ((q / kPerLane) & 7)] = v;
+        const float x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          f2 = fmaxf(f2, fminf(f1, x[e]));
+          f1 = fmaxf(f1, x[e]);
+        }
+      }
+      const uint32_t top1 = f1 == -INFINITY ? 0u : order_key(f1), top2 = f2 == -INFINITY ? 0u : order_key(f2);
+      uint32_t low = 0u;
+#pragma unroll 1
+      for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t c = low | (1u << bit);
+        if (__popc(__ballot_sync(0xffffffffu, top1 >= c)) + __popc(__ballot_sync(0xffffffffu, top2 >= c)) >= k_hat) low = c;
+      }
+      __syncwarp();
+      if (low != 0u) {
+        // L is the key of one of the 64 values: back to that value
+        const float low_f = __uint_as_float((low & 0x80000000u) ? (low ^ 0x80000000u) : ~low);
+        uint64_t cand = 0ull;
+#pragma unroll
+        for (int j = 0; j < kPerLane; ++j) {
+          const float4 v = stage[(lane * kPerLane + j) ^ (lane & 7)];
+          cand |= (uint64_t)((v.x >= low_f ? 1u : 0u) | (v.y >= low_f ? 2u : 0u) | (v.z >= low_f ? 4u : 0u) | (v.w >= low_f ? 8u : 0u))
+                  << (4 * j);
+        }
+        if (__reduce_max_sync(0xffffffffu, __popcll(cand)) <= kCandSlots) {
+          const float* words = reinterpret_cast<const float*>(stage);
+          CandKeys<kCandSlots> ck;
+#pragma unroll
+          for (int j = 0; j < kCandSlots; ++j) {
+            ck.k[j] = 0u;
+            ck.c[j] = 0;
+            if (cand != 0ull) {
+              const int t = __ffsll((long long)cand) - 1;
+              cand &= cand - 1ull;
+              ck.k[j] = order_key(words[4 * ((lane * kPerLane + (t >> 2)) ^ (lane & 7)) + (t & 3)]);
+              ck.c[j] = col0 + t;
+            }
+          }
+          select_row(ck, hist_all[warp], lane, k_hat, out);
+          return;
+        }
+      }
+      __syncwarp();  // the keys below go where the values were
+    }
+    // every key of the row, lane l's t-th at word l (VPL + 1) + t
     if (Kc_all % 4 == 0) {
 #pragma unroll 4
       for (int c = 4 * lane; c < 32 * VPL; c += 128) {
@@ -305,46 +384,6 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
   } else {
 #pragma unroll
     for (int t = 0; t < VPL; ++t) key.set(t, col0 + t < Kc ? order_key(__ldg(a + col0 + t)) : 0u);
-  }
-  RowOut out;
-  out.sel = sel != nullptr ? sel + (size_t)row * k_all : nullptr;
-  out.n_words = (Kc_all + 31) / 32;
-  out.words = mask_bits != nullptr ? mask_bits + (size_t)row * out.n_words : nullptr;
-  out.count = row_counts != nullptr ? row_counts + row : nullptr;
-  out.i = row % seq_len;
-  out.r = r;
-  out.causal = causal;
-
-  if constexpr (kShared) {
-    // A wide row first sheds most of its keys.  When every lane holds a column of the row, the
-    // smallest of the lanes' largest keys, L, has at least 32 keys at or above it, so with
-    // k_hat <= 32 every selected key is >= L; usually only a few keys per lane are.  They go, with
-    // their columns and in column order, through the same selection on kCandSlots slots per lane.
-    if (k_hat <= 32 && 31 * VPL < Kc) {
-      uint32_t lane_top = 0u;
-#pragma unroll 8
-      for (int t = 0; t < VPL; ++t) lane_top = max(lane_top, key.get(t));
-      const uint32_t low = __reduce_min_sync(0xffffffffu, lane_top);
-      uint64_t cand = 0ull;
-#pragma unroll 8
-      for (int t = 0; t < VPL; ++t) cand |= (uint64_t)(key.get(t) >= low) << t;
-      if (__reduce_max_sync(0xffffffffu, __popcll(cand)) <= kCandSlots && low != 0u) {
-        CandKeys<kCandSlots> ck;
-#pragma unroll
-        for (int j = 0; j < kCandSlots; ++j) {
-          ck.k[j] = 0u;
-          ck.c[j] = 0;
-          if (cand != 0ull) {
-            const int t = __ffsll((long long)cand) - 1;
-            cand &= cand - 1ull;
-            ck.k[j] = key.get(t);
-            ck.c[j] = col0 + t;
-          }
-        }
-        select_row(ck, hist_all[warp], lane, k_hat, out);
-        return;
-      }
-    }
   }
   select_row(key, hist_all[warp], lane, k_hat, out);
 }
