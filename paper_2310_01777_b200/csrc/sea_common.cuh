@@ -167,8 +167,9 @@ size_t mlp_tc_weight_bytes(int n3);
 sea_status launch_mlp_tc(const sea_shape& s, const sea_decoder& dec, const float* c_first, const float* c_value, const void* V, float* Z,
                          void* act, void* w_tiles, int32_t* status, cudaStream_t st);
 // Tensor-core form of a 3 x 3 convolution layer (sea_conv_tc.cu).
-bool conv_tc_shape_ok(int c_in, int c_out, int h_in, int w_in, int up_h, int up_w, int stride_h);
-size_t conv_tc_weight_bytes(int c_in, int c_out, int up_h, int up_w);
+int conv_tc_channels(int c);  // channel stride of the bf16 planes: c rounded up to a multiple of 64
+bool conv_tc_shape_ok(int c_in, int c_out, int h_in, int w_in, int up_h, int up_w, int stride_h, bool logits);
+size_t conv_tc_weight_bytes(int c_in);
 sea_status launch_nchw_to_nhwc_split(const float* in, void* out, int batch, int C, int h, int w, cudaStream_t st);
 sea_status launch_conv_tc(const void* act_in, int batch, int c_in, int h_in, int w_in, int up_h, int up_w, int stride_h,
                           int pad_top, const float* w, const float* bias, int c_out, int relu, void* w_tiles, void* out_split,

@@ -38,7 +38,8 @@ constexpr int kCtMaxN = 128;
 
 struct ConvTcParams {
   int n_cblk;             // C_in / 64
-  int n_out;              // accumulator columns N (a multiple of 32)
+  int n_out;              // accumulator columns N (a multiple of 32): n_real outputs and columns of zeros
+  int n_real;
   int bw, bh;             // pixel tile: bh rows of bw columns, bh * bw = 128
   int tiles_x, tiles_y;   // tiles_y counts groups of kCtTiles tile rows
   int n_items;
@@ -48,7 +49,7 @@ struct ConvTcParams {
   int tap_s[3], tap_y[3], tap_x[3];
   const float* bias;      // [c_out]
   int c_out, relu;
-  __nv_bfloat16* out_split;  // [2][batch][h_out][w_out][c_out]   (kLogits == false)
+  __nv_bfloat16* out_split;  // [2][batch][h_out][w_out][n_out]   (kLogits == false; channels c_out .. n_out - 1 are zero)
   float* out_logits;         // [batch][c_out][h_out up_h][w_out up_w]   (kLogits == true)
   int up_h, up_w;
   int32_t* status;
@@ -87,7 +88,7 @@ conv_taps_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     *abort_flag = 0;
     mbar_init_fence();
   }
-  for (int n = tid; n < kCtMaxN; n += kCtThreads) bias_s[n] = n < p.n_out ? p.bias[n % p.c_out] : 0.f;
+  for (int n = tid; n < kCtMaxN; n += kCtThreads) bias_s[n] = n < p.n_real ? p.bias[n % p.c_out] : 0.f;
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
   fence_before();
   __syncthreads();
@@ -208,8 +209,8 @@ conv_taps_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             uint32_t hi[16], lo[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) split_pair(vals[2 * i], vals[2 * i + 1], hi[i], lo[i]);
-            const size_t plane_elems = (size_t)p.batch * p.h_out * p.w_out * p.c_out;
-            __nv_bfloat16* dst = p.out_split + (((size_t)b * p.h_out + y) * p.w_out + x) * p.c_out + 32 * c;
+            const size_t plane_elems = (size_t)p.batch * p.h_out * p.w_out * p.n_out;
+            __nv_bfloat16* dst = p.out_split + (((size_t)b * p.h_out + y) * p.w_out + x) * p.n_out + 32 * c;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
               reinterpret_cast<uint4*>(dst)[q] = make_uint4(hi[4 * q], hi[4 * q + 1], hi[4 * q + 2], hi[4 * q + 3]);
@@ -221,7 +222,8 @@ conv_taps_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const int py = ph / p.up_w, px = ph - py * p.up_w;
-              p.out_logits[(((size_t)b * p.c_out + co) * h_full + (size_t)y * p.up_h + py) * w_full + (size_t)x * p.up_w + px] = vals[i];
+              if (32 * c + i < p.n_real)
+                p.out_logits[(((size_t)b * p.c_out + co) * h_full + (size_t)y * p.up_h + py) * w_full + (size_t)x * p.up_w + px] = vals[i];
               if (++co == p.c_out) {
                 co = 0;
                 ++ph;
@@ -245,13 +247,15 @@ conv_taps_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 }
 
 // ---- operand preparation -----------------------------------------------------------------------
-// Weights [c_out][c_in][3][3] fp32 -> tiles [ny nx][c_in / 64][hi, lo][n_out][64] bf16 of the
-// effective taps: column n = phase (py, px) * c_out + co takes, at tap (a, bx), the sum of the
-// original taps (ky, kx) whose logical input pixel falls on stored offset (min_y + a, min_x + bx).
-__global__ void conv_weights_split_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ out, int c_in, int c_out,
-                                          int n_out, int ny, int nx, int up_h, int up_w, int pad_top) {
+// Weights [c_out][c_in][3][3] fp32 -> tiles [ny nx][cs_in / 64][hi, lo][n_out][64] bf16 of the
+// effective taps (cs_in = c_in rounded up to whole blocks of 64 channels): column n = phase
+// (py, px) * c_out + co takes, at tap (a, bx), the sum of the original taps (ky, kx) whose logical
+// input pixel falls on stored offset (min_y + a, min_x + bx); columns n >= n_real and channels
+// >= c_in hold zeros.
+__global__ void conv_weights_split_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ out, int c_in, int cs_in,
+                                          int c_out, int n_real, int n_out, int ny, int nx, int up_h, int up_w, int pad_top) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const int half_c = c_in / 2;
+  const int half_c = cs_in / 2;
   if (idx >= (long long)ny * nx * n_out * half_c) return;
   const int cpair = (int)(idx % half_c);
   const int n = (int)((idx / half_c) % n_out), tap = (int)(idx / ((long long)half_c * n_out));
@@ -259,26 +263,29 @@ __global__ void conv_weights_split_kernel(const float* __restrict__ w, __nv_bflo
   const int ph = n / c_out, co = n - ph * c_out, py = ph / up_w, px = ph - py * up_w;
   const int min_y = floor_div(-pad_top, up_h), min_x = floor_div(-1, up_w);
   float sum[2] = {0.f, 0.f};
-  for (int ky = 0; ky < 3; ++ky) {
-    if (floor_div(py + ky - pad_top, up_h) - min_y != a) continue;
-    for (int kx = 0; kx < 3; ++kx) {
-      if (floor_div(px + kx - 1, up_w) - min_x != bx) continue;
-      for (int q = 0; q < 2; ++q) sum[q] += w[(((size_t)co * c_in + 2 * cpair + q) * 3 + ky) * 3 + kx];
+  if (n < n_real)
+    for (int ky = 0; ky < 3; ++ky) {
+      if (floor_div(py + ky - pad_top, up_h) - min_y != a) continue;
+      for (int kx = 0; kx < 3; ++kx) {
+        if (floor_div(px + kx - 1, up_w) - min_x != bx) continue;
+        for (int q = 0; q < 2; ++q)
+          if (2 * cpair + q < c_in) sum[q] += w[(((size_t)co * c_in + 2 * cpair + q) * 3 + ky) * 3 + kx];
+      }
     }
-  }
   uint32_t hi, lo;
   split_pair(sum[0], sum[1], hi, lo);
   const int ci = 2 * cpair, cb = ci / 64, within = ci % 64;
-  const size_t tile = ((size_t)tap * (c_in / 64) + cb) * 2;
+  const size_t tile = ((size_t)tap * (cs_in / 64) + cb) * 2;
   uint32_t* o = reinterpret_cast<uint32_t*>(out);
   o[((tile * n_out + n) * 64 + within) / 2] = hi;
   o[(((tile + 1) * n_out + n) * 64 + within) / 2] = lo;
 }
 
-// Feature map [batch][C][h][w] fp32 -> [hi, lo][batch][h][w][C] bf16.  A block: 64 channels x 32
-// columns of one row through shared memory (reads run along w, writes along C).
+// Feature map [batch][C][h][w] fp32 -> [hi, lo][batch][h][w][cs] bf16, cs = C rounded up to whole
+// blocks of 64 channels (the added channels are zero).  A block: 64 channels x 32 columns of one row
+// through shared memory (reads run along w, writes along the channels).
 __global__ void __launch_bounds__(256)
-nchw_to_nhwc_split_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, int C, int h, int w, int batch) {
+nchw_to_nhwc_split_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, int C, int cs, int h, int w, int batch) {
   __shared__ float t[64][33];
   const int tiles_w = (w + 31) / 32;
   const int x0 = (blockIdx.x % tiles_w) * 32, y = blockIdx.x / tiles_w, c0 = blockIdx.y * 64, b = blockIdx.z;
@@ -286,10 +293,10 @@ nchw_to_nhwc_split_kernel(const float* __restrict__ in, __nv_bfloat16* __restric
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int c = grp + 8 * i;
-    t[c][lane] = (x0 + lane < w) ? in[(((size_t)b * C + c0 + c) * h + y) * w + x0 + lane] : 0.f;
+    t[c][lane] = (x0 + lane < w && c0 + c < C) ? in[(((size_t)b * C + c0 + c) * h + y) * w + x0 + lane] : 0.f;
   }
   __syncthreads();
-  const size_t plane_words = (size_t)batch * h * w * C / 2;
+  const size_t plane_words = (size_t)batch * h * w * cs / 2;
   uint32_t* o = reinterpret_cast<uint32_t*>(out);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -297,7 +304,7 @@ nchw_to_nhwc_split_kernel(const float* __restrict__ in, __nv_bfloat16* __restric
     if (x0 + xl >= w) continue;
     uint32_t hi, lo;
     split_pair(t[2 * lane][xl], t[2 * lane + 1][xl], hi, lo);
-    const size_t word = ((((size_t)b * h + y) * w + x0 + xl) * C + c0 + 2 * lane) / 2;
+    const size_t word = ((((size_t)b * h + y) * w + x0 + xl) * cs + c0 + 2 * lane) / 2;
     o[word] = hi;
     o[plane_words + word] = lo;
   }
@@ -319,39 +326,51 @@ bool make_map_bf16_5d(CUtensorMap* map, const void* ptr, unsigned long long d0, 
 
 }  // namespace
 
-// Shapes this form takes: whole blocks of 64 input channels, at most 128 accumulator columns in
-// whole chunks of 32, a row of the stored map made of whole boxes of min(w, 128) columns that
-// divide 128, and (strided layer) a height that is a multiple of the stride.
-bool conv_tc_shape_ok(int c_in, int c_out, int h_in, int w_in, int up_h, int up_w, int stride_h) {
-  const int n_out = up_h * up_w * c_out;
-  const int bw = w_in < 128 ? w_in : 128;
-  if (c_in <= 0 || c_in % 64 != 0 || n_out <= 0 || n_out > kCtMaxN || n_out % 32 != 0) return false;
-  if (w_in <= 0 || 128 % bw != 0 || w_in % bw != 0) return false;
-  if (stride_h != 1 && (up_h != 1 || up_w != 1 || h_in % stride_h != 0)) return false;
-  return h_in > 0 && up_h >= 1 && up_w >= 1 && stride_h >= 1;
+// Channel strides and accumulator widths: channels come in whole blocks of 64 (a row of an operand
+// tile), accumulator columns in whole chunks of 32; what is added holds zeros.
+int conv_tc_channels(int c) { return (c + 63) / 64 * 64; }
+static int conv_tc_columns(int c_out, int up_h, int up_w, bool logits) {
+  return logits ? (up_h * up_w * c_out + 31) / 32 * 32 : conv_tc_channels(c_out);
 }
 
-size_t conv_tc_weight_bytes(int c_in, int c_out, int up_h, int up_w) {
-  return (size_t)9 * (c_in / 64) * 2 * (size_t)(up_h * up_w * c_out) * 64 * sizeof(__nv_bfloat16);
+// Shapes this form takes: at most 128 input channels and 128 accumulator columns after rounding
+// up, a row of the stored map made of whole boxes of min(w, 128) columns that divide 128, and
+// (strided layer) a height that is a multiple of the stride.  `logits`: the layer writes fp32 logits
+// with the resize's phases scattered; else bf16 planes for the next layer (no resize).
+bool conv_tc_shape_ok(int c_in, int c_out, int h_in, int w_in, int up_h, int up_w, int stride_h, bool logits) {
+  if (c_in <= 0 || c_out <= 0 || up_h < 1 || up_w < 1 || stride_h < 1 || h_in <= 0 || w_in <= 0) return false;
+  if (!logits && (up_h != 1 || up_w != 1)) return false;
+  const int bw = w_in < 128 ? w_in : 128;
+  if (conv_tc_channels(c_in) > 128 || conv_tc_columns(c_out, up_h, up_w, logits) > kCtMaxN) return false;
+  if (128 % bw != 0 || w_in % bw != 0) return false;
+  if (stride_h != 1 && (up_h != 1 || up_w != 1 || h_in % stride_h != 0)) return false;
+  return true;
 }
+
+size_t conv_tc_weight_bytes(int c_in) { return (size_t)9 * (conv_tc_channels(c_in) / 64) * 2 * kCtMaxN * 64 * sizeof(__nv_bfloat16); }
 
 sea_status launch_nchw_to_nhwc_split(const float* in, void* out, int batch, int C, int h, int w, cudaStream_t st) {
-  const dim3 grid(((w + 31) / 32) * h, C / 64, batch);
-  nchw_to_nhwc_split_kernel<<<grid, 256, 0, st>>>(in, static_cast<__nv_bfloat16*>(out), C, h, w, batch);
+  const int cs = conv_tc_channels(C);
+  const dim3 grid(((w + 31) / 32) * h, cs / 64, batch);
+  nchw_to_nhwc_split_kernel<<<grid, 256, 0, st>>>(in, static_cast<__nv_bfloat16*>(out), C, cs, h, w, batch);
   return check_launch();
 }
 
-// One layer.  act_in: [hi, lo][batch][h_in][w_in][c_in] bf16; the layer's logical input is its
-// nearest resize by (up_h, up_w), padded by pad_top rows above (2 - pad_top below) and one column
-// on either side, read at row stride stride_h.  Output: out_split ([hi, lo][batch][h_out][w_in][c_out]
-// bf16, ReLU per `relu`) or, when out_logits is given, fp32 [batch][c_out][h_in up_h][w_in up_w].
+// One layer.  act_in: [hi, lo][batch][h_in][w_in][cs_in] bf16 (cs_in = c_in rounded up to a multiple of
+// 64, the added channels zero); the layer's logical input is its nearest resize by (up_h, up_w),
+// padded by pad_top rows above (2 - pad_top below) and one column on either side, read at row stride
+// stride_h.  Output: out_split ([hi, lo][batch][h_out][w_in][cs_out] bf16, ReLU per `relu`, added
+// channels zero) or, when out_logits is given, fp32 [batch][c_out][h_in up_h][w_in up_w].
 sea_status launch_conv_tc(const void* act_in, int batch, int c_in, int h_in, int w_in, int up_h, int up_w, int stride_h,
                           int pad_top, const float* w, const float* bias, int c_out, int relu, void* w_tiles, void* out_split,
                           float* out_logits, int32_t* status, cudaStream_t st) {
-  if (!conv_tc_shape_ok(c_in, c_out, h_in, w_in, up_h, up_w, stride_h)) return SEA_ERR_UNSUPPORTED;
+  const bool logits = out_logits != nullptr;
+  if (!conv_tc_shape_ok(c_in, c_out, h_in, w_in, up_h, up_w, stride_h, logits)) return SEA_ERR_UNSUPPORTED;
+  const int cs_in = conv_tc_channels(c_in);
   ConvTcParams p{};
-  p.n_cblk = c_in / 64;
-  p.n_out = up_h * up_w * c_out;
+  p.n_cblk = cs_in / 64;
+  p.n_real = up_h * up_w * c_out;
+  p.n_out = conv_tc_columns(c_out, up_h, up_w, logits);
   p.bw = w_in < 128 ? w_in : 128;
   p.bh = 128 / p.bw;
   p.h_out = stride_h > 1 ? h_in / stride_h : h_in;
@@ -379,14 +398,14 @@ sea_status launch_conv_tc(const void* act_in, int batch, int c_in, int h_in, int
   p.up_w = up_w;
   p.status = status;
 
-  const long long w_threads = (long long)p.ny * p.nx * p.n_out * (c_in / 2);
-  conv_weights_split_kernel<<<(unsigned)((w_threads + 255) / 256), 256, 0, st>>>(w, static_cast<__nv_bfloat16*>(w_tiles), c_in, c_out,
-                                                                               p.n_out, p.ny, p.nx, up_h, up_w, pad_top);
+  const long long w_threads = (long long)p.ny * p.nx * p.n_out * (cs_in / 2);
+  conv_weights_split_kernel<<<(unsigned)((w_threads + 255) / 256), 256, 0, st>>>(w, static_cast<__nv_bfloat16*>(w_tiles), c_in, cs_in,
+                                                                               c_out, p.n_real, p.n_out, p.ny, p.nx, up_h, up_w, pad_top);
   sea_status rc = check_launch();
   if (rc != SEA_OK) return rc;
 
   CUtensorMap map_a, map_w;
-  if (!make_map_bf16_5d(&map_a, act_in, c_in, w_in, stride_h, h_in / stride_h, 2ull * batch, p.bw, p.bh)) return SEA_ERR_CUDA;
+  if (!make_map_bf16_5d(&map_a, act_in, cs_in, w_in, stride_h, h_in / stride_h, 2ull * batch, p.bw, p.bh)) return SEA_ERR_CUDA;
   if (!make_map_bf16_3d(&map_w, w_tiles, 64, p.n_out, (unsigned long long)p.ny * p.nx * p.n_cblk * 2, 64, p.n_out)) return SEA_ERR_CUDA;
   const size_t smem = 1024 + (size_t)kCtStages * kCtStageBytes + 128 + kCtMaxN * sizeof(float);
   int dev = 0, sms = 0;

@@ -318,8 +318,8 @@ static bool decoder_conv_tc(const sea_shape& s, const sea_decoder& dec) {
   const int stride1 = s.causal ? 1 : dec.c_s;
   const int t1 = conv_out_h(s.T, stride1);
   if (t1 <= 0 || s.T % t1 != 0) return false;
-  return conv_tc_shape_ok(C, C, s.T, wr, 1, 1, stride1) && conv_tc_shape_ok(C, C, t1, wr, 1, 1, 1) &&
-         conv_tc_shape_ok(C, s.H, t1, wr, s.T / t1, dec.c_s, 1);
+  return conv_tc_shape_ok(C, C, s.T, wr, 1, 1, stride1, false) && conv_tc_shape_ok(C, C, t1, wr, 1, 1, 1, false) &&
+         conv_tc_shape_ok(C, s.H, t1, wr, s.T / t1, dec.c_s, 1, true);
 }
 
 // Buffers of the decoder path inside its part of the workspace (all offsets 256-byte aligned).
@@ -342,14 +342,16 @@ DecoderLayout decoder_layout(const sea_shape& s, const sea_decoder& dec) {
   L.z = take(rows * (size_t)dec.d_hidden * sizeof(float));
   L.hidden = take(rows * (size_t)dec.d_hidden * sizeof(float));
   L.image = take((size_t)s.B * C * s.T * wr * sizeof(float));
-  L.conv_a = take((size_t)s.B * C * t1 * wr * sizeof(float));
-  L.conv_b = take((size_t)s.B * C * t1 * wr * sizeof(float));
+  // (in the tensor-core form the buffers hold bf16 head / remainder planes of whole blocks of 64 channels)
+  const size_t Cs = decoder_conv_tc(s, dec) ? (size_t)conv_tc_channels((int)C) : C;
+  L.conv_a = take((size_t)s.B * Cs * t1 * wr * sizeof(float));
+  L.conv_b = take((size_t)s.B * Cs * t1 * wr * sizeof(float));
   L.s_prob = take(rows * sizeof(float));
   L.s_mix = take(rows * sizeof(float));
   L.c_avg = take((s.causal ? rows : (size_t)s.B * s.H) * kHeadDim * sizeof(float));
   if (decoder_conv_tc(s, dec)) {
-    L.act0 = take((size_t)s.B * C * s.T * wr * 2 * sizeof(__nv_bfloat16));
-    L.w_tiles = take(3 * align_up(conv_tc_weight_bytes((int)C, 128, 1, 1), 256));  // 128: the most accumulator columns of a layer
+    L.act0 = take((size_t)s.B * Cs * s.T * wr * 2 * sizeof(__nv_bfloat16));
+    L.w_tiles = take(3 * align_up(conv_tc_weight_bytes((int)C), 256));
     if (mlp_tc_shape_ok(dec.d_hidden, (int)wr * dec.c_h)) L.mlp_w = take(mlp_tc_weight_bytes((int)wr * dec.c_h));
   }
   L.total = off;
@@ -408,7 +410,7 @@ static sea_status estimate_decoder_typed(const sea_shape& s, const sea_decoder& 
     // tensor-core form: activations as bf16 head / remainder planes, pixel-major
     char* act0 = dws + L.act0;
     char* wt = dws + L.w_tiles;
-    const size_t wt_step = align_up(conv_tc_weight_bytes(C, 128, 1, 1), 256);
+    const size_t wt_step = align_up(conv_tc_weight_bytes(C), 256);
     if (!mlp_tc && (rc = launch_nchw_to_nhwc_split(image, act0, s.B, C, s.T, wr, st)) != SEA_OK) return rc;
     if ((rc = launch_conv_tc(act0, s.B, C, s.T, wr, 1, 1, stride1, pad_top, dec.conv1_w, dec.conv1_b, C, 1, wt, conv_a, nullptr,
                              status, st)) != SEA_OK)

@@ -36,10 +36,11 @@ struct MlpTcParams {
   const void* V;                    // [rows][64], io dtype
   const float *b_mu, *b_1, *b_2;
   float* Z;                         // [rows][64]
-  __nv_bfloat16* act;               // [2][B][T][wr][H c_h]
+  __nv_bfloat16* act;               // [2][B][T][wr][cs]
   long long rows;
   int n_tiles, n3, n_chunks, chunk;
   int H, seq_len, c_h, wr, batch;
+  int cs;                           // channels per pixel of act: H c_h rounded up to a multiple of 64 (the rest stays zero)
   int hg, tiles_t;                  // heads per tile (a power of two dividing H, at most 32); tiles along the sequence per group of heads
   int32_t* status;
 };
@@ -199,7 +200,7 @@ mlp_tc_kernel(const __grid_constant__ CUtensorMap map_wmu, const __grid_constant
     const int r = warp * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
     const T* V = static_cast<const T*>(p.V);
-    const int C = p.H * p.c_h;
+    const int C = p.cs;  // channel stride of the feature map (H c_h rounded up to a multiple of 64)
     const size_t plane_elems = (size_t)p.batch * p.seq_len * p.wr * C;
     const bool fast = p.n_chunks == 1 && p.c_h == 4 && p.wr % 16 == 0;
     bool ok = true;
@@ -419,6 +420,10 @@ static sea_status launch_mlp_tc_typed(const sea_shape& s, const sea_decoder& dec
   p.wr = wr;
   p.batch = s.B;
   p.status = status;
+  p.cs = conv_tc_channels(s.H * dec.c_h);
+  if (p.cs != s.H * dec.c_h &&  // the channels beyond H c_h are written by nobody: zero
+      cudaMemsetAsync(act, 0, (size_t)2 * s.B * s.T * wr * p.cs * sizeof(__nv_bfloat16), st) != cudaSuccess)
+    return SEA_ERR_CUDA;
   CUtensorMap map_wmu, map_w1, map_w2;
   if (!make_map_bf16_3d(&map_wmu, wmu, 64, kMlHidden, 6, 64, kMlHidden) || !make_map_bf16_3d(&map_w1, w1, 64, kMlHidden, 2, 64, kMlHidden) ||
       !make_map_bf16_3d(&map_w2, w2, 64, n3, 2, 64, p.chunk))

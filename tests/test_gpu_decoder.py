@@ -83,12 +83,15 @@ def check_batch(run, b, check_z=True):
         check_float(np64(run.P[lo:hi]), P2, w.dtype, "P")
 
 
+# Images whose width divides 128 (or is a multiple of it) run the tensor-core convolutions with their
+# few channels in one block of 64; the others (12 columns) the fp32 ones.
 CASES = [
     small("dec_causal"),
     small("dec_nc", causal=False, H=3, T=96, Kc=24, k_hat=5),
     small("dec_f32", dtype="f32", T=64, Kc=8, k_hat=2, m=16),
     small("dec_nc_f32", dtype="f32", causal=False, T=64, Kc=16, k_hat=4, m=16, B=2),
     small("dec_wide", T=256, Kc=128, k_hat=9, H=4, m=64),       # image 64 columns wide: two column tiles, 16 channels
+    small("dec_causal_w12", T=96, Kc=24, k_hat=5),              # image 12 columns wide: the fp32 convolutions, causal
 ]
 
 
@@ -118,6 +121,8 @@ TC_CASES = [
     small("dec_tc_nc_ragged", causal=False, H=16, T=80, Kc=16, k_hat=3),
     small("dec_tc_causal_ragged", H=16, T=80, Kc=16, k_hat=3, B=2),
     small("dec_tc_wide", H=16, T=512, Kc=256, k_hat=8),   # Z_hat 512 wide: two chunks of W_2; image rows of 128 pixels
+    small("dec_tc_h12_nc", causal=False, H=12, T=128, Kc=32, k_hat=4),  # 48 channels in a block of 64, 48 of 64 logit columns
+    small("dec_tc_h12", H=12, T=160, Kc=32, k_hat=4, dtype="f32"),      # fp32 I/O; 24 of 32 logit columns; tiles of 4 heads
 ]
 
 
