@@ -335,7 +335,7 @@ static int conv_tc_columns(int c_out, int up_h, int up_w, bool logits) {
 
 // Shapes this form takes: at most 128 input channels and 128 accumulator columns after rounding
 // up, a row of the stored map made of whole boxes of min(w, 128) columns that divide 128, and
-// (strided layer) a height that is a multiple of the stride.  `logits`: the layer writes fp32 logits
+// (strided layer) a height that is a multiple of the stride, at least as many rows as a box has.  `logits`: the layer writes fp32 logits
 // with the resize's phases scattered; else bf16 planes for the next layer (no resize).
 bool conv_tc_shape_ok(int c_in, int c_out, int h_in, int w_in, int up_h, int up_w, int stride_h, bool logits) {
   if (c_in <= 0 || c_out <= 0 || up_h < 1 || up_w < 1 || stride_h < 1 || h_in <= 0 || w_in <= 0) return false;
@@ -344,6 +344,7 @@ bool conv_tc_shape_ok(int c_in, int c_out, int h_in, int w_in, int up_h, int up_
   if (conv_tc_channels(c_in) > 128 || conv_tc_columns(c_out, up_h, up_w, logits) > kCtMaxN) return false;
   if (128 % bw != 0 || w_in % bw != 0) return false;
   if (stride_h != 1 && (up_h != 1 || up_w != 1 || h_in % stride_h != 0)) return false;
+  if (h_in / stride_h < 128 / bw) return false;  // a copy box (128 / bw rows) no taller than the map
   return true;
 }
 
