@@ -602,7 +602,7 @@ def main():
                                   "sparse_attn_masked": sum(e[1].elapsed_time(e[2]) for e in gsev) / args.steps},
                     "nnz": int(row_ptr[-1])}
 
-        if w.Kc % 4 == 0 and w.H * w.Kc <= 32768:
+        if w.Kc % 4 == 0 and w.H * ((w.Kc + 31) // 32 + 1) <= 12288:
             grouped = time_bits_mode("causal-per-batch", sea.sea_attention_grouped, sea.sea_topk_mask_grouped)
         if w.causal:
             causal_aware = time_bits_mode("causal-aware per-query", sea.sea_attention_causal_aware,

@@ -179,7 +179,9 @@ sea_status sea_attention(const sea_shape* shape, const void* Q, const void* K, c
  * entries A_hat[b, :, t, :] are selected, with no exchange along T.  Equal values
  * (including -0 and +0) go to the lower flattened index h*Kc + c.  A row (b, h, t)
  * therefore keeps between 0 and min(Kc, H*k_hat) columns, and every (b, t) keeps
- * exactly H*k_hat over its heads.  Requires Kc % 4 == 0 and H*Kc <= 32768.
+ * exactly H*k_hat over its heads.  Requires Kc % 4 == 0 and H*(ceil(Kc/32) + 1) <=
+ * 12288 (the position's bit strings in shared memory); positions of more than 32768
+ * values are read several times instead of being kept in registers.
  *
  * mask_bits [rows, ceil(Kc/32)] uint32 receives the selection (bit c%32 of word
  * c/32 of a row is set when column c is kept; may be NULL).  The up-sampling and the

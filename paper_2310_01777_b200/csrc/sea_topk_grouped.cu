@@ -74,11 +74,16 @@ constexpr int kBins = 1 << kBinBits;
 constexpr uint32_t kFineMask = (1u << kFineBits) - 1u;
 constexpr int kListCap = 1024;
 
-template <int VI, int kThreadsMax, int kMinCtas>
+//
+// kStream: the position holds more keys than VI groups per thread (H * Kc > 4 VI blockDim.x).  The
+// threads then take the groups in n_pass passes of VI, and every step below that walks the keys
+// fetches them again pass by pass (from L2: a position's values are a few hundred KB) instead of
+// keeping them in registers; group (pass VI + i) blockDim.x + tid keeps the flattened order.
+template <int VI, int kThreadsMax, int kMinCtas, bool kStream>
 __global__ void __launch_bounds__(kThreadsMax, kMinCtas)
 topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask_bits,
                     int32_t* __restrict__ row_counts, int32_t* __restrict__ park_off, int H, int T, int Kc, int log2Kc,
-                    int k_sel, int r, int causal) {
+                    int k_sel, int r, int causal, int n_pass) {
   extern __shared__ uint32_t sh_dyn[];  // [H][words] bits, then [H] selected columns per head
   __shared__ int hist[kBins];
   __shared__ uint32_t list[kListCap];
@@ -116,21 +121,31 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
   const int per = 1 << log2per, log2owners = kBinBits - log2per, owners = 1 << log2owners;
 
   uint32_t key[VI][4];
-  uint32_t top = 0u;
+  // the keys of the thread's groups of pass `pass` (all of its groups when the keys stay in registers)
+  auto load_keys = [&](int pass) {
 #pragma unroll
-  for (int i = 0; i < VI; ++i) {
-    const int q = i * nthreads + tid;
-    key[i][0] = key[i][1] = key[i][2] = key[i][3] = 0u;  // below the key of every finite value
-    if (q < n4) {
-      int h, c;
-      split(4 * q, h, c);
-      const float4 v = __ldg(reinterpret_cast<const float4*>(A_hat + ((size_t)(b * H + h) * T + t) * Kc + c));
-      key[i][0] = order_key(v.x);
-      key[i][1] = order_key(v.y);
-      key[i][2] = order_key(v.z);
-      key[i][3] = order_key(v.w);
+    for (int i = 0; i < VI; ++i) {
+      const int q = (pass * VI + i) * nthreads + tid;
+      key[i][0] = key[i][1] = key[i][2] = key[i][3] = 0u;  // below the key of every finite value
+      if (q < n4) {
+        int h, c;
+        split(4 * q, h, c);
+        const float4 v = __ldg(reinterpret_cast<const float4*>(A_hat + ((size_t)(b * H + h) * T + t) * Kc + c));
+        key[i][0] = order_key(v.x);
+        key[i][1] = order_key(v.y);
+        key[i][2] = order_key(v.z);
+        key[i][3] = order_key(v.w);
+      }
     }
-    top = max(max(top, key[i][0]), max(key[i][1], max(key[i][2], key[i][3])));
+  };
+  const int passes = kStream ? n_pass : 1;
+  // SEA_EACH_PASS { body }: the body once per pass, with that pass's keys in key[][]
+#define SEA_EACH_PASS for (int pass = 0; pass < passes; ++pass) if (kStream ? (load_keys(pass), true) : true)
+  uint32_t top = 0u;
+  for (int pass = 0; pass < passes; ++pass) {
+    load_keys(pass);
+#pragma unroll
+    for (int i = 0; i < VI; ++i) top = max(max(top, key[i][0]), max(key[i][1], max(key[i][2], key[i][3])));
   }
   // ---- 1: the largest key
   top = __reduce_max_sync(0xffffffffu, top);
@@ -138,15 +153,17 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
   __syncthreads();  // also: the counters are zero
   top = __reduce_max_sync(0xffffffffu, lane < nwarps ? (uint32_t)red[0][lane] : 0u);
   // ---- 2: histogram of (top - key) >> kFineBits over the keys less than kBins steps below top
+  SEA_EACH_PASS {
 #pragma unroll
-  for (int i = 0; i < VI; ++i)
-    if (i * nthreads + tid < n4) {
+    for (int i = 0; i < VI; ++i)
+      if ((pass * VI + i) * nthreads + tid < n4) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const uint32_t x = (top - key[i][e]) >> kFineBits;
-        if (x < (uint32_t)kBins) atomicAdd(&hist[((x & (per - 1)) << log2owners) + (x >> log2per)], 1);
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t x = (top - key[i][e]) >> kFineBits;
+          if (x < (uint32_t)kBins) atomicAdd(&hist[((x & (per - 1)) << log2owners) + (x >> log2per)], 1);
+        }
       }
-    }
+  }
   __syncthreads();
   int n_gt = 0, n_eq = 0;
   uint32_t tau = 0u;
@@ -170,20 +187,24 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
       const uint32_t step = found[0];
       const int above = (int)found[1];
       int inside = 0;
+      SEA_EACH_PASS {
 #pragma unroll
-      for (int i = 0; i < VI; ++i)
+        for (int i = 0; i < VI; ++i)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) inside += key[i][e] != 0u && ((top - key[i][e]) >> kFineBits) == step;  // 0: a padding slot
+          for (int e = 0; e < 4; ++e) inside += key[i][e] != 0u && ((top - key[i][e]) >> kFineBits) == step;
+  }  // 0: a padding slot
       if (inside > 0) {
         int at = atomicAdd(&list_n, inside);
         if (at + inside <= kListCap) {
+          SEA_EACH_PASS {
 #pragma unroll
-          for (int i = 0; i < VI; ++i)
+            for (int i = 0; i < VI; ++i)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const uint32_t rel = top - key[i][e];
-              if (key[i][e] != 0u && (rel >> kFineBits) == step) list[at++] = kFineMask - (rel & kFineMask);  // grows with the key
-            }
+              for (int e = 0; e < 4; ++e) {
+                const uint32_t rel = top - key[i][e];
+                if (key[i][e] != 0u && (rel >> kFineBits) == step) list[at++] = kFineMask - (rel & kFineMask);  // grows with the key
+              }
+  }
         }
       }
       __syncthreads();  // also: every thread has read found[] before it is written again
@@ -236,61 +257,72 @@ topk_grouped_kernel(const float* __restrict__ A_hat, uint32_t* __restrict__ mask
     for (int bit = 31; bit >= 0; --bit) {
       const uint32_t cand = tau | (1u << bit);
       int c = 0;
+      SEA_EACH_PASS {
 #pragma unroll
-      for (int i = 0; i < VI; ++i)
+        for (int i = 0; i < VI; ++i)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) c += key[i][e] >= cand;
+          for (int e = 0; e < 4; ++e) c += key[i][e] >= cand;
+  }
       if (block_sum(c, red[rb], nwarps) >= k_sel) tau = cand;
       rb ^= 1;
     }
+    SEA_EACH_PASS {
 #pragma unroll
-    for (int i = 0; i < VI; ++i)
+      for (int i = 0; i < VI; ++i)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        n_gt += key[i][e] > tau;
-        n_eq += key[i][e] == tau;
-      }
+        for (int e = 0; e < 4; ++e) {
+          n_gt += key[i][e] > tau;
+          n_eq += key[i][e] == tau;
+        }
+  }
     n_gt = block_sum(n_gt, red[rb], nwarps);
     n_eq = block_sum(n_eq, red[rb ^ 1], nwarps);
   }
   const int need = k_sel - n_gt;  // how many keys equal to tau are taken (lowest flattened index first)
 
-  uint32_t taken = 0u;  // bit 4 i + e: element e of group i is selected
-  if (n_eq == need) {
-#pragma unroll
-    for (int i = 0; i < VI; ++i)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) taken |= (key[i][e] >= tau ? 1u : 0u) << (4 * i + e);
-  } else {
-    // more equal keys than places: rank them in flattened order (group index i-major, then thread)
-    int seen = 0;
-#pragma unroll
-    for (int i = 0; i < VI; ++i) {
-      int mine = 0;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) mine += key[i][e] == tau;
-      int total;
-      int rank = seen + block_exclusive_scan(mine, scan_tot, nwarps, total);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const bool eq = key[i][e] == tau;
-        const bool take = key[i][e] > tau || (eq && rank < need);
-        rank += eq;
-        taken |= (take ? 1u : 0u) << (4 * i + e);
-      }
-      seen += total;
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < VI; ++i) {
-    const uint32_t nib = (taken >> (4 * i)) & 15u;
-    const int q = i * nthreads + tid;
+  // the selected elements of a group, as bits of its head's string
+  auto emit = [&](int q, uint32_t nib) {
     if (nib != 0u && q < n4) {
       int h, c;
       split(4 * q, h, c);
       atomicOr(&sh_bits[h * words + (c >> 5)], nib << (c & 31));
     }
+  };
+  if (n_eq == need) {
+    SEA_EACH_PASS {
+#pragma unroll
+      for (int i = 0; i < VI; ++i) {
+        uint32_t nib = 0u;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) nib |= (key[i][e] >= tau ? 1u : 0u) << e;
+        emit((pass * VI + i) * nthreads + tid, nib);
+      }
   }
+  } else {
+    // more equal keys than places: rank them in flattened order (group index major, then thread)
+    int seen = 0;
+    SEA_EACH_PASS {
+#pragma unroll
+      for (int i = 0; i < VI; ++i) {
+        int mine = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mine += key[i][e] == tau;
+        int total;
+        int rank = seen + block_exclusive_scan(mine, scan_tot, nwarps, total);
+        uint32_t nib = 0u;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const bool eq = key[i][e] == tau;
+          const bool take = key[i][e] > tau || (eq && rank < need);
+          rank += eq;
+          nib |= (take ? 1u : 0u) << e;
+        }
+        emit((pass * VI + i) * nthreads + tid, nib);
+        seen += total;
+      }
+  }
+  }
+#undef SEA_EACH_PASS
   __syncthreads();
 
   // a thread per head: the row's bit string and its number of keys after up-sampling.  Column c
@@ -397,21 +429,24 @@ __global__ void park_offsets_kernel(const uint32_t* __restrict__ mask_bits, int3
   if (over) atomicOr(status, SEA_DEV_ROW_OVERFLOW);
 }
 
-template <int VI, int kThreadsMax, int kMinCtas>
+template <int VI, int kThreadsMax, int kMinCtas, bool kStream = false>
 void launch_grouped(const float* A_hat, uint32_t* mask_bits, int32_t* counts, int32_t* park_off, const sea_shape& s,
                     int threads, cudaStream_t st) {
   const size_t smem = ((size_t)s.H * ((s.Kc + 31) / 32) + s.H) * sizeof(uint32_t);
   int log2Kc = -1;
   for (int l = 0; l < 31; ++l)
     if ((1 << l) == s.Kc) log2Kc = l;
-  topk_grouped_kernel<VI, kThreadsMax, kMinCtas><<<s.B * s.T, threads, smem, st>>>(
-      A_hat, mask_bits, counts, park_off, s.H, s.T, s.Kc, log2Kc, s.H * s.k_hat, s.T / s.Kc, s.causal);
+  const int n_pass = (s.H * s.Kc / 4 + VI * threads - 1) / (VI * threads);
+  topk_grouped_kernel<VI, kThreadsMax, kMinCtas, kStream><<<s.B * s.T, threads, smem, st>>>(
+      A_hat, mask_bits, counts, park_off, s.H, s.T, s.Kc, log2Kc, s.H * s.k_hat, s.T / s.Kc, s.causal, n_pass);
 }
 
 }  // namespace
 
+// Rows of whole 16-byte groups, and the position's bit strings (with a word per head) within the
+// 48 KB of dynamic shared memory a kernel gets without asking.
 bool topk_grouped_supported(const sea_shape& s) {
-  return s.Kc % 4 == 0 && (long long)s.H * s.Kc <= 4ll * kMaxVI * kMaxThreads;
+  return s.Kc % 4 == 0 && ((long long)s.H * ((s.Kc + 31) / 32) + s.H) * 4 <= 48 * 1024 && (long long)s.H * s.Kc < (1ll << 30);
 }
 
 sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint32_t* mask_bits, int32_t* row_ptr,
@@ -432,8 +467,10 @@ sea_status launch_topk_mask_grouped(const sea_shape& s, const float* A_hat, uint
     else launch_grouped<4, 256, 6>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
   } else if (vi <= 4) {
     launch_grouped<4, kMaxThreads, 1>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
-  } else {
+  } else if (vi <= kMaxVI) {
     launch_grouped<8, kMaxThreads, 1>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
+  } else {  // more keys than a CTA's registers hold: several passes over the position's values
+    launch_grouped<8, kMaxThreads, 1, true>(A_hat, mask_bits, row_counts, park_off, s, threads, st);
   }
   sea_status rc = check_launch();
   if (rc != SEA_OK) return rc;

@@ -101,7 +101,7 @@ def test_grouped_entry_points_reject_bad_arguments_before_launch(lib):
     assert rc == binding.SEA_ERR_INVALID_ARG  # misaligned mask_bits
     rc = lib.sea_topk_mask_grouped(ctypes.byref(shp), fake, None, fake, None, 0, fake, 1024, None)
     assert rc == binding.SEA_ERR_WORKSPACE
-    big = sea.make_shape(WORKLOADS["long_32k"])  # H * Kc = 65536 values per position
+    big = sea.make_shape(WORKLOADS["long_32k"].scaled(H=256, T=2048, k_hat=1))  # a position's bit strings: 256 x 65 words > 48 KB
     rc = lib.sea_topk_mask_grouped(ctypes.byref(big), fake, None, fake, None, 0, fake, 1 << 40, None)
     assert rc == binding.SEA_ERR_UNSUPPORTED
     rc = lib.sea_sparse_attn_masked(ctypes.byref(shp), fake, fake, fake, fake, None, None, fake, None, None, 0, None)

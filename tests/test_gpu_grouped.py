@@ -152,6 +152,7 @@ GROUPED_CASES = [
     small("g_wide", dtype="bf16", H=4, T=2048, Kc=512, k_hat=24, causal=True, m=64), # 2048 values per position, 16 words per row
     small("g_many_heads", dtype="bf16", H=32, T=256, Kc=64, k_hat=8, causal=True, m=64),      # 2048 values, 4 groups per thread
     small("g_eight_per_thread", dtype="bf16", H=16, T=2048, Kc=512, k_hat=16, causal=True, m=64),  # 8192 values: 1024 threads x 2 groups
+    small("g_two_passes", H=36, T=1024, Kc=1024, k_hat=16, causal=True, m=64),  # 36864 values: more than a CTA's registers hold (fp32 I/O: with one key per column, O is as large as V and bf16 rounding alone would pass the absolute bound)
 ]
 
 
@@ -226,6 +227,25 @@ def test_grouped_ties_zeros_and_dominating_head():
     assert list(cols0[0]) == list(range(w.H * w.k_hat))
     for h in (0, 2):
         assert bool((run.O[0, h, 2:10] == 0).all())
+
+
+def test_grouped_ties_across_passes():
+    """A position with more values than the CTA keeps in registers (two passes over them) and many
+    duplicates: equal values still go to the lower flattened index, whichever pass holds them."""
+    w = small("g_ties_stream", H=36, T=1024, Kc=1024, k_hat=16, m=0)
+    host = make_inputs(w)
+    g = torch.Generator().manual_seed(6)
+    A = torch.round(torch.randn((w.B, w.H, w.T, w.Kc), generator=g) * 1.5) / 2
+    A[0, :, 0, :] = 0.25           # an all-equal position: the first H * k_hat flattened indices win
+    A[0, :, 1, :] = -3.0           # ... and one whose k-th largest value sits far below the largest
+    A[0, 35, 1, 1000:] = 7.0
+    host["A_hat"] = A.contiguous()
+    run = GroupedRun(w, inputs=host)
+    run.fused(); run.sync()
+    assert run.status() == 0
+    check_batch_against_oracle(run, 0, check_estimate=False)
+    cols0 = run.cols_of(0, 0)
+    assert list(cols0[0]) == list(range(w.H * w.k_hat))
 
 
 def test_grouped_with_one_head_equals_per_query_calls_bitwise():
