@@ -63,16 +63,6 @@ struct RowKeys<VPL, true> {
   // the key of column `col`, whichever lane owns it
   __device__ __forceinline__ void put(int col, uint32_t v) { base[(col / VPL) * kStride + (col % VPL)] = v; }
 };
-// A few keys of the lane's columns with their columns (ascending), the rest of the slots empty.
-template <int N>
-struct CandKeys {
-  static constexpr int kSlots = N;
-  static constexpr bool kDense = false;
-  uint32_t k[N];
-  int c[N];
-  __device__ __forceinline__ uint32_t get(int t) const { return k[t]; }
-};
-
 struct RowOut {
   int32_t* sel;      // the row's part of sel, or null
   uint32_t* words;   // the row's part of mask_bits, or null
@@ -217,7 +207,7 @@ __device__ __forceinline__ void select_row(const Keys& key, int* hist, int lane,
 
   int cnt = 0;
   int32_t* my_sel = out.sel != nullptr ? out.sel + taken_before : nullptr;
-  if constexpr (Keys::kDense) {
+  {
     for (uint64_t tk = take; tk != 0ull; tk &= tk - 1ull) {
       const int col = key.col0 + __ffsll((long long)tk) - 1;
       if (my_sel != nullptr) *my_sel++ = col;
@@ -237,23 +227,6 @@ __device__ __forceinline__ void select_row(const Keys& key, int* hist, int lane,
         if (lane % kLanes == 0 && lane / kLanes < out.n_words) out.words[lane / kLanes] = word;
       }
     }
-  } else {
-    // scattered columns: the bits are gathered in the warp's shared memory first
-    uint32_t* words = reinterpret_cast<uint32_t*>(hist);
-    __syncwarp();
-    for (int wv = lane; wv < out.n_words; wv += 32) words[wv] = 0u;
-    __syncwarp();
-#pragma unroll
-    for (int t = 0; t < N; ++t)
-      if ((take >> t) & 1ull) {
-        const int col = key.c[t];
-        if (my_sel != nullptr) *my_sel++ = col;
-        cnt += out.causal ? max(0, min(out.r, out.i + 1 - col * out.r)) : out.r;
-        if (out.words != nullptr) atomicOr(&words[col >> 5], 1u << (col & 31));
-      }
-    __syncwarp();
-    if (out.words != nullptr)
-      for (int wv = lane; wv < out.n_words; wv += 32) out.words[wv] = words[wv];
   }
   if (out.count != nullptr) {
     cnt = __reduce_add_sync(0xffffffffu, cnt);
@@ -261,7 +234,65 @@ __device__ __forceinline__ void select_row(const Keys& key, int* hist, int lane,
   }
 }
 
-constexpr int kCandSlots = 8;  // candidate keys a lane may bring to the second round
+// Selection among a short list of candidates (a wide row's entries at or above a lower bound of
+// its k_hat-th largest value): `list_key` / `list_col` hold n_c <= kListMax of them in ascending
+// column order, at least k_hat.  The smallest keys are struck off, all entries of a value at a
+// time, while k_hat would still remain: the value at which that stops is the k_hat-th largest key;
+// entries above it are selected, and of those equal to it the first (lowest columns) that are still
+// needed.  Lane l looks after entries l, l + 32, l + 64.
+constexpr int kListMax = 96;
+__device__ __forceinline__ void select_from_list(const uint32_t* list_key, const int* list_col, int n_c, uint32_t* words,
+                                                 int lane, int k_hat, const RowOut& out) {
+  constexpr uint32_t kGone = 0xffffffffu;  // no finite value has this key
+  uint32_t a[3];
+  int col[3];
+#pragma unroll
+  for (int i = 0; i < 3; ++i) {
+    const int idx = lane + 32 * i;
+    a[i] = idx < n_c ? list_key[idx] : kGone;
+    col[i] = idx < n_c ? list_col[idx] : 0;
+  }
+  int remaining = n_c;
+  uint32_t tau;
+  int ties_needed;
+  for (;;) {
+    tau = __reduce_min_sync(0xffffffffu, min(a[0], min(a[1], a[2])));
+    const int c = __popc(__ballot_sync(0xffffffffu, a[0] == tau)) + __popc(__ballot_sync(0xffffffffu, a[1] == tau)) +
+                  __popc(__ballot_sync(0xffffffffu, a[2] == tau));
+    if (remaining - c < k_hat) {
+      ties_needed = k_hat - (remaining - c);
+      break;
+    }
+    remaining -= c;
+#pragma unroll
+    for (int i = 0; i < 3; ++i) a[i] = a[i] == tau ? kGone : a[i];
+  }
+  for (int wv = lane; wv < out.n_words; wv += 32) words[wv] = 0u;
+  __syncwarp();
+  const uint32_t below = (1u << lane) - 1u;
+  int ties_before = 0, taken_before = 0, cnt = 0;
+#pragma unroll
+  for (int i = 0; i < 3; ++i) {
+    const bool alive = a[i] != kGone;
+    const uint32_t eq = __ballot_sync(0xffffffffu, alive && a[i] == tau);
+    const bool take = alive && (a[i] > tau || (a[i] == tau && ties_before + __popc(eq & below) < ties_needed));
+    const uint32_t tk = __ballot_sync(0xffffffffu, take);
+    if (take) {
+      if (out.sel != nullptr) out.sel[taken_before + __popc(tk & below)] = col[i];
+      cnt += out.causal ? max(0, min(out.r, out.i + 1 - col[i] * out.r)) : out.r;
+      if (out.words != nullptr) atomicOr(&words[col[i] >> 5], 1u << (col[i] & 31));
+    }
+    ties_before += __popc(eq);
+    taken_before += __popc(tk);
+  }
+  __syncwarp();
+  if (out.words != nullptr)
+    for (int wv = lane; wv < out.n_words; wv += 32) out.words[wv] = words[wv];
+  if (out.count != nullptr) {
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if (lane == 0) *out.count = cnt;
+  }
+}
 
 template <int VPL, bool kShared>
 __global__ void __launch_bounds__(kWarpsPerCta * 32, kShared ? 3 : 4)
@@ -292,12 +323,12 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
     // A wide row first sheds most of its values.  The row is fetched as 16-byte pieces (lane l takes
     // pieces l, l + 32, ...) and parked in the warp's shared memory as it is; while fetching, every
     // lane keeps the two largest values it met.  Those are 64 different entries of the row, so the
-    // k_hat-th largest of the 64, L (found bit by bit with ballots on their keys), has at least
-    // k_hat entries at or above it: every selected entry is >= L, and usually few more than k_hat
-    // are (L = 0 when fewer than k_hat of the 64 hold a column: no shortcut then).  Each lane then
-    // reads back its own VPL consecutive columns (piece q sits at q ^ (owner lane & 7): neither the
-    // writes nor these reads meet bank conflicts), and the entries >= L go, with their columns and in
-    // column order, through the same selection on kCandSlots slots per lane.
+    // k_hat-th largest of the 64 (found bit by bit with ballots on their keys) has at least k_hat
+    // entries at or above it, and so has any bound L below it: every selected entry is >= L, and few
+    // more than k_hat entries are (L = 0 when fewer than k_hat of the 64 hold a column: no shortcut
+    // then).  Each lane then reads back its own VPL consecutive columns (piece q sits at q ^ (owner
+    // lane & 7): neither the writes nor these reads meet bank conflicts); the entries >= L go, in
+    // column order, to a short list and select_from_list finishes the row.
     if (k_hat <= 32 && Kc_all % 4 == 0) {
       constexpr int kPerLane = VPL / 4;  // pieces of a lane's own columns
       static_assert(kPerLane >= 8, "the swizzle takes the owner's low three bits");
@@ -321,15 +352,17 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
         }
       }
       const uint32_t top1 = f1 == -INFINITY ? 0u : order_key(f1), top2 = f2 == -INFINITY ? 0u : order_key(f2);
+      // (the upper 16 bits of the k_hat-th largest key are bound enough: the values between that and
+      // the key itself are a 128th of an octave)
       uint32_t low = 0u;
 #pragma unroll 1
-      for (int bit = 31; bit >= 0; --bit) {
+      for (int bit = 31; bit >= 16; --bit) {
         const uint32_t c = low | (1u << bit);
         if (__popc(__ballot_sync(0xffffffffu, top1 >= c)) + __popc(__ballot_sync(0xffffffffu, top2 >= c)) >= k_hat) low = c;
       }
       __syncwarp();
       if (low != 0u) {
-        // L is the key of one of the 64 values: back to that value
+        // from the key back to the value it stands for
         const float low_f = __uint_as_float((low & 0x80000000u) ? (low ^ 0x80000000u) : ~low);
         uint64_t cand = 0ull;
 #pragma unroll
@@ -338,21 +371,29 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
           cand |= (uint64_t)((v.x >= low_f ? 1u : 0u) | (v.y >= low_f ? 2u : 0u) | (v.z >= low_f ? 4u : 0u) | (v.w >= low_f ? 8u : 0u))
                   << (4 * j);
         }
-        if (__reduce_max_sync(0xffffffffu, __popcll(cand)) <= kCandSlots) {
-          const float* words = reinterpret_cast<const float*>(stage);
-          CandKeys<kCandSlots> ck;
+        // the candidates in column order: lane by lane, each lane's in ascending order
+        const int mine = __popcll(cand);
+        int inc = mine;
 #pragma unroll
-          for (int j = 0; j < kCandSlots; ++j) {
-            ck.k[j] = 0u;
-            ck.c[j] = 0;
-            if (cand != 0ull) {
-              const int t = __ffsll((long long)cand) - 1;
-              cand &= cand - 1ull;
-              ck.k[j] = order_key(words[4 * ((lane * kPerLane + (t >> 2)) ^ (lane & 7)) + (t & 3)]);
-              ck.c[j] = col0 + t;
-            }
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += v;
+        }
+        const int n_c = __shfl_sync(0xffffffffu, inc, 31);
+        if (n_c <= kListMax) {
+          const float* vals = reinterpret_cast<const float*>(stage);
+          uint32_t* list_key = reinterpret_cast<uint32_t*>(hist_all[warp]);
+          int* list_col = hist_all[warp] + kListMax;
+          uint32_t* words = reinterpret_cast<uint32_t*>(hist_all[warp]) + 2 * kListMax;
+          static_assert(2 * kListMax + 64 <= kHistBins, "the lists and the row's bit words share the histogram's words");
+          int at = inc - mine;
+          for (; cand != 0ull; cand &= cand - 1ull, ++at) {
+            const int t = __ffsll((long long)cand) - 1;
+            list_key[at] = order_key(vals[4 * ((lane * kPerLane + (t >> 2)) ^ (lane & 7)) + (t & 3)]);
+            list_col[at] = col0 + t;
           }
-          select_row(ck, hist_all[warp], lane, k_hat, out);
+          __syncwarp();
+          select_from_list(list_key, list_col, n_c, words, lane, k_hat, out);
           return;
         }
       }
