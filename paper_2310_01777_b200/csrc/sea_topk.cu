@@ -331,7 +331,10 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
     // column order, to a short list and select_from_list finishes the row.
     if (k_hat <= 32 && Kc_all % 4 == 0) {
       constexpr int kPerLane = VPL / 4;  // pieces of a lane's own columns
-      static_assert(kPerLane >= 8, "the swizzle takes the owner's low three bits");
+      static_assert(kPerLane >= 4, "the swizzle needs at least four pieces per lane");
+      // where piece q is parked: eight neighbouring pieces, and the j-th pieces of eight neighbouring
+      // lanes, fall on eight different 16-byte bank groups
+      auto parked = [](int q) { return kPerLane >= 8 ? q ^ ((q / kPerLane) & 7) : q ^ ((q >> 3) & 3); };
       float4* stage = reinterpret_cast<float4*>(keys_all + warp * (VPL + 1) * 32);
       float f1 = -INFINITY, f2 = -INFINITY;  // columns that do not compete count as -inf (inputs are finite)
 #pragma unroll 4
@@ -343,7 +346,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
           if (4 * q + 2 >= Kc) v.z = -INFINITY;
           v.w = -INFINITY;
         }
-        stage[q ^ ((q / kPerLane) & 7)] = v;
+        stage[parked(q)] = v;
         const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -367,7 +370,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
         uint64_t cand = 0ull;
 #pragma unroll
         for (int j = 0; j < kPerLane; ++j) {
-          const float4 v = stage[(lane * kPerLane + j) ^ (lane & 7)];
+          const float4 v = stage[parked(lane * kPerLane + j)];
           cand |= (uint64_t)((v.x >= low_f ? 1u : 0u) | (v.y >= low_f ? 2u : 0u) | (v.z >= low_f ? 4u : 0u) | (v.w >= low_f ? 8u : 0u))
                   << (4 * j);
         }
@@ -389,7 +392,7 @@ topk_rows_kernel(const float* __restrict__ A_hat, int32_t* __restrict__ sel,
           int at = inc - mine;
           for (; cand != 0ull; cand &= cand - 1ull, ++at) {
             const int t = __ffsll((long long)cand) - 1;
-            list_key[at] = order_key(vals[4 * ((lane * kPerLane + (t >> 2)) ^ (lane & 7)) + (t & 3)]);
+            list_key[at] = order_key(vals[4 * parked(lane * kPerLane + (t >> 2)) + (t & 3)]);
             list_col[at] = col0 + t;
           }
           __syncwarp();
@@ -657,7 +660,7 @@ template <int VPL>
 bool launch_topk(const float* A_hat, int32_t* sel, int32_t* counts, uint32_t* mask_bits, int rows,
                  const sea_shape& s, bool aware, cudaStream_t st) {
   const int grid = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
-  constexpr bool kShared = VPL >= 32;  // beyond 512 columns the keys no longer fit the registers
+  constexpr bool kShared = VPL >= 16;  // from 512 columns on the row is parked in shared memory (beyond that its keys would not fit the registers)
   const size_t smem = kShared ? (size_t)kWarpsPerCta * (VPL + 1) * 32 * sizeof(uint32_t) : 0;
   auto kern = topk_rows_kernel<VPL, kShared>;
   if (smem > 40 * 1024 && cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
