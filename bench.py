@@ -32,8 +32,9 @@ metric is quoted.  One JSON line is printed by rank 0.
   structured_mask
              the mask and sparse stages when the caller gives a banded estimate (the structure of
              trained SEA masks): the tile kernel skips the key tiles nothing was selected in.
-  decoder_head  (--decoder) the layer with the paper's estimator head (MLPs + three-layer CNN, random-init
-             weights) and output mixing through sea_attention_decoder: MLPs and convolutions on tcgen05.
+  decoder_head  the layer with the paper's estimator head (MLPs + three-layer CNN, random-init
+             weights) and output mixing through sea_attention_decoder, MLPs and convolutions on
+             tcgen05 (timed by default up to T = 2048; longer shapes with --decoder).
   cpu_baseline  the fp64 oracle on a bounded sample of heads, one head per host core at a time.
 
 With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no
@@ -392,7 +393,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-modes", action="store_true", help="skip the grouped / causal-aware / lean regions")
     ap.add_argument("--soak-s", type=float, default=1.2, help="seconds of steps the clock sampler watches")
-    ap.add_argument("--decoder", action="store_true", help="also time the paper's MLP + CNN estimator head (a few ms per step)")
+    ap.add_argument("--decoder", action="store_true",
+                    help="time the paper's MLP + CNN estimator head (a few ms per step) even with --no-modes; without "
+                         "--no-modes it is timed anyway on the workloads of up to 2048 tokens per sequence")
+    ap.add_argument("--no-decoder", action="store_true", help="skip the estimator-head region")
     ap.add_argument("--capped-sweep", action="store_true", help="time the paper's long-sequence sweep shape instead")
     ap.add_argument("--sweep-B", type=int, default=1)
     ap.add_argument("--sweep-H", type=int, default=12)
@@ -640,7 +644,8 @@ def main():
         torch.cuda.synchronize(dev)
 
     decoder = None
-    if args.decoder:
+    # the estimator head's buffers grow with T * Kc per head and channel: the long-context shapes only on request
+    if (args.decoder or (not args.no_modes and w.T <= 2048)) and not args.no_decoder:
         # ---- timed region 6: the paper's estimator head (MLPs + three-layer CNN) with random-init weights ----
         from paper_2310_01777_b200.inputs import make_decoder_params
 
