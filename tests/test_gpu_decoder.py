@@ -152,3 +152,49 @@ def test_causal_decoder_on_device_does_not_look_ahead():
     b.fused(); b.done()
     assert torch.equal(a.A_hat[:, :, :t + 1], b.A_hat[:, :, :t + 1])
     assert torch.equal(a.O[:, :, :t + 1], b.O[:, :, :t + 1])
+
+
+def test_decoder_head_full_size_on_row_windows():
+    """The OPT-1.3B-shaped workload with d' = 64, c_s = 2, c_h = 4 (128 channels: the shape the
+    benchmark times, both blocks of input channels, two-row pixel tiles): Z for every row of one
+    batch element, the estimate on two windows of rows.  A causal layer's row depends on the rows
+    above it only, so the oracle's CNN runs on crops: the first rows as they are, later rows with
+    six rows of context above them (three layers, two rows each)."""
+    from paper_2310_01777_b200.inputs import WORKLOADS
+    w = WORKLOADS["opt_1p3b"]
+    a = Run(w, d_hidden=64, c_s=2, c_h=4)
+    d = a.d
+    sea.sea_estimate_decoder(a.shape, a.dec, d["Q"], d["K"], d["V"], d["omega"], a.A_hat, a.Z, a.ws)
+    a.done()
+    assert bool(torch.isfinite(a.A_hat).all())
+    b = w.B - 1
+    prm = {k: np64(v) for k, v in a.hp.items()}
+    Q, K, V = (np64(a.host[n][b]) for n in ("Q", "K", "V"))
+    omega = np64(a.host["omega"])
+    Z = np.stack([dec.mlp_mu(dec.performer_cat(Q[h], K[h], V[h], prm["pos_emb"], omega, True), V[h], prm["W_mu"], prm["b_mu"])
+                  for h in range(w.H)])
+    check_a_hat(a.Z[b].cpu().numpy().reshape(w.H * w.T, -1), Z.reshape(w.H * w.T, -1))
+    Z_hat = np.stack([dec.mlp_nu(Z[h], prm["W_nu1"], prm["b_nu1"], prm["W_nu2"], prm["b_nu2"]) for h in range(w.H)])
+    image = dec.to_image(Z_hat, a.c_h)
+    A = a.A_hat[b].cpu().numpy()
+    for lo, hi in ((0, 200), (w.T - 150, w.T)):
+        top = max(0, lo - 6)
+        ref = dec.cnn_decoder(image[:, top:hi], prm, hi - top, w.Kc, a.c_s, True)[:, lo - top:]
+        check_a_hat(A[:, lo:hi].reshape(-1, w.Kc), ref.reshape(-1, w.Kc))
+
+
+def test_decoder_head_full_size_not_causal():
+    """The BERT-base-shaped workload (12 heads: 48 channels in one block of 64; strided first layer,
+    four phases of the folded resize): estimate and Z of one batch element, element by element."""
+    from paper_2310_01777_b200.inputs import WORKLOADS
+    w = WORKLOADS["bert_base"]
+    a = Run(w, d_hidden=64, c_s=2, c_h=4)
+    d = a.d
+    sea.sea_estimate_decoder(a.shape, a.dec, d["Q"], d["K"], d["V"], d["omega"], a.A_hat, a.Z, a.ws)
+    a.done()
+    b = w.B - 1
+    prm = {k: np64(v) for k, v in a.hp.items()}
+    Q, K, V = (np64(a.host[n][b]) for n in ("Q", "K", "V"))
+    A_ref, Z_ref = dec.decoder_estimate(Q, K, V, np64(a.host["omega"]), prm, w.Kc, a.c_s, a.c_h, False)
+    check_a_hat(a.A_hat[b].cpu().numpy().reshape(-1, w.Kc), A_ref.reshape(-1, w.Kc))
+    check_a_hat(a.Z[b].cpu().numpy().reshape(w.H * w.T, -1), Z_ref.reshape(w.H * w.T, -1))
