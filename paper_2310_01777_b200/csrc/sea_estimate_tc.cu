@@ -422,9 +422,9 @@ enum {
   kO_Phi,                  // phi(Q): every row warp has written its first chunk of features ...
   kO_Phi2,                 // ... and all of them
   kO_A, kO_P, kO_Num, kO_C,
-  kO_W,                    // [2] decoder columns staged
-  kO_WDone = kO_W + 2,     // [2] the MMAs that read them are complete
-  kO_Ahat = kO_WDone + 2,  // [2] A_hat tile in tensor memory
+  kO_W,                    // [3] decoder columns staged (the third place only when a row of A_hat takes three passes or more)
+  kO_WDone = kO_W + 3,     // [3] the MMAs that read them are complete
+  kO_Ahat = kO_WDone + 3,  // [2] A_hat tile in tensor memory
   kO_AFree = kO_Ahat + 2,  // [2] rows have read it
   kO_Drain = kO_AFree + 2,
   kO_NumBars
@@ -565,7 +565,22 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       bool ok = true;
       uint32_t it = 0;          // items done: parity of the per-item barriers
       uint32_t g = 0;           // decoder passes issued so far: pass g uses buffers g & 1
-      uint32_t w_next = 0;      // decoder passes whose columns have been requested
+      // Places for the decoder's column tiles: the two halves of phi(K)'s area, and - when a row of
+      // A_hat takes three passes or more - omega's, which is free between an item's projections and
+      // the next item's: the passes ct = om_ct (mod 3) read from there, the last of them is pass
+      // n_ct - 2, and omega' is copied in again once that pass's products are complete.  With three
+      // places a tile is asked for two passes before its turn instead of one.
+      const bool three = n_ct >= 3;
+      const int om_ct = three ? (n_ct - 2) % 3 : -1;
+      auto slot_of = [&](int ct, uint32_t pass) -> int {  // pass: the running number of the pass (for the two-place rotation)
+        if (!three) return (int)(pass & 1u);
+        const int q = (ct - om_ct + 3) % 3;
+        return q == 0 ? 2 : q - 1;
+      };
+      uint32_t w_loads[3] = {0u, 0u, 0u};  // tiles requested per place
+      uint32_t w_uses[3] = {0u, 0u, 0u};   // passes issued per place
+      uint32_t w_next = 0;                 // decoder passes whose columns have been requested
+      uint32_t om_loads = 1;               // copies of omega' requested
       uint32_t afree_next = 0;  // decoder passes whose tile the rows are known to have read
       auto load_qk = [&](int item) {
         if (!leader) return;
@@ -596,17 +611,25 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
           bulk_load(smem_u32(z_s), p.z_prefix + (size_t)(state_idx / 2) * MP, MP * 4, bar(kO_VS));
         }
       };
-      // decoder columns of pass number w_next (column tile ct of its item) into buffer w_next & 1
+      // decoder columns of column tile ct of the current item into their place
       auto load_w = [&](int ct) {
-        const int b = w_next & 1;
-        const uint32_t dst = smem_u32(sPhi) + b * 2 * kTileBytes;
+        const int sl = slot_of(ct, w_next);
+        const uint32_t dst = sl < 2 ? smem_u32(sPhi) + sl * 2 * kTileBytes : smem_u32(sOm);
         if (leader) {
-          mbar_expect_tx(bar(kO_W + b), 4 * 8192);
+          mbar_expect_tx(bar(kO_W + sl), 4 * 8192);
           for (int part = 0; part < 2; ++part)
             for (int atom = 0; atom < 2; ++atom)
-              tma_load_3d(dst + part * kTileBytes + atom * 8192, &map_w, ct * kWTile + 64 * atom, 0, part, bar(kO_W + b));
+              tma_load_3d(dst + part * kTileBytes + atom * 8192, &map_w, ct * kWTile + 64 * atom, 0, part, bar(kO_W + sl));
         }
+        ++w_loads[sl];
         ++w_next;
+      };
+      auto load_om = [&]() {
+        if (leader) {
+          mbar_expect_tx(bar(kO_Om), 2 * MP * 128);
+          tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kO_Om));
+          tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kO_Om));
+        }
       };
       auto wait_afree_upto = [&](uint32_t upto) {  // the rows have read the tiles of passes 0 .. upto-1
         while (ok && afree_next < upto) {
@@ -616,11 +639,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       };
       const int first = blockIdx.x;
       if (first < n_items) {
-        if (leader) {
-          mbar_expect_tx(bar(kO_Om), 2 * MP * 128);
-          tma_load_3d(smem_u32(sOm), &map_om, 0, 0, 0, bar(kO_Om));
-          tma_load_3d(smem_u32(sOm) + kTileBytes, &map_om, 0, 0, 1, bar(kO_Om));
-        }
+        load_om();
         load_qk(first);
         load_vs(first);
         __syncwarp();
@@ -637,7 +656,12 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         // columns were: the rows have read the former (which also means the MMAs that read the
         // latter are complete); with a tile region of its own only the MMAs matter
         if (!single) wait_afree_upto(g);
-        else if (ok && g > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_WDone + ((g - 1) & 1)), ((g - 1) >> 1) & 1, abort_flag));
+        else if (ok && g > 0) {
+          const int ps = (int)((g - 1) & 1u);
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_WDone + ps), (w_uses[ps] - 1) & 1, abort_flag));
+        }
+        // omega' is back (it made room for decoder columns during the previous item's passes)
+        if (ok && three) ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_Om), (om_loads - 1) & 1, abort_flag));
         if (!ok) break;
         fence_after();
         if (causal) load_phik(item);
@@ -717,6 +741,7 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         // decoder columns of this item's first passes
         load_w(0);
         if (n_ct > 1) load_w(1);
+        if (three) load_w(2);  // omega's place: the projections were complete before the rows wrote phi(Q)
         if (causal) {
           constexpr uint32_t idN = idesc_bf16(64, false, true);
           const uint64_t bv0 = smem_desc(smem_u32(sV), kTileBytes, 1024);
@@ -741,13 +766,14 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         constexpr uint32_t idW = idesc_bf16(kWTile, false, true);
         for (int ct = 0; ct < n_ct && ok; ++ct, ++g) {
           const uint32_t b = g & 1;
-          ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_W + b), (g >> 1) & 1, abort_flag));
+          const int sl = slot_of(ct, g);
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_W + sl), w_uses[sl] & 1, abort_flag));
           // the rows have read the tile that was in this buffer
           if (single) wait_afree_upto(g);
           else if (g >= 2) wait_afree_upto(g - 1);
           if (!ok) break;
           fence_after();
-          const uint32_t wbase = smem_u32(sPhi) + b * 2 * kTileBytes;
+          const uint32_t wbase = sl < 2 ? smem_u32(sPhi) + sl * 2 * kTileBytes : smem_u32(sOm);
           const uint32_t d = tmem + (single ? kColAh : (b ? kColA : kColQ));
           const uint64_t wh0 = smem_desc(wbase, 8192, 1024), wl0 = smem_desc(wbase + kTileBytes, 8192, 1024);
           if (leader) {
@@ -759,13 +785,26 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
               mma_ts(d, a + 16, wh0 + 128 * k, idW, 1);
             }
             mma_commit(bar(kO_Ahat + b));
-            mma_commit(bar(kO_WDone + b));
+            mma_commit(bar(kO_WDone + sl));
           }
+          ++w_uses[sl];
           __syncwarp();
-          if (ct >= 1 && ct + 1 < n_ct) {
-            // columns of the next pass go where the previous pass read from
-            ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_WDone + (b ^ 1)), ((g - 1) >> 1) & 1, abort_flag));
-            if (ok) load_w(ct + 1);
+          if (ct >= 1 && (three || ct + 1 < n_ct)) {
+            // the place the previous pass read from takes the columns of the pass that comes
+            // round to it next (one pass on with two places, two with three), or omega' again
+            const int ps = slot_of(ct - 1, g - 1);
+            const int ct_new = ct + (three ? 2 : 1);
+            if (ct_new < n_ct || (ps == 2 && next < n_items)) {
+              ok = __all_sync(0xffffffffu, mbar_wait(bar(kO_WDone + ps), (w_uses[ps] - 1) & 1, abort_flag));
+              if (ok) {
+                if (ct_new < n_ct) {
+                  load_w(ct_new);
+                } else {
+                  load_om();
+                  ++om_loads;
+                }
+              }
+            }
           }
         }
       }
@@ -775,11 +814,12 @@ favor_output_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       // copies still in flight must land before the CTA may leave (only after a wait ran out can
       // any be outstanding here: every armed phase is waited for in the loop above)
       if (!ok) {
-        mbar_wait_drain(bar(kO_Om), 0);
+        mbar_wait_drain(bar(kO_Om), (om_loads - 1) & 1);
         mbar_wait_drain(bar(kO_QK), it & 1);
         mbar_wait_drain(bar(kO_VS), it & 1);
         if (causal) mbar_wait_drain(bar(kO_PhiK), it & 1);
-        for (uint32_t w = (w_next >= 2 ? w_next - 2 : 0); w < w_next; ++w) mbar_wait_drain(bar(kO_W + (w & 1)), (w >> 1) & 1);
+        for (int sl = 0; sl < 3; ++sl)
+          if (w_loads[sl] > 0) mbar_wait_drain(bar(kO_W + sl), (w_loads[sl] - 1) & 1);
       }
     }
   } else {
