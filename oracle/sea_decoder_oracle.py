@@ -30,7 +30,7 @@ Steps, in the paper's order (readings where the paper is silent are marked R):
                     attention's output; the CSR probabilities are s_prob * softmax.
 
 Parity unpinned: the weight draws (only their seed is fixed); the readings marked R are choices
-where the paper gives no detail (they are listed in the design doc), pinned only in the sense that the
+where the paper gives no detail (each is stated in the list of steps above), pinned only in the sense that the
 library routines used here are checked against explicit loops.
 """
 from __future__ import annotations
