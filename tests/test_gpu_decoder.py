@@ -121,6 +121,7 @@ TC_CASES = [
     small("dec_tc_nc_ragged", causal=False, H=16, T=80, Kc=16, k_hat=3),
     small("dec_tc_causal_ragged", H=16, T=80, Kc=16, k_hat=3, B=2),
     small("dec_tc_wide", H=16, T=512, Kc=256, k_hat=8),   # Z_hat 512 wide: two chunks of W_2; image rows of 128 pixels
+    small("dec_tc_two_tiles", H=16, T=512, Kc=512, k_hat=8),  # image 256 pixels wide: two column tiles per row, Z_hat in four chunks
     small("dec_tc_h12_nc", causal=False, H=12, T=128, Kc=32, k_hat=4),  # 48 channels in a block of 64, 48 of 64 logit columns
     small("dec_tc_h12", H=12, T=160, Kc=32, k_hat=4, dtype="f32"),      # fp32 I/O; 24 of 32 logit columns; tiles of 4 heads
 ]
